@@ -1,0 +1,145 @@
+"""TEST INFRASTRUCTURE — Python entry to the CPU oracle (oracle/ccr_oracle.cpp).
+
+Only tests, the smoke check and the benchmark's cpu_baseline / reference legs may import this.
+It does not import the product package and the product package never imports it; the oracle
+takes plain numpy arrays (or any object with the attribute names used below).
+
+`build()` compiles the C++ with g++ into oracle/libccr_oracle.so (building the checker is not
+using it); `join(...)` runs Eq. 1 / Algorithm 1 steps 2-4 of the paper plus the doc-row gather and
+request broadcast for a ragged batch and returns (out_rows uint8[C, out_b], out_mask uint8[C]).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ccr_oracle.cpp")
+_LIB = os.path.join(_HERE, "libccr_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    with _lock:
+        stale = force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if stale:
+            tmp = _LIB + ".tmp.%d" % os.getpid()
+            cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fPIC", "-shared", "-pthread", _SRC, "-o", tmp]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, i64, i32, u64 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint64
+        lib.ccr_oracle_join.restype = ctypes.c_int
+        lib.ccr_oracle_join.argtypes = [
+            i64, vp, i64, vp, i32, vp, vp, i32, i32, u64,
+            i32, vp, vp, vp, vp, vp, vp, i64, i32, vp, vp, i32,
+        ]
+        lib.ccr_oracle_half_to_float_bits.restype = ctypes.c_uint32
+        lib.ccr_oracle_half_to_float_bits.argtypes = [ctypes.c_uint16]
+        lib.ccr_oracle_float_bits_to_half.restype = ctypes.c_uint16
+        lib.ccr_oracle_float_bits_to_half.argtypes = [ctypes.c_uint32]
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype=None):
+    if a is None:
+        return None
+    a = np.ascontiguousarray(a) if dtype is None else np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def out_row_bytes(doc_feats, edge_feats, req_feats, max_actors: int, first_degree_only: bool) -> int:
+    doc_b = doc_feats.shape[1] * doc_feats.dtype.itemsize
+    edge_b = edge_feats.shape[1] * edge_feats.dtype.itemsize
+    req_b = 0 if req_feats is None else req_feats.shape[1] * req_feats.dtype.itemsize
+    second = max_actors > 0 and not first_degree_only
+    return doc_b + edge_b + (edge_b if second else 0) + req_b
+
+
+def join(
+    doc_feats: np.ndarray,
+    author_ids: np.ndarray,
+    edge_keys: np.ndarray,
+    edge_feats: np.ndarray,
+    edge_offsets: np.ndarray,
+    cand_idx: np.ndarray,
+    cand_offsets: np.ndarray,
+    req_feats: Optional[np.ndarray] = None,
+    actor_ids: Optional[np.ndarray] = None,
+    actor_types: Optional[np.ndarray] = None,
+    reduce_sum_mask: int = 0,
+    first_degree_only: bool = False,
+    n_threads: int = 1,
+) -> Tuple[np.ndarray, np.ndarray]:
+    lib = _load()
+    doc_feats = _c(doc_feats)
+    author_ids = _c(author_ids, np.int64)
+    edge_keys = _c(edge_keys, np.int64)
+    edge_feats = _c(edge_feats)
+    edge_offsets = _c(edge_offsets, np.int64)
+    cand_idx = _c(cand_idx, np.int32)
+    cand_offsets = _c(cand_offsets, np.int64)
+    req_feats = _c(req_feats)
+    max_actors = 0
+    if actor_ids is not None:
+        actor_ids = _c(actor_ids, np.int64)
+        actor_types = _c(actor_types, np.uint8)
+        max_actors = int(actor_ids.shape[1])
+    if doc_feats.ndim != 2 or edge_feats.ndim != 2:
+        raise ValueError("doc_feats and edge_feats are 2-D")
+    n_docs = int(doc_feats.shape[0])
+    if author_ids.shape[0] != n_docs:
+        raise ValueError("author_ids length differs from the store's row count")
+    n_req = int(len(cand_offsets) - 1)
+    if len(edge_offsets) != n_req + 1:
+        raise ValueError("offset arrays disagree on the request count")
+    total = int(cand_offsets[-1]) if n_req > 0 else 0
+    out_b = out_row_bytes(doc_feats, edge_feats, req_feats, max_actors, first_degree_only)
+    out_rows = np.full((total, out_b), 0xCD, dtype=np.uint8)  # poison: every byte must be written
+    out_mask = np.full(total, 0xCD, dtype=np.uint8)
+    rc = lib.ccr_oracle_join(
+        n_docs, _ptr(doc_feats), doc_feats.shape[1] * doc_feats.dtype.itemsize, _ptr(author_ids),
+        max_actors, _ptr(actor_ids), _ptr(actor_types),
+        int(edge_feats.shape[1]), int(edge_feats.dtype.itemsize), int(reduce_sum_mask) & (2**64 - 1),
+        n_req, _ptr(edge_keys), _ptr(edge_feats), _ptr(edge_offsets), _ptr(cand_idx), _ptr(cand_offsets),
+        _ptr(req_feats), 0 if req_feats is None else req_feats.shape[1] * req_feats.dtype.itemsize,
+        1 if first_degree_only else 0, _ptr(out_rows), _ptr(out_mask), int(n_threads),
+    )
+    if rc != 0:
+        raise ValueError("the oracle does not define this case (code %d)" % rc)
+    return out_rows, out_mask
+
+
+def join_workload(wl, first_degree_only: bool = False, n_threads: int = 1):
+    """Convenience for objects with `.store` and `.batch` attributes (duck-typed, nothing imported)."""
+    s, b = wl.store, wl.batch
+    return join(
+        s.doc_feats, s.author_ids, b.edge_keys, b.edge_feats, b.edge_offsets, b.cand_idx, b.cand_offsets,
+        req_feats=b.req_feats, actor_ids=s.actor_ids, actor_types=s.actor_types,
+        reduce_sum_mask=s.reduce_sum_mask, first_degree_only=first_degree_only, n_threads=n_threads,
+    )
+
+
+def half_to_float_bits(h: int) -> int:
+    return int(_load().ccr_oracle_half_to_float_bits(int(h)))
+
+
+def float_bits_to_half(b: int) -> int:
+    return int(_load().ccr_oracle_float_bits_to_half(int(b)))

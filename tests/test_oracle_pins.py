@@ -1,0 +1,348 @@
+"""Pins for the CPU oracle: checks against things other than itself.
+
+  * the naive O(N*K) scan of Section 3.1 (pure Python, tiny inputs, hypothesis-generated);
+  * Algorithm 1 steps 2-4 restated literally with library ops (torch.searchsorted / index_select / where);
+  * the worked batching example of Section 6.3.1 (tests/golden/batching_example.txt);
+  * set-intersection and concatenation invariants; boundary cases of Algorithm 1 step 3;
+  * the oracle's fp16 <-> fp32 conversions against numpy's float16, exhaustively;
+  * second-degree reduction special cases (the paper prints nothing for it).
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+from hypothesis import HealthCheck, given, settings
+from hypothesis import strategies as st
+
+from oracle import brute_force, oracle
+from paper_2609_22441_b200 import workloads as W
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ---------------------------------------------------------------- fp16 conversions
+def test_half_to_float_exhaustive_against_numpy():
+    h = np.arange(65536, dtype=np.uint16)
+    ref = h.view(np.float16).astype(np.float32)
+    ref_bits = ref.view(np.uint32)
+    got = np.array([oracle.half_to_float_bits(int(x)) for x in h], dtype=np.uint32)
+    nan = np.isnan(ref)
+    assert np.array_equal(got[~nan], ref_bits[~nan])
+    assert np.all(np.isnan(got[nan].view(np.float32)))
+    # round trip is the identity on every non-NaN half
+    back = np.array([oracle.float_bits_to_half(int(b)) for b in got[~nan]], dtype=np.uint16)
+    assert np.array_equal(back, h[~nan])
+
+
+def test_float_to_half_rne_against_numpy():
+    rng = np.random.default_rng(5)
+    bits = [rng.integers(0, 2**32, size=120_000, dtype=np.uint64).astype(np.uint32)]
+    # every tie between adjacent halves, and its two float neighbours (normal and subnormal range)
+    h = np.arange(0, 0x7C00, dtype=np.uint16)
+    lo = h.view(np.float16).astype(np.float64)
+    hi = (h + 1).astype(np.uint16).view(np.float16).astype(np.float64)
+    hi[-1] = 65536.0  # the "next half" after 65504 for rounding purposes
+    mid = ((lo + hi) / 2).astype(np.float32)
+    mb = mid.view(np.uint32)
+    bits += [mb, mb + 1, mb - 1, mb | 0x80000000]
+    # around the subnormal floor and the overflow threshold
+    for v in (2.0**-25, 2.0**-24, 2.0**-26, 65504.0, 65519.99, 65520.0, 65536.0, 1e30, 1e-30, 0.0):
+        f = np.array([v, -v], dtype=np.float32).view(np.uint32)
+        bits += [f, f + 1, f - 1]
+    bits = np.concatenate(bits).astype(np.uint32)
+    f = bits.view(np.float32)
+    keep = ~np.isnan(f)
+    with np.errstate(over="ignore"):
+        ref = f[keep].astype(np.float16).view(np.uint16)
+    got = np.array([oracle.float_bits_to_half(int(b)) for b in bits[keep]], dtype=np.uint16)
+    assert np.array_equal(got, ref)
+    assert oracle.float_bits_to_half(0x7FC00000) == 0x7FFF  # NaN is stored canonically
+
+
+# ---------------------------------------------------------------- helpers
+def _oracle(wl, **kw):
+    return oracle.join_workload(wl, **kw)
+
+
+def _brute(wl, **kw):
+    s, b = wl.store, wl.batch
+    return brute_force.join(
+        s.doc_feats, s.author_ids, b.edge_keys, b.edge_feats, b.edge_offsets, b.cand_idx, b.cand_offsets,
+        req_feats=b.req_feats, actor_ids=s.actor_ids, actor_types=s.actor_types,
+        reduce_sum_mask=s.reduce_sum_mask, **kw)
+
+
+def _tiny(seed, n_docs, alphabet, n_req, kmax, nmax, second, req_dim, doc_dtype=np.float32):
+    """Tiny problem with ids from a tiny alphabet so that hits, misses and repeats are all common."""
+    rng = np.random.default_rng(seed)
+    store = W.make_store(rng, n_docs, alphabet, 4, doc_dtype, max_actors=4 if second else 0,
+                         reduce_sum_mask=0b10110100 if second else 0)
+    keys_l, feats_l, cands_l = [], [], []
+    for _ in range(n_req):
+        k = int(rng.integers(0, min(kmax, alphabet) + 1))
+        keys, _ = W.make_viewer(rng, alphabet, k, 8, np.float16)
+        # edge values include negatives, repeats and exact ties so that max / sum rules matter
+        feats = rng.choice(np.array([-2.0, -0.5, 0.0, 0.25, 0.5, 1.0, 1.5, 3.0, 1000.0, 6e-5], np.float16),
+                           size=(k, 8))
+        n = int(rng.integers(0, nmax + 1))
+        cands_l.append(rng.integers(-1, n_docs + 1, size=n).astype(np.int32))  # includes -1 and n_docs
+        keys_l.append(keys)
+        feats_l.append(feats)
+    req = rng.standard_normal((n_req, req_dim)).astype(np.float32) if req_dim else None
+    batch = W.assemble_batch(keys_l, feats_l, cands_l, req, 8, np.float16, req_dim, np.float32)
+    return W.Workload("tiny", seed, store, batch)
+
+
+# ---------------------------------------------------------------- brute force (naive scan) == oracle
+@settings(max_examples=60, deadline=None, suppress_health_check=list(HealthCheck))
+@given(seed=st.integers(0, 2**31), n_docs=st.integers(1, 40), alphabet=st.integers(1, 24),
+       n_req=st.integers(0, 4), second=st.booleans(), req_dim=st.sampled_from([0, 4]))
+def test_oracle_equals_naive_scan(seed, n_docs, alphabet, n_req, second, req_dim):
+    wl = _tiny(seed, n_docs, alphabet, n_req, 16, 48, second, req_dim)
+    rows, mask = _oracle(wl)
+    brows, bmask = _brute(wl)
+    assert np.array_equal(mask, bmask)
+    if len(mask):
+        assert rows.shape == brows.shape
+        assert np.array_equal(rows, brows)
+    if second:  # ignoring the engager slots must reproduce the first-degree result
+        r1, m1 = _oracle(wl, first_degree_only=True)
+        b1, bm1 = _brute(wl, first_degree_only=True)
+        assert np.array_equal(m1, bm1) and (len(m1) == 0 or np.array_equal(r1, b1))
+        assert np.array_equal(m1, mask & 1)
+
+
+# ---------------------------------------------------------------- Algorithm 1 with library ops
+def _alg1_torch(keys, feats, d):
+    """Steps 2-4 of Algorithm 1 for one request, restated with the library ops the paper names."""
+    K = keys.shape[0]
+    if K == 0:
+        return torch.zeros((d.shape[0], feats.shape[1]), dtype=feats.dtype), torch.zeros(d.shape[0], dtype=torch.bool)
+    pos = torch.searchsorted(keys, d, right=False)
+    pos_safe = torch.clamp(pos, max=K - 1)
+    valid = (pos < K) & (keys[pos_safe] == d)
+    O = torch.zeros((d.shape[0], feats.shape[1]), dtype=feats.dtype)
+    O[valid] = feats.index_select(0, pos_safe[valid])
+    return O, valid
+
+
+@pytest.mark.parametrize("maker", [
+    lambda: W.config0(n_docs=20_000, n_cand=6_000, k=500),
+    lambda: W.config1(n_docs=40_000, n_req=6, n_cand=3_000),
+])
+def test_oracle_equals_algorithm1_library_ops(maker):
+    wl = maker()
+    s, b = wl.store, wl.batch
+    rows, mask = _oracle(wl)
+    doc_b, edge_b = s.doc_row_bytes, b.edge_row_bytes
+    for r in range(b.n_req):
+        e0, e1 = int(b.edge_offsets[r]), int(b.edge_offsets[r + 1])
+        c0, c1 = int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])
+        d = torch.from_numpy(s.author_ids[b.cand_idx[c0:c1].astype(np.int64)])
+        O, valid = _alg1_torch(torch.from_numpy(b.edge_keys[e0:e1]),
+                               torch.from_numpy(b.edge_feats[e0:e1].view(np.int16)), d)
+        got = rows[c0:c1, doc_b:doc_b + edge_b].copy().view(np.int16)
+        assert np.array_equal(got, O.numpy())
+        assert np.array_equal(mask[c0:c1], valid.numpy().astype(np.uint8))
+        # doc section is a plain gather by position, request section a broadcast
+        gathered = torch.from_numpy(s.doc_feats.view(np.uint8).reshape(s.n_docs, -1)).index_select(
+            0, torch.from_numpy(b.cand_idx[c0:c1].astype(np.int64))).numpy()
+        assert np.array_equal(rows[c0:c1, :doc_b], gathered)
+        if b.req_feats is not None:
+            want = np.broadcast_to(b.req_feats[r].view(np.uint8), (c1 - c0, b.req_row_bytes))
+            assert np.array_equal(rows[c0:c1, doc_b + edge_b:], want)
+
+
+# ---------------------------------------------------------------- the paper's worked example
+def test_worked_batching_example_from_the_paper():
+    req, flat = [], None
+    for line in open(os.path.join(GOLDEN, "batching_example.txt")):
+        if line.startswith("request"):
+            req.append([int(x) for x in line.split(":")[1].split()])
+        elif line.startswith("flattened"):
+            flat = [int(x) for x in line.split(":")[1].split()]
+    assert flat == sum(req, [])
+    rng = np.random.default_rng(1)
+    store = W.make_store(rng, 100, 50, 8, np.float32, tagged=True)
+    keys, feats = W.make_viewer(rng, 50, 5, 8, np.float16)
+    batch = W.assemble_batch([keys, keys], [feats, feats], [np.array(x, np.int32) for x in req], None,
+                             8, np.float16, 0, np.float32)
+    rows, _ = _oracle(W.Workload("example", 1, store, batch))
+    doc_b = store.doc_row_bytes
+    assert list(batch.cand_offsets) == [0, 3, 5]
+    for k, p in enumerate(flat):
+        assert np.array_equal(rows[k, :doc_b], store.doc_feats[p].view(np.uint8))
+        # tagged store: the first value of row p is p * doc_dim
+        assert rows[k, :4].copy().view(np.float32)[0] == (p * 8) % 2048
+
+
+# ---------------------------------------------------------------- invariants at realistic shapes
+def _check_invariants(wl):
+    s, b = wl.store, wl.batch
+    rows, mask = _oracle(wl)
+    doc_b, edge_b, req_b = s.doc_row_bytes, b.edge_row_bytes, b.req_row_bytes
+    assert rows.shape == (b.total_cands, wl.out_row_bytes())
+    docs_u8 = s.doc_feats.view(np.uint8).reshape(s.n_docs, -1)
+    edge_u8 = b.edge_feats.view(np.uint8).reshape(len(b.edge_keys), -1)
+    for r in range(b.n_req):
+        e0, e1 = int(b.edge_offsets[r]), int(b.edge_offsets[r + 1])
+        c0, c1 = int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])
+        keyset = {int(k): i for i, k in enumerate(b.edge_keys[e0:e1])}
+        cand = b.cand_idx[c0:c1].astype(np.int64)
+        auth = s.author_ids[cand]
+        member = np.array([int(a) in keyset for a in auth], dtype=bool)
+        # found count = size of the intersection (as a multiset over candidates)
+        assert int((mask[c0:c1] & 1).sum()) == int(member.sum())
+        assert np.array_equal((mask[c0:c1] & 1).astype(bool), member)
+        # every row is the concatenation of its source rows (or zeros)
+        assert np.array_equal(rows[c0:c1, :doc_b], docs_u8[cand])
+        src = np.array([keyset.get(int(a), 0) for a in auth]) + e0
+        want_edge = np.where(member[:, None], edge_u8[src], 0)
+        assert np.array_equal(rows[c0:c1, doc_b:doc_b + edge_b], want_edge)
+        if req_b:
+            assert np.all(rows[c0:c1, -req_b:] == b.req_feats[r].view(np.uint8)[None, :])
+    return rows, mask
+
+
+def test_invariants_config0_full_size():
+    wl = W.config0()
+    assert wl.batch.total_cands == 20_000 and wl.batch.max_edge_len == 500
+    assert wl.out_row_bytes() == 320
+    assert len(np.unique(wl.batch.cand_idx)) == 20_000  # drawn without replacement
+    rows, mask = _check_invariants(wl)
+    frac = float((mask & 1).mean())
+    assert 0.69 < frac < 0.72, frac  # 70 % forced plus a few chance hits
+
+
+def test_invariants_config1_scaled():
+    wl = W.config1(n_docs=60_000, n_req=8, n_cand=4_000)
+    assert wl.out_row_bytes() == 384
+    _check_invariants(wl)
+
+
+def test_batch_equals_single_requests_and_permutation_equivariance():
+    wl = W.config1(n_docs=30_000, n_req=5, n_cand=700)
+    s, b = wl.store, wl.batch
+    rows, mask = _oracle(wl)
+    for r in range(b.n_req):
+        e0, e1 = int(b.edge_offsets[r]), int(b.edge_offsets[r + 1])
+        c0, c1 = int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])
+        one = W.assemble_batch([b.edge_keys[e0:e1]], [b.edge_feats[e0:e1]], [b.cand_idx[c0:c1]],
+                               b.req_feats[r:r + 1], b.edge_dim, b.edge_dtype, b.req_dim, b.req_dtype)
+        r1, m1 = _oracle(W.Workload("one", 0, s, one))
+        assert np.array_equal(r1, rows[c0:c1]) and np.array_equal(m1, mask[c0:c1])
+    perm = np.random.default_rng(0).permutation(int(b.cand_offsets[1]))
+    cand2 = b.cand_idx.copy()
+    cand2[: len(perm)] = b.cand_idx[: len(perm)][perm]
+    r2, m2 = _oracle(W.Workload("perm", 0, s, W.Batch(**{**b.__dict__, "cand_idx": cand2})))
+    assert np.array_equal(r2[: len(perm)], rows[: len(perm)][perm])
+    assert np.array_equal(m2[: len(perm)], mask[: len(perm)][perm])
+    assert np.array_equal(r2[len(perm):], rows[len(perm):])
+    # a threaded run partitions candidates only
+    r3, m3 = _oracle(wl, n_threads=3)
+    assert np.array_equal(r3, rows) and np.array_equal(m3, mask)
+
+
+# ---------------------------------------------------------------- boundary cases of Algorithm 1 step 3
+def test_search_boundaries():
+    imax = np.iinfo(np.int64).max
+    author_ids = np.array([0, 5, 7, 9, imax, imax - 1, -3, 6], dtype=np.int64)
+    docs = np.arange(8 * 4, dtype=np.float32).reshape(8, 4)
+    keys = np.array([0, 7, imax], dtype=np.int64)
+    feats = np.array([[1, 2], [3, 4], [5, 6]], dtype=np.float16)
+    cand = np.array([0, 1, 2, 3, 4, 5, 6, 7, 2, 2, -1, 8], dtype=np.int32)
+    rows, mask = oracle.join(docs, author_ids, keys, feats, np.array([0, 3]), cand, np.array([0, len(cand)]))
+    assert list(mask) == [1, 0, 1, 0, 1, 0, 0, 0, 1, 1, 0, 0]
+    edge = rows[:, 16:].copy().view(np.float16)
+    assert edge.tolist() == [[1, 2], [0, 0], [3, 4], [0, 0], [5, 6], [0, 0], [0, 0], [0, 0], [3, 4], [3, 4], [0, 0], [0, 0]]
+    assert not rows[10].any() and not rows[11].any()  # unresolved / out-of-range position: zero row
+    # K == 0 and K == 1
+    r0, m0 = oracle.join(docs, author_ids, keys[:0], feats[:0], np.array([0, 0]), cand, np.array([0, len(cand)]))
+    assert not m0.any() and not r0[:, 16:].any()
+    r1, m1 = oracle.join(docs, author_ids, keys[1:2], feats[1:2], np.array([0, 1]), cand, np.array([0, len(cand)]))
+    assert list(m1) == [0, 0, 1, 0, 0, 0, 0, 0, 1, 1, 0, 0]
+    # requests with no candidates in the middle of a batch
+    r2, m2 = oracle.join(docs, author_ids, np.concatenate([keys, keys]), np.concatenate([feats, feats]),
+                         np.array([0, 3, 3, 6]), cand, np.array([0, 0, 5, len(cand)]))
+    assert list(m2) == [0, 0, 0, 0, 0, 0, 0, 0, 1, 1, 0, 0]
+
+
+# ---------------------------------------------------------------- second-degree reduction (unpinned by the paper)
+def _second_case(actor_rows, types, keys, feats, sum_mask, author=999):
+    n = len(actor_rows)
+    docs = np.zeros((n, 2), dtype=np.float32)
+    author_ids = np.full(n, author, dtype=np.int64)
+    return oracle.join(docs, author_ids, np.asarray(keys, np.int64), np.asarray(feats, np.float16),
+                       np.array([0, len(keys)]), np.arange(n, dtype=np.int32), np.array([0, n]),
+                       actor_ids=np.asarray(actor_rows, np.int64), actor_types=np.asarray(types, np.uint8),
+                       reduce_sum_mask=sum_mask)
+
+
+def test_second_degree_special_cases():
+    keys = [10, 20, 30, 40]
+    feats = [[1.0, 8.0, -1.0, 2.0], [3.0, 0.5, -4.0, 2.0], [2.0, 0.25, -0.0, 2.0], [0.5, 100.0, 5.0, 2.0]]
+    actors = [[-1, -1, -1, -1],      # nothing to look up
+              [11, 21, -1, -1],      # engagers present, none is a key
+              [-1, 30, -1, -1],      # exactly one found: edge2 is that row, bit for bit, for max and for sum
+              [10, 20, 30, 40],      # all four found
+              [40, 20, 40, 5],       # a key found twice is counted twice; slot 3 misses
+              [20, 10, -1, -1]]      # order of slots is the order of reduction
+    types = [[0, 0, 0, 0], [1, 2, 0, 0], [0, 2, 0, 0], [0, 1, 2, 0], [1, 1, 1, 2], [2, 2, 0, 0]]
+    sum_mask = 0b1010  # dims 1 and 3 summed, dims 0 and 2 max
+    rows, mask = _second_case(actors, types, keys, feats, sum_mask)
+    e1 = rows[:, 8:16].copy().view(np.float16)
+    e2 = rows[:, 16:24].copy().view(np.float16)
+    assert not e1.any()  # author 999 is not a key
+    assert list(mask) == [0, 0, 0b10000100, 0b11111110, 0b01001110, 0b10000110]
+    assert e2[0].tolist() == [0, 0, 0, 0] and e2[1].tolist() == [0, 0, 0, 0]
+    # one found slot: bit-identical copy (the -0.0 in a max dim keeps its sign bit)
+    assert np.array_equal(e2[2].view(np.uint16), np.asarray(feats[2], np.float16).view(np.uint16))
+    assert e2[3].tolist() == [3.0, 108.75, 5.0, 8.0]
+    assert e2[4].tolist() == [3.0, 200.5, 5.0, 6.0]
+    assert e2[5].tolist() == [3.0, 8.5, -1.0, 4.0]
+
+
+def test_second_degree_sum_matches_float64_when_partial_sums_are_exact():
+    rng = np.random.default_rng(11)
+    K, n = 64, 500
+    keys = np.arange(0, 2 * K, 2)
+    feats = rng.integers(-64, 65, size=(K, 8)).astype(np.float16)  # small integers: every fp32 partial sum is exact
+    actors = rng.integers(0, 2 * K, size=(n, 4))
+    actors[rng.random((n, 4)) < 0.2] = -1
+    types = rng.integers(0, 3, size=(n, 4))
+    rows, mask = _second_case(actors, types, keys, feats, 0xFF)
+    e2 = rows[:, 8 + 16: 8 + 32].copy().view(np.float16)
+    for j in range(n):
+        hit = [int(a) // 2 for a in actors[j] if a >= 0 and a % 2 == 0]
+        want = np.zeros(8) if not hit else feats[hit].astype(np.float64).sum(axis=0)
+        assert np.array_equal(e2[j].astype(np.float64), want)
+        bits = sum(1 << (1 + s) for s, a in enumerate(actors[j]) if a >= 0 and a % 2 == 0)
+        assert (int(mask[j]) & 0b11110) == bits
+
+
+def test_second_degree_max_is_an_input_and_dominates():
+    rng = np.random.default_rng(12)
+    K, n = 40, 400
+    keys = np.arange(K)
+    feats = rng.standard_normal((K, 8)).astype(np.float16)
+    actors = rng.integers(-1, K + 10, size=(n, 4))
+    rows, mask = _second_case(actors, np.zeros((n, 4)), keys, feats, 0)
+    e2 = rows[:, 8 + 16: 8 + 32].copy().view(np.float16)
+    for j in range(n):
+        hit = [int(a) for a in actors[j] if 0 <= a < K]
+        if not hit:
+            assert not e2[j].any()
+            continue
+        assert np.array_equal(e2[j], feats[hit].max(axis=0))
+
+
+def test_generators_are_deterministic():
+    a = W.config1(n_docs=20_000, n_req=3, n_cand=500)
+    b = W.config1(n_docs=20_000, n_req=3, n_cand=500)
+    for x, y in ((a.store.author_ids, b.store.author_ids), (a.store.doc_feats, b.store.doc_feats),
+                 (a.batch.edge_keys, b.batch.edge_keys), (a.batch.cand_idx, b.batch.cand_idx)):
+        assert W.checksum64(x) == W.checksum64(y)
+    for r in range(3):
+        k = a.batch.edge_keys[a.batch.edge_offsets[r]:a.batch.edge_offsets[r + 1]]
+        assert np.all(np.diff(k) > 0)
