@@ -1,0 +1,177 @@
+/* ccr.h — C ABI of the sorted-search edge-feature join for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one operation of the paper "Connected Content Retriever": the join of a
+ * viewer's dense edge features onto a request's candidate documents at scoring time
+ * (Section 3.1, Eq. 1 and Algorithm 1), fused with the gather of the candidates' document features
+ * from the GPU-resident index (Section 6.3, "Feat. gather"; Section 6.3.1, "Batching and Padding")
+ * and with the broadcast of the request-level features (Section 3), for a ragged batch of requests
+ * in one kernel launch.
+ *
+ * Conventions
+ *   - Plain C.  Every call returns a ccr_status; nothing throws across the boundary.
+ *   - Pointers are marked HOST or DEVICE.  DEVICE pointers must belong to the store's device.
+ *   - The caller owns every buffer it passes; the library keeps none of them after a call returns
+ *     (asynchronous work enqueued on `stream` still reads/writes them until the stream reaches it).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Feature, key and output buffers must be 16-byte aligned; section widths (dim * element size)
+ *     must be multiples of 16 bytes.
+ *   - There is no CPU fallback: without a CUDA device every compute entry returns CCR_ERR_CUDA.
+ */
+#ifndef CCR_H_
+#define CCR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ccr_docstore ccr_docstore;   /* opaque; owns its device memory */
+typedef struct ccr_workspace ccr_workspace; /* opaque; device staging for the host-buffer entry */
+
+typedef enum {
+  CCR_OK = 0,
+  CCR_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, negative size, misaligned buffer   */
+  CCR_ERR_UNSUPPORTED = 2, /* a width, dtype or size outside what the kernels handle               */
+  CCR_ERR_OOM = 3,         /* device (or pinned host) allocation failed or would not fit           */
+  CCR_ERR_CUDA = 4,        /* a CUDA runtime call failed, or no usable device                      */
+  CCR_ERR_BAD_HANDLE = 5,  /* handle is NULL, freed or not one of ours                             */
+  CCR_ERR_VALIDATION = 6,  /* CCR_FLAG_VALIDATE found a broken precondition                        */
+  CCR_ERR_DEVICE_WAIT = 7  /* a bounded device-side wait ran out (reported by device_status)       */
+} ccr_status;
+
+typedef enum { CCR_F16 = 0, CCR_F32 = 1 } ccr_dtype;
+
+/* Store schema.  One store is one GPU's shard of the document index (Section 6.3, Eq. 5):
+ * per-document feature rows addressed by position, plus the ids the join needs.                    */
+typedef struct {
+  int64_t  n_docs;          /* capacity in rows; valid positions are 0 .. n_docs-1                  */
+  int32_t  doc_dim;         /* document features per row                                            */
+  int32_t  doc_dtype;       /* ccr_dtype                                                            */
+  int32_t  edge_dim;        /* D of Eq. 1: features per viewer-author affinity record               */
+  int32_t  edge_dtype;      /* ccr_dtype (second-degree reduction needs CCR_F16)                    */
+  int32_t  req_dim;         /* request-level features per request, 0 = none                         */
+  int32_t  req_dtype;       /* ccr_dtype                                                            */
+  int32_t  max_actors;      /* engager slots per document: 0 = first-degree store, else 1..4        */
+  int32_t  device;          /* CUDA device ordinal                                                  */
+  uint64_t reduce_sum_mask; /* second-degree: bit d set = edge dim d is summed over the found
+                               engagers, clear = elementwise max (edge_dim <= 64 when max_actors>0) */
+} ccr_docstore_desc;
+
+/* Flags of ccr_join_batch. */
+enum {
+  CCR_FLAG_FORCE_SMEM        = 1u << 0, /* stage every request's full key list in shared memory
+                                           (CCR_ERR_UNSUPPORTED if max_edge_len does not fit)       */
+  CCR_FLAG_FORCE_GLOBAL      = 1u << 1, /* never stage keys: search them in global memory / L2      */
+  CCR_FLAG_CANDS_SORTED      = 1u << 2, /* caller promises that, inside each request, the candidates'
+                                           author ids are non-decreasing: use the merge-path kernel  */
+  CCR_FLAG_VALIDATE          = 1u << 3, /* check offsets, key order (and candidate order) on the
+                                           device first; synchronises the stream                     */
+  CCR_FLAG_FIRST_DEGREE_ONLY = 1u << 4, /* ignore engager slots of a second-degree store: no edge2
+                                           section, mask is 0/1                                      */
+  CCR_FLAG_FORCE_SAMPLED     = 1u << 5  /* stage only every s-th key (a sampled top of the search
+                                           tree) even when the list would fit; testing aid          */
+};
+
+/* Create an empty store on desc->device.  Allocates doc_feats [n_docs, doc_dim], author_ids
+ * int64[n_docs] and, when max_actors > 0, actor_ids int64[n_docs, max_actors] and actor_types
+ * uint8[n_docs, max_actors].  Rows are uninitialised until uploaded.  The required bytes are compared
+ * with the device's free memory before anything is allocated (CCR_ERR_OOM).  HOST call.            */
+ccr_status ccr_docstore_create(const ccr_docstore_desc* desc, ccr_docstore** out);
+
+/* Write rows [first_doc, first_doc + n) of the store (Section 6.2: features are written into the GPU
+ * index by position).  Sources are HOST pointers when src_on_device == 0, DEVICE pointers otherwise;
+ * doc_feats is [n, doc_dim] in doc_dtype, author_ids int64[n]; actor_ids int64[n, max_actors] and
+ * actor_types uint8[n, max_actors] (engagement type 0 reacted, 1 commented, 2 reshared; values are
+ * taken modulo 3) are required when max_actors > 0, an empty slot is any negative id.  A NULL source
+ * leaves that array untouched.  Copies are enqueued on `stream`; the store must not be joined
+ * against concurrently with an upload (the paper's index read/write lock, Section 6.3.1, is the
+ * caller's job).                                                                                   */
+ccr_status ccr_docstore_upload(ccr_docstore* store, int64_t first_doc, int64_t n,
+                               const void* doc_feats, const int64_t* author_ids,
+                               const int64_t* actor_ids, const uint8_t* actor_types,
+                               int src_on_device, void* stream);
+
+/* Free the store and its device memory.  A second free of the same handle returns
+ * CCR_ERR_BAD_HANDLE as long as the freed block has not been reused by the allocator.              */
+ccr_status ccr_docstore_free(ccr_docstore* store);
+
+/* Bytes of one output row for this store and these flags:
+ * doc_dim*sizeof(doc) + edge_dim*sizeof(edge) [+ edge_dim*sizeof(edge) if max_actors > 0 and not
+ * FIRST_DEGREE_ONLY] + req_dim*sizeof(req).  0 for a bad handle.                                    */
+size_t ccr_out_row_bytes(const ccr_docstore* store, uint32_t flags);
+
+/* The join (Eq. 1 / Algorithm 1 steps 2-4, fused with the document gather and request broadcast).
+ *
+ * For request r = 0 .. n_req-1, with keys = edge_keys[edge_offsets[r] .. edge_offsets[r+1]) (K of
+ * them, ascending and unique) and candidates j in [cand_offsets[r], cand_offsets[r+1]):
+ *     p   = cand_idx[j]                       position in the store
+ *     d   = author_id[p]                      Algorithm 1's d_j
+ *     pos = lower bound of d in keys;  found = pos < K and keys[pos] == d
+ *     out_rows[j] = [ doc_feats[p] | found ? edge_feats[edge_offsets[r]+pos] : 0
+ *                   | edge2 (second-degree stores) | req_feats[r] ]
+ *     out_mask[j] = bit0 found; bits1-4 engager slot 0-3 found; bits5-7 OR of 1<<type over found slots
+ * edge2[dim] reduces, over the found engager slots in ascending slot order, the matched edge rows:
+ * max (strict > on the fp32 values, earlier slot wins ties, the winner's bits are kept) or sum (fp32
+ * accumulator from +0, one rounded add per slot, rounded once to fp16 with ties to even; NaN is stored
+ * as 0x7fff); all zero when no slot is found.  A position p < 0 or p >= n_docs gives zero doc/edge/
+ * edge2 sections and mask 0 (the request section is still written).  Values are moved bit for bit.
+ *
+ * All array arguments are DEVICE pointers.  n_req, total_cands (= cand_offsets[n_req]) and
+ * max_edge_len (>= every request's K) are HOST scalars: the offsets live on the device and the call
+ * never synchronises.  cand_offsets[0] must be 0 and both offset arrays non-decreasing; they and the
+ * key order are trusted unless CCR_FLAG_VALIDATE is given.  With unsorted keys or an untruthful
+ * CCR_FLAG_CANDS_SORTED the values are unspecified but every access stays in bounds.
+ * The call allocates nothing, clears nothing and is asynchronous: one kernel on `stream`.          */
+ccr_status ccr_join_batch(const ccr_docstore* store,
+                          int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                          const int64_t* edge_keys,    /* DEVICE [E]                               */
+                          const void*    edge_feats,   /* DEVICE [E, edge_dim]                     */
+                          const int64_t* edge_offsets, /* DEVICE [n_req + 1]                       */
+                          const int32_t* cand_idx,     /* DEVICE [total_cands]                     */
+                          const int64_t* cand_offsets, /* DEVICE [n_req + 1]                       */
+                          const void*    req_feats,    /* DEVICE [n_req, req_dim]; NULL if req_dim == 0 */
+                          void*          out_rows,     /* DEVICE [total_cands, out_row_bytes]      */
+                          uint8_t*       out_mask,     /* DEVICE [total_cands]                     */
+                          uint32_t       flags,
+                          void*          stream);
+
+/* Device staging buffers for ccr_join_batch_host, sized for the largest batch the caller will pass.
+ * HOST calls; allocation happens here, never inside the join.                                      */
+ccr_status ccr_workspace_create(const ccr_docstore* store, int32_t max_req, int64_t max_cands,
+                                int64_t max_edges, ccr_workspace** out);
+ccr_status ccr_workspace_free(ccr_workspace* ws);
+
+/* The same join with HOST buffers (the request payload of Section 6.1.3 arrives in host memory):
+ * copies the inputs to the workspace, runs ccr_join_batch, copies rows and mask back — all enqueued
+ * on `stream`, nothing synchronised.  Pinned host memory makes the copies asynchronous.
+ * total_edges = edge_offsets[n_req].  Sizes beyond the workspace give CCR_ERR_INVALID_ARG.          */
+ccr_status ccr_join_batch_host(const ccr_docstore* store, ccr_workspace* ws,
+                               int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                               int64_t total_edges,
+                               const int64_t* edge_keys, const void* edge_feats,
+                               const int64_t* edge_offsets, const int32_t* cand_idx,
+                               const int64_t* cand_offsets, const void* req_feats,
+                               void* out_rows, uint8_t* out_mask, /* HOST */
+                               uint32_t flags, void* stream);
+
+/* Synchronise `stream` and report the store's device-side status word: CCR_OK, or
+ * CCR_ERR_DEVICE_WAIT if a kernel gave up a bounded wait for a shared-memory bulk copy since the
+ * last call (the affected rows of that launch were not written).  Clears the word.                 */
+ccr_status ccr_docstore_device_status(ccr_docstore* store, void* stream);
+
+/* Tuning knobs of the join kernels (0 keeps the current value): candidates per thread block, and
+ * the largest number of keys (or sampled keys) a block stages in shared memory per request.        */
+ccr_status ccr_docstore_set_tuning(ccr_docstore* store, int32_t tile_cands, int32_t key_capacity);
+
+/* Number of kernels the library has launched on behalf of this store since creation.               */
+int64_t ccr_docstore_launch_count(const ccr_docstore* store);
+
+const char* ccr_status_str(ccr_status s);
+int         ccr_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CCR_H_ */

@@ -1,0 +1,295 @@
+"""Thin ctypes binding of the C ABI in include/ccr.h (same names, argument marshalling only).
+
+Every step of the join runs in the CUDA library; torch is used here only for device memory, streams
+and pointer/size bookkeeping.  There is no CPU fallback: if the shared object is missing or no CUDA
+device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libccr.so")
+
+CCR_OK = 0
+CCR_ERR_INVALID_ARG = 1
+CCR_ERR_UNSUPPORTED = 2
+CCR_ERR_OOM = 3
+CCR_ERR_CUDA = 4
+CCR_ERR_BAD_HANDLE = 5
+CCR_ERR_VALIDATION = 6
+CCR_ERR_DEVICE_WAIT = 7
+
+CCR_F16 = 0
+CCR_F32 = 1
+
+CCR_FLAG_FORCE_SMEM = 1 << 0
+CCR_FLAG_FORCE_GLOBAL = 1 << 1
+CCR_FLAG_CANDS_SORTED = 1 << 2
+CCR_FLAG_VALIDATE = 1 << 3
+CCR_FLAG_FIRST_DEGREE_ONLY = 1 << 4
+CCR_FLAG_FORCE_SAMPLED = 1 << 5
+
+EXPORTS = (
+    "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
+    "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
+    "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
+)
+
+
+class ccr_docstore_desc(ctypes.Structure):
+    _fields_ = [
+        ("n_docs", ctypes.c_int64),
+        ("doc_dim", ctypes.c_int32), ("doc_dtype", ctypes.c_int32),
+        ("edge_dim", ctypes.c_int32), ("edge_dtype", ctypes.c_int32),
+        ("req_dim", ctypes.c_int32), ("req_dtype", ctypes.c_int32),
+        ("max_actors", ctypes.c_int32), ("device", ctypes.c_int32),
+        ("reduce_sum_mask", ctypes.c_uint64),
+    ]
+
+
+class CcrError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        msg = lib().ccr_status_str(self.status).decode() if _lib is not None else "?"
+        super().__init__("%s: %s (status %d)" % (where, msg, self.status))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (built in-tree by `paper_2609_22441_b200.build`); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "CUDA library %s is not built; run `python -m paper_2609_22441_b200.build` "
+            "(there is no CPU fallback)" % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, u32, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_uint64
+    L.ccr_docstore_create.restype = ctypes.c_int
+    L.ccr_docstore_create.argtypes = [ctypes.POINTER(ccr_docstore_desc), ctypes.POINTER(vp)]
+    L.ccr_docstore_upload.restype = ctypes.c_int
+    L.ccr_docstore_upload.argtypes = [vp, i64, i64, vp, vp, vp, vp, ctypes.c_int, vp]
+    L.ccr_docstore_free.restype = ctypes.c_int
+    L.ccr_docstore_free.argtypes = [vp]
+    L.ccr_out_row_bytes.restype = ctypes.c_size_t
+    L.ccr_out_row_bytes.argtypes = [vp, u32]
+    L.ccr_join_batch.restype = ctypes.c_int
+    L.ccr_join_batch.argtypes = [vp, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
+    L.ccr_workspace_create.restype = ctypes.c_int
+    L.ccr_workspace_create.argtypes = [vp, i32, i64, i64, ctypes.POINTER(vp)]
+    L.ccr_workspace_free.restype = ctypes.c_int
+    L.ccr_workspace_free.argtypes = [vp]
+    L.ccr_join_batch_host.restype = ctypes.c_int
+    L.ccr_join_batch_host.argtypes = [vp, vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
+    L.ccr_docstore_device_status.restype = ctypes.c_int
+    L.ccr_docstore_device_status.argtypes = [vp, vp]
+    L.ccr_docstore_set_tuning.restype = ctypes.c_int
+    L.ccr_docstore_set_tuning.argtypes = [vp, i32, i32]
+    L.ccr_docstore_launch_count.restype = i64
+    L.ccr_docstore_launch_count.argtypes = [vp]
+    L.ccr_status_str.restype = ctypes.c_char_p
+    L.ccr_status_str.argtypes = [ctypes.c_int]
+    L.ccr_version.restype = ctypes.c_int
+    L.ccr_version.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(status: int, where: str) -> None:
+    if status != CCR_OK:
+        raise CcrError(status, where)
+
+
+def _dtype_code(dt) -> int:
+    dt = np.dtype(dt)
+    if dt == np.float16:
+        return CCR_F16
+    if dt == np.float32:
+        return CCR_F32
+    raise ValueError("feature dtype must be float16 or float32")
+
+
+def _ptr(x) -> Optional[int]:
+    """Address of a torch tensor (device or host) or numpy array; None stays NULL."""
+    if x is None:
+        return None
+    if isinstance(x, torch.Tensor):
+        if not x.is_contiguous():
+            raise ValueError("tensors passed to the library must be contiguous")
+        return x.data_ptr()
+    if isinstance(x, np.ndarray):
+        if not x.flags["C_CONTIGUOUS"]:
+            raise ValueError("arrays passed to the library must be contiguous")
+        return x.ctypes.data
+    raise TypeError(type(x))
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream or None
+    return int(stream) or None
+
+
+class Docstore:
+    """ccr_docstore handle: the GPU-resident document-feature store of one shard."""
+
+    def __init__(self, n_docs: int, doc_dim: int, doc_dtype, edge_dim: int, edge_dtype=np.float16,
+                 req_dim: int = 0, req_dtype=np.float32, max_actors: int = 0, reduce_sum_mask: int = 0,
+                 device: int = 0):
+        self._h = ctypes.c_void_p()
+        self.desc = ccr_docstore_desc(
+            int(n_docs), int(doc_dim), _dtype_code(doc_dtype), int(edge_dim), _dtype_code(edge_dtype),
+            int(req_dim), _dtype_code(req_dtype), int(max_actors), int(device),
+            int(reduce_sum_mask) & (2**64 - 1))
+        self.device = int(device)
+        _check(lib().ccr_docstore_create(ctypes.byref(self.desc), ctypes.byref(self._h)), "ccr_docstore_create")
+
+    @property
+    def handle(self) -> ctypes.c_void_p:
+        return self._h
+
+    def upload(self, first_doc: int, doc_feats=None, author_ids=None, actor_ids=None, actor_types=None,
+               stream=None) -> None:
+        """ccr_docstore_upload: rows [first_doc, first_doc + n); sources all on the host or all on the device."""
+        given = [x for x in (doc_feats, author_ids, actor_ids, actor_types) if x is not None]
+        if not given:
+            return
+        n = int(given[0].shape[0])
+        on_dev = [isinstance(x, torch.Tensor) and x.is_cuda for x in given]
+        if any(on_dev) != all(on_dev):
+            raise ValueError("upload sources must be all on the host or all on the device")
+        _check(lib().ccr_docstore_upload(self._h, int(first_doc), n, _ptr(doc_feats), _ptr(author_ids),
+                                         _ptr(actor_ids), _ptr(actor_types), 1 if all(on_dev) else 0,
+                                         _stream_ptr(stream)), "ccr_docstore_upload")
+
+    def out_row_bytes(self, flags: int = 0) -> int:
+        return int(lib().ccr_out_row_bytes(self._h, int(flags)))
+
+    def set_tuning(self, tile_cands: int = 0, key_capacity: int = 0) -> None:
+        _check(lib().ccr_docstore_set_tuning(self._h, int(tile_cands), int(key_capacity)), "ccr_docstore_set_tuning")
+
+    def launch_count(self) -> int:
+        return int(lib().ccr_docstore_launch_count(self._h))
+
+    def device_status(self, stream=None) -> int:
+        return int(lib().ccr_docstore_device_status(self._h, _stream_ptr(stream)))
+
+    def free(self) -> None:
+        if self._h:
+            _check(lib().ccr_docstore_free(self._h), "ccr_docstore_free")
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            if self._h:
+                lib().ccr_docstore_free(self._h)
+                self._h = ctypes.c_void_p()
+        except Exception:
+            pass
+
+
+def ccr_join_batch(store: Docstore, n_req: int, total_cands: int, max_edge_len: int,
+                   edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets, req_feats,
+                   out_rows, out_mask, flags: int = 0, stream=None) -> int:
+    """Raw call, device tensors in, status out (raises on error)."""
+    st = lib().ccr_join_batch(store.handle, int(n_req), int(total_cands), int(max_edge_len), _ptr(edge_keys),
+                              _ptr(edge_feats), _ptr(edge_offsets), _ptr(cand_idx), _ptr(cand_offsets),
+                              _ptr(req_feats), _ptr(out_rows), _ptr(out_mask), int(flags), _stream_ptr(stream))
+    _check(st, "ccr_join_batch")
+    return st
+
+
+class DeviceBatch:
+    """A ragged batch resident on the device (torch tensors), plus the host scalars the call needs."""
+
+    def __init__(self, batch, device: int = 0):
+        dev = torch.device("cuda", device)
+        self.n_req = int(batch.n_req)
+        self.total_cands = int(batch.total_cands)
+        self.max_edge_len = int(batch.max_edge_len)
+        self.total_edges = int(len(batch.edge_keys))
+
+        def up(a):
+            if a is None:
+                return None
+            t = torch.from_numpy(np.ascontiguousarray(a))
+            return t.to(dev) if t.numel() else torch.empty(t.shape, dtype=t.dtype, device=dev)
+
+        self.edge_keys = up(batch.edge_keys)
+        self.edge_feats = up(batch.edge_feats)
+        self.edge_offsets = up(batch.edge_offsets)
+        self.cand_idx = up(batch.cand_idx)
+        self.cand_offsets = up(batch.cand_offsets)
+        self.req_feats = up(batch.req_feats)
+
+
+def join_batch(store: Docstore, db: DeviceBatch, flags: int = 0, out_rows: Optional[torch.Tensor] = None,
+               out_mask: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Allocate outputs if needed (torch, outside the library) and call ccr_join_batch."""
+    out_b = store.out_row_bytes(flags)
+    dev = torch.device("cuda", store.device)
+    if out_rows is None:
+        out_rows = torch.empty((db.total_cands, out_b), dtype=torch.uint8, device=dev)
+    if out_mask is None:
+        out_mask = torch.empty((db.total_cands,), dtype=torch.uint8, device=dev)
+    ccr_join_batch(store, db.n_req, db.total_cands, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets,
+                   db.cand_idx, db.cand_offsets, db.req_feats, out_rows, out_mask, flags, stream)
+    return out_rows, out_mask
+
+
+class Workspace:
+    """ccr_workspace handle: device staging for ccr_join_batch_host."""
+
+    def __init__(self, store: Docstore, max_req: int, max_cands: int, max_edges: int):
+        self._h = ctypes.c_void_p()
+        self.store = store
+        _check(lib().ccr_workspace_create(store.handle, int(max_req), int(max_cands), int(max_edges),
+                                          ctypes.byref(self._h)), "ccr_workspace_create")
+
+    @property
+    def handle(self):
+        return self._h
+
+    def free(self) -> None:
+        if self._h:
+            _check(lib().ccr_workspace_free(self._h), "ccr_workspace_free")
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def ccr_join_batch_host(store: Docstore, ws: Workspace, n_req: int, total_cands: int, max_edge_len: int,
+                        total_edges: int, edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets, req_feats,
+                        out_rows, out_mask, flags: int = 0, stream=None) -> int:
+    """Raw call with HOST buffers (numpy arrays or pinned CPU tensors); copies are inside the call."""
+    st = lib().ccr_join_batch_host(store.handle, ws.handle, int(n_req), int(total_cands), int(max_edge_len),
+                                   int(total_edges), _ptr(edge_keys), _ptr(edge_feats), _ptr(edge_offsets),
+                                   _ptr(cand_idx), _ptr(cand_offsets), _ptr(req_feats), _ptr(out_rows),
+                                   _ptr(out_mask), int(flags), _stream_ptr(stream))
+    _check(st, "ccr_join_batch_host")
+    return st
+
+
+def store_from_workload(wl, device: int = 0, upload_doc_feats: bool = True) -> Docstore:
+    """Create a store with the workload's schema and upload its arrays (host sources)."""
+    s, b = wl.store, wl.batch
+    st = Docstore(s.n_docs, s.doc_dim, s.doc_dtype, b.edge_dim, b.edge_dtype, b.req_dim, b.req_dtype,
+                  s.max_actors, s.reduce_sum_mask, device)
+    st.upload(0, s.doc_feats if upload_doc_feats else None, s.author_ids, s.actor_ids, s.actor_types)
+    torch.cuda.synchronize(device)
+    return st

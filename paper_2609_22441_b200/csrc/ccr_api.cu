@@ -1,0 +1,512 @@
+// Host side of the C ABI declared in include/ccr.h: handles, argument checks, kernel selection, launches.
+// No CPU fallback exists: when CUDA is unavailable every compute entry fails with CCR_ERR_CUDA.
+#include "../../include/ccr.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "ccr_join.cuh"
+#include "ccr_merge.cuh"
+
+namespace {
+
+constexpr uint64_t kStoreMagic = 0x43435253544f5245ull;  // "CCRSTORE"
+constexpr uint64_t kWsMagic = 0x4343525753504143ull;     // "CCRWSPAC"
+constexpr int kMaxSmemBytes = 227 * 1024;
+constexpr int kDefaultTile = 1024;
+constexpr int kDefaultKeyCap = 4096;
+constexpr int kMaxTile = 4096;
+
+inline size_t dtype_size(int32_t dt) { return dt == CCR_F16 ? 2 : (dt == CCR_F32 ? 4 : 0); }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Sets the store's device for the scope of a call and restores the caller's device afterwards.
+struct DeviceScope {
+  int prev = -1;
+  bool ok = false;
+  explicit DeviceScope(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) return;
+    ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+    if (prev == dev) prev = -1;
+  }
+  ~DeviceScope() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+}  // namespace
+
+struct ccr_docstore {
+  uint64_t magic;
+  ccr_docstore_desc desc;
+  int doc_b, edge_b, req_b;  // section widths in bytes
+  uint8_t* doc_feats;
+  int64_t* author_ids;
+  int64_t* actor_ids;
+  uint8_t* actor_types;
+  int* status;        // device: [0] wait expiry, [1] validation code
+  int* status_host;   // pinned host copy
+  int tile;
+  int key_cap;
+  int64_t launches;
+};
+
+struct ccr_workspace {
+  uint64_t magic;
+  int device;
+  int32_t max_req;
+  int64_t max_cands, max_edges;
+  size_t out_b_max, edge_b, req_b;
+  int64_t* edge_keys;
+  uint8_t* edge_feats;
+  int64_t* edge_offsets;
+  int32_t* cand_idx;
+  int64_t* cand_offsets;
+  uint8_t* req_feats;
+  uint8_t* out_rows;
+  uint8_t* out_mask;
+};
+
+namespace {
+
+inline bool good(const ccr_docstore* s) { return s != nullptr && s->magic == kStoreMagic; }
+
+// ---------------------------------------------------------------------------------------------------
+// Precondition check behind CCR_FLAG_VALIDATE: one block per request.
+//   code 1: cand_offsets malformed   2: edge_offsets malformed / longer than max_edge_len
+//   code 3: keys not strictly ascending or negative   4: candidates not sorted by author (CANDS_SORTED)
+__global__ void validate_kernel(const ccr::JoinArgs a, int check_sorted, int* code) {
+  const int r = blockIdx.x;
+  const int64_t c0 = a.cand_offsets[r], c1 = a.cand_offsets[r + 1];
+  const int64_t e0 = a.edge_offsets[r], e1 = a.edge_offsets[r + 1];
+  int bad = 0;
+  if (threadIdx.x == 0) {
+    if (c0 > c1 || c0 < 0 || (r == 0 && c0 != 0) || (r == a.n_req - 1 && c1 != a.total)) bad = 1;
+    else if (e0 > e1 || e0 < 0 || e1 - e0 > a.max_edge_len) bad = 2;
+  }
+  bad = __syncthreads_or(bad) ? (bad ? bad : -1) : 0;
+  if (bad != 0) {
+    if (bad > 0) atomicCAS(code, 0, bad);
+    return;
+  }
+  for (int64_t i = e0 + threadIdx.x; i < e1; i += blockDim.x) {
+    const int64_t k = a.edge_keys[i];
+    if (k < 0 || (i > e0 && a.edge_keys[i - 1] >= k)) atomicCAS(code, 0, 3);
+  }
+  if (check_sorted) {
+    for (int64_t j = c0 + 1 + threadIdx.x; j < c1; j += blockDim.x) {
+      const int p = a.cand_idx[j - 1], q = a.cand_idx[j];
+      const bool pin = p >= 0 && p < a.n_docs, qin = q >= 0 && q < a.n_docs;
+      const long long ap = pin ? a.author_ids[p] : ccr::kNoAuthor;
+      const long long aq = qin ? a.author_ids[q] : ccr::kNoAuthor;
+      if (ap > aq) atomicCAS(code, 0, 4);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Kernel variants: section widths fixed at compile time for the layouts the benchmark configurations
+// use (256-byte doc rows; 64- or 128-byte edge rows; 0 or 64 bytes of request features), and a generic
+// variant with run-time widths for everything else.
+using KernelFn = void (*)(const ccr::JoinArgs);
+
+struct Variant {
+  int doc_ch, edge_ch, req_ch;
+  KernelFn first, second, merge;
+};
+
+#define CCR_VARIANT(D, E, R)                                                                        \
+  Variant {                                                                                         \
+    D, E, R, ccr::join_kernel<D, E, R, false>, ccr::join_kernel<D, E, R, true>, ccr::join_merge_kernel<D, E, R> \
+  }
+
+const Variant kVariants[] = {
+    CCR_VARIANT(16, 4, 0),
+    CCR_VARIANT(16, 4, 4),
+    CCR_VARIANT(16, 8, 0),
+    CCR_VARIANT(16, 8, 4),
+    CCR_VARIANT(0, 0, 0),  // generic: must stay last
+};
+constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
+
+const Variant& pick_variant(int doc_ch, int edge_ch, int req_ch) {
+  for (int i = 0; i < kNumVariants - 1; ++i) {
+    const Variant& v = kVariants[i];
+    if (v.doc_ch == doc_ch && v.edge_ch == edge_ch && v.req_ch == req_ch) return v;
+  }
+  return kVariants[kNumVariants - 1];
+}
+
+ccr_status allow_large_smem() {
+  for (int i = 0; i < kNumVariants; ++i) {
+    const KernelFn fns[3] = {kVariants[i].first, kVariants[i].second, kVariants[i].merge};
+    for (KernelFn f : fns) {
+      if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemBytes) != cudaSuccess) {
+        cudaGetLastError();
+        return CCR_ERR_CUDA;
+      }
+    }
+  }
+  return CCR_OK;
+}
+
+size_t out_row_bytes(const ccr_docstore* s, uint32_t flags) {
+  const bool second = s->desc.max_actors > 0 && !(flags & CCR_FLAG_FIRST_DEGREE_ONLY);
+  return static_cast<size_t>(s->doc_b) + s->edge_b * (second ? 2 : 1) + s->req_b;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ccr_version(void) { return 100; }
+
+const char* ccr_status_str(ccr_status s) {
+  switch (s) {
+    case CCR_OK: return "ok";
+    case CCR_ERR_INVALID_ARG: return "invalid argument";
+    case CCR_ERR_UNSUPPORTED: return "unsupported width, dtype or size";
+    case CCR_ERR_OOM: return "out of device memory";
+    case CCR_ERR_CUDA: return "CUDA runtime error or no usable device";
+    case CCR_ERR_BAD_HANDLE: return "bad handle";
+    case CCR_ERR_VALIDATION: return "input validation failed";
+    case CCR_ERR_DEVICE_WAIT: return "a bounded device-side wait expired";
+  }
+  return "unknown status";
+}
+
+ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
+  if (out == nullptr) return CCR_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (d == nullptr) return CCR_ERR_INVALID_ARG;
+  if (d->n_docs < 0 || d->doc_dim <= 0 || d->edge_dim <= 0 || d->req_dim < 0 || d->max_actors < 0 || d->device < 0)
+    return CCR_ERR_INVALID_ARG;
+  const size_t dsz = dtype_size(d->doc_dtype), esz = dtype_size(d->edge_dtype), rsz = dtype_size(d->req_dtype);
+  if (dsz == 0 || esz == 0 || (d->req_dim > 0 && rsz == 0)) return CCR_ERR_INVALID_ARG;
+  const size_t doc_b = d->doc_dim * dsz, edge_b = d->edge_dim * esz, req_b = d->req_dim * rsz;
+  if (doc_b % 16 || edge_b % 16 || req_b % 16) return CCR_ERR_UNSUPPORTED;
+  if (doc_b > (1u << 20) || edge_b > (1u << 20) || req_b > (1u << 20)) return CCR_ERR_UNSUPPORTED;
+  if (d->n_docs > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;  // positions are int32
+  if (d->max_actors > 4) return CCR_ERR_UNSUPPORTED;
+  if (d->max_actors > 0 && (d->edge_dtype != CCR_F16 || d->edge_dim > 64)) return CCR_ERR_UNSUPPORTED;
+
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || d->device >= n_dev) {
+    cudaGetLastError();
+    return CCR_ERR_CUDA;
+  }
+  DeviceScope scope(d->device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+
+  const size_t n = static_cast<size_t>(d->n_docs);
+  const size_t need = n * doc_b + n * 8 + (d->max_actors ? n * d->max_actors * 9 : 0) + 4096;
+  size_t free_b = 0, total_b = 0;
+  if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return CCR_ERR_CUDA;
+  if (need > free_b) return CCR_ERR_OOM;
+
+  ccr_docstore* s = new (std::nothrow) ccr_docstore();
+  if (s == nullptr) return CCR_ERR_OOM;
+  std::memset(s, 0, sizeof(*s));
+  s->desc = *d;
+  s->doc_b = static_cast<int>(doc_b);
+  s->edge_b = static_cast<int>(edge_b);
+  s->req_b = static_cast<int>(req_b);
+  s->tile = kDefaultTile;
+  s->key_cap = kDefaultKeyCap;
+  bool ok = true;
+  // n == 0 still allocates a token block so that every pointer is valid and aligned
+  ok = ok && cudaMalloc(&s->doc_feats, n * doc_b + 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->author_ids, n * 8 + 256) == cudaSuccess;
+  if (d->max_actors > 0) {
+    ok = ok && cudaMalloc(&s->actor_ids, n * d->max_actors * 8 + 256) == cudaSuccess;
+    ok = ok && cudaMalloc(&s->actor_types, n * d->max_actors + 256) == cudaSuccess;
+  }
+  ok = ok && cudaMalloc(&s->status, 4 * sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemset(s->status, 0, 4 * sizeof(int)) == cudaSuccess;
+  ok = ok && cudaHostAlloc(&s->status_host, 4 * sizeof(int), cudaHostAllocDefault) == cudaSuccess;
+  ccr_status st = ok ? allow_large_smem() : CCR_ERR_OOM;
+  if (st != CCR_OK) {
+    cudaGetLastError();
+    cudaFree(s->doc_feats);
+    cudaFree(s->author_ids);
+    cudaFree(s->actor_ids);
+    cudaFree(s->actor_types);
+    cudaFree(s->status);
+    if (s->status_host) cudaFreeHost(s->status_host);
+    delete s;
+    return st;
+  }
+  s->magic = kStoreMagic;
+  *out = s;
+  return CCR_OK;
+}
+
+ccr_status ccr_docstore_free(ccr_docstore* s) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  DeviceScope scope(s->desc.device);
+  s->magic = 0;
+  cudaFree(s->doc_feats);
+  cudaFree(s->author_ids);
+  cudaFree(s->actor_ids);
+  cudaFree(s->actor_types);
+  cudaFree(s->status);
+  cudaFreeHost(s->status_host);
+  delete s;
+  return CCR_OK;
+}
+
+ccr_status ccr_docstore_upload(ccr_docstore* s, int64_t first_doc, int64_t n, const void* doc_feats,
+                               const int64_t* author_ids, const int64_t* actor_ids, const uint8_t* actor_types,
+                               int src_on_device, void* stream) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  if (first_doc < 0 || n < 0 || first_doc + n > s->desc.n_docs) return CCR_ERR_INVALID_ARG;
+  if (n == 0) return CCR_OK;
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const cudaMemcpyKind kind = src_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  const size_t un = static_cast<size_t>(n), uf = static_cast<size_t>(first_doc);
+  const int ma = s->desc.max_actors;
+  bool ok = true;
+  if (doc_feats) ok = ok && cudaMemcpyAsync(s->doc_feats + uf * s->doc_b, doc_feats, un * s->doc_b, kind, st) == cudaSuccess;
+  if (author_ids) ok = ok && cudaMemcpyAsync(s->author_ids + uf, author_ids, un * 8, kind, st) == cudaSuccess;
+  if (ma > 0 && actor_ids) ok = ok && cudaMemcpyAsync(s->actor_ids + uf * ma, actor_ids, un * ma * 8, kind, st) == cudaSuccess;
+  if (ma > 0 && actor_types) ok = ok && cudaMemcpyAsync(s->actor_types + uf * ma, actor_types, un * ma, kind, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return CCR_ERR_CUDA;
+  }
+  return CCR_OK;
+}
+
+size_t ccr_out_row_bytes(const ccr_docstore* s, uint32_t flags) { return good(s) ? out_row_bytes(s, flags) : 0; }
+
+ccr_status ccr_docstore_set_tuning(ccr_docstore* s, int32_t tile_cands, int32_t key_capacity) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  if (tile_cands < 0 || key_capacity < 0) return CCR_ERR_INVALID_ARG;
+  if (tile_cands > 0) {
+    if (tile_cands % 32 || tile_cands > kMaxTile) return CCR_ERR_INVALID_ARG;
+    s->tile = tile_cands;
+  }
+  if (key_capacity > 0) {
+    if (static_cast<size_t>(key_capacity + 2) * 8 + ccr::kSmemHeader > static_cast<size_t>(kMaxSmemBytes)) return CCR_ERR_INVALID_ARG;
+    s->key_cap = key_capacity;
+  }
+  return CCR_OK;
+}
+
+int64_t ccr_docstore_launch_count(const ccr_docstore* s) { return good(s) ? s->launches : -1; }
+
+ccr_status ccr_docstore_device_status(ccr_docstore* s, void* stream) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool ok = cudaMemcpyAsync(s->status_host, s->status, 4 * sizeof(int), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(s->status, 0, 4 * sizeof(int), st) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return CCR_ERR_CUDA;
+  }
+  return s->status_host[0] == ccr::kDevWaitExpired ? CCR_ERR_DEVICE_WAIT : CCR_OK;
+}
+
+ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                          const int64_t* edge_keys, const void* edge_feats, const int64_t* edge_offsets,
+                          const int32_t* cand_idx, const int64_t* cand_offsets, const void* req_feats,
+                          void* out_rows, uint8_t* out_mask, uint32_t flags, void* stream) {
+  if (!good(cs)) return CCR_ERR_BAD_HANDLE;
+  ccr_docstore* s = const_cast<ccr_docstore*>(cs);  // only the launch counter and status words change
+  if (n_req < 0 || total_cands < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
+  if (max_edge_len > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;
+  const uint32_t path = flags & (CCR_FLAG_FORCE_SMEM | CCR_FLAG_FORCE_GLOBAL | CCR_FLAG_FORCE_SAMPLED);
+  if (path & (path - 1)) return CCR_ERR_INVALID_ARG;  // at most one forced path
+  if (n_req == 0 || total_cands == 0) return (n_req == 0 && total_cands != 0) ? CCR_ERR_INVALID_ARG : CCR_OK;
+  if (!edge_offsets || !cand_offsets || !cand_idx || !out_rows || !out_mask) return CCR_ERR_INVALID_ARG;
+  if (max_edge_len > 0 && (!edge_keys || !edge_feats)) return CCR_ERR_INVALID_ARG;
+  if (s->req_b > 0 && !req_feats) return CCR_ERR_INVALID_ARG;
+  if (!aligned16(edge_keys) || !aligned16(edge_feats) || !aligned16(req_feats) || !aligned16(out_rows))
+    return CCR_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(edge_offsets) & 7u) || (reinterpret_cast<uintptr_t>(cand_offsets) & 7u) ||
+      (reinterpret_cast<uintptr_t>(cand_idx) & 3u))
+    return CCR_ERR_INVALID_ARG;
+
+  const bool second = s->desc.max_actors > 0 && !(flags & CCR_FLAG_FIRST_DEGREE_ONLY);
+  // engager ids are not sorted, so the merge path serves first-degree joins only; a second-degree join
+  // on sorted candidates takes the binary-search kernel (same result by definition)
+  const bool merge = (flags & CCR_FLAG_CANDS_SORTED) && !second;
+
+  int key_cap;
+  if (flags & CCR_FLAG_FORCE_GLOBAL) key_cap = 0;
+  else if (flags & CCR_FLAG_FORCE_SMEM) key_cap = static_cast<int>(max_edge_len);
+  else key_cap = static_cast<int>(max_edge_len < s->key_cap ? max_edge_len : s->key_cap);
+  size_t smem = ccr::kSmemHeader + static_cast<size_t>(key_cap + 2) * 8;
+  if (merge) smem += static_cast<size_t>(s->tile) * 8 + static_cast<size_t>((s->tile + 3) & ~3) * 4;
+  if (smem > static_cast<size_t>(kMaxSmemBytes)) return CCR_ERR_UNSUPPORTED;
+
+  ccr::JoinArgs a;
+  a.doc_feats = s->doc_feats;
+  a.author_ids = s->author_ids;
+  a.actor_ids = s->actor_ids;
+  a.actor_types = s->actor_types;
+  a.n_docs = s->desc.n_docs;
+  a.max_actors = s->desc.max_actors;
+  a.reduce_sum_mask = s->desc.reduce_sum_mask;
+  a.doc_ch = s->doc_b / 16;
+  a.edge_ch = s->edge_b / 16;
+  a.req_ch = s->req_b / 16;
+  a.n_req = n_req;
+  a.total = total_cands;
+  a.max_edge_len = static_cast<int>(max_edge_len);
+  a.edge_keys = edge_keys;
+  a.edge_feats = static_cast<const uint8_t*>(edge_feats);
+  a.edge_offsets = edge_offsets;
+  a.cand_idx = cand_idx;
+  a.cand_offsets = cand_offsets;
+  a.req_feats = static_cast<const uint8_t*>(req_feats);
+  a.out_rows = static_cast<uint8_t*>(out_rows);
+  a.out_mask = out_mask;
+  a.tile = s->tile;
+  a.key_cap = key_cap;
+  a.min_stride_log2 = (flags & CCR_FLAG_FORCE_SAMPLED) ? 2 : 0;
+  a.status = s->status;
+
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  if (flags & CCR_FLAG_VALIDATE) {
+    validate_kernel<<<n_req, 256, 0, st>>>(a, (flags & CCR_FLAG_CANDS_SORTED) ? 1 : 0, s->status + 1);
+    s->launches++;
+    bool ok = cudaMemcpyAsync(s->status_host + 1, s->status + 1, sizeof(int), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(s->status + 1, 0, sizeof(int), st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
+    if (s->status_host[1] != 0) return CCR_ERR_VALIDATION;
+  }
+
+  const Variant& v = pick_variant(a.doc_ch, a.edge_ch, a.req_ch);
+  const KernelFn fn = merge ? v.merge : (second ? v.second : v.first);
+  const long long blocks = (total_cands + a.tile - 1) / a.tile;
+  if (blocks > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;
+  fn<<<static_cast<unsigned>(blocks), ccr::kThreads, smem, st>>>(a);
+  s->launches++;
+  if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+  return CCR_OK;
+}
+
+ccr_status ccr_workspace_create(const ccr_docstore* s, int32_t max_req, int64_t max_cands, int64_t max_edges,
+                                ccr_workspace** out) {
+  if (out == nullptr) return CCR_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  if (max_req <= 0 || max_cands <= 0 || max_edges < 0) return CCR_ERR_INVALID_ARG;
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  ccr_workspace* w = new (std::nothrow) ccr_workspace();
+  if (w == nullptr) return CCR_ERR_OOM;
+  std::memset(w, 0, sizeof(*w));
+  w->device = s->desc.device;
+  w->max_req = max_req;
+  w->max_cands = max_cands;
+  w->max_edges = max_edges;
+  w->out_b_max = out_row_bytes(s, 0);
+  w->edge_b = s->edge_b;
+  w->req_b = s->req_b;
+  const size_t need = (max_edges + 2) * (8 + w->edge_b) + (max_req + 1) * (16 + w->req_b) + max_cands * (5 + w->out_b_max);
+  size_t free_b = 0, total_b = 0;
+  if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess || need + (64u << 20) > free_b) {
+    cudaGetLastError();
+    delete w;
+    return CCR_ERR_OOM;
+  }
+  bool ok = true;
+  ok = ok && cudaMalloc(&w->edge_keys, (max_edges + 2) * 8) == cudaSuccess;
+  ok = ok && cudaMalloc(&w->edge_feats, (max_edges + 2) * w->edge_b) == cudaSuccess;
+  ok = ok && cudaMalloc(&w->edge_offsets, (max_req + 1) * 8) == cudaSuccess;
+  ok = ok && cudaMalloc(&w->cand_idx, max_cands * 4) == cudaSuccess;
+  ok = ok && cudaMalloc(&w->cand_offsets, (max_req + 1) * 8) == cudaSuccess;
+  ok = ok && cudaMalloc(&w->req_feats, (max_req + 1) * (w->req_b ? w->req_b : 16)) == cudaSuccess;
+  ok = ok && cudaMalloc(&w->out_rows, max_cands * w->out_b_max) == cudaSuccess;
+  ok = ok && cudaMalloc(&w->out_mask, max_cands) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    w->magic = kWsMagic;
+    ccr_workspace_free(w);
+    return CCR_ERR_OOM;
+  }
+  w->magic = kWsMagic;
+  *out = w;
+  return CCR_OK;
+}
+
+ccr_status ccr_workspace_free(ccr_workspace* w) {
+  if (w == nullptr || w->magic != kWsMagic) return CCR_ERR_BAD_HANDLE;
+  DeviceScope scope(w->device);
+  w->magic = 0;
+  cudaFree(w->edge_keys);
+  cudaFree(w->edge_feats);
+  cudaFree(w->edge_offsets);
+  cudaFree(w->cand_idx);
+  cudaFree(w->cand_offsets);
+  cudaFree(w->req_feats);
+  cudaFree(w->out_rows);
+  cudaFree(w->out_mask);
+  delete w;
+  return CCR_OK;
+}
+
+ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t n_req, int64_t total_cands,
+                               int64_t max_edge_len, int64_t total_edges, const int64_t* edge_keys,
+                               const void* edge_feats, const int64_t* edge_offsets, const int32_t* cand_idx,
+                               const int64_t* cand_offsets, const void* req_feats, void* out_rows,
+                               uint8_t* out_mask, uint32_t flags, void* stream) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  if (w == nullptr || w->magic != kWsMagic || w->device != s->desc.device) return CCR_ERR_BAD_HANDLE;
+  if (n_req < 0 || total_cands < 0 || total_edges < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
+  if (n_req > w->max_req || total_cands > w->max_cands || total_edges > w->max_edges) return CCR_ERR_INVALID_ARG;
+  if (n_req == 0 || total_cands == 0) return (n_req == 0 && total_cands != 0) ? CCR_ERR_INVALID_ARG : CCR_OK;
+  if (!edge_offsets || !cand_offsets || !cand_idx || !out_rows || !out_mask) return CCR_ERR_INVALID_ARG;
+  if (total_edges > 0 && (!edge_keys || !edge_feats)) return CCR_ERR_INVALID_ARG;
+  if (s->req_b > 0 && !req_feats) return CCR_ERR_INVALID_ARG;
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t out_b = out_row_bytes(s, flags);
+  bool ok = true;
+  if (total_edges > 0) {
+    ok = ok && cudaMemcpyAsync(w->edge_keys, edge_keys, total_edges * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(w->edge_feats, edge_feats, total_edges * w->edge_b, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(w->edge_offsets, edge_offsets, (n_req + 1) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(w->cand_idx, cand_idx, total_cands * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(w->cand_offsets, cand_offsets, (n_req + 1) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (s->req_b > 0)
+    ok = ok && cudaMemcpyAsync(w->req_feats, req_feats, static_cast<size_t>(n_req) * w->req_b, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return CCR_ERR_CUDA;
+  }
+  const ccr_status js = ccr_join_batch(s, n_req, total_cands, max_edge_len, w->edge_keys, w->edge_feats, w->edge_offsets,
+                                       w->cand_idx, w->cand_offsets, s->req_b ? w->req_feats : nullptr, w->out_rows,
+                                       w->out_mask, flags, stream);
+  if (js != CCR_OK) return js;
+  ok = ok && cudaMemcpyAsync(out_rows, w->out_rows, total_cands * out_b, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(out_mask, w->out_mask, total_cands, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return CCR_ERR_CUDA;
+  }
+  return CCR_OK;
+}
+
+}  // extern "C"

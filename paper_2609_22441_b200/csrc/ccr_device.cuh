@@ -1,0 +1,133 @@
+// Device-side building blocks of the join kernels (sm_100a): bulk-copy + mbarrier wrappers,
+// cache-hinted 128-bit loads/stores and the branch-free lower-bound searches.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace ccr {
+
+constexpr int kThreads = 256;            // threads per block of every join kernel
+constexpr int kWarps = kThreads / 32;
+constexpr int kSmemHeader = 16;          // one mbarrier (8 B) + padding so that keys start 16-B aligned
+constexpr unsigned kFull = 0xffffffffu;
+
+// Device status word values (written to JoinArgs::status[0]).
+constexpr int kDevOk = 0;
+constexpr int kDevWaitExpired = 1;
+
+// Everything a join launch needs, passed by value as the kernel argument.
+struct JoinArgs {
+  // store
+  const uint8_t* doc_feats;
+  const int64_t* author_ids;
+  const int64_t* actor_ids;   // [n_docs, max_actors] or null
+  const uint8_t* actor_types; // [n_docs, max_actors] or null
+  long long n_docs;
+  int max_actors;
+  unsigned long long reduce_sum_mask;
+  // section widths in 16-byte chunks
+  int doc_ch, edge_ch, req_ch;
+  // batch
+  int n_req;
+  long long total;            // candidates in the launch
+  int max_edge_len;           // host-promised bound on every request's key count
+  const int64_t* edge_keys;
+  const uint8_t* edge_feats;
+  const int64_t* edge_offsets;
+  const int32_t* cand_idx;
+  const int64_t* cand_offsets;
+  const uint8_t* req_feats;
+  uint8_t* out_rows;
+  uint8_t* out_mask;
+  // launch shape
+  int tile;                   // candidates per block
+  int key_cap;                // keys (or sampled keys) a block may stage per request; 0 = search global memory
+  int min_stride_log2;        // >0 forces sampling with at least this stride (testing aid)
+  int* status;                // device status words
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+// Make generic-proxy writes to shared memory (the barrier's initial state) visible to the async proxy.
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// 1-D bulk copy global -> this block's shared memory through the TMA engine; completion is signalled
+// on `bar` as `bytes` of transaction count.  Both addresses 16-B aligned, bytes a multiple of 16.
+// No multicast: one block, one destination.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+      "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      " selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait: gives up after kWaitTries polls (each poll may itself suspend for a short,
+// hardware-defined time).  Returns false when the phase never completed.
+constexpr int kWaitTries = 1 << 22;
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (int i = 0; i < kWaitTries; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+
+__device__ __forceinline__ uint4 ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+
+// Output rows are written once and never read back by the kernel: streaming (evict-first) stores keep
+// them from displacing the keys, edge tables and id arrays that live in L2.
+__device__ __forceinline__ void st128_stream(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
+
+// Branch-free lower bound over n ascending keys: number of keys < id.  Every lane of a warp runs the
+// same trip count when n is warp-uniform.
+__device__ __forceinline__ int lower_bound_smem(const int64_t* s, int n, int64_t id) {
+  int lo = 0;
+  while (n > 1) {
+    const int half = n >> 1;
+    lo = (s[lo + half - 1] < id) ? lo + half : lo;
+    n -= half;
+  }
+  if (n == 1) lo += (s[lo] < id) ? 1 : 0;
+  return lo;
+}
+
+__device__ __forceinline__ int lower_bound_global(const int64_t* g, int n, int64_t id) {
+  int lo = 0;
+  while (n > 1) {
+    const int half = n >> 1;
+    lo = (__ldg(g + lo + half - 1) < id) ? lo + half : lo;
+    n -= half;
+  }
+  if (n == 1) lo += (__ldg(g + lo) < id) ? 1 : 0;
+  return lo;
+}
+
+}  // namespace ccr

@@ -1,0 +1,51 @@
+"""Shared test helpers: tiny random problems and the GPU call with guard bytes around the outputs."""
+import numpy as np
+
+from paper_2609_22441_b200 import workloads as W
+
+GUARD = 256
+
+
+def tiny_workload(seed, n_docs, alphabet, n_req, kmax, nmax, second, req_dim, doc_dim=4, doc_dtype=np.float32,
+                  edge_dim=8, sum_mask=0b10110100):
+    """Tiny problem with ids from a tiny alphabet so that hits, misses, repeats, empty requests and
+    unresolved / out-of-range positions are all common."""
+    rng = np.random.default_rng(seed)
+    store = W.make_store(rng, n_docs, alphabet, doc_dim, doc_dtype, max_actors=4 if second else 0,
+                         reduce_sum_mask=sum_mask if second else 0)
+    keys_l, feats_l, cands_l = [], [], []
+    vals = np.array([-2.0, -0.5, 0.0, 0.25, 0.5, 1.0, 1.5, 3.0, 1000.0, 6e-5, 60000.0, -0.0], np.float16)
+    for _ in range(n_req):
+        k = int(rng.integers(0, min(kmax, alphabet) + 1))
+        keys, _ = W.make_viewer(rng, alphabet, k, edge_dim, np.float16)
+        feats = rng.choice(vals, size=(k, edge_dim))
+        n = int(rng.integers(0, nmax + 1))
+        cands_l.append(rng.integers(-1, n_docs + 1, size=n).astype(np.int32))
+        keys_l.append(keys)
+        feats_l.append(feats)
+    req = rng.standard_normal((n_req, req_dim)).astype(np.float32) if req_dim else None
+    batch = W.assemble_batch(keys_l, feats_l, cands_l, req, edge_dim, np.float16, req_dim, np.float32)
+    return W.Workload("tiny", seed, store, batch)
+
+
+def gpu_join(store, db, flags=0):
+    """Run ccr_join_batch into buffers framed by guard bytes; returns numpy (rows, mask) after checking
+    that no byte outside the output ranges was written."""
+    import torch
+
+    from paper_2609_22441_b200 import binding as B
+
+    out_b = store.out_row_bytes(flags)
+    n = db.total_cands
+    dev = torch.device("cuda", store.device)
+    rows_buf = torch.full((GUARD + n * out_b + GUARD,), 0xA5, dtype=torch.uint8, device=dev)
+    mask_buf = torch.full((GUARD + n + GUARD,), 0xA5, dtype=torch.uint8, device=dev)
+    rows = rows_buf[GUARD:GUARD + n * out_b].view(n, out_b) if n else rows_buf[GUARD:GUARD].view(0, out_b)
+    mask = mask_buf[GUARD:GUARD + n]
+    B.ccr_join_batch(store, db.n_req, n, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets, db.cand_idx,
+                     db.cand_offsets, db.req_feats, rows, mask, flags)
+    torch.cuda.synchronize(dev)
+    rb, mb = rows_buf.cpu().numpy(), mask_buf.cpu().numpy()
+    assert (rb[:GUARD] == 0xA5).all() and (rb[GUARD + n * out_b:] == 0xA5).all(), "write outside out_rows"
+    assert (mb[:GUARD] == 0xA5).all() and (mb[GUARD + n:] == 0xA5).all(), "write outside out_mask"
+    return rb[GUARD:GUARD + n * out_b].reshape(n, out_b), mb[GUARD:GUARD + n]

@@ -1,0 +1,325 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, byte for byte.
+
+The join is indexing and copying (plus a fixed-order fp16 reduction for second-degree stores whose
+rounding both sides take in fp32 with one final round-to-nearest-even), so the bar is bit-exact equality
+of every output row and mask byte."""
+import ctypes
+
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2609_22441_b200 import workloads as W
+
+from helpers import gpu_join, tiny_workload
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2609_22441_b200 import binding, build
+
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _variants(B, include_smem=True):
+    v = [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL), ("sampled", B.CCR_FLAG_FORCE_SAMPLED)]
+    if include_smem:
+        v.append(("smem", B.CCR_FLAG_FORCE_SMEM))
+    return v
+
+
+def _check(B, wl, flag_sets, first_degree_only=False, tunings=((0, 0),)):
+    want_rows, want_mask = oracle.join_workload(wl, first_degree_only=first_degree_only, n_threads=4)
+    store = B.store_from_workload(wl)
+    db = B.DeviceBatch(wl.batch)
+    try:
+        for tile, cap in tunings:
+            if tile or cap:
+                store.set_tuning(tile, cap)
+            for name, flags in flag_sets:
+                if first_degree_only:
+                    flags |= B.CCR_FLAG_FIRST_DEGREE_ONLY
+                rows, mask = gpu_join(store, db, flags)
+                assert np.array_equal(mask, want_mask), (wl.name, name, tile, cap)
+                assert rows.shape == want_rows.shape
+                if not np.array_equal(rows, want_rows):
+                    bad = np.nonzero((rows != want_rows).any(axis=1))[0]
+                    raise AssertionError("%s/%s tile=%d cap=%d: %d rows differ, first %d" %
+                                         (wl.name, name, tile, cap, len(bad), bad[0]))
+        assert store.device_status() == B.CCR_OK
+    finally:
+        store.free()
+    return want_rows, want_mask
+
+
+# ------------------------------------------------------------------ the benchmark configurations
+def test_config0_single_tiny_request_all_search_paths(B):
+    wl = W.config0()
+    _check(B, wl, _variants(B))
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
+
+
+def test_config1_batched_first_degree_full_size(B):
+    wl = W.config1()
+    assert wl.batch.total_cands == 64 * 30_000 and wl.out_row_bytes() == 384
+    _check(B, wl, _variants(B))
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
+
+
+def test_config2a_second_degree_on_config0_shape(B):
+    wl = W.config0(second_degree=True)
+    assert wl.out_row_bytes() == 384
+    _, mask = _check(B, wl, _variants(B))
+    assert (mask >> 1).any() and (mask >> 5).any()
+    _check(B, wl, [("auto", 0)], first_degree_only=True)
+    ws = W.sort_candidates_by_author(wl)
+    _check(B, ws, [("sorted-second", B.CCR_FLAG_CANDS_SORTED)])
+    _check(B, ws, [("merge", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=True)
+
+
+def test_config2b_second_degree_on_config1_shape_full_size(B):
+    wl = W.config1(second_degree=True)
+    assert wl.out_row_bytes() == 448
+    _check(B, wl, [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL)])
+
+
+def test_config3_scaled_store_long_edge_lists(B):
+    # production shape at 1/25 of the store: K log-uniform up to 20000 (longer than the default staging
+    # budget, so the sampled top-of-tree path runs), 128-byte edge rows, second-degree store joined
+    # first-degree-only as in the headline run, then fully
+    wl = W.config3(n_docs=2_000_000, n_req=12, n_cand=20_000, gen_doc_feats=True, extra_pools=0)
+    assert wl.batch.max_edge_len > 4096
+    _check(B, wl, _variants(B), first_degree_only=True, tunings=((0, 0), (512, 1000), (2048, 20_000)))
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=True,
+           tunings=((0, 0), (256, 64)))
+    _check(B, wl, [("auto", 0)])
+
+
+# ------------------------------------------------------------------ ragged / degenerate inputs
+@pytest.mark.parametrize("seed", range(12))
+def test_tiny_random_batches(B, seed):
+    second = bool(seed % 2)
+    wl = tiny_workload(seed, n_docs=37 + seed, alphabet=20 + 3 * seed, n_req=1 + seed, kmax=16, nmax=70,
+                       second=second, req_dim=4 * (seed % 3 == 0))
+    _check(B, wl, _variants(B), tunings=((32, 0), (0, 0)))
+    if second:
+        _check(B, wl, [("auto", 0)], first_degree_only=True)
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=second,
+           tunings=((64, 0),))
+
+
+def test_generic_widths_take_the_runtime_variant(B):
+    # 96-byte doc rows, 16-byte edge rows, 16 bytes of request features: none of the compiled-in layouts
+    wl = tiny_workload(99, n_docs=500, alphabet=300, n_req=7, kmax=120, nmax=900, second=False, req_dim=4,
+                       doc_dim=24, edge_dim=8)
+    _check(B, wl, _variants(B))
+    wl2 = tiny_workload(98, n_docs=500, alphabet=300, n_req=7, kmax=120, nmax=900, second=True, req_dim=0,
+                        doc_dim=24, edge_dim=8)
+    _check(B, wl2, _variants(B))
+
+
+def _manual(keys_l, cand_l, author_ids, n_docs=None, edge_dim=32, doc_dim=64, seed=0):
+    rng = np.random.default_rng(seed)
+    n_docs = n_docs or len(author_ids)
+    store = W.Store(n_docs=n_docs, doc_dim=doc_dim, doc_dtype=np.dtype(np.float32),
+                    author_ids=np.asarray(author_ids, np.int64),
+                    doc_feats=rng.standard_normal((n_docs, doc_dim)).astype(np.float32))
+    feats_l = [rng.random((len(k), edge_dim), dtype=np.float32).astype(np.float16) for k in keys_l]
+    batch = W.assemble_batch([np.asarray(k, np.int64) for k in keys_l], feats_l,
+                             [np.asarray(c, np.int32) for c in cand_l], None, edge_dim, np.float16, 0, np.float32)
+    return W.Workload("manual", seed, store, batch)
+
+
+def test_search_boundaries_and_empty_requests(B):
+    imax = np.iinfo(np.int64).max
+    authors = [0, 5, 7, 9, imax, imax - 1, -3, 6, 7, 7]
+    keys = [[0, 7, imax], [], [7], [0, 7, imax], [5, 6, 9, imax - 1]]
+    cands = [[0, 1, 2, 3, 4, 5, 6, 7, 2, 2, -1, 10], [1, 2, 3], [2, 8, 9, 0], [], [1, 7, 3, 5, 4, 2]]
+    wl = _manual(keys, cands, authors)
+    rows, mask = _check(B, wl, _variants(B), tunings=((32, 0), (0, 0)))
+    assert list(mask[:12]) == [1, 0, 1, 0, 1, 0, 0, 0, 1, 1, 0, 0]
+    assert list(mask[12:15]) == [0, 0, 0] and list(mask[15:19]) == [1, 1, 1, 0] and list(mask[19:]) == [1, 1, 1, 1, 0, 0]
+
+
+def test_all_found_none_found_and_duplicates(B):
+    rng = np.random.default_rng(3)
+    authors = rng.integers(0, 1000, size=4000)
+    all_keys = np.unique(authors)
+    none_keys = np.arange(2000, 2600)
+    cand = rng.integers(0, 4000, size=5000)  # with repeats
+    wl = _manual([all_keys, none_keys, all_keys[::2]], [cand, cand, cand[:1]], authors)
+    rows, mask = _check(B, wl, _variants(B))
+    assert mask[:5000].all() and not mask[5000:10000].any()
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 255, 256, 257, 4095, 4096, 4097, 8191, 29_000, 65_536, 100_000])
+def test_edge_list_lengths_around_every_path_threshold(B, k):
+    # two requests so that the second one's keys start at an odd (8-byte aligned only) offset when k is odd
+    rng = np.random.default_rng(k)
+    n_docs = 30_000
+    authors = rng.integers(0, 4 * k + 10, size=n_docs)
+    keys1 = W.sorted_unique_sample(rng, 4 * k + 10, k)
+    keys2 = W.sorted_unique_sample(rng, 4 * k + 10, k)
+    cand = [rng.integers(0, n_docs, size=3000), rng.integers(0, n_docs, size=2500)]
+    wl = _manual([keys1, keys2], cand, authors, edge_dim=8)
+    fits_smem = k <= 29_000
+    _check(B, wl, _variants(B, include_smem=fits_smem))
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
+    if not fits_smem:
+        store = B.store_from_workload(wl)
+        db = B.DeviceBatch(wl.batch)
+        with pytest.raises(B.CcrError) as e:
+            gpu_join(store, db, B.CCR_FLAG_FORCE_SMEM)
+        assert e.value.status == B.CCR_ERR_UNSUPPORTED
+        store.free()
+
+
+def test_many_small_requests_in_one_launch(B):
+    # hundreds of requests of 0..40 candidates: most blocks serve many request segments
+    wl = tiny_workload(7, n_docs=3000, alphabet=900, n_req=700, kmax=300, nmax=40, second=False, req_dim=4,
+                       doc_dim=64, edge_dim=32)
+    _check(B, wl, _variants(B))
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
+
+
+def test_batch_equals_single_request_launches(B):
+    wl = W.config1(n_docs=50_000, n_req=6, n_cand=1500)
+    s, b = wl.store, wl.batch
+    store = B.store_from_workload(wl)
+    rows, mask = gpu_join(store, B.DeviceBatch(b))
+    for r in range(b.n_req):
+        e0, e1 = int(b.edge_offsets[r]), int(b.edge_offsets[r + 1])
+        c0, c1 = int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])
+        one = W.assemble_batch([b.edge_keys[e0:e1]], [b.edge_feats[e0:e1]], [b.cand_idx[c0:c1]],
+                               b.req_feats[r:r + 1], b.edge_dim, b.edge_dtype, b.req_dim, b.req_dtype)
+        r1, m1 = gpu_join(store, B.DeviceBatch(one))
+        assert np.array_equal(r1, rows[c0:c1]) and np.array_equal(m1, mask[c0:c1])
+    store.free()
+
+
+# ------------------------------------------------------------------ host-buffer entry, validation, errors
+def test_host_buffer_entry_matches_device_entry(B):
+    wl = W.config1(n_docs=80_000, n_req=9, n_cand=4000)
+    b = wl.batch
+    want_rows, want_mask = oracle.join_workload(wl)
+    store = B.store_from_workload(wl)
+    ws = B.Workspace(store, b.n_req, b.total_cands, len(b.edge_keys))
+    out_rows = torch.empty((b.total_cands, store.out_row_bytes()), dtype=torch.uint8).pin_memory()
+    out_mask = torch.empty((b.total_cands,), dtype=torch.uint8).pin_memory()
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    args = [pin(b.edge_keys), pin(b.edge_feats.view(np.uint8)), pin(b.edge_offsets), pin(b.cand_idx),
+            pin(b.cand_offsets), pin(b.req_feats.view(np.uint8))]
+    for _ in range(2):
+        out_rows.fill_(7)
+        B.ccr_join_batch_host(store, ws, b.n_req, b.total_cands, b.max_edge_len, len(b.edge_keys), *args,
+                              out_rows, out_mask)
+        torch.cuda.synchronize()
+        assert np.array_equal(out_rows.numpy(), want_rows) and np.array_equal(out_mask.numpy(), want_mask)
+    with pytest.raises(B.CcrError) as e:
+        B.ccr_join_batch_host(store, ws, b.n_req, b.total_cands + 1, b.max_edge_len, len(b.edge_keys), *args,
+                              out_rows, out_mask)
+    assert e.value.status == B.CCR_ERR_INVALID_ARG
+    ws.free()
+    store.free()
+
+
+def test_validate_flag_reports_broken_preconditions(B):
+    wl = W.config1(n_docs=20_000, n_req=4, n_cand=500)
+    store = B.store_from_workload(wl)
+    good = B.DeviceBatch(wl.batch)
+    gpu_join(store, good, B.CCR_FLAG_VALIDATE)
+
+    def expect_validation(batch, flags=0):
+        with pytest.raises(B.CcrError) as e:
+            gpu_join(store, B.DeviceBatch(batch), B.CCR_FLAG_VALIDATE | flags)
+        assert e.value.status == B.CCR_ERR_VALIDATION
+
+    b = wl.batch
+    keys = b.edge_keys.copy()
+    e0 = int(b.edge_offsets[2])
+    keys[e0], keys[e0 + 1] = keys[e0 + 1], keys[e0]  # one inversion inside request 2
+    expect_validation(W.Batch(**{**b.__dict__, "edge_keys": keys}))
+    keys = b.edge_keys.copy()
+    keys[e0 + 1] = keys[e0]  # duplicate key
+    expect_validation(W.Batch(**{**b.__dict__, "edge_keys": keys}))
+    co = b.cand_offsets.copy()
+    co[2], co[3] = co[3], co[2]  # non-monotone candidate offsets
+    expect_validation(W.Batch(**{**b.__dict__, "cand_offsets": co}))
+    # CANDS_SORTED on unsorted candidates is caught; on sorted ones it passes
+    expect_validation(b, B.CCR_FLAG_CANDS_SORTED)
+    gpu_join(store, B.DeviceBatch(W.sort_candidates_by_author(wl).batch), B.CCR_FLAG_VALIDATE | B.CCR_FLAG_CANDS_SORTED)
+    # the store stays usable after a rejected call
+    rows, mask = gpu_join(store, good)
+    want_rows, want_mask = oracle.join_workload(wl)
+    assert np.array_equal(rows, want_rows) and np.array_equal(mask, want_mask)
+    store.free()
+
+
+def test_unsorted_keys_and_false_sorted_promise_stay_in_bounds(B):
+    # values are unspecified here; the guard bytes and a clean device status are what is checked
+    wl = W.config1(n_docs=20_000, n_req=4, n_cand=3000)
+    b = wl.batch
+    rng = np.random.default_rng(0)
+    keys = b.edge_keys.copy()
+    rng.shuffle(keys)
+    store = B.store_from_workload(wl)
+    bad = B.DeviceBatch(W.Batch(**{**b.__dict__, "edge_keys": keys}))
+    for _, flags in _variants(B):
+        gpu_join(store, bad, flags)
+    gpu_join(store, B.DeviceBatch(b), B.CCR_FLAG_CANDS_SORTED)  # candidates are not sorted
+    gpu_join(store, bad, B.CCR_FLAG_CANDS_SORTED)
+    assert store.device_status() == B.CCR_OK
+    store.free()
+
+
+def test_argument_errors_on_a_live_store(B):
+    wl = W.config0(n_docs=5000, n_cand=1000, k=50)
+    store = B.store_from_workload(wl)
+    db = B.DeviceBatch(wl.batch)
+    L = B.lib()
+    out_rows = torch.empty((db.total_cands, 320), dtype=torch.uint8, device="cuda")
+    out_mask = torch.empty((db.total_cands,), dtype=torch.uint8, device="cuda")
+
+    def call(**kw):
+        a = dict(n_req=db.n_req, total=db.total_cands, maxk=db.max_edge_len, keys=db.edge_keys.data_ptr(),
+                 feats=db.edge_feats.data_ptr(), eo=db.edge_offsets.data_ptr(), ci=db.cand_idx.data_ptr(),
+                 co=db.cand_offsets.data_ptr(), rows=out_rows.data_ptr(), mask=out_mask.data_ptr(), flags=0)
+        a.update(kw)
+        return L.ccr_join_batch(store.handle, a["n_req"], a["total"], a["maxk"], a["keys"], a["feats"], a["eo"], a["ci"],
+                                a["co"], None, a["rows"], a["mask"], a["flags"], None)
+
+    assert call() == B.CCR_OK
+    assert call(n_req=-1) == B.CCR_ERR_INVALID_ARG
+    assert call(total=-5) == B.CCR_ERR_INVALID_ARG
+    assert call(rows=None) == B.CCR_ERR_INVALID_ARG
+    assert call(rows=out_rows.data_ptr() + 8) == B.CCR_ERR_INVALID_ARG  # misaligned
+    assert call(keys=db.edge_keys.data_ptr() + 8) == B.CCR_ERR_INVALID_ARG
+    assert call(flags=B.CCR_FLAG_FORCE_SMEM | B.CCR_FLAG_FORCE_GLOBAL) == B.CCR_ERR_INVALID_ARG
+    assert call(total=0) == B.CCR_OK and call(n_req=0, total=0) == B.CCR_OK
+    assert store.out_row_bytes() == 320
+    torch.cuda.synchronize()
+    h = ctypes.c_void_p(store.handle.value)
+    store.free()
+    assert L.ccr_docstore_free(h) == B.CCR_ERR_BAD_HANDLE  # double free
+
+
+def test_upload_in_pieces_from_device_memory(B):
+    wl = W.config0(n_docs=10_000, n_cand=3000, k=200, second_degree=True)
+    s = wl.store
+    store = B.Docstore(s.n_docs, s.doc_dim, s.doc_dtype, 32, np.float16, 0, np.float32, s.max_actors, s.reduce_sum_mask)
+    for a in range(0, s.n_docs, 3333):
+        z = min(s.n_docs, a + 3333)
+        dev = lambda x: torch.from_numpy(np.ascontiguousarray(x[a:z])).cuda()
+        store.upload(a, dev(s.doc_feats), dev(s.author_ids), dev(s.actor_ids), dev(s.actor_types))
+    torch.cuda.synchronize()
+    rows, mask = gpu_join(store, B.DeviceBatch(wl.batch))
+    want_rows, want_mask = oracle.join_workload(wl)
+    assert np.array_equal(rows, want_rows) and np.array_equal(mask, want_mask)
+    assert store.launch_count() == 1
+    store.free()
