@@ -1,0 +1,426 @@
+#!/usr/bin/env python
+"""Benchmark of the batched sorted-search join on B200: `python bench.py --gpus N --steps K --warmup W`.
+
+One step = one pass of the whole hot path (key staging, search, validate, edge/doc gather, request
+broadcast, row store) over one ragged batch of synthetic requests, i.e. one `ccr_join_batch` call.
+The default workload is the batched first-degree configuration (1M-doc store of 128 fp16 features, 64
+requests x 30,000 candidates, Zipf(1.2) edge lists clipped to 50..5000 with 32 fp16 features, 16 fp32
+request features).  Rank 0 prints ONE JSON line:
+
+  value      candidates joined per second, whole job, inputs resident in HBM (CUDA events, max over ranks)
+  e2e        the same through ccr_join_batch_host: pinned host inputs copied in, rows and mask copied out
+  roofline   compulsory bytes of one launch / average launch time, against the measured HBM copy peak
+  cpu_baseline  the CPU oracle as it stands, timed on this machine's host cores (rank 0, N = 1 only)
+
+With N > 1 (torchrun, one rank per GPU) every rank joins its own batch against its own replica of the
+store: the path has no exchange step, so there is no collective in the data path (weak scaling).
+`--impl reference` times the CPU oracle alone on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "candidates_joined_per_sec"
+UNIT = "candidates/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
+# summarised under profiles/ (bytes per launch; None until a capture of that workload exists)
+NCU_TRAFFIC_BYTES = {"config1": None, "config2b": None}
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=2000)
+    p.add_argument("--warmup", type=int, default=10)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--config", default="1", choices=["1", "2b"])
+    p.add_argument("--e2e-steps", type=int, default=0, help="0 = min(steps, 10)")
+    p.add_argument("--flags", type=int, default=0, help="extra CCR_FLAG_* bits (experiments)")
+    p.add_argument("--tile", type=int, default=0)
+    p.add_argument("--key-cap", type=int, default=0)
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    return p.parse_args()
+
+
+def make_workload(config: str, rank: int):
+    from paper_2609_22441_b200 import workloads as W
+
+    if config == "1":
+        return W.config1(seed=W.config_seed(1, 0) + 17 * rank)
+    return W.config1(seed=W.config_seed(2, 1) + 17 * rank, second_degree=True)
+
+
+def workload_label(wl) -> str:
+    b = wl.batch
+    return "%s: %d docs x %d %s, %d requests x %d candidates, edge lists %d..%d (mean %.0f) x %d fp16, %d fp32 request features" % (
+        wl.name, wl.store.n_docs, wl.store.doc_dim, wl.store.doc_dtype.name, b.n_req, b.total_cands // max(b.n_req, 1),
+        wl.meta["edge_len_min"], wl.meta["edge_len_max"], wl.meta["edge_len_mean"], b.edge_dim, b.req_dim)
+
+
+def byte_counts(wl, mask: np.ndarray, out_b: int, second: bool):
+    """Algorithmic bytes of one launch.  logical: every candidate pays for its own doc row, ids and matched
+    edge rows.  compulsory: doc rows / ids once per distinct doc of the launch and edge rows once per
+    distinct matched key of a request (what must cross HBM at least once); outputs are always per candidate."""
+    s, b = wl.store, wl.batch
+    doc_b, edge_b, req_b = s.doc_row_bytes, b.edge_row_bytes, b.req_row_bytes
+    C = b.total_cands
+    ids_b = 8 + (36 if second else 0)
+    per_req = int(8 * len(b.edge_keys) + (req_b + 16) * b.n_req)
+    found_slots = int((mask & 1).sum())
+    if second:
+        for sft in range(1, 5):
+            found_slots += int(((mask >> sft) & 1).sum())
+    logical = C * (4 + ids_b + doc_b + out_b + 1) + found_slots * edge_b + per_req
+    cand = b.cand_idx.astype(np.int64)
+    distinct_docs = int(len(np.unique(cand)))
+    matched_keys = 0
+    for r in range(b.n_req):
+        c0, c1 = int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])
+        hit = (mask[c0:c1] & 1).astype(bool)
+        ids = [s.author_ids[cand[c0:c1][hit]]]
+        if second:
+            for sft in range(4):
+                h = ((mask[c0:c1] >> (1 + sft)) & 1).astype(bool)
+                ids.append(s.actor_ids[cand[c0:c1][h], sft])
+        matched_keys += int(len(np.unique(np.concatenate(ids))))
+    compulsory = C * (4 + out_b + 1) + distinct_docs * (ids_b + doc_b) + matched_keys * edge_b + per_req
+    return {"logical": int(logical), "compulsory": int(compulsory), "distinct_docs": distinct_docs,
+            "match_rate": float((mask & 1).mean())}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples while the GPU is under load (one subprocess, 100 ms period)."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        sm, mx, reasons = [], [], set()
+        for t, line in self.samples:
+            if t < t0 or t > t1 + 0.15:
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measured_peak_gbs():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(wl, n_threads: int, repeats: int, max_cands: int = 0):
+    """Seconds per pass of the CPU oracle over the first `max_cands` candidates (0 = the whole batch)."""
+    from oracle import oracle
+    from paper_2609_22441_b200 import workloads as W
+
+    b = wl.batch
+    if max_cands and max_cands < b.total_cands:
+        co = np.minimum(b.cand_offsets, max_cands)
+        b = W.Batch(**{**b.__dict__, "cand_offsets": co, "cand_idx": b.cand_idx[:max_cands]})
+    s = wl.store
+    best = float("inf")
+    for _ in range(repeats):
+        t = time.perf_counter()
+        oracle.join(s.doc_feats, s.author_ids, b.edge_keys, b.edge_feats, b.edge_offsets, b.cand_idx, b.cand_offsets,
+                    req_feats=b.req_feats, actor_ids=s.actor_ids, actor_types=s.actor_types,
+                    reduce_sum_mask=s.reduce_sum_mask, n_threads=n_threads)
+        best = min(best, time.perf_counter() - t)
+    return best, int(b.total_cands)
+
+
+def run_reference(args, rank: int):
+    """The reference arm of this tier is the CPU oracle: rank 0 times it, the other ranks do nothing."""
+    if rank != 0:
+        return
+    from oracle import oracle
+
+    oracle.build()
+    wl = make_workload(args.config, 0)
+    cores = host_cores()
+    t_probe, n_probe = time_oracle(wl, cores, 1, max_cands=200_000)
+    rate = n_probe / t_probe
+    budget_s = 60.0
+    sample = int(min(wl.batch.total_cands, max(30_000, rate * budget_s / max(args.steps + args.warmup, 1))))
+    for _ in range(args.warmup):
+        time_oracle(wl, cores, 1, max_cands=sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time_oracle(wl, cores, 1, max_cands=sample)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    desc = "first %d of %d candidates of the batch per step" % (sample, wl.batch.total_cands)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": workload_label(wl), "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the join has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2609_22441_b200 import binding as B
+    from paper_2609_22441_b200 import build as lib_build
+
+    if rank == 0:
+        lib_build.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def sum_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
+    wl = make_workload(args.config, rank)
+    b = wl.batch
+    second = wl.store.max_actors > 0
+    store = B.store_from_workload(wl, device=local_rank)
+    if args.tile or args.key_cap:
+        store.set_tuning(args.tile, args.key_cap)
+    db = B.DeviceBatch(b, device=local_rank)
+    flags = args.flags
+    out_b = store.out_row_bytes(flags)
+    C = b.total_cands
+    n_buf = 2  # outputs rotate so that consecutive steps do not rewrite lines still in L2
+    outs = [(torch.empty((C, out_b), dtype=torch.uint8, device=dev), torch.empty((C,), dtype=torch.uint8, device=dev))
+            for _ in range(n_buf)]
+
+    def step(i: int):
+        rows, mask = outs[i % n_buf]
+        B.ccr_join_batch(store, db.n_req, C, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets, db.cand_idx,
+                         db.cand_offsets, db.req_feats, rows, mask, flags)
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    launches0 = store.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    barrier()
+    launches = store.launch_count() - launches0
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    # keep the same kernel running until the loaded window is long enough for clock samples
+    while time.time() - t_wall0 < 1.2:
+        for i in range(50):
+            step(i)
+        torch.cuda.synchronize(dev)
+    t_wall1 = time.time()
+    ms_per_step = ms_total / max(args.steps, 1)
+    total_cands_job = sum_over_ranks(float(C))
+    value = total_cands_job / (ms_per_step * 1e-3)
+    if store.device_status() != B.CCR_OK:
+        raise SystemExit("device status not clean after the timed region")
+
+    # ---- end to end: pinned host inputs in, rows + mask out, through ccr_join_batch_host
+    ws = B.Workspace(store, b.n_req, C, len(b.edge_keys))
+    pin = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h_in = [pin(b.edge_keys), pin(b.edge_feats.view(np.uint8)), pin(b.edge_offsets), pin(b.cand_idx), pin(b.cand_offsets),
+            pin(None if b.req_feats is None else b.req_feats.view(np.uint8))]
+    h_rows = torch.empty((C, out_b), dtype=torch.uint8).pin_memory()
+    h_mask = torch.empty((C,), dtype=torch.uint8).pin_memory()
+    h2d = int(sum(t.numel() * t.element_size() for t in h_in if t is not None))
+    d2h = int(h_rows.numel() + h_mask.numel())
+
+    def e2e_step():
+        B.ccr_join_batch_host(store, ws, b.n_req, C, b.max_edge_len, len(b.edge_keys), *h_in, h_rows, h_mask, flags)
+
+    e2e_steps = args.e2e_steps or max(1, min(args.steps, 10))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
+    e2e_value = total_cands_job / (e2e_ms * 1e-3)
+    mask_host = h_mask.numpy().copy()
+    ws.free()
+
+    # ---- per-request latency on this batch's requests (one request per launch, device-resident inputs)
+    lat = []
+    if rank == 0:
+        rows0, mask0 = outs[0]
+        evs = []
+        for rep in range(4):
+            for r in range(b.n_req):
+                e0, e1 = int(b.edge_offsets[r]), int(b.edge_offsets[r + 1])
+                c0, c1 = int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])
+                a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                one_eo = torch.tensor([0, e1 - e0], dtype=torch.int64, device=dev)
+                one_co = torch.tensor([0, c1 - c0], dtype=torch.int64, device=dev)
+                # 16-byte alignment of the key slice: start on an even key index
+                e0a = e0 - (e0 & 1)
+                one_eo[0] = e0 - e0a
+                one_eo[1] = e1 - e0a
+                if (db.edge_feats[e0a:].data_ptr() % 16) or (db.req_feats is not None and db.req_feats[r:].data_ptr() % 16):
+                    continue
+                torch.cuda.synchronize(dev)
+                a.record()
+                B.ccr_join_batch(store, 1, c1 - c0, e1 - e0a, db.edge_keys[e0a:], db.edge_feats[e0a:], one_eo,
+                                 db.cand_idx[c0:], one_co, None if db.req_feats is None else db.req_feats[r:],
+                                 rows0, mask0, flags)
+                z.record()
+                evs.append((a, z))
+        torch.cuda.synchronize(dev)
+        lat = sorted(a.elapsed_time(z) for a, z in evs[len(evs) // 4:])
+
+    def pct(v, q):
+        return None if not v else float(v[max(0, int(np.ceil(q * len(v))) - 1)])
+
+    if sampler is not None:
+        sampler.stop()
+
+    line = None
+    if rank == 0:
+        peak, peak_kind = measured_peak_gbs()
+        bc = byte_counts(wl, mask_host, out_b, second and not (flags & B.CCR_FLAG_FIRST_DEGREE_ONLY))
+        launch_s = ms_per_step * 1e-3  # one kernel launch per step
+        achieved = bc["compulsory"] / launch_s / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8", "data": "synthetic",
+            "config": {"workload": workload_label(wl), "l2": "inputs and outputs of a step (%.2f GB) exceed the 126 MB L2; "
+                       "outputs rotate over %d buffers" % (bc["compulsory"] / 1e9, n_buf),
+                       "match_rate": bc["match_rate"], "seed": wl.seed, "tile": args.tile or 1024, "key_cap": args.key_cap or 4096,
+                       "flags": flags, "replicas": world},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_kind": "of " + peak_kind,
+                         "bytes_per_launch": bc["compulsory"], "logical_bytes_per_launch": bc["logical"],
+                         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                         "logical_gbs": bc["logical"] / launch_s / 1e9},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "latency_ms": {"what": "one request (%d candidates) per launch, CUDA events" % (C // max(b.n_req, 1)),
+                           "p50": pct(lat, 0.50), "p99": pct(lat, 0.99), "n": len(lat)},
+            "clocks": sampler.summary(t_wall0, t_wall1) if sampler is not None else None,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            from oracle import oracle
+
+            oracle.build()
+            cores = host_cores()
+            t_mt, n_mt = time_oracle(wl, cores, 3)
+            t_st, n_st = time_oracle(wl, 1, 1, max_cands=600_000)
+            line["cpu_baseline"] = {"value": n_mt / t_mt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": "the whole batch (%d candidates), best of 3 passes" % n_mt,
+                                    "single_thread_value": n_st / t_st,
+                                    "gbs_compulsory": bc["compulsory"] / t_mt / 1e9}
+        else:
+            line["cpu_baseline"] = None
+    store.free()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()
