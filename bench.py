@@ -51,9 +51,13 @@ def parse_args():
     p.add_argument("--config", default="1", choices=["1", "2b"])
     p.add_argument("--e2e-steps", type=int, default=0, help="0 = min(steps, 10)")
     p.add_argument("--flags", type=int, default=0, help="extra CCR_FLAG_* bits (experiments)")
-    p.add_argument("--tile", type=int, default=0)
-    p.add_argument("--key-cap", type=int, default=0)
+    p.add_argument("--tile", type=int, default=0, help="candidates per ring slot (0 = library default)")
+    p.add_argument("--key-cap", type=int, default=0, help="keys staged per request (0 = library default)")
+    p.add_argument("--streamers", type=int, default=0)
+    p.add_argument("--resolvers", type=int, default=0)
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--timed-only", action="store_true",
+                   help="only warm-up and the timed region (for profiler captures): no sustain loop, e2e, latency or CPU legs")
     return p.parse_args()
 
 
@@ -273,8 +277,9 @@ def main():
     b = wl.batch
     second = wl.store.max_actors > 0
     store = B.store_from_workload(wl, device=local_rank)
-    if args.tile or args.key_cap:
-        store.set_tuning(args.tile, args.key_cap)
+    if args.tile or args.key_cap or args.streamers or args.resolvers:
+        store.set_tuning(tile_cands=args.tile, key_capacity=args.key_cap, ws_streamers=args.streamers,
+                         ws_resolvers=args.resolvers)
     db = B.DeviceBatch(b, device=local_rank)
     flags = args.flags
     out_b = store.out_row_bytes(flags)
@@ -303,7 +308,7 @@ def main():
     launches = store.launch_count() - launches0
     ms_total = max_over_ranks(ev0.elapsed_time(ev1))
     # keep the same kernel running until the loaded window is long enough for clock samples
-    while time.time() - t_wall0 < 1.2:
+    while not args.timed_only and time.time() - t_wall0 < 1.2:
         for i in range(50):
             step(i)
         torch.cuda.synchronize(dev)
@@ -328,7 +333,9 @@ def main():
         B.ccr_join_batch_host(store, ws, b.n_req, C, b.max_edge_len, len(b.edge_keys), *h_in, h_rows, h_mask, flags)
 
     e2e_steps = args.e2e_steps or max(1, min(args.steps, 10))
-    for _ in range(3):
+    if args.timed_only:
+        e2e_steps = 1
+    for _ in range(0 if args.timed_only else 3):
         e2e_step()
     barrier()
     ev0.record()
@@ -343,7 +350,7 @@ def main():
 
     # ---- per-request latency on this batch's requests (one request per launch, device-resident inputs)
     lat = []
-    if rank == 0:
+    if rank == 0 and not args.timed_only:
         rows0, mask0 = outs[0]
         evs = []
         for rep in range(4):
@@ -387,7 +394,7 @@ def main():
             "dtype": "u8", "data": "synthetic",
             "config": {"workload": workload_label(wl), "l2": "inputs and outputs of a step (%.2f GB) exceed the 126 MB L2; "
                        "outputs rotate over %d buffers" % (bc["compulsory"] / 1e9, n_buf),
-                       "match_rate": bc["match_rate"], "seed": wl.seed, "tile": args.tile or 1024, "key_cap": args.key_cap or 4096,
+                       "match_rate": bc["match_rate"], "seed": wl.seed, "tile": args.tile or "default", "key_cap": args.key_cap or "default",
                        "flags": flags, "replicas": world},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_kind": "of " + peak_kind,
@@ -401,7 +408,7 @@ def main():
                            "p50": pct(lat, 0.50), "p99": pct(lat, 0.99), "n": len(lat)},
             "clocks": sampler.summary(t_wall0, t_wall1) if sampler is not None else None,
         }
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and not args.timed_only:
             from oracle import oracle
 
             oracle.build()

@@ -70,8 +70,12 @@ enum {
                                            device first; synchronises the stream                     */
   CCR_FLAG_FIRST_DEGREE_ONLY = 1u << 4, /* ignore engager slots of a second-degree store: no edge2
                                            section, mask is 0/1                                      */
-  CCR_FLAG_FORCE_SAMPLED     = 1u << 5  /* stage only every s-th key (a sampled top of the search
+  CCR_FLAG_FORCE_SAMPLED     = 1u << 5, /* stage only every s-th key (a sampled top of the search
                                            tree) even when the list would fit; testing aid          */
+  CCR_FLAG_STATIC_SPLIT      = 1u << 6, /* warp-specialised kernel: give every block one equal contiguous
+                                           slice instead of drawing chunks from a device-side counter */
+  CCR_FLAG_TWO_PHASE         = 1u << 7  /* use the two-phase kernel (every warp alternates search and
+                                           row streaming) instead of the warp-specialised kernel      */
 };
 
 /* Create an empty store on desc->device.  Allocates doc_feats [n_docs, doc_dim], author_ids
@@ -161,9 +165,16 @@ ccr_status ccr_join_batch_host(const ccr_docstore* store, ccr_workspace* ws,
  * last call (the affected rows of that launch were not written).  Clears the word.                 */
 ccr_status ccr_docstore_device_status(ccr_docstore* store, void* stream);
 
-/* Tuning knobs of the join kernels (0 keeps the current value): candidates per thread block, and
- * the largest number of keys (or sampled keys) a block stages in shared memory per request.        */
-ccr_status ccr_docstore_set_tuning(ccr_docstore* store, int32_t tile_cands, int32_t key_capacity);
+/* Tuning knobs of the join kernels; a field that is 0 keeps the store's current value.              */
+typedef struct {
+  int32_t tile_cands;         /* candidates per ring slot / search-copy phase pair: multiple of 256, <= 4096 */
+  int32_t key_capacity;       /* most keys (or sampled keys) a block stages in shared memory per request;
+                                 unset = as many as fit (warp-specialised kernel) or 4096 (the others)       */
+  int32_t ws_streamers;       /* warp-specialised kernel: row-streaming warps per block (1..14)              */
+  int32_t ws_resolvers;       /* warp-specialised kernel: search warps per block (1..8); sum <= 16           */
+  int32_t blocks_per_sm;      /* two-phase kernel: cap on resident blocks per SM (1..8)                      */
+} ccr_tuning;
+ccr_status ccr_docstore_set_tuning(ccr_docstore* store, const ccr_tuning* tuning);
 
 /* Number of kernels the library has launched on behalf of this store since creation.               */
 int64_t ccr_docstore_launch_count(const ccr_docstore* store);

@@ -14,7 +14,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libccr.so")
+LIB_PATH = os.environ.get("CCR_LIB_OVERRIDE") or os.path.join(_HERE, "libccr.so")
 
 CCR_OK = 0
 CCR_ERR_INVALID_ARG = 1
@@ -34,6 +34,8 @@ CCR_FLAG_CANDS_SORTED = 1 << 2
 CCR_FLAG_VALIDATE = 1 << 3
 CCR_FLAG_FIRST_DEGREE_ONLY = 1 << 4
 CCR_FLAG_FORCE_SAMPLED = 1 << 5
+CCR_FLAG_STATIC_SPLIT = 1 << 6
+CCR_FLAG_TWO_PHASE = 1 << 7
 
 EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
@@ -51,6 +53,11 @@ class ccr_docstore_desc(ctypes.Structure):
         ("max_actors", ctypes.c_int32), ("device", ctypes.c_int32),
         ("reduce_sum_mask", ctypes.c_uint64),
     ]
+
+
+class ccr_tuning(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "tile_cands", "key_capacity", "ws_streamers", "ws_resolvers", "blocks_per_sm")]
 
 
 class CcrError(RuntimeError):
@@ -93,7 +100,7 @@ def lib() -> ctypes.CDLL:
     L.ccr_docstore_device_status.restype = ctypes.c_int
     L.ccr_docstore_device_status.argtypes = [vp, vp]
     L.ccr_docstore_set_tuning.restype = ctypes.c_int
-    L.ccr_docstore_set_tuning.argtypes = [vp, i32, i32]
+    L.ccr_docstore_set_tuning.argtypes = [vp, ctypes.POINTER(ccr_tuning)]
     L.ccr_docstore_launch_count.restype = i64
     L.ccr_docstore_launch_count.argtypes = [vp]
     L.ccr_status_str.restype = ctypes.c_char_p
@@ -176,8 +183,10 @@ class Docstore:
     def out_row_bytes(self, flags: int = 0) -> int:
         return int(lib().ccr_out_row_bytes(self._h, int(flags)))
 
-    def set_tuning(self, tile_cands: int = 0, key_capacity: int = 0) -> None:
-        _check(lib().ccr_docstore_set_tuning(self._h, int(tile_cands), int(key_capacity)), "ccr_docstore_set_tuning")
+    def set_tuning(self, tile_cands: int = 0, key_capacity: int = 0, ws_streamers: int = 0, ws_resolvers: int = 0,
+                   blocks_per_sm: int = 0) -> None:
+        t = ccr_tuning(int(tile_cands), int(key_capacity), int(ws_streamers), int(ws_resolvers), int(blocks_per_sm))
+        _check(lib().ccr_docstore_set_tuning(self._h, ctypes.byref(t)), "ccr_docstore_set_tuning")
 
     def launch_count(self) -> int:
         return int(lib().ccr_docstore_launch_count(self._h))

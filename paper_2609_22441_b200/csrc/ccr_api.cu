@@ -11,16 +11,19 @@
 #include <new>
 
 #include "ccr_join.cuh"
-#include "ccr_merge.cuh"
+#include "ccr_ws.cuh"
 
 namespace {
 
 constexpr uint64_t kStoreMagic = 0x43435253544f5245ull;  // "CCRSTORE"
 constexpr uint64_t kWsMagic = 0x4343525753504143ull;     // "CCRWSPAC"
 constexpr int kMaxSmemBytes = 227 * 1024;
-constexpr int kDefaultTile = 1024;
+constexpr int kDefaultTile = 512;
+constexpr int kSmemPerSm = 228 * 1024;
 constexpr int kDefaultKeyCap = 4096;
 constexpr int kMaxTile = 4096;
+constexpr int kSchedRegions = 64;                    // launches of one store that may be in flight at once
+constexpr int kStatusInts = 4 + 2 * kSchedRegions;   // [0] wait expiry, [1] validation code, [4..] scheduling words
 
 inline size_t dtype_size(int32_t dt) { return dt == CCR_F16 ? 2 : (dt == CCR_F32 ? 4 : 0); }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -53,6 +56,9 @@ struct ccr_docstore {
   int* status_host;   // pinned host copy
   int tile;
   int key_cap;
+  int blocks_per_sm;  // cap on resident blocks per SM of the two-phase kernel (0 = as many as fit)
+  int ws_streamers, ws_resolvers;  // warp split of the warp-specialised kernel
+  int n_sms;
   int64_t launches;
 };
 
@@ -114,15 +120,19 @@ __global__ void validate_kernel(const ccr::JoinArgs a, int check_sorted, int* co
 // use (256-byte doc rows; 64- or 128-byte edge rows; 0 or 64 bytes of request features), and a generic
 // variant with run-time widths for everything else.
 using KernelFn = void (*)(const ccr::JoinArgs);
+using WsKernelFn = void (*)(const ccr::JoinArgs, int);
 
 struct Variant {
   int doc_ch, edge_ch, req_ch;
   KernelFn first, second, merge;
+  WsKernelFn ws_first, ws_second;
 };
 
-#define CCR_VARIANT(D, E, R)                                                                        \
-  Variant {                                                                                         \
-    D, E, R, ccr::join_kernel<D, E, R, false>, ccr::join_kernel<D, E, R, true>, ccr::join_merge_kernel<D, E, R> \
+#define CCR_VARIANT(D, E, R)                                                                                      \
+  Variant {                                                                                                       \
+    D, E, R, ccr::join_kernel<D, E, R, false, false>, ccr::join_kernel<D, E, R, true, false>,                     \
+        ccr::join_kernel<D, E, R, false, true>,                                                                   \
+        ccr::join_ws_kernel<D, E, R, false>, ccr::join_ws_kernel<D, E, R, true>                                   \
   }
 
 const Variant kVariants[] = {
@@ -146,6 +156,13 @@ ccr_status allow_large_smem() {
   for (int i = 0; i < kNumVariants; ++i) {
     const KernelFn fns[3] = {kVariants[i].first, kVariants[i].second, kVariants[i].merge};
     for (KernelFn f : fns) {
+      if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemBytes) != cudaSuccess) {
+        cudaGetLastError();
+        return CCR_ERR_CUDA;
+      }
+    }
+    const WsKernelFn ws[2] = {kVariants[i].ws_first, kVariants[i].ws_second};
+    for (WsKernelFn f : ws) {
       if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemBytes) != cudaSuccess) {
         cudaGetLastError();
         return CCR_ERR_CUDA;
@@ -217,7 +234,14 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   s->edge_b = static_cast<int>(edge_b);
   s->req_b = static_cast<int>(req_b);
   s->tile = kDefaultTile;
-  s->key_cap = kDefaultKeyCap;
+  s->key_cap = 0;  // automatic
+  s->ws_streamers = 12;
+  s->ws_resolvers = 4;
+  if (cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, d->device) != cudaSuccess || s->n_sms <= 0) {
+    cudaGetLastError();
+    delete s;
+    return CCR_ERR_CUDA;
+  }
   bool ok = true;
   // n == 0 still allocates a token block so that every pointer is valid and aligned
   ok = ok && cudaMalloc(&s->doc_feats, n * doc_b + 256) == cudaSuccess;
@@ -226,8 +250,8 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
     ok = ok && cudaMalloc(&s->actor_ids, n * d->max_actors * 8 + 256) == cudaSuccess;
     ok = ok && cudaMalloc(&s->actor_types, n * d->max_actors + 256) == cudaSuccess;
   }
-  ok = ok && cudaMalloc(&s->status, 4 * sizeof(int)) == cudaSuccess;
-  ok = ok && cudaMemset(s->status, 0, 4 * sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->status, kStatusInts * sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemset(s->status, 0, kStatusInts * sizeof(int)) == cudaSuccess;
   ok = ok && cudaHostAlloc(&s->status_host, 4 * sizeof(int), cudaHostAllocDefault) == cudaSuccess;
   ccr_status st = ok ? allow_large_smem() : CCR_ERR_OOM;
   if (st != CCR_OK) {
@@ -286,17 +310,24 @@ ccr_status ccr_docstore_upload(ccr_docstore* s, int64_t first_doc, int64_t n, co
 
 size_t ccr_out_row_bytes(const ccr_docstore* s, uint32_t flags) { return good(s) ? out_row_bytes(s, flags) : 0; }
 
-ccr_status ccr_docstore_set_tuning(ccr_docstore* s, int32_t tile_cands, int32_t key_capacity) {
+ccr_status ccr_docstore_set_tuning(ccr_docstore* s, const ccr_tuning* t) {
   if (!good(s)) return CCR_ERR_BAD_HANDLE;
-  if (tile_cands < 0 || key_capacity < 0) return CCR_ERR_INVALID_ARG;
-  if (tile_cands > 0) {
-    if (tile_cands % 32 || tile_cands > kMaxTile) return CCR_ERR_INVALID_ARG;
-    s->tile = tile_cands;
-  }
-  if (key_capacity > 0) {
-    if (static_cast<size_t>(key_capacity + 2) * 8 + ccr::kSmemHeader > static_cast<size_t>(kMaxSmemBytes)) return CCR_ERR_INVALID_ARG;
-    s->key_cap = key_capacity;
-  }
+  if (t == nullptr) return CCR_ERR_INVALID_ARG;
+  if (t->tile_cands < 0 || t->key_capacity < 0 || t->ws_streamers < 0 || t->ws_resolvers < 0 || t->blocks_per_sm < 0)
+    return CCR_ERR_INVALID_ARG;
+  if (t->tile_cands % 256 || t->tile_cands > kMaxTile) return CCR_ERR_INVALID_ARG;
+  if (t->key_capacity > 0 &&
+      static_cast<size_t>(ccr::search_bytes(t->key_capacity, true)) + ccr::kSmemHeader > static_cast<size_t>(kMaxSmemBytes))
+    return CCR_ERR_INVALID_ARG;
+  const int st = t->ws_streamers > 0 ? t->ws_streamers : s->ws_streamers;
+  const int rs = t->ws_resolvers > 0 ? t->ws_resolvers : s->ws_resolvers;
+  if (st > 14 || rs > 8 || (st + rs) * 32 > ccr::kWsMaxThreads) return CCR_ERR_INVALID_ARG;
+  if (t->blocks_per_sm > 8) return CCR_ERR_INVALID_ARG;
+  if (t->tile_cands > 0) s->tile = t->tile_cands;
+  if (t->key_capacity > 0) s->key_cap = t->key_capacity;
+  s->ws_streamers = st;
+  s->ws_resolvers = rs;
+  if (t->blocks_per_sm > 0) s->blocks_per_sm = t->blocks_per_sm;
   return CCR_OK;
 }
 
@@ -342,12 +373,37 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
   // on sorted candidates takes the binary-search kernel (same result by definition)
   const bool merge = (flags & CCR_FLAG_CANDS_SORTED) && !second;
 
+  // which kernel: the merge path and CCR_FLAG_TWO_PHASE take the two-phase kernel, everything else the
+  // warp-specialised kernel
+  const bool use_ws = !merge && !(flags & CCR_FLAG_TWO_PHASE);
+  auto smem_for = [&](int t, int cap) -> size_t {
+    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, cap).bytes)
+                  : static_cast<size_t>(ccr::TileLayout(t, second, merge, cap).bytes);
+  };
+  // Keys staged per request.  The warp-specialised kernel runs one block per SM, so by default it stages
+  // as many keys as fit next to its ring (whole lists of up to ~20,000 ids); the kernels that keep several
+  // blocks per SM default to kDefaultKeyCap.  A configured key_capacity overrides both.
+  int tile = s->tile;
   int key_cap;
-  if (flags & CCR_FLAG_FORCE_GLOBAL) key_cap = 0;
-  else if (flags & CCR_FLAG_FORCE_SMEM) key_cap = static_cast<int>(max_edge_len);
-  else key_cap = static_cast<int>(max_edge_len < s->key_cap ? max_edge_len : s->key_cap);
-  size_t smem = ccr::kSmemHeader + static_cast<size_t>(key_cap + 2) * 8;
-  if (merge) smem += static_cast<size_t>(s->tile) * 8 + static_cast<size_t>((s->tile + 3) & ~3) * 4;
+  if (flags & CCR_FLAG_FORCE_GLOBAL) {
+    key_cap = 0;
+  } else if (flags & CCR_FLAG_FORCE_SMEM) {
+    key_cap = static_cast<int>(max_edge_len);
+  } else if (s->key_cap > 0 || !use_ws) {
+    const long long cap = s->key_cap > 0 ? s->key_cap : kDefaultKeyCap;
+    key_cap = static_cast<int>(max_edge_len < cap ? max_edge_len : cap);
+  } else {
+    key_cap = static_cast<int>(max_edge_len);
+    // shrink the ring first; if the longest list still does not fit, stage a sampled top of the tree
+    while (tile > 256 && smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) tile -= 256;
+    if (smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) {
+      tile = s->tile;
+      key_cap = kDefaultKeyCap;
+    }
+  }
+  // sub-tile size: the configured one, shrunk (in steps of 256) until the kernel's arrays fit next to the keys
+  while (tile > 256 && smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) tile -= 256;
+  const size_t smem = smem_for(tile, key_cap);
   if (smem > static_cast<size_t>(kMaxSmemBytes)) return CCR_ERR_UNSUPPORTED;
 
   ccr::JoinArgs a;
@@ -372,10 +428,11 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
   a.req_feats = static_cast<const uint8_t*>(req_feats);
   a.out_rows = static_cast<uint8_t*>(out_rows);
   a.out_mask = out_mask;
-  a.tile = s->tile;
+  a.tile = tile;
   a.key_cap = key_cap;
   a.min_stride_log2 = (flags & CCR_FLAG_FORCE_SAMPLED) ? 2 : 0;
   a.status = s->status;
+  a.sched = nullptr;
 
   DeviceScope scope(s->desc.device);
   if (!scope.ok) return CCR_ERR_CUDA;
@@ -395,10 +452,29 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
   }
 
   const Variant& v = pick_variant(a.doc_ch, a.edge_ch, a.req_ch);
-  const KernelFn fn = merge ? v.merge : (second ? v.second : v.first);
-  const long long blocks = (total_cands + a.tile - 1) / a.tile;
-  if (blocks > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;
-  fn<<<static_cast<unsigned>(blocks), ccr::kThreads, smem, st>>>(a);
+  const long long groups = (total_cands + 31) / 32;
+  if (use_ws) {
+    // one persistent warp-specialised block per SM (fewer when there are fewer 32-row groups than SMs)
+    long long blocks = s->n_sms;
+    if (blocks > groups) blocks = groups;
+    const WsKernelFn fn = second ? v.ws_second : v.ws_first;
+    // dynamic chunk scheduling through a pair of device words; each launch takes the next pair in turn, so
+    // up to kSchedRegions launches of one store may be in flight at once (on any streams)
+    if (!(flags & CCR_FLAG_STATIC_SPLIT)) a.sched = s->status + 4 + 2 * static_cast<int>(s->launches % kSchedRegions);
+    fn<<<static_cast<unsigned>(blocks), (s->ws_streamers + s->ws_resolvers) * 32, smem, st>>>(a, s->ws_streamers);
+  } else {
+    // persistent two-phase kernel: as many blocks as stay resident, each with at least 256 candidates
+    const KernelFn fn = merge ? v.merge : (second ? v.second : v.first);
+    const int by_regs = ccr::kJoinMinBlocks;  // matches the kernel's __launch_bounds__
+    int per_sm = static_cast<int>(kSmemPerSm / (smem + 1024));
+    if (per_sm > by_regs) per_sm = by_regs;
+    if (s->blocks_per_sm > 0 && per_sm > s->blocks_per_sm) per_sm = s->blocks_per_sm;
+    if (per_sm < 1) per_sm = 1;
+    long long blocks = static_cast<long long>(s->n_sms) * per_sm;
+    const long long most = (groups + ccr::kWarps - 1) / ccr::kWarps;
+    if (blocks > most) blocks = most;
+    fn<<<static_cast<unsigned>(blocks), ccr::kThreads, smem, st>>>(a);
+  }
   s->launches++;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
   return CCR_OK;

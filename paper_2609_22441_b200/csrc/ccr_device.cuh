@@ -47,6 +47,7 @@ struct JoinArgs {
   int key_cap;                // keys (or sampled keys) a block may stage per request; 0 = search global memory
   int min_stride_log2;        // >0 forces sampling with at least this stride (testing aid)
   int* status;                // device status words
+  int* sched;                 // two scheduling words (next tile, finished blocks), zero between launches; or null
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -2,116 +2,90 @@
 // document-row gather from the resident index (Section 6.3.1) and the request-feature broadcast
 // (Section 3), for a ragged batch of requests in one launch.
 //
-// Work split.  The flat candidate range [0, total) is cut into tiles of `tile` candidates, one thread
-// block each, so the grid is known on the host without reading the offsets.  A block walks the request
-// segments that intersect its tile (usually one); per segment it stages that request's sorted keys in
-// shared memory and its warps take groups of 32 consecutive candidates:
-//   lane-per-candidate : position -> author id (8-B gather) -> branch-free lower bound in the staged keys
-//   warp-cooperative   : rows are moved as 16-byte chunks, consecutive lanes on consecutive chunks of
-//                        the same row, the owning lane's position / match broadcast with __shfl_sync;
-//                        every output byte is written exactly once with full-sector streaming stores.
-// Key staging.  K <= key_cap: the whole list, by one 1-D TMA bulk copy (plus at most one scalar key at
-// either end when the request's first key is only 8-byte aligned).  K > key_cap: every 2^s-th key is
-// staged as the top of the search tree and the last <= 2^s keys of a search are read from global
-// memory (one 128-byte line at s = 4, L2 resident).  key_cap == 0: the whole search runs on global memory.
+// Work split.  The kernel is persistent: the grid is a multiple of the SM count, every block owns one
+// contiguous slice of the flat candidate range and walks the request segments inside it, so a request's
+// keys are staged once per block.  Inside a segment the block alternates two phases over sub-tiles of
+// `tile` candidates:
+//   phase A, lane-per-candidate : position -> author id (8-byte gather) -> branch-free lower bound in the
+//            staged keys -> (position, match index) into shared memory, mask byte to global memory.
+//            Several candidates per thread are in flight at once, so the dependent chain
+//            position -> id -> search is paid once per sub-tile, not once per row group.
+//   phase B, warp-cooperative   : pure streaming.  Rows move as 16-byte chunks, consecutive lanes on
+//            consecutive chunks of a row (the row's position / match index is a shared-memory broadcast);
+//            all loads of a 32-row group are issued before its stores; every output byte is written
+//            exactly once with full-sector streaming stores.
+// Several blocks are resident per SM, so one block's phase A overlaps other blocks' phase B.
+//
+// Key staging and the search itself are in ccr_search.cuh (TMA bulk copy of the request's keys, bucket
+// index, sampled top-of-tree for lists longer than the staging budget, global-memory search).
+//
+// Merge-path mode (MERGE = true; not in the paper) serves candidates whose author ids are non-decreasing
+// inside each request: phase A gathers the sub-tile's author ids, finds with a block-cooperative k-ary
+// search the window of keys the sub-tile can touch, stages only that window, and merges the two sorted
+// runs along merge-path diagonals (O(n + w) comparisons instead of O(n log K)); phase B is unchanged.
 #pragma once
 
 #include "ccr_device.cuh"
+#include "ccr_search.cuh"
 
 namespace ccr {
 
-// Keys of the request a block is currently serving.
-struct StagedKeys {
-  const int64_t* sk;  // shared-memory copy (index i = key i when s_log == 0, sample i otherwise)
-  const int64_t* gk;  // the request's keys in global memory
-  int K;              // keys in the request
-  int M;              // staged entries (0 = nothing staged)
-  int s_log;          // log2 of the sampling stride
+constexpr long long kNoAuthor = static_cast<long long>(0x8000000000000000ull);  // below every key (keys are >= 0)
 
-  // Algorithm 1 steps 2-3 for one id: pos = lower bound, found = pos < K and keys[pos] == id.
-  __device__ __forceinline__ bool find(int64_t id, int& pos) const {
-    if (K == 0) {
-      pos = 0;
-      return false;
-    }
-    if (M > 0 && s_log == 0) {
-      pos = lower_bound_smem(sk, M, id);
-      return pos < K && sk[pos] == id;
-    }
-    int lo = 0, n = K;
-    if (M > 0) {
-      // sample i is key (i+1)*2^s - 1: c samples below id means blocks 0..c-1 are entirely below it
-      const int c = lower_bound_smem(sk, M, id);
-      lo = c << s_log;
-      n = min(1 << s_log, K - lo);
-    }
-    pos = lo + lower_bound_global(gk + lo, n, id);
-    return pos < K && __ldg(gk + pos) == id;
-  }
-};
-
-// Stage request keys [kb, kb+K) for the whole block.  Returns false if the bounded wait for the bulk
-// copy expired (block-uniform).  Ends with a __syncthreads.
-__device__ __forceinline__ bool stage_keys(const JoinArgs& a, int64_t* skeys, uint32_t bar, uint32_t& phase,
-                                           long long kb, int K, StagedKeys& st) {
-  const int tid = threadIdx.x;
-  st.gk = a.edge_keys + kb;
-  st.K = K;
-  st.M = 0;
-  st.s_log = 0;
-  st.sk = skeys;
-  int expired = 0;
-  if (a.key_cap > 0 && K > 0) {
-    if (K <= a.key_cap && a.min_stride_log2 == 0) {
-      // slot of key i is i + shift, so that 16-byte aligned global addresses land on 16-byte aligned slots
-      const int shift = static_cast<int>(kb & 1);
-      const int i0 = shift;                       // first key whose address is 16-byte aligned
-      const int nb = (K - i0) & ~1;               // keys moved by the bulk copy (even count)
-      st.sk = skeys + shift;
-      st.M = K;
-      if (tid == 0 && nb > 0) {
-        mbar_arrive_expect_tx(bar, static_cast<uint32_t>(nb) * 8u);
-        bulk_copy_g2s(smem_u32(skeys + i0 + shift), a.edge_keys + kb + i0, static_cast<uint32_t>(nb) * 8u, bar);
-      }
-      if (tid == 32 && shift) skeys[shift] = __ldg(a.edge_keys + kb);
-      if (tid == 64 && ((K - i0) & 1)) skeys[K - 1 + shift] = __ldg(a.edge_keys + kb + K - 1);
-      if (nb > 0) {
-        expired = mbar_wait_bounded(bar, phase) ? 0 : 1;
-        phase ^= 1u;
-      }
-    } else {
-      int s_log = a.min_stride_log2;
-      while ((K >> s_log) > a.key_cap) ++s_log;
-      st.s_log = s_log;
-      st.M = K >> s_log;
-      for (int i = tid; i < st.M; i += kThreads)
-        skeys[i] = __ldg(a.edge_keys + kb + ((static_cast<long long>(i) + 1) << s_log) - 1);
-    }
-  }
-  return __syncthreads_or(expired) == 0;
-}
-
-// Copy one section of the 32 rows of a warp's group: `ch` 16-byte chunks per row, source row given by
-// `src(row)` (nullptr = zeros), destination out + row*out_b.  Uniform trip count: safe for shuffles in src.
-template <typename SrcFn>
-__device__ __forceinline__ void copy_chunk(int i, int ch, int lane, int cnt, uint8_t* out, long long out_b, SrcFn& src) {
-  const int c = i * 32 + lane;
-  const int row = c / ch;
-  const int piece = c - row * ch;
-  const uint8_t* s = src(row);
-  uint4 v = make_uint4(0u, 0u, 0u, 0u);
-  if (s != nullptr) v = ldg128(s + piece * 16);
-  if (row < cnt) st128_stream(out + row * out_b + piece * 16, v);
-}
-
-template <int CH, typename SrcFn>
-__device__ __forceinline__ void copy_section(int ch_rt, int lane, int cnt, uint8_t* out, long long out_b, SrcFn src) {
-  if constexpr (CH > 0) {
+// One 16-byte chunk (8 fp16 dims, starting at dim piece*8) of the edge2 section of one candidate: the
+// matched edge rows of its found engager slots (rp[s] >= 0 is the row index, < 0 = slot not found)
+// reduced per dim in ascending slot order.  max: strict > on the fp32 values, the winner's 16 bits are
+// kept.  sum: fp32 accumulator from +0, one rounded add per slot, one round-to-nearest-even conversion;
+// a NaN sum is stored as 0x7fff.
+__device__ __forceinline__ uint4 edge2_chunk(unsigned long long reduce_sum_mask, const uint8_t* edge_base, int edge_b,
+                                             int piece, const int (&rp)[4]) {
+  uint4 q[4];
 #pragma unroll
-    for (int i = 0; i < CH; ++i) copy_chunk(i, CH, lane, cnt, out, out_b, src);
-  } else {
-    for (int i = 0; i < ch_rt; ++i) copy_chunk(i, ch_rt, lane, cnt, out, out_b, src);
+  for (int s = 0; s < 4; ++s) {
+    q[s] = make_uint4(0u, 0u, 0u, 0u);
+    if (rp[s] >= 0) q[s] = ldg128(edge_base + static_cast<long long>(rp[s]) * edge_b + piece * 16);
   }
+  float acc[8], bestf[8];
+  unsigned short best[8];
+#pragma unroll
+  for (int h = 0; h < 8; ++h) {
+    acc[h] = 0.0f;
+    bestf[h] = 0.0f;
+    best[h] = 0;
+  }
+  bool any = false;
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    if (rp[s] >= 0) {
+      const unsigned w[4] = {q[s].x, q[s].y, q[s].z, q[s].w};
+#pragma unroll
+      for (int h = 0; h < 8; ++h) {
+        const unsigned short bits = static_cast<unsigned short>((w[h >> 1] >> (16 * (h & 1))) & 0xffffu);
+        const float f = __half2float(__ushort_as_half(bits));
+        acc[h] = __fadd_rn(acc[h], f);  // one rounded fp32 add per found slot, never fused
+        if (!any || f > bestf[h]) {     // strict >: the earlier slot keeps a tie
+          bestf[h] = f;
+          best[h] = bits;
+        }
+      }
+      any = true;
+    }
+  }
+  unsigned short res[8];
+#pragma unroll
+  for (int h = 0; h < 8; ++h) {
+    const int d = piece * 8 + h;
+    const bool is_sum = (reduce_sum_mask >> (d & 63)) & 1ull;
+    unsigned short sum_bits = __half_as_ushort(__float2half_rn(acc[h]));
+    if (acc[h] != acc[h]) sum_bits = 0x7fffu;
+    res[h] = any ? (is_sum ? sum_bits : best[h]) : static_cast<unsigned short>(0);
+  }
+  uint4 v;
+  v.x = res[0] | (static_cast<unsigned>(res[1]) << 16);
+  v.y = res[2] | (static_cast<unsigned>(res[3]) << 16);
+  v.z = res[4] | (static_cast<unsigned>(res[5]) << 16);
+  v.w = res[6] | (static_cast<unsigned>(res[7]) << 16);
+  return v;
 }
 
 // Section widths of a launch, in 16-byte chunks and bytes (compile-time where the variant fixes them).
@@ -129,166 +103,6 @@ struct RowShape {
     out_b = doc_b + edge_b * (SECOND ? 2 : 1) + req_b;
   }
 };
-
-// One warp, one group of up to 32 consecutive candidates [jg, jg+cnt) of request r.
-// `lookup(inr, author, pos)` returns whether the author id is among the request's keys and its index.
-template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, typename Lookup>
-__device__ __forceinline__ void process_group(const JoinArgs& a, const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND>& sh,
-                                              const StagedKeys& keys, int r, long long kb, long long jg, int cnt,
-                                              int lane, Lookup lookup) {
-  const int doc_b = sh.doc_b, edge_b = sh.edge_b;
-  const long long out_b = sh.out_b;
-  uint8_t* out = a.out_rows + jg * out_b;
-
-  // ---- lane-per-candidate: position, ids
-  const int idx = (lane < cnt) ? __ldg(a.cand_idx + jg + lane) : -1;
-  const bool inr = idx >= 0 && idx < a.n_docs;
-  const int64_t auth = inr ? __ldg(a.author_ids + idx) : -1;
-  int64_t actor[4] = {-1, -1, -1, -1};
-  unsigned types = 0;
-  if (SECOND && inr) {
-    if (a.max_actors == 4) {
-      const longlong2* ap = reinterpret_cast<const longlong2*>(a.actor_ids + 4LL * idx);
-      const longlong2 p0 = __ldg(ap);
-      const longlong2 p1 = __ldg(ap + 1);
-      actor[0] = p0.x;
-      actor[1] = p0.y;
-      actor[2] = p1.x;
-      actor[3] = p1.y;
-      types = __ldg(reinterpret_cast<const unsigned*>(a.actor_types + 4LL * idx));
-    } else {
-      for (int s = 0; s < a.max_actors; ++s) {
-        actor[s] = __ldg(a.actor_ids + static_cast<long long>(a.max_actors) * idx + s);
-        types |= static_cast<unsigned>(__ldg(a.actor_types + static_cast<long long>(a.max_actors) * idx + s)) << (8 * s);
-      }
-    }
-  }
-
-  // ---- document rows: issued before the search so that both latencies overlap
-  auto doc_src = [&](int row) -> const uint8_t* {
-    const int ridx = __shfl_sync(kFull, idx, row);
-    return (ridx >= 0 && ridx < a.n_docs) ? a.doc_feats + static_cast<long long>(ridx) * doc_b : nullptr;
-  };
-  constexpr int kDocRegs = DOC_CH ? DOC_CH : 1;
-  uint4 dv[kDocRegs];
-  if constexpr (DOC_CH > 0) {
-#pragma unroll
-    for (int i = 0; i < DOC_CH; ++i) {
-      const int c = i * 32 + lane;
-      const int row = c / kDocRegs;
-      const int piece = c - row * kDocRegs;
-      const uint8_t* s = doc_src(row);
-      dv[i] = make_uint4(0u, 0u, 0u, 0u);
-      if (s != nullptr) dv[i] = ldg128(s + piece * 16);
-    }
-  }
-
-  // ---- search (Algorithm 1 steps 2-3)
-  int pos = 0;
-  const bool found = lookup(inr, auth, pos);
-  unsigned m = found ? 1u : 0u;
-  int apos[4] = {0, 0, 0, 0};
-  if (SECOND) {
-#pragma unroll
-    for (int s = 0; s < 4; ++s) {
-      if (actor[s] >= 0 && keys.find(actor[s], apos[s])) {
-        m |= 1u << (1 + s);
-        m |= 1u << (5 + ((types >> (8 * s)) & 0xffu) % 3u);
-      }
-    }
-  }
-
-  // ---- doc section
-  if constexpr (DOC_CH > 0) {
-#pragma unroll
-    for (int i = 0; i < DOC_CH; ++i) {
-      const int c = i * 32 + lane;
-      const int row = c / kDocRegs;
-      const int piece = c - row * kDocRegs;
-      if (row < cnt) st128_stream(out + row * out_b + piece * 16, dv[i]);
-    }
-  } else {
-    copy_section<0>(sh.doc_ch, lane, cnt, out, out_b, doc_src);
-  }
-
-  // ---- edge section (Eq. 1: the matched row, or zeros)
-  const uint8_t* edge_base = a.edge_feats + kb * edge_b;
-  copy_section<EDGE_CH>(sh.edge_ch, lane, cnt, out + doc_b, out_b, [&](int row) -> const uint8_t* {
-    const int rpos = __shfl_sync(kFull, pos, row);
-    const unsigned rm = __shfl_sync(kFull, m, row);
-    return (rm & 1u) ? edge_base + static_cast<long long>(rpos) * edge_b : nullptr;
-  });
-
-  // ---- edge2 section: the matched rows of the found engager slots, reduced per dim in slot order
-  if (SECOND) {
-    uint8_t* out2 = out + doc_b + edge_b;
-    for (int ii = 0; ii < sh.edge_ch; ++ii) {
-      const int c = ii * 32 + lane;
-      const int row = c / sh.edge_ch;
-      const int piece = c - row * sh.edge_ch;
-      const unsigned rm = __shfl_sync(kFull, m, row);
-      int rp[4];
-#pragma unroll
-      for (int s = 0; s < 4; ++s) rp[s] = __shfl_sync(kFull, apos[s], row);
-      uint4 q[4];
-#pragma unroll
-      for (int s = 0; s < 4; ++s) {
-        q[s] = make_uint4(0u, 0u, 0u, 0u);
-        if ((rm >> (1 + s)) & 1u) q[s] = ldg128(edge_base + static_cast<long long>(rp[s]) * edge_b + piece * 16);
-      }
-      float acc[8], bestf[8];
-      unsigned short best[8];
-#pragma unroll
-      for (int h = 0; h < 8; ++h) {
-        acc[h] = 0.0f;
-        bestf[h] = 0.0f;
-        best[h] = 0;
-      }
-      bool any = false;
-#pragma unroll
-      for (int s = 0; s < 4; ++s) {
-        if ((rm >> (1 + s)) & 1u) {
-          const unsigned w[4] = {q[s].x, q[s].y, q[s].z, q[s].w};
-#pragma unroll
-          for (int h = 0; h < 8; ++h) {
-            const unsigned short bits = static_cast<unsigned short>((w[h >> 1] >> (16 * (h & 1))) & 0xffffu);
-            const float f = __half2float(__ushort_as_half(bits));
-            acc[h] = __fadd_rn(acc[h], f);  // one rounded fp32 add per found slot, never fused
-            if (!any || f > bestf[h]) {     // strict >: the earlier slot keeps a tie
-              bestf[h] = f;
-              best[h] = bits;
-            }
-          }
-          any = true;
-        }
-      }
-      unsigned short res[8];
-#pragma unroll
-      for (int h = 0; h < 8; ++h) {
-        const int d = piece * 8 + h;
-        const bool is_sum = (a.reduce_sum_mask >> (d & 63)) & 1ull;
-        unsigned short sum_bits = __half_as_ushort(__float2half_rn(acc[h]));
-        if (acc[h] != acc[h]) sum_bits = 0x7fffu;
-        res[h] = any ? (is_sum ? sum_bits : best[h]) : static_cast<unsigned short>(0);
-      }
-      uint4 v;
-      v.x = res[0] | (static_cast<unsigned>(res[1]) << 16);
-      v.y = res[2] | (static_cast<unsigned>(res[3]) << 16);
-      v.z = res[4] | (static_cast<unsigned>(res[5]) << 16);
-      v.w = res[6] | (static_cast<unsigned>(res[7]) << 16);
-      if (row < cnt) st128_stream(out2 + row * out_b + piece * 16, v);
-    }
-  }
-
-  // ---- request section (one source row for the whole request)
-  if (sh.req_ch) {
-    const uint8_t* req_src = a.req_feats + static_cast<long long>(r) * sh.req_b;
-    copy_section<((DOC_CH || EDGE_CH) ? REQ_CH : 0)>(sh.req_ch, lane, cnt, out + doc_b + edge_b * (SECOND ? 2 : 1), out_b,
-                                                     [&](int) -> const uint8_t* { return req_src; });
-  }
-
-  if (lane < cnt) a.out_mask[jg + lane] = static_cast<uint8_t>(m);
-}
 
 // Index of the request that holds flat candidate j0 = number of requests that end at or before j0.
 __device__ __forceinline__ int request_of(const int64_t* co, int n_req, long long j0) {
@@ -323,10 +137,129 @@ __device__ __forceinline__ void give_up_wait(const JoinArgs& a, uint32_t bar, ui
   __syncthreads();
 }
 
+// Block-wide lower bound of `id` in ascending g[0..K): every thread probes one pivot per round.
+// All threads must call; returns the same value in every thread.  Result is always within [0, K].
+__device__ __forceinline__ int block_lower_bound(const int64_t* g, int K, int64_t id) {
+  int lo = 0, n = K;
+  while (n > 0) {
+    const int step = (n + kThreads - 1) / kThreads;
+    const long long p = static_cast<long long>(lo) + static_cast<long long>(threadIdx.x + 1) * step - 1;
+    const int below = (p < lo + n) && (__ldg(g + p) < id);
+    const int c = __syncthreads_count(below);
+    const int nlo = min(lo + c * step, lo + n);
+    n = min(step - 1, lo + n - nlo);
+    lo = nlo;
+  }
+  return lo;
+}
+
+// Shared-memory layout of join_kernel, shared by host (sizing) and device (carving).
+struct TileLayout {
+  int off_idx, off_pos, off_apos, off_auth, off_keys, bytes;
+  __host__ __device__ TileLayout(int tile, bool second, bool merge, int key_cap) {
+    off_idx = kSmemHeader;
+    off_pos = off_idx + tile * 4;
+    off_apos = off_pos + tile * 4;
+    off_auth = off_apos + (second ? tile * 16 : 0);
+    off_keys = off_auth + (merge ? tile * 8 : 0);
+    off_keys = (off_keys + 15) & ~15;
+    bytes = off_keys + search_bytes(key_cap, !merge);
+  }
+};
+
+// ---- phase B: 32 rows of one warp, everything already resolved in shared memory -------------------
 template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND>
-__global__ void __launch_bounds__(kThreads, 2) join_kernel(const JoinArgs a) {
+__device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND>& sh,
+                                           const int* s_idx, const int* s_pos, const int4* s_apos,
+                                           const uint8_t* edge_base, const uint8_t* req_src, uint8_t* out, int cnt,
+                                           int lane) {
+  const long long out_b = sh.out_b;
+  if constexpr (DOC_CH > 0 && EDGE_CH > 0) {
+    // every load of the group is issued before its first store
+    uint4 dv[DOC_CH], ev[EDGE_CH];
+#pragma unroll
+    for (int i = 0; i < DOC_CH; ++i) {
+      const int c = i * 32 + lane, row = c / DOC_CH, piece = c % DOC_CH;
+      const int ridx = row < cnt ? s_idx[row] : -1;
+      dv[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (ridx >= 0) dv[i] = ldg128(a.doc_feats + static_cast<long long>(ridx) * (DOC_CH * 16) + piece * 16);
+    }
+#pragma unroll
+    for (int i = 0; i < EDGE_CH; ++i) {
+      const int c = i * 32 + lane, row = c / EDGE_CH, piece = c % EDGE_CH;
+      const int rpos = row < cnt ? s_pos[row] : -1;
+      ev[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (rpos >= 0) ev[i] = ldg128(edge_base + static_cast<long long>(rpos) * (EDGE_CH * 16) + piece * 16);
+    }
+#pragma unroll
+    for (int i = 0; i < DOC_CH; ++i) {
+      const int c = i * 32 + lane, row = c / DOC_CH, piece = c % DOC_CH;
+      if (row < cnt) st128_stream(out + row * out_b + piece * 16, dv[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < EDGE_CH; ++i) {
+      const int c = i * 32 + lane, row = c / EDGE_CH, piece = c % EDGE_CH;
+      if (row < cnt) st128_stream(out + row * out_b + DOC_CH * 16 + piece * 16, ev[i]);
+    }
+  } else {
+    for (int i = 0; i < sh.doc_ch; ++i) {
+      const int c = i * 32 + lane, row = c / sh.doc_ch, piece = c - row * sh.doc_ch;
+      const int ridx = row < cnt ? s_idx[row] : -1;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (ridx >= 0) v = ldg128(a.doc_feats + static_cast<long long>(ridx) * sh.doc_b + piece * 16);
+      if (row < cnt) st128_stream(out + row * out_b + piece * 16, v);
+    }
+    for (int i = 0; i < sh.edge_ch; ++i) {
+      const int c = i * 32 + lane, row = c / sh.edge_ch, piece = c - row * sh.edge_ch;
+      const int rpos = row < cnt ? s_pos[row] : -1;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (rpos >= 0) v = ldg128(edge_base + static_cast<long long>(rpos) * sh.edge_b + piece * 16);
+      if (row < cnt) st128_stream(out + row * out_b + sh.doc_b + piece * 16, v);
+    }
+  }
+  // edge2 section: the matched rows of the found engager slots, reduced per dim in slot order
+  if constexpr (SECOND) {
+    for (int i = 0; i < sh.edge_ch; ++i) {
+      const int c = i * 32 + lane, row = c / sh.edge_ch, piece = c - row * sh.edge_ch;
+      int rp[4] = {-1, -1, -1, -1};
+      if (row < cnt) {
+        const int4 p = s_apos[row];
+        rp[0] = p.x;
+        rp[1] = p.y;
+        rp[2] = p.z;
+        rp[3] = p.w;
+      }
+      const uint4 v = edge2_chunk(a.reduce_sum_mask, edge_base, sh.edge_b, piece, rp);
+      if (row < cnt) st128_stream(out + row * out_b + sh.doc_b + sh.edge_b + piece * 16, v);
+    }
+  }
+  // request section: one source row for the whole request (L1/L2 hits)
+  if (sh.req_ch) {
+    const int off = sh.doc_b + sh.edge_b * (SECOND ? 2 : 1);
+    for (int i = 0; i < sh.req_ch; ++i) {
+      const int c = i * 32 + lane, row = c / sh.req_ch, piece = c - row * sh.req_ch;
+      const uint4 v = ldg128(req_src + piece * 16);
+      if (row < cnt) st128_stream(out + row * out_b + off + piece * 16, v);
+    }
+  }
+}
+
+constexpr int kUnroll = 8;  // candidates a thread keeps in flight in phase A
+#ifndef CCR_JOIN_MIN_BLOCKS
+#define CCR_JOIN_MIN_BLOCKS 2
+#endif
+constexpr int kJoinMinBlocks = CCR_JOIN_MIN_BLOCKS;  // resident blocks per SM the register budget is set for
+
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, bool MERGE>
+__global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const JoinArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
-  int64_t* skeys = reinterpret_cast<int64_t*>(smem + kSmemHeader);
+  const TileLayout lay(a.tile, SECOND, MERGE, a.key_cap);
+  int* s_idx = reinterpret_cast<int*>(smem + lay.off_idx);
+  int* s_pos = reinterpret_cast<int*>(smem + lay.off_pos);
+  int4* s_apos = reinterpret_cast<int4*>(smem + lay.off_apos);
+  int64_t* s_auth = reinterpret_cast<int64_t*>(smem + lay.off_auth);
+  const SearchSmem ssm = carve_search(smem + lay.off_keys, a.key_cap, !MERGE);
+  const BlockGroup grp;
   const uint32_t bar = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND> sh(a);
@@ -338,8 +271,12 @@ __global__ void __launch_bounds__(kThreads, 2) join_kernel(const JoinArgs a) {
   __syncthreads();
   uint32_t phase = 0;
 
-  const long long j0 = static_cast<long long>(blockIdx.x) * a.tile;
-  const long long j1 = min(j0 + a.tile, a.total);
+  // this block's contiguous slice of the flat candidate range, in whole groups of 32
+  const long long groups = (a.total + 31) >> 5;
+  const long long per = (groups + gridDim.x - 1) / gridDim.x;
+  const long long j0 = min(a.total, static_cast<long long>(blockIdx.x) * per * 32);
+  const long long j1 = min(a.total, j0 + per * 32);
+  if (j0 >= j1) return;
   int r = request_of(a.cand_offsets, a.n_req, j0);
 
   long long seg = j0;
@@ -352,21 +289,163 @@ __global__ void __launch_bounds__(kThreads, 2) join_kernel(const JoinArgs a) {
     const long long seg_end = min(rend, j1);
     long long kb;
     const int K = request_keys(a, r, kb);
+    const uint8_t* edge_base = a.edge_feats + kb * sh.edge_b;
+    const uint8_t* req_src = sh.req_ch ? a.req_feats + static_cast<long long>(r) * sh.req_b : nullptr;
 
     StagedKeys keys;
-    if (!stage_keys(a, skeys, bar, phase, kb, K, keys)) {
-      give_up_wait(a, bar, phase);
-      return;
+    if (!MERGE) {
+      if (!stage_keys(a, ssm, bar, phase, kb, K, true, keys, grp)) {
+        give_up_wait(a, bar, phase);
+        return;
+      }
     }
 
-    const long long nseg = seg_end - seg;
-    for (long long g = static_cast<long long>(warp) * 32; g < nseg; g += kWarps * 32) {
-      const int cnt = static_cast<int>(min(32LL, nseg - g));
-      process_group<DOC_CH, EDGE_CH, REQ_CH, SECOND>(
-          a, sh, keys, r, kb, seg + g, cnt, lane,
-          [&](bool inr, int64_t auth, int& pos) -> bool { return inr && keys.find(auth, pos); });
+    for (long long sub = seg; sub < seg_end; sub += a.tile) {
+      const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_end - sub));
+
+      // ================= phase A: resolve every candidate of the sub-tile =================
+      if (!MERGE) {
+        for (int base = 0; base < n; base += kThreads * kUnroll) {
+          int idx[kUnroll];
+          int64_t auth[kUnroll];
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            const int i = base + u * kThreads + tid;
+            idx[u] = i < n ? __ldg(a.cand_idx + sub + i) : -1;
+          }
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;  // unresolved / out-of-range position
+            auth[u] = idx[u] >= 0 ? __ldg(a.author_ids + idx[u]) : -1;
+          }
+          bool found[kUnroll];
+          int pos[kUnroll];
+          static_assert(kUnroll % 4 == 0, "lookups are interleaved four at a time");
+#pragma unroll
+          for (int h = 0; h < kUnroll; h += 4) {
+            const int64_t id4[4] = {auth[h], auth[h + 1], auth[h + 2], auth[h + 3]};
+            bool f4[4];
+            int p4[4];
+            keys.find_batch<4>(id4, f4, p4);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              found[h + q] = f4[q];
+              pos[h + q] = p4[q];
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            const int i = base + u * kThreads + tid;
+            if (i >= n) continue;
+            unsigned m = found[u] ? 1u : 0u;
+            if (SECOND) {
+              int64_t act[4] = {-1, -1, -1, -1};
+              unsigned types = 0;
+              if (idx[u] >= 0) {
+                for (int sl = 0; sl < a.max_actors; ++sl) {
+                  const long long e = static_cast<long long>(a.max_actors) * idx[u] + sl;
+                  act[sl] = __ldg(a.actor_ids + e);
+                  types |= (__ldg(a.actor_types + e) % 3u) << (2 * sl);
+                }
+              }
+              bool af[4];
+              int ap[4];
+              keys.find_batch<4>(act, af, ap);
+#pragma unroll
+              for (int sl = 0; sl < 4; ++sl) {
+                if (af[sl]) {
+                  m |= 1u << (1 + sl);
+                  m |= 1u << (5 + ((types >> (2 * sl)) & 3u));
+                } else {
+                  ap[sl] = -1;
+                }
+              }
+              s_apos[i] = make_int4(ap[0], ap[1], ap[2], ap[3]);
+            }
+            s_idx[i] = idx[u];
+            s_pos[i] = found[u] ? pos[u] : -1;
+            a.out_mask[sub + i] = static_cast<uint8_t>(m);
+          }
+        }
+      } else {
+        // 1. author ids of the sub-tile
+        for (int base = 0; base < n; base += kThreads * kUnroll) {
+          int idx[kUnroll];
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            const int i = base + u * kThreads + tid;
+            idx[u] = i < n ? __ldg(a.cand_idx + sub + i) : -1;
+          }
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            const int i = base + u * kThreads + tid;
+            if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;
+            if (i < n) {
+              s_idx[i] = idx[u];
+              s_auth[i] = idx[u] >= 0 ? __ldg(a.author_ids + idx[u]) : kNoAuthor;
+            }
+          }
+        }
+        __syncthreads();
+        // 2. the only keys this sub-tile can touch: window [lo, hi)
+        const int64_t* gk = a.edge_keys + kb;
+        const int lo = block_lower_bound(gk, K, s_auth[0]);
+        const int hi = min(K, block_lower_bound(gk, K, s_auth[n - 1]) + 1);
+        const int w = max(hi - lo, 0);
+        const bool windowed = (a.key_cap > 0) && (w <= a.key_cap) && (a.min_stride_log2 == 0);
+        // 3. stage the window (or, if it is too long, the request's keys as the binary-search mode does)
+        if (!stage_keys(a, ssm, bar, phase, windowed ? kb + lo : kb, windowed ? w : K, false, keys, grp)) {
+          give_up_wait(a, bar, phase);
+          return;
+        }
+        if (windowed) {
+          // 4. merge path over (s_auth[0..n), window[0..w)); a candidate goes before an equal key, so the
+          //    keys consumed when it is emitted are exactly the keys below it
+          const int64_t* B = keys.sk;
+          const int total = n + w;
+          const int L = (total + kThreads - 1) / kThreads;
+          const int diag = min(tid * L, total);
+          int ab = max(0, diag - w), ae = min(diag, n);
+          while (ab < ae) {
+            const int mid = (ab + ae) >> 1;
+            if (s_auth[mid] <= B[diag - 1 - mid]) ab = mid + 1; else ae = mid;
+          }
+          int ai = ab, bi = diag - ab;
+          for (int step = 0; step < L && (ai < n || bi < w); ++step) {
+            if (ai < n && (bi >= w || s_auth[ai] <= B[bi])) {
+              const bool hit = bi < w && B[bi] == s_auth[ai] && s_idx[ai] >= 0;
+              s_pos[ai] = hit ? lo + bi : -1;
+              ++ai;
+            } else {
+              ++bi;
+            }
+          }
+          __syncthreads();
+          // under a broken sortedness promise a slot may not have been written by the merge: bound it
+          for (int i = tid; i < n; i += kThreads) {
+            int p = s_pos[i];
+            if (p >= K) p = -1;
+            s_pos[i] = p;
+            a.out_mask[sub + i] = p >= 0 ? 1 : 0;
+          }
+        } else {
+          for (int i = tid; i < n; i += kThreads) {
+            int pos = 0;
+            const bool found = s_idx[i] >= 0 && keys.find(s_auth[i], pos);
+            s_pos[i] = found ? pos : -1;
+            a.out_mask[sub + i] = found ? 1 : 0;
+          }
+        }
+      }
+      __syncthreads();
+
+      // ================= phase B: stream the rows =================
+      for (int g = warp * 32; g < n; g += kWarps * 32) {
+        emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND>(a, sh, s_idx + g, s_pos + g, s_apos + g, edge_base, req_src,
+                                                    a.out_rows + (sub + g) * sh.out_b, min(32, n - g), lane);
+      }
+      __syncthreads();  // phase A of the next sub-tile overwrites the resolved arrays (and, in merge mode, the keys)
     }
-    __syncthreads();  // every warp is done with the staged keys before the next request overwrites them
     seg = seg_end;
     ++r;
   }

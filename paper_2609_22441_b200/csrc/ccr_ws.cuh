@@ -1,0 +1,303 @@
+// Warp-specialised variant of the fused join (same result as join_kernel).
+//
+// In join_kernel every warp alternates between resolving candidates (position -> author id -> search: two
+// dependent memory accesses plus a shared-memory search) and streaming rows; while a block resolves, its
+// share of the memory pipeline idles.  Here the two jobs run concurrently in one persistent block per SM:
+//   resolver warps : take chunks of the flat candidate range, stage each request's keys (TMA bulk copy +
+//                    mbarrier, waited on by the resolvers only), and fill a ring of sub-tile buffers in
+//                    shared memory with (position, match index) per candidate; they also write the mask
+//                    bytes.  Their latency (ids are 8-byte gathers, key staging) hides behind the streaming.
+//   streamer warps : consume the ring; for every 32-row group all loads are issued, then all stores —
+//                    nothing else.  They never touch keys, ids or barriers other than the ring's.
+// Ring slots are handed over with shared-memory mbarriers: full[slot] (one arrival, by the resolvers, once the
+// slot is written) and empty[slot] (one arrival per streamer warp, once it has taken its last group of the
+// slot).  Warps wait on them individually — a streamer warp that is done with a slot moves on to the next
+// full slot without waiting for its siblings — and every wait is bounded: on expiry the warp records
+// kDevWaitExpired and leaves.  A slot with n == 0 tells the streamers to stop.  Inside a slot the streamer
+// warps take 32-row groups one at a time from a shared-memory counter.
+//
+// Work distribution.  With a scheduling word (JoinArgs::sched) the resolvers of all blocks draw chunks of
+// consecutive tiles from one global counter; the chunk shrinks from kMaxChunk tiles to one tile as the
+// launch drains (guided self-scheduling), so blocks on slower SMs or with costlier requests simply take
+// fewer chunks and all blocks finish within about one tile of each other.  The last block to finish puts
+// the two scheduling words back to zero for the next launch.  Without a scheduling word every block takes
+// one equal contiguous slice.
+#pragma once
+
+#include "ccr_join.cuh"
+
+namespace ccr {
+
+constexpr int kWsSlots = 8;        // ring depth
+constexpr int kWsMaxThreads = 512;
+constexpr int kMaxChunk = 8;       // most tiles a block draws at once
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+struct WsSlot {          // descriptor of one ring slot
+  long long sub;         // first flat candidate of the sub-tile
+  long long kb;          // first key / edge row of its request
+  int n;                 // candidates in the sub-tile (0 = stop)
+  int r;                 // request index
+  int next;              // next 32-row group a streamer warp may take (reset by the resolvers)
+  int pad;
+};
+
+struct WsLayout {
+  int off_full, off_empty, off_slots, off_grab, off_idx, off_pos, off_apos, off_keys, bytes;
+  __host__ __device__ WsLayout(int tile, bool second, int key_cap) {
+    off_full = kSmemHeader;                 // after the key-staging mbarrier
+    off_empty = off_full + kWsSlots * 8;
+    off_slots = off_empty + kWsSlots * 8;
+    off_grab = off_slots + kWsSlots * static_cast<int>(sizeof(WsSlot));
+    off_idx = off_grab + 16;
+    off_pos = off_idx + kWsSlots * tile * 4;
+    off_apos = off_pos + kWsSlots * tile * 4;
+    off_keys = off_apos + (second ? kWsSlots * tile * 16 : 0);
+    bytes = off_keys + search_bytes(key_cap, true);
+  }
+};
+
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND>
+__global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArgs a, int n_streamers) {
+  extern __shared__ __align__(16) unsigned char smem_ws[];
+  unsigned char* smem = smem_ws;
+  const WsLayout lay(a.tile, SECOND, a.key_cap);
+  WsSlot* slots = reinterpret_cast<WsSlot*>(smem + lay.off_slots);
+  int* grab = reinterpret_cast<int*>(smem + lay.off_grab);
+  int* s_idx = reinterpret_cast<int*>(smem + lay.off_idx);
+  int* s_pos = reinterpret_cast<int*>(smem + lay.off_pos);
+  int4* s_apos = reinterpret_cast<int4*>(smem + lay.off_apos);
+  const SearchSmem ssm = carve_search(smem + lay.off_keys, a.key_cap, true);
+  const uint32_t bar = smem_u32(smem);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_threads = blockDim.x;
+  const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND> sh(a);
+  const uint32_t full0 = smem_u32(smem + lay.off_full), empty0 = smem_u32(smem + lay.off_empty);
+  const int kBarGroup = 1;  // named barrier of the resolver group
+
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    for (int s = 0; s < kWsSlots; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, static_cast<uint32_t>(n_streamers));
+    }
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+
+  // static split (no scheduling word): this block's contiguous slice, in whole groups of 32
+  const long long groups = (a.total + 31) >> 5;
+  const long long per = (groups + gridDim.x - 1) / gridDim.x;
+  const long long slice0 = min(a.total, static_cast<long long>(blockIdx.x) * per * 32);
+  const long long slice1 = min(a.total, slice0 + per * 32);
+  if (a.sched == nullptr && slice0 >= slice1) return;  // block-uniform, before any named barrier
+
+  if (warp < n_streamers) {
+    // ============================ streamers ============================
+    for (unsigned it = 0;; ++it) {
+      const int s = it % kWsSlots;
+      if (!mbar_wait_bounded(full0 + 8 * s, (it / kWsSlots) & 1u)) {
+        if (lane == 0) atomicExch(a.status, kDevWaitExpired);
+        return;
+      }
+      const WsSlot d = slots[s];
+      if (d.n == 0) break;
+      const uint8_t* edge_base = a.edge_feats + d.kb * sh.edge_b;
+      const uint8_t* req_src = sh.req_ch ? a.req_feats + static_cast<long long>(d.r) * sh.req_b : nullptr;
+      const int* idx = s_idx + s * a.tile;
+      const int* pos = s_pos + s * a.tile;
+      const int4* apos = s_apos + s * a.tile;
+      // groups are handed out one at a time, so a warp that finishes early simply takes more
+      for (;;) {
+        int g = 0;
+        if (lane == 0) g = atomicAdd(&slots[s].next, 1);
+        g = __shfl_sync(kFull, g, 0) * 32;
+        if (g >= d.n) break;
+        emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND>(a, sh, idx + g, pos + g, apos + g, edge_base, req_src,
+                                                    a.out_rows + (d.sub + g) * sh.out_b, min(32, d.n - g), lane);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8 * s);
+    }
+    return;
+  }
+
+  // ============================ resolvers ============================
+  const int gsize = n_threads - n_streamers * 32;
+  const int gtid = tid - n_streamers * 32;
+  const NamedGroup grp(gtid, gsize, kBarGroup);
+  uint32_t phase = 0;
+  unsigned it = 0;       // ring slots published so far
+  bool failed = false;
+  int staged_r = -1;     // request whose keys are in shared memory
+  StagedKeys keys;
+  const long long n_tiles = (a.total + a.tile - 1) / a.tile;
+
+  for (bool more = true; more && !failed;) {
+    long long j0, j1;
+    if (a.sched != nullptr) {
+      if (gtid == 0) {
+        const long long rem = n_tiles - *reinterpret_cast<volatile int*>(a.sched);
+        long long c = rem / (2LL * gridDim.x);
+        c = c < 1 ? 1 : (c > kMaxChunk ? kMaxChunk : c);
+        grab[0] = atomicAdd(a.sched, static_cast<int>(c));
+        grab[1] = static_cast<int>(c);
+      }
+      grp.sync();
+      const long long t = grab[0], c = grab[1];
+      grp.sync();
+      if (t >= n_tiles) break;
+      j0 = t * a.tile;
+      j1 = min(a.total, (t + c) * a.tile);
+    } else {
+      j0 = slice0;
+      j1 = slice1;
+      more = false;
+    }
+
+    int r = request_of(a.cand_offsets, a.n_req, j0);
+    long long seg = j0;
+    while (seg < j1 && r < a.n_req && !failed) {
+      const long long rend = __ldg(a.cand_offsets + r + 1);
+      if (rend <= seg) {  // request without candidates here
+        ++r;
+        continue;
+      }
+      const long long seg_end = min(rend, j1);
+      long long kb;
+      const int K = request_keys(a, r, kb);
+      if (r != staged_r) {
+        if (!stage_keys(a, ssm, bar, phase, kb, K, true, keys, grp)) {
+          if (gtid == 0) {
+            atomicExch(a.status, kDevWaitExpired);
+            mbar_wait_bounded(bar, phase ^ 1u);
+          }
+          failed = true;
+          break;
+        }
+        staged_r = r;
+      }
+      for (long long sub = seg; sub < seg_end; sub += a.tile, ++it) {
+        const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_end - sub));
+        const int s = it % kWsSlots;
+        if (it >= static_cast<unsigned>(kWsSlots) && !mbar_wait_bounded(empty0 + 8 * s, (it / kWsSlots - 1) & 1u)) {
+          failed = true;  // the streamers are gone: every resolver thread times out on the same barrier
+          break;
+        }
+        int* out_idx = s_idx + s * a.tile;
+        int* out_pos = s_pos + s * a.tile;
+        int4* out_apos = s_apos + s * a.tile;
+        for (int base = 0; base < n; base += gsize * kUnroll) {
+          int idx[kUnroll];
+          int64_t auth[kUnroll];
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            const int i = base + u * gsize + gtid;
+            idx[u] = i < n ? __ldg(a.cand_idx + sub + i) : -1;
+          }
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;  // unresolved / out-of-range position
+            auth[u] = idx[u] >= 0 ? __ldg(a.author_ids + idx[u]) : -1;
+          }
+          bool found[kUnroll];
+          int pos[kUnroll];
+          static_assert(kUnroll % 4 == 0, "lookups are interleaved four at a time");
+#pragma unroll
+          for (int h = 0; h < kUnroll; h += 4) {
+            const int64_t id4[4] = {auth[h], auth[h + 1], auth[h + 2], auth[h + 3]};
+            bool f4[4];
+            int p4[4];
+            keys.find_batch<4>(id4, f4, p4);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              found[h + q] = f4[q];
+              pos[h + q] = p4[q];
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {
+            const int i = base + u * gsize + gtid;
+            if (i >= n) continue;
+            unsigned m = found[u] ? 1u : 0u;
+            if (SECOND) {
+              int64_t act[4] = {-1, -1, -1, -1};
+              unsigned types = 0;
+              if (idx[u] >= 0) {
+                for (int sl = 0; sl < a.max_actors; ++sl) {
+                  const long long e = static_cast<long long>(a.max_actors) * idx[u] + sl;
+                  act[sl] = __ldg(a.actor_ids + e);
+                  types |= (__ldg(a.actor_types + e) % 3u) << (2 * sl);
+                }
+              }
+              bool af[4];
+              int ap[4];
+              keys.find_batch<4>(act, af, ap);
+#pragma unroll
+              for (int sl = 0; sl < 4; ++sl) {
+                if (af[sl]) {
+                  m |= 1u << (1 + sl);
+                  m |= 1u << (5 + ((types >> (2 * sl)) & 3u));
+                } else {
+                  ap[sl] = -1;
+                }
+              }
+              out_apos[i] = make_int4(ap[0], ap[1], ap[2], ap[3]);
+            }
+            out_idx[i] = idx[u];
+            out_pos[i] = found[u] ? pos[u] : -1;
+            a.out_mask[sub + i] = static_cast<uint8_t>(m);
+          }
+        }
+        if (gtid == 0) {
+          WsSlot d;
+          d.sub = sub;
+          d.kb = kb;
+          d.n = n;
+          d.r = r;
+          d.next = 0;
+          d.pad = 0;
+          slots[s] = d;
+        }
+        grp.sync();  // every resolver's part of the slot is written
+        if (gtid == 0) mbar_arrive(full0 + 8 * s);
+      }
+      if (failed) break;
+      seg = seg_end;
+      ++r;
+    }
+  }
+
+  // stop slot
+  if (failed) {
+    if (gtid == 0) atomicExch(a.status, kDevWaitExpired);
+  } else {
+    const int s = it % kWsSlots;
+    if (it >= static_cast<unsigned>(kWsSlots)) failed = !mbar_wait_bounded(empty0 + 8 * s, (it / kWsSlots - 1) & 1u);
+    if (gtid == 0) {
+      WsSlot d;
+      d.sub = 0;
+      d.kb = 0;
+      d.n = 0;
+      d.r = 0;
+      d.next = 0;
+      d.pad = 0;
+      slots[s] = d;
+      mbar_arrive(full0 + 8 * s);
+    }
+  }
+  // the last block to stop drawing tiles zeroes the scheduling words for the next launch
+  if (a.sched != nullptr && gtid == 0) {
+    __threadfence();
+    if (atomicAdd(a.sched + 1, 1) == static_cast<int>(gridDim.x) - 1) {
+      a.sched[0] = 0;
+      a.sched[1] = 0;
+      __threadfence();
+    }
+  }
+}
+
+}  // namespace ccr

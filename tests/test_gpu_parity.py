@@ -28,10 +28,13 @@ def B():
 
 
 def _variants(B, include_smem=True):
+    """Every key-search path, each through the warp-specialised kernel (default: dynamic chunks; and with the
+    static split) and the two-phase kernel."""
     v = [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL), ("sampled", B.CCR_FLAG_FORCE_SAMPLED)]
     if include_smem:
         v.append(("smem", B.CCR_FLAG_FORCE_SMEM))
-    return v
+    return (v + [(n + "+2phase", f | B.CCR_FLAG_TWO_PHASE) for n, f in v] +
+            [(n + "+static", f | B.CCR_FLAG_STATIC_SPLIT) for n, f in v])
 
 
 def _check(B, wl, flag_sets, first_degree_only=False, tunings=((0, 0),)):
@@ -39,9 +42,10 @@ def _check(B, wl, flag_sets, first_degree_only=False, tunings=((0, 0),)):
     store = B.store_from_workload(wl)
     db = B.DeviceBatch(wl.batch)
     try:
-        for tile, cap in tunings:
-            if tile or cap:
-                store.set_tuning(tile, cap)
+        for tuning in tunings:
+            tile, cap = tuning[0], tuning[1]
+            if any(tuning):
+                store.set_tuning(*tuning)
             for name, flags in flag_sets:
                 if first_degree_only:
                     flags |= B.CCR_FLAG_FIRST_DEGREE_ONLY
@@ -68,7 +72,7 @@ def test_config0_single_tiny_request_all_search_paths(B):
 def test_config1_batched_first_degree_full_size(B):
     wl = W.config1()
     assert wl.batch.total_cands == 64 * 30_000 and wl.out_row_bytes() == 384
-    _check(B, wl, _variants(B))
+    _check(B, wl, _variants(B), tunings=((0, 0), (512, 0, 1, 1, 1), (2048, 0, 14, 2, 3), (768, 0, 5, 8, 2)))
     _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
 
 
@@ -95,7 +99,7 @@ def test_config3_scaled_store_long_edge_lists(B):
     # first-degree-only as in the headline run, then fully
     wl = W.config3(n_docs=2_000_000, n_req=12, n_cand=20_000, gen_doc_feats=True, extra_pools=0)
     assert wl.batch.max_edge_len > 4096
-    _check(B, wl, _variants(B), first_degree_only=True, tunings=((0, 0), (512, 1000), (2048, 20_000)))
+    _check(B, wl, _variants(B), first_degree_only=True, tunings=((0, 0), (512, 1000), (2048, 20_000), (256, 7)))
     _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=True,
            tunings=((0, 0), (256, 64)))
     _check(B, wl, [("auto", 0)])
@@ -107,11 +111,11 @@ def test_tiny_random_batches(B, seed):
     second = bool(seed % 2)
     wl = tiny_workload(seed, n_docs=37 + seed, alphabet=20 + 3 * seed, n_req=1 + seed, kmax=16, nmax=70,
                        second=second, req_dim=4 * (seed % 3 == 0))
-    _check(B, wl, _variants(B), tunings=((32, 0), (0, 0)))
+    _check(B, wl, _variants(B), tunings=((256, 0), (0, 0)))
     if second:
         _check(B, wl, [("auto", 0)], first_degree_only=True)
     _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=second,
-           tunings=((64, 0),))
+           tunings=((256, 3),))
 
 
 def test_generic_widths_take_the_runtime_variant(B):
@@ -142,7 +146,7 @@ def test_search_boundaries_and_empty_requests(B):
     keys = [[0, 7, imax], [], [7], [0, 7, imax], [5, 6, 9, imax - 1]]
     cands = [[0, 1, 2, 3, 4, 5, 6, 7, 2, 2, -1, 10], [1, 2, 3], [2, 8, 9, 0], [], [1, 7, 3, 5, 4, 2]]
     wl = _manual(keys, cands, authors)
-    rows, mask = _check(B, wl, _variants(B), tunings=((32, 0), (0, 0)))
+    rows, mask = _check(B, wl, _variants(B), tunings=((256, 0), (0, 0)))
     assert list(mask[:12]) == [1, 0, 1, 0, 1, 0, 0, 0, 1, 1, 0, 0]
     assert list(mask[12:15]) == [0, 0, 0] and list(mask[15:19]) == [1, 1, 1, 0] and list(mask[19:]) == [1, 1, 1, 1, 0, 0]
 
@@ -158,7 +162,7 @@ def test_all_found_none_found_and_duplicates(B):
     assert mask[:5000].all() and not mask[5000:10000].any()
 
 
-@pytest.mark.parametrize("k", [1, 2, 3, 255, 256, 257, 4095, 4096, 4097, 8191, 29_000, 65_536, 100_000])
+@pytest.mark.parametrize("k", [1, 2, 3, 255, 256, 257, 4095, 4096, 4097, 8191, 20_000, 65_536, 100_000])
 def test_edge_list_lengths_around_every_path_threshold(B, k):
     # two requests so that the second one's keys start at an odd (8-byte aligned only) offset when k is odd
     rng = np.random.default_rng(k)
@@ -168,7 +172,7 @@ def test_edge_list_lengths_around_every_path_threshold(B, k):
     keys2 = W.sorted_unique_sample(rng, 4 * k + 10, k)
     cand = [rng.integers(0, n_docs, size=3000), rng.integers(0, n_docs, size=2500)]
     wl = _manual([keys1, keys2], cand, authors, edge_dim=8)
-    fits_smem = k <= 29_000
+    fits_smem = k <= 20_000
     _check(B, wl, _variants(B, include_smem=fits_smem))
     _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
     if not fits_smem:
