@@ -48,7 +48,11 @@ def parse_args():
     p.add_argument("--steps", type=int, default=2000)
     p.add_argument("--warmup", type=int, default=10)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--config", default="1", choices=["1", "2b"])
+    p.add_argument("--config", default="1", choices=["1", "2b", "3", "3b", "3s", "4"],
+                   help="1 batched first-degree (default, the headline); 2b second-degree on the same shape; 3 production-scale "
+                        "store, first-degree; 3b the same on candidates sorted by author (merge path); 3s production scale, "
+                        "second-degree; 4 single-request latency sweep on the production-scale store")
+    p.add_argument("--sweep-requests", type=int, default=1000, help="requests per cell of the latency sweep")
     p.add_argument("--e2e-steps", type=int, default=0, help="0 = min(steps, 10)")
     p.add_argument("--flags", type=int, default=0, help="extra CCR_FLAG_* bits (experiments)")
     p.add_argument("--tile", type=int, default=0, help="candidates per ring slot (0 = library default)")
@@ -62,11 +66,20 @@ def parse_args():
 
 
 def make_workload(config: str, rank: int):
+    """(workload, extra join flags) of a benchmark configuration; rank shifts the seed so replicas differ."""
+    from paper_2609_22441_b200 import binding as B
     from paper_2609_22441_b200 import workloads as W
 
     if config == "1":
-        return W.config1(seed=W.config_seed(1, 0) + 17 * rank)
-    return W.config1(seed=W.config_seed(2, 1) + 17 * rank, second_degree=True)
+        return W.config1(seed=W.config_seed(1, 0) + 17 * rank), 0
+    if config == "2b":
+        return W.config1(seed=W.config_seed(2, 1) + 17 * rank, second_degree=True), 0
+    wl = W.config3(seed=W.config_seed(3, 0) + 17 * rank)
+    if config == "3":
+        return wl, B.CCR_FLAG_FIRST_DEGREE_ONLY
+    if config == "3b":
+        return W.sort_candidates_by_author(wl), B.CCR_FLAG_FIRST_DEGREE_ONLY | B.CCR_FLAG_CANDS_SORTED
+    return wl, 0
 
 
 def workload_label(wl) -> str:
@@ -194,6 +207,107 @@ def time_oracle(wl, n_threads: int, repeats: int, max_cands: int = 0):
     return best, int(b.total_cands)
 
 
+def compact_sample(wl, kept, n_cands: int, flags: int):
+    """The first n_cands candidates as a self-contained problem for the oracle: store = the rows of exactly
+    those docs (kept on the host when the store was generated), candidates renumbered 0..n-1."""
+    from paper_2609_22441_b200 import binding as B
+    from paper_2609_22441_b200 import workloads as W
+
+    s, b = wl.store, wl.batch
+    docs = b.cand_idx[:n_cands].astype(np.int64)
+    where = np.searchsorted(kept["idx"], docs)
+    n_req = int(np.searchsorted(b.cand_offsets, n_cands, side="left"))
+    first_only = bool(flags & B.CCR_FLAG_FIRST_DEGREE_ONLY)
+    store = W.Store(n_docs=n_cands, doc_dim=s.doc_dim, doc_dtype=s.doc_dtype, author_ids=s.author_ids[docs],
+                    doc_feats=kept["rows"][where], max_actors=0 if first_only else s.max_actors,
+                    actor_ids=None if first_only else s.actor_ids[docs],
+                    actor_types=None if first_only else s.actor_types[docs], reduce_sum_mask=s.reduce_sum_mask)
+    batch = W.Batch(**{**b.__dict__, "cand_idx": np.arange(n_cands, dtype=np.int32),
+                       "cand_offsets": b.cand_offsets[:n_req + 1].copy(), "edge_offsets": b.edge_offsets[:n_req + 1].copy(),
+                       "req_feats": None if b.req_feats is None else b.req_feats[:n_req]})
+    return W.Workload(wl.name + "-sample", wl.seed, store, batch, dict(wl.meta))
+
+
+def latency_sweep(args, B, device: int):
+    """Config 4: one request per launch on one stream, candidates x edge-list length grid on the
+    production-scale store; p50 / p99 of the CUDA-event time and of the host time from call to stream sync."""
+    import torch
+
+    from paper_2609_22441_b200 import workloads as W
+
+    dev = torch.device("cuda", device)
+    wl = W.config3()
+    s = wl.store
+    n_values = (1_000, 5_000, 20_000, 50_000, 100_000)
+    k_values = (10, 100, 1_000, 10_000, 20_000)
+    per_k = 32
+    tpl = W.make_latency_templates(s, W.config_seed(4), k_values, per_k, first_pool=256, n_pools=wl.meta["n_pools"],
+                                   forced_per_template=70_000, edge_dim=wl.batch.edge_dim, n_authors=wl.meta["n_authors"])
+    store, _, _ = B.store_from_generated(wl, device=device)
+    flags = B.CCR_FLAG_FIRST_DEGREE_ONLY | args.flags
+    out_b = store.out_row_bytes(flags)
+    rows = torch.empty((max(n_values), out_b), dtype=torch.uint8, device=dev)
+    mask = torch.empty((max(n_values),), dtype=torch.uint8, device=dev)
+    mark = np.zeros(s.n_docs, dtype=bool)
+    n_per_cell = args.sweep_requests
+    cells = []
+    launches0 = store.launch_count()
+    t_all = 0.0
+    c_all = 0
+    for k in k_values:
+        dev_tpl = [(torch.from_numpy(t.keys).to(dev), torch.from_numpy(t.feats).to(dev),
+                    torch.tensor([0, len(t.keys)], dtype=torch.int64, device=dev)) for t in tpl[k]]
+        for n in n_values:
+            rng = np.random.default_rng(W.config_seed(4, 1000 * k_values.index(k) + n_values.index(n)))
+            co = torch.tensor([0, n], dtype=torch.int64, device=dev)
+            # candidate lists of the cell, pre-staged on the device
+            cand = np.empty((n_per_cell, n), dtype=np.int32)
+            for i in range(n_per_cell):
+                t = tpl[k][i % per_k]
+                n_f = min(int(round(0.7 * n)), len(t.forced_docs))
+                f = t.forced_docs[rng.integers(0, len(t.forced_docs), size=n_f)] if n_f < len(t.forced_docs) else t.forced_docs
+                row = np.concatenate([f[:n_f], rng.integers(0, s.n_docs, size=n - n_f)])
+                rng.shuffle(row)
+                cand[i] = row
+            cand_dev = torch.from_numpy(cand).to(dev)
+            ev, wall = [], []
+            for i in range(-50, n_per_cell):  # 50 warm-up requests per cell
+                j = i % n_per_cell
+                keys, feats, eo = dev_tpl[j % per_k]
+                a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize(dev)
+                t0 = time.perf_counter()
+                a.record()
+                B.ccr_join_batch(store, 1, n, k, keys, feats, eo, cand_dev[j], co, None, rows, mask, flags)
+                z.record()
+                torch.cuda.synchronize(dev)
+                t1 = time.perf_counter()
+                if i >= 0:
+                    ev.append(a.elapsed_time(z))
+                    wall.append((t1 - t0) * 1e3)
+            ev.sort()
+            wall.sort()
+            q = lambda v, p: float(v[max(0, int(np.ceil(p * len(v))) - 1)])
+            cells.append({"candidates": n, "edge_len": k, "event_ms_p50": q(ev, 0.5), "event_ms_p99": q(ev, 0.99),
+                          "host_ms_p50": q(wall, 0.5), "host_ms_p99": q(wall, 0.99)})
+            t_all += sum(ev) * 1e-3
+            c_all += n * n_per_cell
+            del cand_dev
+    if store.device_status() != B.CCR_OK:
+        raise SystemExit("device status not clean after the sweep")
+    print(json.dumps({
+        "metric": METRIC, "value": c_all / t_all, "unit": UNIT, "n_gpus": 1, "steps": n_per_cell * len(cells), "warmup": 50,
+        "ms_per_step": 1e3 * t_all / (n_per_cell * len(cells)), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "config4: latency sweep, one request per launch on one stream, 50,000,000-doc store x 128 fp16, "
+                   "384-byte rows, %d requests per cell (32 viewer templates per edge-list length, 70%% forced matches)" % n_per_cell,
+                   "flags": flags},
+        "latency_sweep": cells, "gpu_launches": int(store.launch_count() - launches0),
+        "paper_context": "the paper quotes 5-10 ms for its join on unstated Hopper-class hardware (abstract)",
+    }))
+    store.free()
+
+
 def run_reference(args, rank: int):
     """The reference arm of this tier is the CPU oracle: rank 0 times it, the other ranks do nothing."""
     if rank != 0:
@@ -201,7 +315,11 @@ def run_reference(args, rank: int):
     from oracle import oracle
 
     oracle.build()
-    wl = make_workload(args.config, 0)
+    if args.config not in ("1", "2b"):
+        print(json.dumps({"impl": "reference", "unavailable": "the CPU oracle cannot hold the 12.8 GB feature matrix of the "
+                          "production-scale configurations; it is timed on configs 1 and 2b"}))
+        return
+    wl, _ = make_workload(args.config, 0)
     cores = host_cores()
     t_probe, n_probe = time_oracle(wl, cores, 1, max_cands=200_000)
     rate = n_probe / t_probe
@@ -273,15 +391,26 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.SUM)
         return float(t.item())
 
-    wl = make_workload(args.config, rank)
+    if args.config == "4":
+        if rank == 0:
+            latency_sweep(args, B, local_rank)
+        return
+    wl, cfg_flags = make_workload(args.config, rank)
     b = wl.batch
     second = wl.store.max_actors > 0
-    store = B.store_from_workload(wl, device=local_rank)
+    kept = None
+    if wl.store.doc_feats is None:
+        # production-scale store: features are drawn on the device chunk by chunk; host copies are kept only
+        # for the docs of the first requests, which is what the CPU baseline is timed on
+        n_base = int(b.cand_offsets[min(10, b.n_req)])
+        store, kept, _ = B.store_from_generated(wl, device=local_rank, keep_rows_of=b.cand_idx[:n_base])
+    else:
+        store = B.store_from_workload(wl, device=local_rank)
     if args.tile or args.key_cap or args.streamers or args.resolvers:
         store.set_tuning(tile_cands=args.tile, key_capacity=args.key_cap, ws_streamers=args.streamers,
                          ws_resolvers=args.resolvers)
     db = B.DeviceBatch(b, device=local_rank)
-    flags = args.flags
+    flags = args.flags | cfg_flags
     out_b = store.out_row_bytes(flags)
     C = b.total_cands
     n_buf = 2  # outputs rotate so that consecutive steps do not rewrite lines still in L2
@@ -332,7 +461,7 @@ def main():
     def e2e_step():
         B.ccr_join_batch_host(store, ws, b.n_req, C, b.max_edge_len, len(b.edge_keys), *h_in, h_rows, h_mask, flags)
 
-    e2e_steps = args.e2e_steps or max(1, min(args.steps, 10))
+    e2e_steps = args.e2e_steps or max(1, min(args.steps, 10 if C < 4_000_000 else 2))
     if args.timed_only:
         e2e_steps = 1
     for _ in range(0 if args.timed_only else 3):
@@ -413,12 +542,18 @@ def main():
 
             oracle.build()
             cores = host_cores()
-            t_mt, n_mt = time_oracle(wl, cores, 3)
-            t_st, n_st = time_oracle(wl, 1, 1, max_cands=600_000)
+            if kept is None:
+                t_mt, n_mt = time_oracle(wl, cores, 3)
+                t_st, n_st = time_oracle(wl, 1, 1, max_cands=600_000)
+                sample = "the whole batch (%d candidates), best of 3 passes" % n_mt
+            else:
+                sub = compact_sample(wl, kept, n_base, flags)
+                t_mt, n_mt = time_oracle(sub, cores, 3)
+                t_st, n_st = time_oracle(sub, 1, 1)
+                sample = ("the first %d candidates (%d requests) against a compacted copy of their docs' rows, best of 3 "
+                          "passes" % (n_mt, min(10, b.n_req)))
             line["cpu_baseline"] = {"value": n_mt / t_mt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                    "sample": "the whole batch (%d candidates), best of 3 passes" % n_mt,
-                                    "single_thread_value": n_st / t_st,
-                                    "gbs_compulsory": bc["compulsory"] / t_mt / 1e9}
+                                    "sample": sample, "single_thread_value": n_st / t_st}
         else:
             line["cpu_baseline"] = None
     store.free()

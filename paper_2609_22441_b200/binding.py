@@ -302,3 +302,38 @@ def store_from_workload(wl, device: int = 0, upload_doc_feats: bool = True) -> D
     st.upload(0, s.doc_feats if upload_doc_feats else None, s.author_ids, s.actor_ids, s.actor_types)
     torch.cuda.synchronize(device)
     return st
+
+
+def store_from_generated(wl, device: int = 0, keep_rows_of=None, keep_all: bool = False):
+    """Create the store of a workload whose doc features are generated on the device in chunks
+    (`workloads.doc_feats_chunk_device`): ids are uploaded from the host, features chunk by chunk from device
+    memory.  Returns (store, kept, full): `kept` = {"idx", "rows"} host copies of the rows of the doc
+    positions in `keep_rows_of` (taken from the generator's output before the library sees it), `full` = the
+    whole generated matrix as a device tensor when keep_all is set."""
+    from . import workloads as W
+
+    s, b = wl.store, wl.batch
+    store = Docstore(s.n_docs, s.doc_dim, s.doc_dtype, b.edge_dim, b.edge_dtype, b.req_dim, b.req_dtype,
+                     s.max_actors, s.reduce_sum_mask, device)
+    store.upload(0, None, s.author_ids, s.actor_ids, s.actor_types)
+    want = None if keep_rows_of is None else np.unique(np.asarray(keep_rows_of, dtype=np.int64))
+    kept_idx, kept_rows, full = [], [], []
+    step = W.DOC_DEVICE_CHUNK
+    dev = torch.device("cuda", device)
+    for first in range(0, s.n_docs, step):
+        n = min(step, s.n_docs - first)
+        chunk = W.doc_feats_chunk_device(wl.seed, first, n, s.doc_dim, dev)
+        store.upload(first, chunk)
+        if want is not None:
+            lo, hi = np.searchsorted(want, [first, first + n])
+            if hi > lo:
+                local = torch.from_numpy(want[lo:hi] - first).to(dev)
+                kept_idx.append(want[lo:hi])
+                kept_rows.append(chunk.index_select(0, local).cpu().numpy())
+        if keep_all:
+            full.append(chunk)
+        torch.cuda.synchronize(device)
+    kept = {}
+    if want is not None and kept_idx:
+        kept = {"idx": np.concatenate(kept_idx), "rows": np.concatenate(kept_rows)}
+    return store, kept, (torch.cat(full) if keep_all else None)

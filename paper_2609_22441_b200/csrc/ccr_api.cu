@@ -18,7 +18,7 @@ namespace {
 constexpr uint64_t kStoreMagic = 0x43435253544f5245ull;  // "CCRSTORE"
 constexpr uint64_t kWsMagic = 0x4343525753504143ull;     // "CCRWSPAC"
 constexpr int kMaxSmemBytes = 227 * 1024;
-constexpr int kDefaultTile = 512;
+constexpr int kDefaultTile = 256;
 constexpr int kSmemPerSm = 228 * 1024;
 constexpr int kDefaultKeyCap = 4096;
 constexpr int kMaxTile = 4096;
@@ -235,8 +235,8 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   s->req_b = static_cast<int>(req_b);
   s->tile = kDefaultTile;
   s->key_cap = 0;  // automatic
-  s->ws_streamers = 12;
-  s->ws_resolvers = 4;
+  s->ws_streamers = 10;
+  s->ws_resolvers = 6;
   if (cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, d->device) != cudaSuccess || s->n_sms <= 0) {
     cudaGetLastError();
     delete s;

@@ -36,15 +36,19 @@ constexpr long long kNoAuthor = static_cast<long long>(0x8000000000000000ull);  
 // matched edge rows of its found engager slots (rp[s] >= 0 is the row index, < 0 = slot not found)
 // reduced per dim in ascending slot order.  max: strict > on the fp32 values, the winner's 16 bits are
 // kept.  sum: fp32 accumulator from +0, one rounded add per slot, one round-to-nearest-even conversion;
-// a NaN sum is stored as 0x7fff.
-__device__ __forceinline__ uint4 edge2_chunk(unsigned long long reduce_sum_mask, const uint8_t* edge_base, int edge_b,
-                                             int piece, const int (&rp)[4]) {
-  uint4 q[4];
+// a NaN sum is stored as 0x7fff.  Loading and reducing are separate so that a caller can put the loads of
+// several chunks in flight before it reduces the first.
+__device__ __forceinline__ void edge2_load(const uint8_t* edge_base, int edge_b, int piece, const int (&rp)[4],
+                                           uint4 (&q)[4]) {
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
     q[s] = make_uint4(0u, 0u, 0u, 0u);
     if (rp[s] >= 0) q[s] = ldg128(edge_base + static_cast<long long>(rp[s]) * edge_b + piece * 16);
   }
+}
+
+__device__ __forceinline__ uint4 edge2_reduce(unsigned long long reduce_sum_mask, int piece, const int (&rp)[4],
+                                              const uint4 (&q)[4]) {
   float acc[8], bestf[8];
   unsigned short best[8];
 #pragma unroll
@@ -219,9 +223,8 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
   }
   // edge2 section: the matched rows of the found engager slots, reduced per dim in slot order
   if constexpr (SECOND) {
-    for (int i = 0; i < sh.edge_ch; ++i) {
-      const int c = i * 32 + lane, row = c / sh.edge_ch, piece = c - row * sh.edge_ch;
-      int rp[4] = {-1, -1, -1, -1};
+    auto slots_of = [&](int row, int (&rp)[4]) {
+      rp[0] = rp[1] = rp[2] = rp[3] = -1;
       if (row < cnt) {
         const int4 p = s_apos[row];
         rp[0] = p.x;
@@ -229,7 +232,14 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
         rp[2] = p.z;
         rp[3] = p.w;
       }
-      const uint4 v = edge2_chunk(a.reduce_sum_mask, edge_base, sh.edge_b, piece, rp);
+    };
+    for (int i = 0; i < sh.edge_ch; ++i) {
+      const int c = i * 32 + lane, row = c / sh.edge_ch, piece = c - row * sh.edge_ch;
+      int rp[4];
+      slots_of(row, rp);
+      uint4 q[4];
+      edge2_load(edge_base, sh.edge_b, piece, rp, q);
+      const uint4 v = edge2_reduce(a.reduce_sum_mask, piece, rp, q);
       if (row < cnt) st128_stream(out + row * out_b + sh.doc_b + sh.edge_b + piece * 16, v);
     }
   }

@@ -126,15 +126,22 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   }
 
   // ============================ resolvers ============================
+  // All resolver warps walk the same sequence of sub-tiles; warp q fills every n_resolvers-th one on its own
+  // (own bounded wait for the slot, own publish), so several sub-tiles are being resolved at any time.  They
+  // meet on a named barrier only to draw the next chunk and to stage a new request's keys.
   const int gsize = n_threads - n_streamers * 32;
   const int gtid = tid - n_streamers * 32;
+  const int n_resolvers = gsize >> 5;
+  const int rwarp = gtid >> 5;
   const NamedGroup grp(gtid, gsize, kBarGroup);
   uint32_t phase = 0;
-  unsigned it = 0;       // ring slots published so far
-  bool failed = false;
+  unsigned it = 0;       // sub-tiles walked so far (= ring slots handed out)
+  bool failed = false;   // key staging gave up (group-uniform): stop drawing work
+  bool dead = false;     // this warp's wait for a free slot expired: keep walking (barriers!), fill nothing
   int staged_r = -1;     // request whose keys are in shared memory
   StagedKeys keys;
   const long long n_tiles = (a.total + a.tile - 1) / a.tile;
+  constexpr int U = SECOND ? 4 : 8;  // candidates a lane keeps in flight
 
   for (bool more = true; more && !failed;) {
     long long j0, j1;
@@ -181,33 +188,58 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
         staged_r = r;
       }
       for (long long sub = seg; sub < seg_end; sub += a.tile, ++it) {
+        if (static_cast<int>(it % n_resolvers) != rwarp || dead) continue;
         const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_end - sub));
         const int s = it % kWsSlots;
         if (it >= static_cast<unsigned>(kWsSlots) && !mbar_wait_bounded(empty0 + 8 * s, (it / kWsSlots - 1) & 1u)) {
-          failed = true;  // the streamers are gone: every resolver thread times out on the same barrier
-          break;
+          if (lane == 0) atomicExch(a.status, kDevWaitExpired);
+          dead = true;  // the streamers are gone
+          continue;
         }
         int* out_idx = s_idx + s * a.tile;
         int* out_pos = s_pos + s * a.tile;
         int4* out_apos = s_apos + s * a.tile;
-        for (int base = 0; base < n; base += gsize * kUnroll) {
-          int idx[kUnroll];
-          int64_t auth[kUnroll];
+        for (int base = 0; base < n; base += 32 * U) {
+          int idx[U];
+          int64_t auth[U];
 #pragma unroll
-          for (int u = 0; u < kUnroll; ++u) {
-            const int i = base + u * gsize + gtid;
+          for (int u = 0; u < U; ++u) {
+            const int i = base + u * 32 + lane;
             idx[u] = i < n ? __ldg(a.cand_idx + sub + i) : -1;
           }
+          // every id of the U candidates is requested before the first one is used
+          int64_t act[SECOND ? U : 1][4];
+          unsigned types[SECOND ? U : 1];
 #pragma unroll
-          for (int u = 0; u < kUnroll; ++u) {
+          for (int u = 0; u < U; ++u) {
             if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;  // unresolved / out-of-range position
             auth[u] = idx[u] >= 0 ? __ldg(a.author_ids + idx[u]) : -1;
+            if constexpr (SECOND) {
+              act[u][0] = act[u][1] = act[u][2] = act[u][3] = -1;
+              types[u] = 0;
+              if (idx[u] >= 0) {
+                if (a.max_actors == 4) {
+                  const longlong2* ap = reinterpret_cast<const longlong2*>(a.actor_ids + 4LL * idx[u]);
+                  const longlong2 p0 = __ldg(ap), p1 = __ldg(ap + 1);
+                  act[u][0] = p0.x;
+                  act[u][1] = p0.y;
+                  act[u][2] = p1.x;
+                  act[u][3] = p1.y;
+                  types[u] = __ldg(reinterpret_cast<const unsigned*>(a.actor_types + 4LL * idx[u]));
+                } else {
+                  for (int sl = 0; sl < a.max_actors; ++sl) {
+                    const long long e = static_cast<long long>(a.max_actors) * idx[u] + sl;
+                    act[u][sl] = __ldg(a.actor_ids + e);
+                    types[u] |= static_cast<unsigned>(__ldg(a.actor_types + e)) << (8 * sl);
+                  }
+                }
+              }
+            }
           }
-          bool found[kUnroll];
-          int pos[kUnroll];
-          static_assert(kUnroll % 4 == 0, "lookups are interleaved four at a time");
+          bool found[U];
+          int pos[U];
 #pragma unroll
-          for (int h = 0; h < kUnroll; h += 4) {
+          for (int h = 0; h < U; h += 4) {
             const int64_t id4[4] = {auth[h], auth[h + 1], auth[h + 2], auth[h + 3]};
             bool f4[4];
             int p4[4];
@@ -219,40 +251,33 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
             }
           }
 #pragma unroll
-          for (int u = 0; u < kUnroll; ++u) {
-            const int i = base + u * gsize + gtid;
-            if (i >= n) continue;
+          for (int u = 0; u < U; ++u) {
+            const int i = base + u * 32 + lane;
             unsigned m = found[u] ? 1u : 0u;
-            if (SECOND) {
-              int64_t act[4] = {-1, -1, -1, -1};
-              unsigned types = 0;
-              if (idx[u] >= 0) {
-                for (int sl = 0; sl < a.max_actors; ++sl) {
-                  const long long e = static_cast<long long>(a.max_actors) * idx[u] + sl;
-                  act[sl] = __ldg(a.actor_ids + e);
-                  types |= (__ldg(a.actor_types + e) % 3u) << (2 * sl);
-                }
-              }
+            if constexpr (SECOND) {
               bool af[4];
               int ap[4];
-              keys.find_batch<4>(act, af, ap);
+              keys.find_batch<4>(act[u], af, ap);
 #pragma unroll
               for (int sl = 0; sl < 4; ++sl) {
                 if (af[sl]) {
                   m |= 1u << (1 + sl);
-                  m |= 1u << (5 + ((types >> (2 * sl)) & 3u));
+                  m |= 1u << (5 + ((types[u] >> (8 * sl)) & 0xffu) % 3u);
                 } else {
                   ap[sl] = -1;
                 }
               }
-              out_apos[i] = make_int4(ap[0], ap[1], ap[2], ap[3]);
+              if (i < n) out_apos[i] = make_int4(ap[0], ap[1], ap[2], ap[3]);
             }
-            out_idx[i] = idx[u];
-            out_pos[i] = found[u] ? pos[u] : -1;
-            a.out_mask[sub + i] = static_cast<uint8_t>(m);
+            if (i < n) {
+              out_idx[i] = idx[u];
+              out_pos[i] = found[u] ? pos[u] : -1;
+              a.out_mask[sub + i] = static_cast<uint8_t>(m);
+            }
           }
         }
-        if (gtid == 0) {
+        __syncwarp();  // the whole warp's part of the slot is written
+        if (lane == 0) {
           WsSlot d;
           d.sub = sub;
           d.kb = kb;
@@ -261,23 +286,21 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
           d.next = 0;
           d.pad = 0;
           slots[s] = d;
+          mbar_arrive(full0 + 8 * s);
         }
-        grp.sync();  // every resolver's part of the slot is written
-        if (gtid == 0) mbar_arrive(full0 + 8 * s);
       }
-      if (failed) break;
       seg = seg_end;
       ++r;
     }
   }
 
-  // stop slot
-  if (failed) {
-    if (gtid == 0) atomicExch(a.status, kDevWaitExpired);
-  } else {
+  // stop slot: published by the warp whose turn it is
+  if (static_cast<int>(it % n_resolvers) == rwarp && !dead) {
     const int s = it % kWsSlots;
-    if (it >= static_cast<unsigned>(kWsSlots)) failed = !mbar_wait_bounded(empty0 + 8 * s, (it / kWsSlots - 1) & 1u);
-    if (gtid == 0) {
+    bool ok = true;
+    if (it >= static_cast<unsigned>(kWsSlots)) ok = mbar_wait_bounded(empty0 + 8 * s, (it / kWsSlots - 1) & 1u);
+    if (lane == 0) {
+      if (!ok) atomicExch(a.status, kDevWaitExpired);
       WsSlot d;
       d.sub = 0;
       d.kb = 0;
@@ -285,8 +308,10 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
       d.r = 0;
       d.next = 0;
       d.pad = 0;
-      slots[s] = d;
-      mbar_arrive(full0 + 8 * s);
+      if (ok) {
+        slots[s] = d;
+        mbar_arrive(full0 + 8 * s);
+      }
     }
   }
   // the last block to stop drawing tiles zeroes the scheduling words for the next launch

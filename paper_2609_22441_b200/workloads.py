@@ -461,6 +461,22 @@ def doc_feats_chunk(seed: int, first: int, n: int, doc_dim: int, doc_dtype=np.fl
 DOC_CHUNK_ROWS = 1 << 18
 
 
+def doc_feats_chunk_device(seed: int, first: int, n: int, doc_dim: int, device):
+    """Rows [first, first+n) of a production-scale feature matrix, drawn on the device (torch Philox,
+    one generator seed per DOC_DEVICE_CHUNK-row block, ~N(0,1) in fp16).  Input generation only: the bytes
+    it returns are what both the CUDA path and the oracle's sampled rows are taken from."""
+    import torch
+
+    if first % DOC_DEVICE_CHUNK != 0 or n > DOC_DEVICE_CHUNK:
+        raise ValueError("device chunks start on multiples of DOC_DEVICE_CHUNK and hold at most that many rows")
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed) * 1_000_003 + first // DOC_DEVICE_CHUNK)
+    return torch.randn((n, doc_dim), generator=g, device=device, dtype=torch.float32).to(torch.float16)
+
+
+DOC_DEVICE_CHUNK = 1 << 22
+
+
 # --- latency sweep (config 4): viewer templates on a shared store ----------------------
 @dataclass
 class ViewerTemplate:

@@ -49,3 +49,31 @@ def gpu_join(store, db, flags=0):
     assert (rb[:GUARD] == 0xA5).all() and (rb[GUARD + n * out_b:] == 0xA5).all(), "write outside out_rows"
     assert (mb[:GUARD] == 0xA5).all() and (mb[GUARD + n:] == 0xA5).all(), "write outside out_mask"
     return rb[GUARD:GUARD + n * out_b].reshape(n, out_b), mb[GUARD:GUARD + n]
+
+
+def upload_generated_store(B, wl, device=0, keep_rows_of=None, keep_all=False):
+    return B.store_from_generated(wl, device, keep_rows_of, keep_all)
+
+
+def sampled_oracle_rows(wl, kept, J, first_degree_only):
+    """Oracle rows and mask for the flat candidate indices J (ascending) of a workload whose doc features
+    exist on the host only for the sampled docs: the sample is re-expressed as a compact problem (store =
+    the sampled docs, candidates = 0..len(J)-1, same requests) and given to the unmodified oracle."""
+    from oracle import oracle
+
+    s, b = wl.store, wl.batch
+    J = np.asarray(J, dtype=np.int64)
+    docs = b.cand_idx[J].astype(np.int64)
+    ok = (docs >= 0) & (docs < s.n_docs)
+    where = np.searchsorted(kept["idx"], np.where(ok, docs, kept["idx"][0]))
+    assert np.array_equal(kept["idx"][where][ok], docs[ok])
+    feats = kept["rows"][where]
+    cand = np.where(ok, np.arange(len(J)), -1).astype(np.int32)
+    safe = np.where(ok, docs, 0)
+    req_of = np.searchsorted(b.cand_offsets, J, side="right") - 1
+    co = np.searchsorted(req_of, np.arange(b.n_req + 1), side="left").astype(np.int64)
+    return oracle.join(
+        feats, s.author_ids[safe], b.edge_keys, b.edge_feats, b.edge_offsets, cand, co, req_feats=b.req_feats,
+        actor_ids=None if s.actor_ids is None else s.actor_ids[safe],
+        actor_types=None if s.actor_types is None else s.actor_types[safe],
+        reduce_sum_mask=s.reduce_sum_mask, first_degree_only=first_degree_only, n_threads=4)
