@@ -160,6 +160,47 @@ ccr_status ccr_join_batch_host(const ccr_docstore* store, ccr_workspace* ws,
                                void* out_rows, uint8_t* out_mask, /* HOST */
                                uint32_t flags, void* stream);
 
+/* The join for callers that cannot allocate device memory.  (The paper has no counterpart: this entry exists
+ * for embedding the library, not for the method.)
+ *
+ * Who that is: code that runs after a serving process has handed all of its device memory to its own pool
+ * and must not touch the CUDA allocator again — the paper's server keeps only a few hundred MB of headroom
+ * beside the index and saw allocations fail under fragmentation (Section 6.3.1) — and request handlers on a
+ * latency budget, for which cudaMalloc / cudaFree mean a device-wide synchronisation and an unbounded
+ * stall.  Such a caller creates the store once at start-up (that does allocate) and then uses this call
+ * per request batch: it takes the request payload from HOST memory (pinned memory makes the copies
+ * asynchronous), writes rows and mask to the caller's DEVICE buffers, and calls neither cudaMalloc nor
+ * cudaFree nor any allocating library routine.
+ *
+ * What it uses instead: one fixed 16 MiB block of device memory that belongs to the library image (every GPU
+ * that loads the library holds it until the process exits).  The block carries the kernel's status and
+ * scheduling words and the device copy of the payload (keys, edge rows, offsets, candidate positions, request
+ * rows, each rounded up to 256 bytes).  ccr_static_payload_capacity() returns the bytes available to the
+ * payload; a batch that needs more is refused with CCR_ERR_UNSUPPORTED before anything is enqueued.
+ * CCR_FLAG_VALIDATE is not accepted here (CCR_ERR_UNSUPPORTED).
+ *
+ * Sharing: all calls in a process use the same block on a device and it keeps the previous call's contents.
+ * Each call re-clears the control words on `stream` before use and overwrites the payload area, so calls on
+ * ONE stream are safe back to back; calls that can overlap on the GPU (different streams, or another
+ * thread) race on the block and must be serialised by the caller.  Results, flags and row layout are
+ * those of ccr_join_batch on the same inputs.
+ *
+ * First use on a device looks up the block's device address (once per device, with that device current);
+ * make that first call outside any stream capture.                                                       */
+size_t     ccr_static_payload_capacity(void);
+ccr_status ccr_join_payload_static(const ccr_docstore* store,
+                                   int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                                   int64_t total_edges,          /* = edge_offsets[n_req]                   */
+                                   const int64_t* edge_keys,     /* HOST [total_edges]                      */
+                                   const void*    edge_feats,    /* HOST [total_edges, edge_dim]            */
+                                   const int64_t* edge_offsets,  /* HOST [n_req + 1]                        */
+                                   const int32_t* cand_idx,      /* HOST [total_cands]                      */
+                                   const int64_t* cand_offsets,  /* HOST [n_req + 1]                        */
+                                   const void*    req_feats,     /* HOST [n_req, req_dim] or NULL           */
+                                   void*          out_rows,      /* DEVICE [total_cands, out_row_bytes]     */
+                                   uint8_t*       out_mask,      /* DEVICE [total_cands]                    */
+                                   uint32_t flags, void* stream);
+
 /* Synchronise `stream` and report the store's device-side status word: CCR_OK, or
  * CCR_ERR_DEVICE_WAIT if a kernel gave up a bounded wait for a shared-memory bulk copy since the
  * last call (the affected rows of that launch were not written).  Clears the word.                 */

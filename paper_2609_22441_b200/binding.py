@@ -41,6 +41,7 @@ EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
     "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
+    "ccr_static_payload_capacity", "ccr_join_payload_static",
 )
 
 
@@ -97,6 +98,10 @@ def lib() -> ctypes.CDLL:
     L.ccr_workspace_free.argtypes = [vp]
     L.ccr_join_batch_host.restype = ctypes.c_int
     L.ccr_join_batch_host.argtypes = [vp, vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
+    L.ccr_static_payload_capacity.restype = ctypes.c_size_t
+    L.ccr_static_payload_capacity.argtypes = []
+    L.ccr_join_payload_static.restype = ctypes.c_int
+    L.ccr_join_payload_static.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
     L.ccr_docstore_device_status.restype = ctypes.c_int
     L.ccr_docstore_device_status.argtypes = [vp, vp]
     L.ccr_docstore_set_tuning.restype = ctypes.c_int
@@ -291,6 +296,19 @@ def ccr_join_batch_host(store: Docstore, ws: Workspace, n_req: int, total_cands:
                                    _ptr(cand_idx), _ptr(cand_offsets), _ptr(req_feats), _ptr(out_rows),
                                    _ptr(out_mask), int(flags), _stream_ptr(stream))
     _check(st, "ccr_join_batch_host")
+    return st
+
+
+def ccr_join_payload_static(store: Docstore, n_req: int, total_cands: int, max_edge_len: int, total_edges: int,
+                            edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets, req_feats,
+                            out_rows, out_mask, flags: int = 0, stream=None) -> int:
+    """Raw call of the entry for callers that must not allocate: HOST payload (numpy arrays or pinned CPU
+    tensors), DEVICE outputs; the library stages the payload in its fixed device block."""
+    st = lib().ccr_join_payload_static(store.handle, int(n_req), int(total_cands), int(max_edge_len),
+                                       int(total_edges), _ptr(edge_keys), _ptr(edge_feats), _ptr(edge_offsets),
+                                       _ptr(cand_idx), _ptr(cand_offsets), _ptr(req_feats), _ptr(out_rows),
+                                       _ptr(out_mask), int(flags), _stream_ptr(stream))
+    _check(st, "ccr_join_payload_static")
     return st
 
 

@@ -8,6 +8,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "ccr_join.cuh"
@@ -583,6 +584,99 @@ ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t 
     return CCR_ERR_CUDA;
   }
   return CCR_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// ccr_join_payload_static: the join for callers that must not allocate (declared in ccr.h).
+//
+// Everything the call needs beyond the caller's buffers lives in one fixed block of device memory that is
+// part of the library image: the kernel's status and scheduling words and the device copy of the request
+// payload.  In host code the array's name is only a stand-in for the device symbol, so its device address
+// is looked up once per device with cudaGetSymbolAddress and that pointer is what kernels and copies get.
+constexpr size_t kStaticScratchBytes = 16u << 20;  // 16 MiB, held by every GPU that loads the library
+constexpr size_t kStaticControlBytes = 256;        // status + scheduling words in front of the payload
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_ptr[kMaxDevices] = {};
+std::mutex g_static_mutex;
+
+// Device address of the scratch block on `device` (which must be current); resolved on first use.
+ccr_status static_scratch(int device, unsigned char** out) {
+  if (device < 0 || device >= kMaxDevices) return CCR_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_ptr[device] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
+    g_static_ptr[device] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_ptr[device];
+  return CCR_OK;
+}
+
+inline size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+}  // namespace
+
+size_t ccr_static_payload_capacity(void) { return kStaticScratchBytes - kStaticControlBytes; }
+
+ccr_status ccr_join_payload_static(const ccr_docstore* s, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                                   int64_t total_edges, const int64_t* edge_keys, const void* edge_feats,
+                                   const int64_t* edge_offsets, const int32_t* cand_idx, const int64_t* cand_offsets,
+                                   const void* req_feats, void* out_rows, uint8_t* out_mask, uint32_t flags,
+                                   void* stream) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  if (n_req < 0 || total_cands < 0 || total_edges < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
+  if (n_req == 0 || total_cands == 0) return (n_req == 0 && total_cands != 0) ? CCR_ERR_INVALID_ARG : CCR_OK;
+  if (!edge_offsets || !cand_offsets || !cand_idx || !out_rows || !out_mask) return CCR_ERR_INVALID_ARG;
+  if (total_edges > 0 && (!edge_keys || !edge_feats)) return CCR_ERR_INVALID_ARG;
+  if (s->req_b > 0 && !req_feats) return CCR_ERR_INVALID_ARG;
+  if (flags & CCR_FLAG_VALIDATE) return CCR_ERR_UNSUPPORTED;  // validation synchronises and uses the store's own words
+
+  // device copy of the payload, every piece on a 256-byte boundary behind the control words
+  const size_t n_off = static_cast<size_t>(n_req) + 1;
+  const size_t sz_keys = static_cast<size_t>(total_edges) * 8, sz_feats = static_cast<size_t>(total_edges) * s->edge_b;
+  const size_t sz_off = n_off * 8, sz_idx = static_cast<size_t>(total_cands) * 4;
+  const size_t sz_req = static_cast<size_t>(n_req) * s->req_b;
+  const size_t o_keys = kStaticControlBytes, o_feats = o_keys + round256(sz_keys), o_eo = o_feats + round256(sz_feats);
+  const size_t o_idx = o_eo + round256(sz_off), o_co = o_idx + round256(sz_idx), o_req = o_co + round256(sz_off);
+  const size_t need = o_req + round256(sz_req);
+  if (need > kStaticScratchBytes) return CCR_ERR_UNSUPPORTED;  // payload larger than the fixed block
+
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  unsigned char* base = nullptr;
+  const ccr_status rs = static_scratch(s->desc.device, &base);
+  if (rs != CCR_OK) return rs;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool ok = cudaMemsetAsync(base, 0, kStaticControlBytes, st) == cudaSuccess;  // the words must start at zero
+  if (total_edges > 0) {
+    ok = ok && cudaMemcpyAsync(base + o_keys, edge_keys, sz_keys, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(base + o_feats, edge_feats, sz_feats, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(base + o_eo, edge_offsets, sz_off, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(base + o_idx, cand_idx, sz_idx, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(base + o_co, cand_offsets, sz_off, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (sz_req > 0) ok = ok && cudaMemcpyAsync(base + o_req, req_feats, sz_req, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return CCR_ERR_CUDA;
+  }
+  // a view of the store whose status / scheduling words are the ones in the fixed block
+  ccr_docstore view = *s;
+  view.status = reinterpret_cast<int*>(base);
+  view.launches = 0;  // always the first pair of scheduling words
+  const ccr_status js = ccr_join_batch(&view, n_req, total_cands, max_edge_len,
+                                       reinterpret_cast<const int64_t*>(base + o_keys), base + o_feats,
+                                       reinterpret_cast<const int64_t*>(base + o_eo),
+                                       reinterpret_cast<const int32_t*>(base + o_idx),
+                                       reinterpret_cast<const int64_t*>(base + o_co),
+                                       s->req_b > 0 ? base + o_req : nullptr, out_rows, out_mask, flags, stream);
+  const_cast<ccr_docstore*>(s)->launches += view.launches;
+  return js;
 }
 
 }  // extern "C"
