@@ -53,6 +53,8 @@ def parse_args():
                         "store, first-degree; 3b the same on candidates sorted by author (merge path); 3s production scale, "
                         "second-degree; 4 single-request latency sweep on the production-scale store")
     p.add_argument("--sweep-requests", type=int, default=1000, help="requests per cell of the latency sweep")
+    p.add_argument("--c3-docs", type=int, default=50_000_000, help="store size of configs 3/3b/3s (smaller for profiler captures)")
+    p.add_argument("--c3-requests", type=int, default=256, help="requests of configs 3/3b/3s (smaller for profiler captures)")
     p.add_argument("--e2e-steps", type=int, default=0, help="0 = min(steps, 10)")
     p.add_argument("--flags", type=int, default=0, help="extra CCR_FLAG_* bits (experiments)")
     p.add_argument("--tile", type=int, default=0, help="candidates per ring slot (0 = library default)")
@@ -65,16 +67,18 @@ def parse_args():
     return p.parse_args()
 
 
-def make_workload(config: str, rank: int):
+def make_workload(config: str, rank: int, c3_docs: int = 50_000_000, c3_requests: int = 256):
     """(workload, extra join flags) of a benchmark configuration; rank shifts the seed so replicas differ."""
     from paper_2609_22441_b200 import binding as B
+    from paper_2609_22441_b200 import replicas
     from paper_2609_22441_b200 import workloads as W
 
     if config == "1":
-        return W.config1(seed=W.config_seed(1, 0) + 17 * rank), 0
+        return W.config1(seed=W.config_seed(1, 0) + replicas.rank_seed_offset(rank)), 0
     if config == "2b":
-        return W.config1(seed=W.config_seed(2, 1) + 17 * rank, second_degree=True), 0
-    wl = W.config3(seed=W.config_seed(3, 0) + 17 * rank)
+        return W.config1(seed=W.config_seed(2, 1) + replicas.rank_seed_offset(rank), second_degree=True), 0
+    wl = W.config3(seed=W.config_seed(3, 0) + replicas.rank_seed_offset(rank), n_docs=c3_docs, n_req=c3_requests,
+                   extra_pools=160 if c3_docs >= 50_000_000 else 0)
     if config == "3":
         return wl, B.CCR_FLAG_FIRST_DEGREE_ONLY
     if config == "3b":
@@ -372,30 +376,22 @@ def main():
         dist.barrier()
     B.lib()
 
+    from paper_2609_22441_b200 import replicas
+
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
+        replicas.barrier(dev)
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(x, dev)
 
     def sum_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        return float(t.item())
+        return replicas.sum_over_ranks(x, dev)
 
     if args.config == "4":
         if rank == 0:
             latency_sweep(args, B, local_rank)
         return
-    wl, cfg_flags = make_workload(args.config, rank)
+    wl, cfg_flags = make_workload(args.config, rank, args.c3_docs, args.c3_requests)
     b = wl.batch
     second = wl.store.max_actors > 0
     kept = None
@@ -435,16 +431,14 @@ def main():
     ev1.record()
     barrier()
     launches = store.launch_count() - launches0
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    value, ms_per_step = replicas.job_throughput(float(C), ev0.elapsed_time(ev1), args.steps, dev)
     # keep the same kernel running until the loaded window is long enough for clock samples
     while not args.timed_only and time.time() - t_wall0 < 1.2:
         for i in range(50):
             step(i)
         torch.cuda.synchronize(dev)
     t_wall1 = time.time()
-    ms_per_step = ms_total / max(args.steps, 1)
     total_cands_job = sum_over_ranks(float(C))
-    value = total_cands_job / (ms_per_step * 1e-3)
     if store.device_status() != B.CCR_OK:
         raise SystemExit("device status not clean after the timed region")
 
