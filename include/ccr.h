@@ -78,9 +78,9 @@ enum {
                                            row streaming) instead of the warp-specialised kernel      */
 };
 
-/* Create an empty store on desc->device.  Allocates doc_feats [n_docs, doc_dim], author_ids
- * int64[n_docs] and, when max_actors > 0, actor_ids int64[n_docs, max_actors] and actor_types
- * uint8[n_docs, max_actors].  Rows are uninitialised until uploaded.  The required bytes are compared
+/* Create an empty store on desc->device.  Allocates doc_feats [n_docs, doc_dim] and author ids
+ * int64[n_docs]; when max_actors > 0 the ids of a document (author, engagers, types) are kept in one
+ * 64-byte record instead, plus a 16 MiB staging block for uploads.  Rows are uninitialised until uploaded.  The required bytes are compared
  * with the device's free memory before anything is allocated (CCR_ERR_OOM).  HOST call.            */
 ccr_status ccr_docstore_create(const ccr_docstore_desc* desc, ccr_docstore** out);
 
@@ -208,11 +208,13 @@ ccr_status ccr_docstore_device_status(ccr_docstore* store, void* stream);
 
 /* Tuning knobs of the join kernels; a field that is 0 keeps the store's current value.              */
 typedef struct {
-  int32_t tile_cands;         /* candidates per ring slot / search-copy phase pair: multiple of 256, <= 4096 */
+  int32_t tile_cands;         /* candidates per ring slot / search-copy phase pair: multiple of 256, <= 4096;
+                                 unset = 256 (warp-specialised kernel) / 1024 (two-phase kernel)               */
   int32_t key_capacity;       /* most keys (or sampled keys) a block stages in shared memory per request;
                                  unset = as many as fit (warp-specialised kernel) or 4096 (the others)       */
   int32_t ws_streamers;       /* warp-specialised kernel: row-streaming warps per block (1..14)              */
-  int32_t ws_resolvers;       /* warp-specialised kernel: search warps per block (1..8); sum <= 16           */
+  int32_t ws_resolvers;       /* warp-specialised kernel: search warps per block (1..8); sum <= 16; set both
+                                 or neither (unset = 12 + 4, or 11 + 5 for second-degree joins)              */
   int32_t blocks_per_sm;      /* two-phase kernel: cap on resident blocks per SM (1..8)                      */
 } ccr_tuning;
 ccr_status ccr_docstore_set_tuning(ccr_docstore* store, const ccr_tuning* tuning);

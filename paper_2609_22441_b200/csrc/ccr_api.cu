@@ -19,10 +19,12 @@ namespace {
 constexpr uint64_t kStoreMagic = 0x43435253544f5245ull;  // "CCRSTORE"
 constexpr uint64_t kWsMagic = 0x4343525753504143ull;     // "CCRWSPAC"
 constexpr int kMaxSmemBytes = 227 * 1024;
-constexpr int kDefaultTile = 256;
+constexpr int kDefaultTileWs = 256;        // candidates per ring slot of the warp-specialised kernel
+constexpr int kDefaultTileTwoPhase = 1024; // candidates per search/copy phase pair of the two-phase kernel
 constexpr int kSmemPerSm = 228 * 1024;
 constexpr int kDefaultKeyCap = 4096;
 constexpr int kMaxTile = 4096;
+constexpr size_t kStageBytes = 16u << 20;  // staging block of second-degree stores (ids uploaded from the host)
 constexpr int kSchedRegions = 64;                    // launches of one store that may be in flight at once
 constexpr int kStatusInts = 4 + 2 * kSchedRegions;   // [0] wait expiry, [1] validation code, [4..] scheduling words
 
@@ -50,9 +52,9 @@ struct ccr_docstore {
   ccr_docstore_desc desc;
   int doc_b, edge_b, req_b;  // section widths in bytes
   uint8_t* doc_feats;
-  int64_t* author_ids;
-  int64_t* actor_ids;
-  uint8_t* actor_types;
+  int64_t* author_ids;     // first-degree stores
+  ccr::IdRec* id_recs;     // second-degree stores: author, engagers and types of a doc in one 64-byte record
+  uint8_t* stage;          // second-degree stores: device staging for host-sourced id uploads (kStageBytes)
   int* status;        // device: [0] wait expiry, [1] validation code
   int* status_host;   // pinned host copy
   int tile;
@@ -109,9 +111,27 @@ __global__ void validate_kernel(const ccr::JoinArgs a, int check_sorted, int* co
     for (int64_t j = c0 + 1 + threadIdx.x; j < c1; j += blockDim.x) {
       const int p = a.cand_idx[j - 1], q = a.cand_idx[j];
       const bool pin = p >= 0 && p < a.n_docs, qin = q >= 0 && q < a.n_docs;
-      const long long ap = pin ? a.author_ids[p] : ccr::kNoAuthor;
-      const long long aq = qin ? a.author_ids[q] : ccr::kNoAuthor;
+      const long long ap = pin ? ccr::load_author(a, p) : ccr::kNoAuthor;
+      const long long aq = qin ? ccr::load_author(a, q) : ccr::kNoAuthor;
       if (ap > aq) atomicCAS(code, 0, 4);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Upload path of second-degree stores: scatter the caller's separate id arrays into the packed records.
+// A null source leaves its fields untouched.
+__global__ void pack_ids_kernel(ccr::IdRec* recs, long long n, int max_actors, const int64_t* author_ids,
+                                const int64_t* actor_ids, const uint8_t* actor_types) {
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    ccr::IdRec& r = recs[i];
+    if (author_ids) r.author = author_ids[i];
+    if (actor_ids) {
+      for (int s = 0; s < 4; ++s) r.actor[s] = s < max_actors ? actor_ids[i * max_actors + s] : -1;
+    }
+    if (actor_types) {
+      for (int s = 0; s < 4; ++s) r.type[s] = s < max_actors ? actor_types[i * max_actors + s] : 0;
     }
   }
 }
@@ -222,7 +242,7 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   if (!scope.ok) return CCR_ERR_CUDA;
 
   const size_t n = static_cast<size_t>(d->n_docs);
-  const size_t need = n * doc_b + n * 8 + (d->max_actors ? n * d->max_actors * 9 : 0) + 4096;
+  const size_t need = n * doc_b + (d->max_actors ? n * sizeof(ccr::IdRec) + kStageBytes : n * 8) + 4096;
   size_t free_b = 0, total_b = 0;
   if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return CCR_ERR_CUDA;
   if (need > free_b) return CCR_ERR_OOM;
@@ -234,10 +254,10 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   s->doc_b = static_cast<int>(doc_b);
   s->edge_b = static_cast<int>(edge_b);
   s->req_b = static_cast<int>(req_b);
-  s->tile = kDefaultTile;
+  s->tile = 0;  // automatic: kDefaultTileWs / kDefaultTileTwoPhase
   s->key_cap = 0;  // automatic
-  s->ws_streamers = 10;
-  s->ws_resolvers = 6;
+  s->ws_streamers = 0;  // automatic: 12 + 4 (first-degree joins), 11 + 5 (second-degree joins)
+  s->ws_resolvers = 0;
   if (cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, d->device) != cudaSuccess || s->n_sms <= 0) {
     cudaGetLastError();
     delete s;
@@ -246,10 +266,11 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   bool ok = true;
   // n == 0 still allocates a token block so that every pointer is valid and aligned
   ok = ok && cudaMalloc(&s->doc_feats, n * doc_b + 256) == cudaSuccess;
-  ok = ok && cudaMalloc(&s->author_ids, n * 8 + 256) == cudaSuccess;
   if (d->max_actors > 0) {
-    ok = ok && cudaMalloc(&s->actor_ids, n * d->max_actors * 8 + 256) == cudaSuccess;
-    ok = ok && cudaMalloc(&s->actor_types, n * d->max_actors + 256) == cudaSuccess;
+    ok = ok && cudaMalloc(&s->id_recs, n * sizeof(ccr::IdRec) + 256) == cudaSuccess;
+    ok = ok && cudaMalloc(&s->stage, kStageBytes) == cudaSuccess;
+  } else {
+    ok = ok && cudaMalloc(&s->author_ids, n * 8 + 256) == cudaSuccess;
   }
   ok = ok && cudaMalloc(&s->status, kStatusInts * sizeof(int)) == cudaSuccess;
   ok = ok && cudaMemset(s->status, 0, kStatusInts * sizeof(int)) == cudaSuccess;
@@ -259,8 +280,8 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
     cudaGetLastError();
     cudaFree(s->doc_feats);
     cudaFree(s->author_ids);
-    cudaFree(s->actor_ids);
-    cudaFree(s->actor_types);
+    cudaFree(s->id_recs);
+    cudaFree(s->stage);
     cudaFree(s->status);
     if (s->status_host) cudaFreeHost(s->status_host);
     delete s;
@@ -277,8 +298,8 @@ ccr_status ccr_docstore_free(ccr_docstore* s) {
   s->magic = 0;
   cudaFree(s->doc_feats);
   cudaFree(s->author_ids);
-  cudaFree(s->actor_ids);
-  cudaFree(s->actor_types);
+  cudaFree(s->id_recs);
+  cudaFree(s->stage);
   cudaFree(s->status);
   cudaFreeHost(s->status_host);
   delete s;
@@ -299,9 +320,41 @@ ccr_status ccr_docstore_upload(ccr_docstore* s, int64_t first_doc, int64_t n, co
   const int ma = s->desc.max_actors;
   bool ok = true;
   if (doc_feats) ok = ok && cudaMemcpyAsync(s->doc_feats + uf * s->doc_b, doc_feats, un * s->doc_b, kind, st) == cudaSuccess;
-  if (author_ids) ok = ok && cudaMemcpyAsync(s->author_ids + uf, author_ids, un * 8, kind, st) == cudaSuccess;
-  if (ma > 0 && actor_ids) ok = ok && cudaMemcpyAsync(s->actor_ids + uf * ma, actor_ids, un * ma * 8, kind, st) == cudaSuccess;
-  if (ma > 0 && actor_types) ok = ok && cudaMemcpyAsync(s->actor_types + uf * ma, actor_types, un * ma, kind, st) == cudaSuccess;
+  if (ma == 0) {
+    if (author_ids) ok = ok && cudaMemcpyAsync(s->author_ids + uf, author_ids, un * 8, kind, st) == cudaSuccess;
+  } else if (author_ids || actor_ids || actor_types) {
+    // second-degree store: the ids go into the packed records.  Device sources are packed in place; host
+    // sources pass through the store's staging block, a chunk at a time (stream order keeps the block safe).
+    const size_t per_row = 8 + static_cast<size_t>(ma) * 9;
+    const size_t chunk = src_on_device ? un : (kStageBytes - 4096) / per_row;
+    for (size_t o = 0; o < un && ok; o += chunk) {
+      const size_t m = un - o < chunk ? un - o : chunk;
+      const int64_t* d_auth = author_ids ? author_ids + o : nullptr;
+      const int64_t* d_act = actor_ids ? actor_ids + o * ma : nullptr;
+      const uint8_t* d_typ = actor_types ? actor_types + o * ma : nullptr;
+      if (!src_on_device) {
+        uint8_t* p = s->stage;
+        if (author_ids) {
+          ok = ok && cudaMemcpyAsync(p, d_auth, m * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+          d_auth = reinterpret_cast<const int64_t*>(p);
+          p += (m * 8 + 255) & ~static_cast<size_t>(255);
+        }
+        if (actor_ids) {
+          ok = ok && cudaMemcpyAsync(p, d_act, m * ma * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+          d_act = reinterpret_cast<const int64_t*>(p);
+          p += (m * ma * 8 + 255) & ~static_cast<size_t>(255);
+        }
+        if (actor_types) {
+          ok = ok && cudaMemcpyAsync(p, d_typ, m * ma, cudaMemcpyHostToDevice, st) == cudaSuccess;
+          d_typ = p;
+        }
+      }
+      const unsigned blocks = static_cast<unsigned>((m + 255) / 256 < 4096 ? (m + 255) / 256 : 4096);
+      pack_ids_kernel<<<blocks, 256, 0, st>>>(s->id_recs + uf + o, static_cast<long long>(m), ma, d_auth, d_act, d_typ);
+      s->launches++;
+      ok = ok && cudaGetLastError() == cudaSuccess;
+    }
+  }
   if (!ok) {
     cudaGetLastError();
     return CCR_ERR_CUDA;
@@ -322,6 +375,7 @@ ccr_status ccr_docstore_set_tuning(ccr_docstore* s, const ccr_tuning* t) {
     return CCR_ERR_INVALID_ARG;
   const int st = t->ws_streamers > 0 ? t->ws_streamers : s->ws_streamers;
   const int rs = t->ws_resolvers > 0 ? t->ws_resolvers : s->ws_resolvers;
+  if ((st > 0) != (rs > 0)) return CCR_ERR_INVALID_ARG;  // the warp split is set as a pair
   if (st > 14 || rs > 8 || (st + rs) * 32 > ccr::kWsMaxThreads) return CCR_ERR_INVALID_ARG;
   if (t->blocks_per_sm > 8) return CCR_ERR_INVALID_ARG;
   if (t->tile_cands > 0) s->tile = t->tile_cands;
@@ -378,13 +432,14 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
   // warp-specialised kernel
   const bool use_ws = !merge && !(flags & CCR_FLAG_TWO_PHASE);
   auto smem_for = [&](int t, int cap) -> size_t {
-    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, cap).bytes)
+    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, cap, n_req <= ccr::kWsMaxCachedReq ? n_req : 0).bytes)
                   : static_cast<size_t>(ccr::TileLayout(t, second, merge, cap).bytes);
   };
   // Keys staged per request.  The warp-specialised kernel runs one block per SM, so by default it stages
   // as many keys as fit next to its ring (whole lists of up to ~20,000 ids); the kernels that keep several
   // blocks per SM default to kDefaultKeyCap.  A configured key_capacity overrides both.
-  int tile = s->tile;
+  const int tile_cfg = s->tile > 0 ? s->tile : (use_ws ? kDefaultTileWs : kDefaultTileTwoPhase);
+  int tile = tile_cfg;
   int key_cap;
   if (flags & CCR_FLAG_FORCE_GLOBAL) {
     key_cap = 0;
@@ -398,7 +453,7 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
     // shrink the ring first; if the longest list still does not fit, stage a sampled top of the tree
     while (tile > 256 && smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) tile -= 256;
     if (smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) {
-      tile = s->tile;
+      tile = tile_cfg;
       key_cap = kDefaultKeyCap;
     }
   }
@@ -410,8 +465,7 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
   ccr::JoinArgs a;
   a.doc_feats = s->doc_feats;
   a.author_ids = s->author_ids;
-  a.actor_ids = s->actor_ids;
-  a.actor_types = s->actor_types;
+  a.id_recs = s->id_recs;
   a.n_docs = s->desc.n_docs;
   a.max_actors = s->desc.max_actors;
   a.reduce_sum_mask = s->desc.reduce_sum_mask;
@@ -462,7 +516,9 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
     // dynamic chunk scheduling through a pair of device words; each launch takes the next pair in turn, so
     // up to kSchedRegions launches of one store may be in flight at once (on any streams)
     if (!(flags & CCR_FLAG_STATIC_SPLIT)) a.sched = s->status + 4 + 2 * static_cast<int>(s->launches % kSchedRegions);
-    fn<<<static_cast<unsigned>(blocks), (s->ws_streamers + s->ws_resolvers) * 32, smem, st>>>(a, s->ws_streamers);
+    const int n_str = s->ws_streamers > 0 ? s->ws_streamers : (second ? 11 : 12);
+    const int n_res = s->ws_resolvers > 0 ? s->ws_resolvers : (second ? 5 : 4);
+    fn<<<static_cast<unsigned>(blocks), (n_str + n_res) * 32, smem, st>>>(a, n_str);
   } else {
     // persistent two-phase kernel: as many blocks as stay resident, each with at least 256 candidates
     const KernelFn fn = merge ? v.merge : (second ? v.second : v.first);

@@ -18,13 +18,23 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr int kDevOk = 0;
 constexpr int kDevWaitExpired = 1;
 
+// Ids of one document of a second-degree store, packed so that one 64-byte aligned access (two sectors)
+// brings everything a lookup needs: a random 8-byte read costs HBM about as much as 100+ streamed bytes,
+// and author, engagers and types in three arrays would be three such reads per candidate.
+struct __align__(64) IdRec {
+  long long author;
+  long long actor[4];   // empty slot = negative
+  uint8_t type[4];
+  uint8_t pad[20];
+};
+static_assert(sizeof(IdRec) == 64, "one record per 64-byte line");
+
 // Everything a join launch needs, passed by value as the kernel argument.
 struct JoinArgs {
   // store
   const uint8_t* doc_feats;
-  const int64_t* author_ids;
-  const int64_t* actor_ids;   // [n_docs, max_actors] or null
-  const uint8_t* actor_types; // [n_docs, max_actors] or null
+  const int64_t* author_ids;  // first-degree stores: int64[n_docs]; null when id_recs is used
+  const IdRec* id_recs;       // second-degree stores: one packed record per document; else null
   long long n_docs;
   int max_actors;
   unsigned long long reduce_sum_mask;
@@ -102,6 +112,21 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 }
 
 __device__ __forceinline__ uint4 ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+
+// Author id of the document at position idx (0 <= idx < n_docs).
+__device__ __forceinline__ long long load_author(const JoinArgs& a, int idx) {
+  return a.id_recs != nullptr ? __ldg(&a.id_recs[idx].author) : __ldg(a.author_ids + idx);
+}
+// Engager ids and types (one byte per slot, packed little-endian) of the document at position idx.
+__device__ __forceinline__ void load_actors(const JoinArgs& a, int idx, long long (&act)[4], unsigned& types) {
+  const uint4* r = reinterpret_cast<const uint4*>(a.id_recs + idx);
+  const uint4 w0 = __ldg(r), w1 = __ldg(r + 1), w2 = __ldg(r + 2);  // author|a0, a1|a2, a3|types
+  act[0] = static_cast<long long>(w0.z | (static_cast<unsigned long long>(w0.w) << 32));
+  act[1] = static_cast<long long>(w1.x | (static_cast<unsigned long long>(w1.y) << 32));
+  act[2] = static_cast<long long>(w1.z | (static_cast<unsigned long long>(w1.w) << 32));
+  act[3] = static_cast<long long>(w2.x | (static_cast<unsigned long long>(w2.y) << 32));
+  types = w2.z;
+}
 
 // Output rows are written once and never read back by the kernel: streaming (evict-first) stores keep
 // them from displacing the keys, edge tables and id arrays that live in L2.

@@ -49,47 +49,42 @@ __device__ __forceinline__ void edge2_load(const uint8_t* edge_base, int edge_b,
 
 __device__ __forceinline__ uint4 edge2_reduce(unsigned long long reduce_sum_mask, int piece, const int (&rp)[4],
                                               const uint4 (&q)[4]) {
-  float acc[8], bestf[8];
-  unsigned short best[8];
+  // two fp16 dims per 32-bit word.  max: compare in fp16 (the same order as the fp32 values, conversions
+  // being exact) and keep the winner's bits with a bit select; sum: fp32 accumulators.
+  unsigned best[4] = {0u, 0u, 0u, 0u};
+  float2 acc[4];
 #pragma unroll
-  for (int h = 0; h < 8; ++h) {
-    acc[h] = 0.0f;
-    bestf[h] = 0.0f;
-    best[h] = 0;
-  }
+  for (int w = 0; w < 4; ++w) acc[w] = make_float2(0.0f, 0.0f);
   bool any = false;
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
     if (rp[s] >= 0) {
-      const unsigned w[4] = {q[s].x, q[s].y, q[s].z, q[s].w};
+      const unsigned v[4] = {q[s].x, q[s].y, q[s].z, q[s].w};
 #pragma unroll
-      for (int h = 0; h < 8; ++h) {
-        const unsigned short bits = static_cast<unsigned short>((w[h >> 1] >> (16 * (h & 1))) & 0xffffu);
-        const float f = __half2float(__ushort_as_half(bits));
-        acc[h] = __fadd_rn(acc[h], f);  // one rounded fp32 add per found slot, never fused
-        if (!any || f > bestf[h]) {     // strict >: the earlier slot keeps a tie
-          bestf[h] = f;
-          best[h] = bits;
-        }
+      for (int w = 0; w < 4; ++w) {
+        const __half2 hv = *reinterpret_cast<const __half2*>(&v[w]);
+        const float2 f = __half22float2(hv);
+        acc[w].x = __fadd_rn(acc[w].x, f.x);  // one rounded fp32 add per found slot, never fused
+        acc[w].y = __fadd_rn(acc[w].y, f.y);
+        // strict >: the earlier slot keeps a tie; the first found slot always takes over
+        const unsigned gt = any ? __hgt2_mask(hv, *reinterpret_cast<const __half2*>(&best[w])) : 0xffffffffu;
+        best[w] = (v[w] & gt) | (best[w] & ~gt);
       }
       any = true;
     }
   }
-  unsigned short res[8];
+  const unsigned sum8 = static_cast<unsigned>(reduce_sum_mask >> ((piece * 8) & 63)) & 0xffu;
+  unsigned res[4];
 #pragma unroll
-  for (int h = 0; h < 8; ++h) {
-    const int d = piece * 8 + h;
-    const bool is_sum = (reduce_sum_mask >> (d & 63)) & 1ull;
-    unsigned short sum_bits = __half_as_ushort(__float2half_rn(acc[h]));
-    if (acc[h] != acc[h]) sum_bits = 0x7fffu;
-    res[h] = any ? (is_sum ? sum_bits : best[h]) : static_cast<unsigned short>(0);
+  for (int w = 0; w < 4; ++w) {
+    const __half2 hs = __floats2half2_rn(acc[w].x, acc[w].y);
+    unsigned sb = *reinterpret_cast<const unsigned*>(&hs);
+    if (acc[w].x != acc[w].x) sb = (sb & 0xffff0000u) | 0x7fffu;
+    if (acc[w].y != acc[w].y) sb = (sb & 0x0000ffffu) | 0x7fff0000u;
+    const unsigned sel = (((sum8 >> (2 * w)) & 1u) ? 0x0000ffffu : 0u) | (((sum8 >> (2 * w + 1)) & 1u) ? 0xffff0000u : 0u);
+    res[w] = any ? ((sb & sel) | (best[w] & ~sel)) : 0u;
   }
-  uint4 v;
-  v.x = res[0] | (static_cast<unsigned>(res[1]) << 16);
-  v.y = res[2] | (static_cast<unsigned>(res[3]) << 16);
-  v.z = res[4] | (static_cast<unsigned>(res[5]) << 16);
-  v.w = res[6] | (static_cast<unsigned>(res[7]) << 16);
-  return v;
+  return make_uint4(res[0], res[1], res[2], res[3]);
 }
 
 // Section widths of a launch, in 16-byte chunks and bytes (compile-time where the variant fixes them).
@@ -113,7 +108,7 @@ __device__ __forceinline__ int request_of(const int64_t* co, int n_req, long lon
   int r = 0, n = n_req;
   while (n > 0) {
     const int half = n >> 1;
-    if (__ldg(co + r + half + 1) <= j0) {
+    if (co[r + half + 1] <= j0) {
       r += half + 1;
       n -= half + 1;
     } else {
@@ -326,7 +321,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
 #pragma unroll
           for (int u = 0; u < kUnroll; ++u) {
             if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;  // unresolved / out-of-range position
-            auth[u] = idx[u] >= 0 ? __ldg(a.author_ids + idx[u]) : -1;
+            auth[u] = idx[u] >= 0 ? load_author(a, idx[u]) : -1;
           }
           bool found[kUnroll];
           int pos[kUnroll];
@@ -352,11 +347,10 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
               int64_t act[4] = {-1, -1, -1, -1};
               unsigned types = 0;
               if (idx[u] >= 0) {
-                for (int sl = 0; sl < a.max_actors; ++sl) {
-                  const long long e = static_cast<long long>(a.max_actors) * idx[u] + sl;
-                  act[sl] = __ldg(a.actor_ids + e);
-                  types |= (__ldg(a.actor_types + e) % 3u) << (2 * sl);
-                }
+                long long rec[4];
+                load_actors(a, idx[u], rec, types);
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) act[sl] = sl < a.max_actors ? rec[sl] : -1;
               }
               bool af[4];
               int ap[4];
@@ -365,7 +359,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
               for (int sl = 0; sl < 4; ++sl) {
                 if (af[sl]) {
                   m |= 1u << (1 + sl);
-                  m |= 1u << (5 + ((types >> (2 * sl)) & 3u));
+                  m |= 1u << (5 + ((types >> (8 * sl)) & 0xffu) % 3u);
                 } else {
                   ap[sl] = -1;
                 }
@@ -392,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
             if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;
             if (i < n) {
               s_idx[i] = idx[u];
-              s_auth[i] = idx[u] >= 0 ? __ldg(a.author_ids + idx[u]) : kNoAuthor;
+              s_auth[i] = idx[u] >= 0 ? load_author(a, idx[u]) : kNoAuthor;
             }
           }
         }

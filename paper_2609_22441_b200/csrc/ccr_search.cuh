@@ -86,10 +86,9 @@ struct StagedKeys {
   }
 
   // U independent lookups with their shared-memory accesses interleaved: one round of bucket-index loads,
-  // then one round of up to kProbe key loads per id (a bucket of evenly spread ids holds about one key).
+  // then one round of up to P key loads per id (a bucket of evenly spread ids holds about one key).
   // Ids whose bucket is longer, and lists without an index, take find().  id < 0 is "nothing to look up".
-  static constexpr int kProbe = 4;
-  template <int U>
+  template <int U, int P = 4>
   __device__ __forceinline__ void find_batch(const int64_t (&id)[U], bool (&found)[U], int (&pos)[U]) const {
     if (!(K > 0 && M > 0 && s_log == 0 && nb > 0)) {
 #pragma unroll
@@ -104,24 +103,24 @@ struct StagedKeys {
       lo[u] = min(max(e.x, 0), M);
       n[u] = min(max(e.y, lo[u]), M) - lo[u];
     }
-    int64_t k[U][kProbe];
+    int64_t k[U][P];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
 #pragma unroll
-      for (int j = 0; j < kProbe; ++j) k[u][j] = sk[min(lo[u] + j, M - 1)];
+      for (int j = 0; j < P; ++j) k[u][j] = (j < n[u]) ? sk[lo[u] + j] : 0;  // lo + j < lo + n <= M
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       found[u] = false;
       pos[u] = 0;
 #pragma unroll
-      for (int j = 0; j < kProbe; ++j) {
+      for (int j = 0; j < P; ++j) {
         if (j < n[u] && k[u][j] == id[u]) {
           found[u] = true;
           pos[u] = lo[u] + j;
         }
       }
-      if (n[u] > kProbe && !found[u]) found[u] = find(id[u], pos[u]);  // long bucket: bounded binary search
+      if (n[u] > P && !found[u]) found[u] = find(id[u], pos[u]);  // long bucket: bounded binary search
     }
   }
 };

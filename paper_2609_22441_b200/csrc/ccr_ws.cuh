@@ -17,8 +17,8 @@
 // warps take 32-row groups one at a time from a shared-memory counter.
 //
 // Work distribution.  With a scheduling word (JoinArgs::sched) the resolvers of all blocks draw chunks of
-// consecutive tiles from one global counter; the chunk shrinks from kMaxChunk tiles to one tile as the
-// launch drains (guided self-scheduling), so blocks on slower SMs or with costlier requests simply take
+// consecutive tiles from one global counter; the chunk shrinks from kMaxRounds tiles per resolver warp to one
+// as the launch drains (guided self-scheduling), so blocks on slower SMs or with costlier requests simply take
 // fewer chunks and all blocks finish within about one tile of each other.  The last block to finish puts
 // the two scheduling words back to zero for the next launch.  Without a scheduling word every block takes
 // one equal contiguous slice.
@@ -30,7 +30,8 @@ namespace ccr {
 
 constexpr int kWsSlots = 8;        // ring depth
 constexpr int kWsMaxThreads = 512;
-constexpr int kMaxChunk = 8;       // most tiles a block draws at once
+constexpr int kWsMaxCachedReq = 1024;  // batches up to this many requests keep their offsets in shared memory
+constexpr int kMaxRounds = 4;      // most tiles per resolver warp a block draws at once
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -46,13 +47,16 @@ struct WsSlot {          // descriptor of one ring slot
 };
 
 struct WsLayout {
-  int off_full, off_empty, off_slots, off_grab, off_idx, off_pos, off_apos, off_keys, bytes;
-  __host__ __device__ WsLayout(int tile, bool second, int key_cap) {
+  int off_full, off_empty, off_slots, off_grab, off_offs, off_idx, off_pos, off_apos, off_keys, bytes;
+  // n_req_cached: requests whose offsets are mirrored in shared memory (0 = read them from global memory)
+  __host__ __device__ WsLayout(int tile, bool second, int key_cap, int n_req_cached) {
     off_full = kSmemHeader;                 // after the key-staging mbarrier
     off_empty = off_full + kWsSlots * 8;
     off_slots = off_empty + kWsSlots * 8;
     off_grab = off_slots + kWsSlots * static_cast<int>(sizeof(WsSlot));
-    off_idx = off_grab + 16;
+    off_offs = off_grab + 16;
+    off_idx = off_offs + (n_req_cached > 0 ? 2 * (n_req_cached + 1) * 8 : 0);
+    off_idx = (off_idx + 15) & ~15;
     off_pos = off_idx + kWsSlots * tile * 4;
     off_apos = off_pos + kWsSlots * tile * 4;
     off_keys = off_apos + (second ? kWsSlots * tile * 16 : 0);
@@ -64,7 +68,8 @@ template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND>
 __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArgs a, int n_streamers) {
   extern __shared__ __align__(16) unsigned char smem_ws[];
   unsigned char* smem = smem_ws;
-  const WsLayout lay(a.tile, SECOND, a.key_cap);
+  const int n_req_cached = a.n_req <= kWsMaxCachedReq ? a.n_req : 0;
+  const WsLayout lay(a.tile, SECOND, a.key_cap, n_req_cached);
   WsSlot* slots = reinterpret_cast<WsSlot*>(smem + lay.off_slots);
   int* grab = reinterpret_cast<int*>(smem + lay.off_grab);
   int* s_idx = reinterpret_cast<int*>(smem + lay.off_idx);
@@ -78,6 +83,19 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   const uint32_t full0 = smem_u32(smem + lay.off_full), empty0 = smem_u32(smem + lay.off_empty);
   const int kBarGroup = 1;  // named barrier of the resolver group
 
+  // offsets of the batch, mirrored once per block: every chunk starts with a search over them
+  const int64_t* co = a.cand_offsets;
+  const int64_t* eo = a.edge_offsets;
+  if (n_req_cached > 0) {
+    int64_t* s_co = reinterpret_cast<int64_t*>(smem + lay.off_offs);
+    int64_t* s_eo = s_co + (a.n_req + 1);
+    for (int i = tid; i <= a.n_req; i += n_threads) {
+      s_co[i] = __ldg(a.cand_offsets + i);
+      s_eo[i] = __ldg(a.edge_offsets + i);
+    }
+    co = s_co;
+    eo = s_eo;
+  }
   if (tid == 0) {
     mbar_init(bar, 1);
     for (int s = 0; s < kWsSlots; ++s) {
@@ -95,7 +113,9 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   const long long slice1 = min(a.total, slice0 + per * 32);
   if (a.sched == nullptr && slice0 >= slice1) return;  // block-uniform, before any named barrier
 
-  if (warp < n_streamers) {
+  const int n_res = (n_threads >> 5) - n_streamers;
+  const int role_rank = (n_threads >> 5) - 1 - warp;  // resolvers are the last n_res warps
+  if (role_rank >= n_res) {
     // ============================ streamers ============================
     for (unsigned it = 0;; ++it) {
       const int s = it % kWsSlots;
@@ -129,8 +149,8 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   // All resolver warps walk the same sequence of sub-tiles; warp q fills every n_resolvers-th one on its own
   // (own bounded wait for the slot, own publish), so several sub-tiles are being resolved at any time.  They
   // meet on a named barrier only to draw the next chunk and to stage a new request's keys.
-  const int gsize = n_threads - n_streamers * 32;
-  const int gtid = tid - n_streamers * 32;
+  const int gsize = n_res * 32;
+  const int gtid = role_rank * 32 + lane;
   const int n_resolvers = gsize >> 5;
   const int rwarp = gtid >> 5;
   const NamedGroup grp(gtid, gsize, kBarGroup);
@@ -147,9 +167,12 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
     long long j0, j1;
     if (a.sched != nullptr) {
       if (gtid == 0) {
+        // a chunk is a whole number of rounds (one tile per resolver warp), so the warps meet at the next
+        // draw having done the same amount of work; rounds shrink from kMaxRounds to 1 as the launch drains
         const long long rem = n_tiles - *reinterpret_cast<volatile int*>(a.sched);
-        long long c = rem / (2LL * gridDim.x);
-        c = c < 1 ? 1 : (c > kMaxChunk ? kMaxChunk : c);
+        long long m = rem / (2LL * gridDim.x * n_resolvers);
+        m = m < 1 ? 1 : (m > kMaxRounds ? kMaxRounds : m);
+        const long long c = m * n_resolvers;
         grab[0] = atomicAdd(a.sched, static_cast<int>(c));
         grab[1] = static_cast<int>(c);
       }
@@ -165,17 +188,17 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
       more = false;
     }
 
-    int r = request_of(a.cand_offsets, a.n_req, j0);
+    int r = request_of(co, a.n_req, j0);
     long long seg = j0;
     while (seg < j1 && r < a.n_req && !failed) {
-      const long long rend = __ldg(a.cand_offsets + r + 1);
+      const long long rend = co[r + 1];
       if (rend <= seg) {  // request without candidates here
         ++r;
         continue;
       }
       const long long seg_end = min(rend, j1);
-      long long kb;
-      const int K = request_keys(a, r, kb);
+      const long long kb = eo[r];
+      const int K = static_cast<int>(min(max(eo[r + 1] - kb, 0LL), static_cast<long long>(a.max_edge_len)));
       if (r != staged_r) {
         if (!stage_keys(a, ssm, bar, phase, kb, K, true, keys, grp)) {
           if (gtid == 0) {
@@ -213,26 +236,15 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
 #pragma unroll
           for (int u = 0; u < U; ++u) {
             if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;  // unresolved / out-of-range position
-            auth[u] = idx[u] >= 0 ? __ldg(a.author_ids + idx[u]) : -1;
+            auth[u] = idx[u] >= 0 ? load_author(a, idx[u]) : -1;
             if constexpr (SECOND) {
               act[u][0] = act[u][1] = act[u][2] = act[u][3] = -1;
               types[u] = 0;
               if (idx[u] >= 0) {
-                if (a.max_actors == 4) {
-                  const longlong2* ap = reinterpret_cast<const longlong2*>(a.actor_ids + 4LL * idx[u]);
-                  const longlong2 p0 = __ldg(ap), p1 = __ldg(ap + 1);
-                  act[u][0] = p0.x;
-                  act[u][1] = p0.y;
-                  act[u][2] = p1.x;
-                  act[u][3] = p1.y;
-                  types[u] = __ldg(reinterpret_cast<const unsigned*>(a.actor_types + 4LL * idx[u]));
-                } else {
-                  for (int sl = 0; sl < a.max_actors; ++sl) {
-                    const long long e = static_cast<long long>(a.max_actors) * idx[u] + sl;
-                    act[u][sl] = __ldg(a.actor_ids + e);
-                    types[u] |= static_cast<unsigned>(__ldg(a.actor_types + e)) << (8 * sl);
-                  }
-                }
+                long long rec[4];
+                load_actors(a, idx[u], rec, types[u]);
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) act[u][sl] = sl < a.max_actors ? rec[sl] : -1;
               }
             }
           }
@@ -250,29 +262,52 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
               pos[h + q] = p4[q];
             }
           }
+          if constexpr (SECOND) {
+            // engager lookups, the slots of two candidates (8 ids) interleaved per batch
+            bool af[U][4];
+            int ap[U][4];
 #pragma unroll
-          for (int u = 0; u < U; ++u) {
-            const int i = base + u * 32 + lane;
-            unsigned m = found[u] ? 1u : 0u;
-            if constexpr (SECOND) {
-              bool af[4];
-              int ap[4];
-              keys.find_batch<4>(act[u], af, ap);
+            for (int h = 0; h < U; h += 2) {
+              const int64_t id8[8] = {act[h][0], act[h][1], act[h][2], act[h][3],
+                                      act[h + 1][0], act[h + 1][1], act[h + 1][2], act[h + 1][3]};
+              bool f8[8];
+              int p8[8];
+              keys.find_batch<8, 2>(id8, f8, p8);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                af[h + (q >> 2)][q & 3] = f8[q];
+                ap[h + (q >> 2)][q & 3] = p8[q];
+              }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+              const int i = base + u * 32 + lane;
+              unsigned m = found[u] ? 1u : 0u;
 #pragma unroll
               for (int sl = 0; sl < 4; ++sl) {
-                if (af[sl]) {
+                if (af[u][sl]) {
                   m |= 1u << (1 + sl);
                   m |= 1u << (5 + ((types[u] >> (8 * sl)) & 0xffu) % 3u);
                 } else {
-                  ap[sl] = -1;
+                  ap[u][sl] = -1;
                 }
               }
-              if (i < n) out_apos[i] = make_int4(ap[0], ap[1], ap[2], ap[3]);
+              if (i < n) {
+                out_apos[i] = make_int4(ap[u][0], ap[u][1], ap[u][2], ap[u][3]);
+                out_idx[i] = idx[u];
+                out_pos[i] = found[u] ? pos[u] : -1;
+                a.out_mask[sub + i] = static_cast<uint8_t>(m);
+              }
             }
-            if (i < n) {
-              out_idx[i] = idx[u];
-              out_pos[i] = found[u] ? pos[u] : -1;
-              a.out_mask[sub + i] = static_cast<uint8_t>(m);
+          } else {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+              const int i = base + u * 32 + lane;
+              if (i < n) {
+                out_idx[i] = idx[u];
+                out_pos[i] = found[u] ? pos[u] : -1;
+                a.out_mask[sub + i] = found[u] ? 1 : 0;
+              }
             }
           }
         }

@@ -72,7 +72,7 @@ def test_config0_single_tiny_request_all_search_paths(B):
 def test_config1_batched_first_degree_full_size(B):
     wl = W.config1()
     assert wl.batch.total_cands == 64 * 30_000 and wl.out_row_bytes() == 384
-    _check(B, wl, _variants(B), tunings=((0, 0), (512, 0, 1, 1, 1), (2048, 0, 14, 2, 3), (768, 0, 5, 8, 2)))
+    _check(B, wl, _variants(B), tunings=((0, 0), (512, 0, 1, 1, 1), (2048, 0, 14, 2, 3), (768, 0, 5, 8, 2), (256, 0, 3, 1, 0)))
     _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
 
 
@@ -322,8 +322,18 @@ def test_upload_in_pieces_from_device_memory(B):
         dev = lambda x: torch.from_numpy(np.ascontiguousarray(x[a:z])).cuda()
         store.upload(a, dev(s.doc_feats), dev(s.author_ids), dev(s.actor_ids), dev(s.actor_types))
     torch.cuda.synchronize()
+    before = store.launch_count()  # uploads of a second-degree store launch their own (packing) kernels
     rows, mask = gpu_join(store, B.DeviceBatch(wl.batch))
     want_rows, want_mask = oracle.join_workload(wl)
     assert np.array_equal(rows, want_rows) and np.array_equal(mask, want_mask)
-    assert store.launch_count() == 1
+    assert store.launch_count() == before + 1
+    # a partial upload (only the types of a few docs) leaves the other ids of those docs untouched
+    types2 = s.actor_types.copy()
+    types2[100:200] = (types2[100:200] + 1) % 3
+    store.upload(100, None, None, None, np.ascontiguousarray(types2[100:200]))
+    torch.cuda.synchronize()
+    s2 = W.Store(**{**s.__dict__, "actor_types": types2})
+    rows2, mask2 = gpu_join(store, B.DeviceBatch(wl.batch))
+    want2 = oracle.join_workload(W.Workload("t", 0, s2, wl.batch))
+    assert np.array_equal(rows2, want2[0]) and np.array_equal(mask2, want2[1])
     store.free()
