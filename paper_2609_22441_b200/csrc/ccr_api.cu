@@ -515,7 +515,12 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
     const WsKernelFn fn = second ? v.ws_second : v.ws_first;
     // dynamic chunk scheduling through a pair of device words; each launch takes the next pair in turn, so
     // up to kSchedRegions launches of one store may be in flight at once (on any streams)
-    if (!(flags & CCR_FLAG_STATIC_SPLIT)) a.sched = s->status + 4 + 2 * static_cast<int>(s->launches % kSchedRegions);
+    // Small launches (fewer tiles than two rounds per block) are split evenly instead: drawing whole rounds
+    // from the counter would leave most SMs without work, and a single request is the latency-critical case.
+    const int n_res_auto = s->ws_resolvers > 0 ? s->ws_resolvers : (second ? 5 : 4);
+    const long long n_tiles = (total_cands + a.tile - 1) / a.tile;
+    const bool dynamic = !(flags & CCR_FLAG_STATIC_SPLIT) && n_tiles >= 2LL * blocks * n_res_auto;
+    if (dynamic) a.sched = s->status + 4 + 2 * static_cast<int>(s->launches % kSchedRegions);
     const int n_str = s->ws_streamers > 0 ? s->ws_streamers : (second ? 11 : 12);
     const int n_res = s->ws_resolvers > 0 ? s->ws_resolvers : (second ? 5 : 4);
     fn<<<static_cast<unsigned>(blocks), (n_str + n_res) * 32, smem, st>>>(a, n_str);
