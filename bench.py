@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (bytes per launch; None until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {"config1": 1182251520, "config2b": None}
+NCU_TRAFFIC_BYTES = {"config1": 1184300000, "config2b": 1454900000}
 
 
 def parse_args():
