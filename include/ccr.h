@@ -206,6 +206,12 @@ ccr_status ccr_join_payload_static(const ccr_docstore* store,
  * last call (the affected rows of that launch were not written).  Clears the word.                 */
 ccr_status ccr_docstore_device_status(ccr_docstore* store, void* stream);
 
+/* Self-test of the failure-reporting path (no fault, trap or hang is involved): enqueues a one-block kernel
+ * that waits, with the kernels' bounded wait cut down to a few thousand polls, on a barrier that nothing will
+ * ever complete.  The wait runs out, the kernel records it and returns; the next ccr_docstore_device_status
+ * reports CCR_ERR_DEVICE_WAIT (and clears the word), and the store and the context stay usable.            */
+ccr_status ccr_docstore_selftest_wait(ccr_docstore* store, void* stream);
+
 /* Tuning knobs of the join kernels; a field that is 0 keeps the store's current value.              */
 typedef struct {
   int32_t tile_cands;         /* candidates per ring slot / search-copy phase pair: multiple of 256, <= 4096;

@@ -79,8 +79,11 @@ def join(
                         if (reduce_sum_mask >> d) & 1:
                             acc = np.float32(0.0)
                             for v in col:
-                                acc = np.float32(acc + np.float32(v))
-                            red[d] = np.float16(acc)
+                                with np.errstate(invalid="ignore", over="ignore"):
+                                    acc = np.float32(acc + np.float32(v))
+                            # a NaN sum is stored as the canonical 0x7fff (the join's stated rule)
+                            with np.errstate(over="ignore"):  # a finite fp32 sum above 65504 rounds to infinity
+                                red[d] = np.uint16(0x7FFF).view(np.float16) if np.isnan(acc) else np.float16(acc)
                         else:
                             best = col[0]
                             for v in col[1:]:

@@ -41,7 +41,7 @@ EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
     "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
-    "ccr_static_payload_capacity", "ccr_join_payload_static",
+    "ccr_static_payload_capacity", "ccr_join_payload_static", "ccr_docstore_selftest_wait",
 )
 
 
@@ -102,6 +102,8 @@ def lib() -> ctypes.CDLL:
     L.ccr_static_payload_capacity.argtypes = []
     L.ccr_join_payload_static.restype = ctypes.c_int
     L.ccr_join_payload_static.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
+    L.ccr_docstore_selftest_wait.restype = ctypes.c_int
+    L.ccr_docstore_selftest_wait.argtypes = [vp, vp]
     L.ccr_docstore_device_status.restype = ctypes.c_int
     L.ccr_docstore_device_status.argtypes = [vp, vp]
     L.ccr_docstore_set_tuning.restype = ctypes.c_int
@@ -195,6 +197,9 @@ class Docstore:
 
     def launch_count(self) -> int:
         return int(lib().ccr_docstore_launch_count(self._h))
+
+    def selftest_wait(self, stream=None) -> None:
+        _check(lib().ccr_docstore_selftest_wait(self._h, _stream_ptr(stream)), "ccr_docstore_selftest_wait")
 
     def device_status(self, stream=None) -> int:
         return int(lib().ccr_docstore_device_status(self._h, _stream_ptr(stream)))

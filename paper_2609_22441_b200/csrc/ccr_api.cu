@@ -119,6 +119,21 @@ __global__ void validate_kernel(const ccr::JoinArgs a, int check_sorted, int* co
 }
 
 // ---------------------------------------------------------------------------------------------------
+// Self-test of the failure-reporting path: one block waits, with the kernels' bounded wait, on a barrier that
+// nothing will ever complete.  The wait must run out, the status word must be set, the kernel must return.
+__global__ void selftest_wait_kernel(int* status, int tries) {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  const uint32_t bar = ccr::smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    ccr::mbar_init(bar, 1);
+    ccr::fence_proxy_async_smem();
+  }
+  __syncthreads();
+  const bool completed = ccr::mbar_wait_bounded(bar, 0, tries);
+  if (!completed && threadIdx.x == 0) atomicExch(status, ccr::kDevWaitExpired);
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Upload path of second-degree stores: scatter the caller's separate id arrays into the packed records.
 // A null source leaves its fields untouched.
 __global__ void pack_ids_kernel(ccr::IdRec* recs, long long n, int max_actors, const int64_t* author_ids,
@@ -401,6 +416,16 @@ ccr_status ccr_docstore_device_status(ccr_docstore* s, void* stream) {
     return CCR_ERR_CUDA;
   }
   return s->status_host[0] == ccr::kDevWaitExpired ? CCR_ERR_DEVICE_WAIT : CCR_OK;
+}
+
+ccr_status ccr_docstore_selftest_wait(ccr_docstore* s, void* stream) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  selftest_wait_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(s->status, 2000);
+  s->launches++;
+  if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+  return CCR_OK;
 }
 
 ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,

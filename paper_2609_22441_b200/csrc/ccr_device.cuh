@@ -104,8 +104,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait: gives up after kWaitTries polls (each poll may itself suspend for a short,
 // hardware-defined time).  Returns false when the phase never completed.
 constexpr int kWaitTries = 1 << 22;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (int i = 0; i < kWaitTries; ++i) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int tries = kWaitTries) {
+  for (int i = 0; i < tries; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
   }
   return false;

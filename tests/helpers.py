@@ -14,7 +14,9 @@ def tiny_workload(seed, n_docs, alphabet, n_req, kmax, nmax, second, req_dim, do
     store = W.make_store(rng, n_docs, alphabet, doc_dim, doc_dtype, max_actors=4 if second else 0,
                          reduce_sum_mask=sum_mask if second else 0)
     keys_l, feats_l, cands_l = [], [], []
-    vals = np.array([-2.0, -0.5, 0.0, 0.25, 0.5, 1.0, 1.5, 3.0, 1000.0, 6e-5, 60000.0, -0.0], np.float16)
+    # negatives, ties, +-0, a subnormal, values whose sums overflow, infinities and two NaN encodings
+    vals = np.concatenate([np.array([-2.0, -0.5, 0.0, 0.25, 0.5, 1.0, 1.5, 3.0, 1000.0, 6e-5, 60000.0, -0.0], np.float16),
+                           np.array([0x7C00, 0xFC00, 0x7E00, 0x7C01], np.uint16).view(np.float16)])
     for _ in range(n_req):
         k = int(rng.integers(0, min(kmax, alphabet) + 1))
         keys, _ = W.make_viewer(rng, alphabet, k, edge_dim, np.float16)

@@ -28,6 +28,10 @@ def env():
     if torch.cuda.mem_get_info()[0] < 60 * 2**30:
         pytest.skip("needs ~50 GB of free device memory")
     wl = W.config3()
+    # viewer templates of the latency sweep (config 4) force their docs before the store is uploaded
+    tpl = W.make_latency_templates(wl.store, W.config_seed(4), (10, 1_000, 20_000), 2, first_pool=256,
+                                   n_pools=wl.meta["n_pools"], forced_per_template=70_000,
+                                   edge_dim=wl.batch.edge_dim, n_authors=wl.meta["n_authors"])
     b = wl.batch
     C = b.total_cands
     rng = np.random.default_rng(7)
@@ -37,6 +41,7 @@ def env():
         J += [np.arange(c0, min(c0 + 96, c1)), np.arange(max(c1 - 96, c0), c1)]
     J = np.unique(np.concatenate(J))
     store, kept, full = upload_generated_store(B, wl, keep_rows_of=b.cand_idx[J], keep_all=True)
+    wl.meta["latency_templates"] = tpl
     yield B, wl, store, kept, full, J
     store.free()
 
@@ -124,3 +129,33 @@ def test_config3_second_degree(env):
     assert np.array_equal(m[J], want_mask)
     assert np.array_equal(got, want_rows)
     assert (want_mask >> 1).any()
+
+
+@pytest.mark.parametrize("n_cand,k", [(1_000, 10), (20_000, 1_000), (100_000, 20_000), (5_000, 20_000)])
+def test_config4_single_request_cells(env, n_cand, k):
+    """Cells of the latency sweep: one request per launch on the production-scale store.  Every output of the
+    request is checked: found bits against numpy membership, doc sections against a torch gather of the
+    generated matrix, matched edge sections against torch.searchsorted + index_select (Algorithm 1 with
+    library ops, on the device), unmatched ones against zero."""
+    B, wl, store, kept, full, J = env
+    s = wl.store
+    mark = np.zeros(s.n_docs, dtype=bool)
+    rng = np.random.default_rng(1000 * k + n_cand)
+    for t in wl.meta["latency_templates"][k]:
+        batch = W.draw_latency_request(rng, s, t, n_cand, 0.7, mark, wl.batch.edge_dim)
+        one = W.Workload("cell", 0, s, batch)
+        for flags in (B.CCR_FLAG_FIRST_DEGREE_ONLY, B.CCR_FLAG_FIRST_DEGREE_ONLY | B.CCR_FLAG_TWO_PHASE):
+            rows, mask, _ = _run(B, store, one, flags)
+            member = _membership(one, batch.cand_idx)
+            m = _check_full(one, full, rows, mask, batch.cand_idx, member)
+            assert 0.3 < member.mean() < 0.8
+            # matched edge rows: Algorithm 1 steps 2-4 with library ops
+            keys = torch.from_numpy(batch.edge_keys).cuda()
+            feats = torch.from_numpy(batch.edge_feats.view(np.uint8).reshape(len(batch.edge_keys), -1)).cuda()
+            d = torch.from_numpy(s.author_ids[batch.cand_idx.astype(np.int64)]).cuda()
+            pos = torch.searchsorted(keys, d).clamp(max=len(batch.edge_keys) - 1)
+            valid = keys[pos] == d
+            assert np.array_equal(valid.cpu().numpy(), member)
+            want = torch.where(valid[:, None], feats.index_select(0, pos), torch.zeros_like(feats[:1]))
+            doc_b = s.doc_row_bytes
+            assert torch.equal(rows[:, doc_b:doc_b + batch.edge_row_bytes], want)

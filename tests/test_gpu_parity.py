@@ -313,6 +313,44 @@ def test_argument_errors_on_a_live_store(B):
     assert L.ccr_docstore_free(h) == B.CCR_ERR_BAD_HANDLE  # double free
 
 
+def test_expired_device_wait_is_reported_and_the_store_stays_usable(B):
+    """Failure reporting without a fault: a wait that nothing completes runs out of polls, the kernel returns,
+    the status call reports it once, and the next join is bit-exact."""
+    wl = W.config1(n_docs=30_000, n_req=3, n_cand=2_000)
+    store = B.store_from_workload(wl)
+    assert store.device_status() == B.CCR_OK
+    store.selftest_wait()
+    assert store.device_status() == B.CCR_ERR_DEVICE_WAIT
+    assert store.device_status() == B.CCR_OK  # reading clears the word
+    rows, mask = gpu_join(store, B.DeviceBatch(wl.batch))
+    want_rows, want_mask = oracle.join_workload(wl)
+    assert np.array_equal(rows, want_rows) and np.array_equal(mask, want_mask)
+    assert store.device_status() == B.CCR_OK
+    store.free()
+
+
+def test_joins_in_flight_on_several_streams(B):
+    """Launches of one store on different streams draw their chunks from different scheduling words."""
+    wl = W.config1(n_docs=200_000, n_req=16, n_cand=20_000)
+    b = wl.batch
+    store = B.store_from_workload(wl)
+    db = B.DeviceBatch(b)
+    want_rows, want_mask = oracle.join_workload(wl, n_threads=4)
+    streams = [torch.cuda.Stream() for _ in range(4)]
+    outs = [(torch.full((b.total_cands, 384), 0x11, dtype=torch.uint8, device="cuda"),
+             torch.full((b.total_cands,), 0x11, dtype=torch.uint8, device="cuda")) for _ in range(12)]
+    torch.cuda.synchronize()  # the fills ran on the default stream: finish them before other streams write
+    for i, (rows, mask) in enumerate(outs):
+        st = streams[i % len(streams)]
+        B.ccr_join_batch(store, db.n_req, b.total_cands, db.max_edge_len, db.edge_keys, db.edge_feats,
+                         db.edge_offsets, db.cand_idx, db.cand_offsets, db.req_feats, rows, mask, 0, st)
+    torch.cuda.synchronize()
+    for rows, mask in outs:
+        assert np.array_equal(mask.cpu().numpy(), want_mask) and np.array_equal(rows.cpu().numpy(), want_rows)
+    assert store.device_status() == B.CCR_OK
+    store.free()
+
+
 def test_upload_in_pieces_from_device_memory(B):
     wl = W.config0(n_docs=10_000, n_cand=3000, k=200, second_degree=True)
     s = wl.store

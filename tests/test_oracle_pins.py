@@ -18,6 +18,8 @@ from hypothesis import strategies as st
 from oracle import brute_force, oracle
 from paper_2609_22441_b200 import workloads as W
 
+from helpers import tiny_workload
+
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
 
@@ -73,25 +75,8 @@ def _brute(wl, **kw):
         reduce_sum_mask=s.reduce_sum_mask, **kw)
 
 
-def _tiny(seed, n_docs, alphabet, n_req, kmax, nmax, second, req_dim, doc_dtype=np.float32):
-    """Tiny problem with ids from a tiny alphabet so that hits, misses and repeats are all common."""
-    rng = np.random.default_rng(seed)
-    store = W.make_store(rng, n_docs, alphabet, 4, doc_dtype, max_actors=4 if second else 0,
-                         reduce_sum_mask=0b10110100 if second else 0)
-    keys_l, feats_l, cands_l = [], [], []
-    for _ in range(n_req):
-        k = int(rng.integers(0, min(kmax, alphabet) + 1))
-        keys, _ = W.make_viewer(rng, alphabet, k, 8, np.float16)
-        # edge values include negatives, repeats and exact ties so that max / sum rules matter
-        feats = rng.choice(np.array([-2.0, -0.5, 0.0, 0.25, 0.5, 1.0, 1.5, 3.0, 1000.0, 6e-5], np.float16),
-                           size=(k, 8))
-        n = int(rng.integers(0, nmax + 1))
-        cands_l.append(rng.integers(-1, n_docs + 1, size=n).astype(np.int32))  # includes -1 and n_docs
-        keys_l.append(keys)
-        feats_l.append(feats)
-    req = rng.standard_normal((n_req, req_dim)).astype(np.float32) if req_dim else None
-    batch = W.assemble_batch(keys_l, feats_l, cands_l, req, 8, np.float16, req_dim, np.float32)
-    return W.Workload("tiny", seed, store, batch)
+def _tiny(seed, n_docs, alphabet, n_req, kmax, nmax, second, req_dim):
+    return tiny_workload(seed, n_docs, alphabet, n_req, kmax, nmax, second, req_dim)
 
 
 # ---------------------------------------------------------------- brute force (naive scan) == oracle
