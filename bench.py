@@ -48,10 +48,11 @@ def parse_args():
     p.add_argument("--steps", type=int, default=2000)
     p.add_argument("--warmup", type=int, default=10)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--config", default="1", choices=["1", "2b", "3", "3b", "3s", "4"],
+    p.add_argument("--config", default="1", choices=["1", "2b", "3", "3b", "3s", "4", "sort"],
                    help="1 batched first-degree (default, the headline); 2b second-degree on the same shape; 3 production-scale "
                         "store, first-degree; 3b the same on candidates sorted by author (merge path); 3s production scale, "
-                        "second-degree; 4 single-request latency sweep on the production-scale store")
+                        "second-degree; 4 single-request latency sweep on the production-scale store; sort: Algorithm 1 step 1 "
+                        "(per-request sort of unsorted affinity records) on the payloads of configs 1 and 3")
     p.add_argument("--sweep-requests", type=int, default=1000, help="requests per cell of the latency sweep")
     p.add_argument("--c3-docs", type=int, default=50_000_000, help="store size of configs 3/3b/3s (smaller for profiler captures)")
     p.add_argument("--c3-requests", type=int, default=256, help="requests of configs 3/3b/3s (smaller for profiler captures)")
@@ -312,6 +313,72 @@ def latency_sweep(args, B, device: int):
     store.free()
 
 
+def sort_bench(args, B, device: int):
+    """Algorithm 1 step 1 on the device: the affinity records of every request of a batch, shuffled, are put
+    back in key order by ccr_sort_edges.  Timed on the payloads of config 1 (64 lists of 50..5000 records,
+    64-byte rows) and config 3 (256 lists of 10..20000 records, 128-byte rows)."""
+    import torch
+
+    from oracle import oracle
+    from paper_2609_22441_b200 import workloads as W
+
+    dev = torch.device("cuda", device)
+    peak, peak_kind = measured_peak_gbs()
+    results = []
+    for name, wl in (("config1 payload", W.config1(n_docs=10_000, n_cand=100)),
+                     ("config3 payload", W.config3(n_docs=100_000, n_cand=100, gen_doc_feats=True, extra_pools=0))):
+        b = wl.batch
+        rng = np.random.default_rng(wl.seed)
+        keys, feats = b.edge_keys.copy(), b.edge_feats.copy()
+        for r in range(b.n_req):
+            a, z = int(b.edge_offsets[r]), int(b.edge_offsets[r + 1])
+            p = rng.permutation(z - a)
+            keys[a:z], feats[a:z] = b.edge_keys[a:z][p], b.edge_feats[a:z][p]
+        store = B.store_from_workload(wl, device=device)
+        up = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(dev)
+        k_in, f_in, eo = up(keys), up(feats), up(b.edge_offsets)
+        k_out, f_out = torch.empty_like(k_in), torch.empty_like(f_in)
+        p_out = torch.empty(len(keys), dtype=torch.int32, device=dev)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # larger than L2: written between launches
+        call = lambda: B.ccr_sort_edges(store, b.n_req, b.max_edge_len, k_in, f_in, eo, k_out, f_out, p_out)
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize(dev)
+        times = []
+        for _ in range(max(args.steps // 20, 20)):
+            flush.fill_(1)
+            a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            call()
+            z.record()
+            torch.cuda.synchronize(dev)
+            times.append(a.elapsed_time(z))
+        ms = float(np.median(times))
+        E = len(keys)
+        nbytes = E * (2 * (8 + b.edge_row_bytes) + 4)
+        t0 = time.perf_counter()
+        want = oracle.sort_edges(keys, feats, b.edge_offsets)
+        t_cpu = time.perf_counter() - t0
+        ok = bool(np.array_equal(k_out.cpu().numpy(), want[0]) and np.array_equal(p_out.cpu().numpy(), want[2]))
+        results.append({"payload": name, "requests": b.n_req, "records": E, "longest_list": b.max_edge_len,
+                        "row_bytes": b.edge_row_bytes, "ms": ms, "records_per_s": E / (ms * 1e-3),
+                        "algorithmic_gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / peak,
+                        "oracle_ms_1_core": 1e3 * t_cpu, "matches_oracle": ok})
+        store.free()
+    head = results[-1]
+    print(json.dumps({
+        "metric": "edge_records_sorted_per_sec", "value": head["records_per_s"], "unit": "records/s", "n_gpus": 1,
+        "steps": max(args.steps // 20, 20), "warmup": 3, "ms_per_step": head["ms"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": "Algorithm 1 step 1: per-request sort of shuffled affinity records; L2 flushed between launches",
+                   "peak_kind": "of " + peak_kind},
+        "roofline": {"bound": "hbm", "achieved": head["algorithmic_gbs"], "peak": peak, "unit": "GB/s",
+                     "frac": head["frac_of_hbm_peak"], "traffic": None,
+                     "note": "latency-bound: one block per request, the longest list sets the launch time"},
+        "payloads": results, "gpu_launches": max(args.steps // 20, 20),
+    }))
+
+
 def run_reference(args, rank: int):
     """The reference arm of this tier is the CPU oracle: rank 0 times it, the other ranks do nothing."""
     if rank != 0:
@@ -390,6 +457,10 @@ def main():
     if args.config == "4":
         if rank == 0:
             latency_sweep(args, B, local_rank)
+        return
+    if args.config == "sort":
+        if rank == 0:
+            sort_bench(args, B, local_rank)
         return
     wl, cfg_flags = make_workload(args.config, rank, args.c3_docs, args.c3_requests)
     b = wl.batch

@@ -141,6 +141,18 @@ ccr_status ccr_join_batch(const ccr_docstore* store,
                           uint32_t       flags,
                           void*          stream);
 
+/* Algorithm 1 step 1 for request payloads whose affinity records arrive unsorted: for every request r the
+ * records [edge_offsets[r], edge_offsets[r+1]) — key int64 + feature row of the store's edge width — are put
+ * in ascending key order (records with equal keys keep their input order) into keys_out / feats_out, which
+ * use the same offsets and must not alias the inputs.  perm_out (optional, int32[E]) receives for every
+ * output record the index of its source record inside the request; it is required when max_edge_len exceeds
+ * 19,000, because longer lists are sorted in place in keys_out / perm_out instead of in shared memory.
+ * All pointers DEVICE; one kernel on `stream` (one 1024-thread block per request), no allocation, no sync.
+ * The output is what ccr_join_batch expects as edge_keys / edge_feats.                                    */
+ccr_status ccr_sort_edges(const ccr_docstore* store, int32_t n_req, int64_t max_edge_len,
+                          const int64_t* edge_keys_in, const void* edge_feats_in, const int64_t* edge_offsets,
+                          int64_t* edge_keys_out, void* edge_feats_out, int32_t* perm_out, void* stream);
+
 /* Device staging buffers for ccr_join_batch_host, sized for the largest batch the caller will pass.
  * HOST calls; allocation happens here, never inside the join.                                      */
 ccr_status ccr_workspace_create(const ccr_docstore* store, int32_t max_req, int64_t max_cands,

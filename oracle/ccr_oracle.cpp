@@ -25,6 +25,9 @@
 // out_mask[j]: bit0 author found; bits 1..4 engager slot 0..3 found; bits 5..7 OR of (1 << type) over
 // the found slots (type 0 reacted, 1 commented, 2 reshared).
 //
+//   * Algorithm 1 step 1 (ccr_oracle_sort_edges): a_sorted, idx = sort(a); F_sorted = gather(F, idx), per
+//     request, as std::stable_sort of the record indices by key followed by a row-by-row copy.
+//
 // Plain, slow and unblocked on purpose; single-threaded unless n_threads > 1, in which case the flat
 // candidate range is cut into contiguous chunks, one std::thread each.
 #include <algorithm>
@@ -256,6 +259,30 @@ int ccr_oracle_join(int64_t n_docs, const void* doc_feats, int64_t doc_row_bytes
     if (a < b) pool.emplace_back([&p, a, b] { join_range(p, a, b); });
   }
   for (auto& th : pool) th.join();
+  return 0;
+}
+
+// Algorithm 1 step 1 for a ragged batch: records [edge_offsets[r], edge_offsets[r+1]) of every request are
+// put in ascending key order (equal keys keep their input order).  perm_out (optional) receives, per output
+// record, the index of its source record inside the request.
+int ccr_oracle_sort_edges(int32_t n_req, const int64_t* keys_in, const void* feats_in, const int64_t* edge_offsets,
+                          int64_t row_bytes, int64_t* keys_out, void* feats_out, int32_t* perm_out) {
+  const uint8_t* fin = static_cast<const uint8_t*>(feats_in);
+  uint8_t* fout = static_cast<uint8_t*>(feats_out);
+  for (int32_t r = 0; r < n_req; ++r) {
+    const int64_t e0 = edge_offsets[r], K = edge_offsets[r + 1] - e0;
+    if (K < 0) return -1;
+    std::vector<int32_t> idx(static_cast<size_t>(K));
+    for (int64_t i = 0; i < K; ++i) idx[static_cast<size_t>(i)] = static_cast<int32_t>(i);
+    std::stable_sort(idx.begin(), idx.end(),
+                     [&](int32_t x, int32_t y) { return keys_in[e0 + x] < keys_in[e0 + y]; });
+    for (int64_t i = 0; i < K; ++i) {
+      const int32_t src = idx[static_cast<size_t>(i)];
+      keys_out[e0 + i] = keys_in[e0 + src];
+      std::memcpy(fout + (e0 + i) * row_bytes, fin + (e0 + src) * row_bytes, static_cast<size_t>(row_bytes));
+      if (perm_out) perm_out[e0 + i] = src;
+    }
+  }
   return 0;
 }
 

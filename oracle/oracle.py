@@ -46,6 +46,8 @@ def _load():
             i64, vp, i64, vp, i32, vp, vp, i32, i32, u64,
             i32, vp, vp, vp, vp, vp, vp, i64, i32, vp, vp, i32,
         ]
+        lib.ccr_oracle_sort_edges.restype = ctypes.c_int
+        lib.ccr_oracle_sort_edges.argtypes = [i32, vp, vp, vp, i64, vp, vp, vp]
         lib.ccr_oracle_half_to_float_bits.restype = ctypes.c_uint32
         lib.ccr_oracle_half_to_float_bits.argtypes = [ctypes.c_uint16]
         lib.ccr_oracle_float_bits_to_half.restype = ctypes.c_uint16
@@ -125,6 +127,28 @@ def join(
     if rc != 0:
         raise ValueError("the oracle does not define this case (code %d)" % rc)
     return out_rows, out_mask
+
+
+def sort_edges(edge_keys: np.ndarray, edge_feats: np.ndarray, edge_offsets: np.ndarray):
+    """Algorithm 1 step 1 per request: (keys, rows) in ascending key order, ties in input order.
+    Returns (keys_sorted int64[E], feats_sorted like edge_feats, perm int32[E] = source index inside the request)."""
+    lib = _load()
+    edge_keys = _c(edge_keys, np.int64)
+    edge_feats = _c(edge_feats)
+    edge_offsets = _c(edge_offsets, np.int64)
+    E = len(edge_keys)
+    if edge_feats.shape[0] != E or int(edge_offsets[-1]) != E:
+        raise ValueError("keys, rows and offsets disagree on the record count")
+    keys_out = np.full(E, -0x3232323232323233, dtype=np.int64)
+    feats_out = np.full(edge_feats.shape, 0, dtype=edge_feats.dtype)
+    feats_out.view(np.uint8)[...] = 0xCD
+    perm = np.full(E, -1, dtype=np.int32)
+    row_b = int(edge_feats.shape[1] * edge_feats.dtype.itemsize)
+    rc = lib.ccr_oracle_sort_edges(len(edge_offsets) - 1, _ptr(edge_keys), _ptr(edge_feats), _ptr(edge_offsets), row_b,
+                                   _ptr(keys_out), _ptr(feats_out), _ptr(perm))
+    if rc != 0:
+        raise ValueError("malformed offsets")
+    return keys_out, feats_out, perm
 
 
 def join_workload(wl, first_degree_only: bool = False, n_threads: int = 1):

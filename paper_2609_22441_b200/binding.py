@@ -42,6 +42,7 @@ EXPORTS = (
     "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
     "ccr_static_payload_capacity", "ccr_join_payload_static", "ccr_docstore_selftest_wait",
+    "ccr_sort_edges",
 )
 
 
@@ -102,6 +103,8 @@ def lib() -> ctypes.CDLL:
     L.ccr_static_payload_capacity.argtypes = []
     L.ccr_join_payload_static.restype = ctypes.c_int
     L.ccr_join_payload_static.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
+    L.ccr_sort_edges.restype = ctypes.c_int
+    L.ccr_sort_edges.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, vp, vp]
     L.ccr_docstore_selftest_wait.restype = ctypes.c_int
     L.ccr_docstore_selftest_wait.argtypes = [vp, vp]
     L.ccr_docstore_device_status.restype = ctypes.c_int
@@ -314,6 +317,16 @@ def ccr_join_payload_static(store: Docstore, n_req: int, total_cands: int, max_e
                                        _ptr(cand_idx), _ptr(cand_offsets), _ptr(req_feats), _ptr(out_rows),
                                        _ptr(out_mask), int(flags), _stream_ptr(stream))
     _check(st, "ccr_join_payload_static")
+    return st
+
+
+def ccr_sort_edges(store: Docstore, n_req: int, max_edge_len: int, edge_keys_in, edge_feats_in, edge_offsets,
+                   edge_keys_out, edge_feats_out, perm_out=None, stream=None) -> int:
+    """Raw call: per-request sort of (key, row) records by key on the device (device tensors in and out)."""
+    st = lib().ccr_sort_edges(store.handle, int(n_req), int(max_edge_len), _ptr(edge_keys_in), _ptr(edge_feats_in),
+                              _ptr(edge_offsets), _ptr(edge_keys_out), _ptr(edge_feats_out), _ptr(perm_out),
+                              _stream_ptr(stream))
+    _check(st, "ccr_sort_edges")
     return st
 
 

@@ -12,6 +12,7 @@
 #include <new>
 
 #include "ccr_join.cuh"
+#include "ccr_sort.cuh"
 #include "ccr_ws.cuh"
 
 namespace {
@@ -196,6 +197,11 @@ ccr_status allow_large_smem() {
         cudaGetLastError();
         return CCR_ERR_CUDA;
       }
+    }
+    if (i == 0 && cudaFuncSetAttribute(ccr::sort_edges_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kMaxSmemBytes) != cudaSuccess) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
     }
     const WsKernelFn ws[2] = {kVariants[i].ws_first, kVariants[i].ws_second};
     for (WsKernelFn f : ws) {
@@ -416,6 +422,40 @@ ccr_status ccr_docstore_device_status(ccr_docstore* s, void* stream) {
     return CCR_ERR_CUDA;
   }
   return s->status_host[0] == ccr::kDevWaitExpired ? CCR_ERR_DEVICE_WAIT : CCR_OK;
+}
+
+ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edge_len, const int64_t* keys_in,
+                          const void* feats_in, const int64_t* edge_offsets, int64_t* keys_out, void* feats_out,
+                          int32_t* perm_out, void* stream) {
+  if (!good(cs)) return CCR_ERR_BAD_HANDLE;
+  ccr_docstore* s = const_cast<ccr_docstore*>(cs);  // only the launch counter changes
+  if (n_req < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
+  if (max_edge_len > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;
+  if (n_req == 0 || max_edge_len == 0) return CCR_OK;
+  if (!keys_in || !feats_in || !edge_offsets || !keys_out || !feats_out) return CCR_ERR_INVALID_ARG;
+  if (keys_in == keys_out || feats_in == feats_out) return CCR_ERR_INVALID_ARG;  // not in place
+  if (!aligned16(feats_in) || !aligned16(feats_out) || (reinterpret_cast<uintptr_t>(keys_in) & 7u) ||
+      (reinterpret_cast<uintptr_t>(keys_out) & 7u) || (reinterpret_cast<uintptr_t>(perm_out) & 3u))
+    return CCR_ERR_INVALID_ARG;
+  if (max_edge_len > ccr::kSortSmemMaxKeys && perm_out == nullptr) return CCR_ERR_INVALID_ARG;  // long lists sort in perm_out
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  ccr::SortArgs a;
+  a.n_req = n_req;
+  a.keys_in = keys_in;
+  a.feats_in = static_cast<const uint8_t*>(feats_in);
+  a.edge_offsets = edge_offsets;
+  a.row_ch = s->edge_b / 16;
+  a.keys_out = keys_out;
+  a.feats_out = static_cast<uint8_t*>(feats_out);
+  a.perm_out = perm_out;
+  a.smem_keys = static_cast<int>(max_edge_len < ccr::kSortSmemMaxKeys ? max_edge_len : ccr::kSortSmemMaxKeys);
+  a.smem_keys = (a.smem_keys + 1) & ~1;  // keeps the index array 8-byte aligned behind the keys
+  const size_t smem = static_cast<size_t>(a.smem_keys) * 12;
+  ccr::sort_edges_kernel<<<static_cast<unsigned>(n_req), ccr::kSortThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  s->launches++;
+  if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+  return CCR_OK;
 }
 
 ccr_status ccr_docstore_selftest_wait(ccr_docstore* s, void* stream) {

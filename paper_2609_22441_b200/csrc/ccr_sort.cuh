@@ -1,0 +1,151 @@
+// Algorithm 1 step 1 of the paper on the device: per request, sort the viewer's affinity records by author
+// id (a_sorted, idx = sort(a); F_sorted = gather(F, idx)) so that unsorted request payloads can be joined.
+//
+// One 1024-thread block per request.  Keys and record indices are sorted together in shared memory with a
+// bitonic network written for arbitrary n (flip + disperse steps, every compare-exchange ascending, partners
+// beyond n skipped — equivalent to padding with +infinity); the order is on (key, index), which makes the
+// result the stable sort.  Lists that do not fit shared memory are sorted by the same network directly on the
+// output arrays in global memory (L2).  The rows then follow their keys in 16-byte chunks.
+#pragma once
+
+#include "ccr_device.cuh"
+
+namespace ccr {
+
+constexpr int kSortThreads = 1024;
+constexpr int kSortSmemMaxKeys = 19000;  // 12 bytes per record (int64 key + int32 index) within 227 KB
+
+// One pass structure for both element types: for partner mask j, the pairs (i, i ^ j) with i < i ^ j are
+// exactly the i whose bit `top(j)` is clear; pair number p (0 .. n/2) maps to i by inserting a zero there.
+__device__ __forceinline__ int pair_low_index(int p, int top_bit) {
+  const int low = p & ((1 << top_bit) - 1);
+  return ((p >> top_bit) << (top_bit + 1)) | low;
+}
+
+// (key, index) records in two arrays, ordered by key then index.
+__device__ __forceinline__ void sort_pairs_bitonic(long long* keys, int* idx, int n) {
+  if (n < 2) return;
+  for (int k = 2;; k <<= 1) {
+    // flip: i pairs with its mirror inside the block of k; then disperse at distances k/4, k/8, ..., 1
+    for (int j = k - 1;;) {
+      const int top = 31 - __clz(j);
+      for (int p = threadIdx.x;; p += blockDim.x) {
+        const int i = pair_low_index(p, top), l = i ^ j;
+        if (i >= n) break;  // i grows with p
+        if (l < n) {
+          const long long ki = keys[i], kl = keys[l];
+          const int ii = idx[i], il = idx[l];
+          if (ki > kl || (ki == kl && ii > il)) {
+            keys[i] = kl;
+            keys[l] = ki;
+            idx[i] = il;
+            idx[l] = ii;
+          }
+        }
+      }
+      __syncthreads();
+      if (j == k - 1) j = k >> 2; else j >>= 1;
+      if (j == 0) break;
+    }
+    if (k >= n) break;
+  }
+}
+
+// The same network on single 64-bit words (key << shift | index): half the shared-memory traffic.
+__device__ __forceinline__ void sort_words_bitonic(unsigned long long* w, int n) {
+  if (n < 2) return;
+  for (int k = 2;; k <<= 1) {
+    for (int j = k - 1;;) {
+      const int top = 31 - __clz(j);
+      for (int p = threadIdx.x;; p += blockDim.x) {
+        const int i = pair_low_index(p, top), l = i ^ j;
+        if (i >= n) break;  // i grows with p
+        if (l < n) {
+          const unsigned long long wi = w[i], wl = w[l];
+          if (wi > wl) {
+            w[i] = wl;
+            w[l] = wi;
+          }
+        }
+      }
+      __syncthreads();
+      if (j == k - 1) j = k >> 2; else j >>= 1;
+      if (j == 0) break;
+    }
+    if (k >= n) break;
+  }
+}
+
+struct SortArgs {
+  int n_req;
+  const int64_t* keys_in;
+  const uint8_t* feats_in;
+  const int64_t* edge_offsets;
+  int row_ch;            // 16-byte chunks per feature row
+  int64_t* keys_out;
+  uint8_t* feats_out;
+  int* perm_out;         // may be null when every list fits shared memory
+  int smem_keys;         // records the dynamic shared memory can hold
+};
+
+__global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_sort[];
+  const int r = blockIdx.x;
+  const long long e0 = __ldg(a.edge_offsets + r);
+  const long long Kl = __ldg(a.edge_offsets + r + 1) - e0;
+  if (Kl <= 0) return;
+  const int K = static_cast<int>(Kl);
+  const bool in_smem = K <= a.smem_keys;
+  if (!in_smem && a.perm_out == nullptr) return;  // refused on the host; never reached
+  long long* keys = in_smem ? reinterpret_cast<long long*>(smem_sort) : reinterpret_cast<long long*>(a.keys_out + e0);
+  int* idx = in_smem ? reinterpret_cast<int*>(smem_sort + static_cast<size_t>(a.smem_keys) * 8) : a.perm_out + e0;
+  // keys that leave room for the record index in one 64-bit word (non-negative, below 2^(63 - index bits)) are
+  // sorted as single words: key << shift | index orders like (key, index)
+  int idx_bits = 1;
+  while ((1 << idx_bits) < K) ++idx_bits;
+  long long kmax = 0;
+  int negative = 0;
+  for (int i = threadIdx.x; i < K; i += blockDim.x) {
+    const long long k = __ldg(a.keys_in + e0 + i);
+    kmax = max(kmax, k);
+    negative |= (k < 0);
+  }
+  const bool packable = __syncthreads_or(negative || (kmax >> (63 - idx_bits)) != 0) == 0;
+  if (packable) {
+    unsigned long long* w = reinterpret_cast<unsigned long long*>(keys);
+    for (int i = threadIdx.x; i < K; i += blockDim.x)
+      w[i] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
+    __syncthreads();
+    sort_words_bitonic(w, K);
+    const unsigned long long low = (1ull << idx_bits) - 1;
+    for (int i = threadIdx.x; i < K; i += blockDim.x) {  // unpack; each thread rewrites only its own slots
+      const unsigned long long v = w[i];
+      idx[i] = static_cast<int>(v & low);
+      keys[i] = static_cast<long long>(v >> idx_bits);
+    }
+    __syncthreads();
+  } else {
+    for (int i = threadIdx.x; i < K; i += blockDim.x) {
+      keys[i] = __ldg(a.keys_in + e0 + i);
+      idx[i] = i;
+    }
+    __syncthreads();
+    sort_pairs_bitonic(keys, idx, K);
+  }
+  if (in_smem) {
+    for (int i = threadIdx.x; i < K; i += blockDim.x) {
+      a.keys_out[e0 + i] = keys[i];
+      if (a.perm_out) a.perm_out[e0 + i] = idx[i];
+    }
+  }
+  // rows follow their keys
+  const long long chunks = static_cast<long long>(K) * a.row_ch;
+  const uint4* src = reinterpret_cast<const uint4*>(a.feats_in) + e0 * a.row_ch;
+  uint4* dst = reinterpret_cast<uint4*>(a.feats_out) + e0 * a.row_ch;
+  for (long long c = threadIdx.x; c < chunks; c += blockDim.x) {
+    const int row = static_cast<int>(c / a.row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * a.row_ch);
+    dst[c] = __ldg(src + static_cast<long long>(idx[row]) * a.row_ch + piece);
+  }
+}
+
+}  // namespace ccr

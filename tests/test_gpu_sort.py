@@ -1,0 +1,114 @@
+"""GPU parity of ccr_sort_edges (Algorithm 1 step 1) against the CPU oracle, and of the join fed with
+device-sorted records."""
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2609_22441_b200 import workloads as W
+
+from helpers import gpu_join
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2609_22441_b200 import binding, build
+
+    build.build()
+    return binding
+
+
+def _shuffle_records(batch, seed, duplicate_keys=False):
+    rng = np.random.default_rng(seed)
+    keys, feats = batch.edge_keys.copy(), batch.edge_feats.copy()
+    for r in range(batch.n_req):
+        a, z = int(batch.edge_offsets[r]), int(batch.edge_offsets[r + 1])
+        p = rng.permutation(z - a)
+        keys[a:z], feats[a:z] = batch.edge_keys[a:z][p], batch.edge_feats[a:z][p]
+        if duplicate_keys and z - a > 4:
+            keys[a:z:3] = keys[a]  # many equal keys: the order among them must be the input order
+    return keys, feats
+
+
+def _gpu_sort(B, store, keys, feats, eo, with_perm=True):
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    k_in, f_in, o = dev(keys), dev(feats), dev(eo)
+    guard = 64
+    k_buf = torch.full((len(keys) + 2 * guard,), -7, dtype=torch.int64, device="cuda")
+    f_buf = torch.full((feats.shape[0] + 2 * guard, feats.shape[1]), 7.0, dtype=torch.float16, device="cuda")
+    p_buf = torch.full((len(keys) + 2 * guard,), -7, dtype=torch.int32, device="cuda")
+    E = len(keys)
+    k_out, f_out, p_out = k_buf[guard:guard + E], f_buf[guard:guard + E], p_buf[guard:guard + E]
+    n_req = len(eo) - 1
+    max_len = int(np.max(np.diff(eo))) if n_req else 0
+    B.ccr_sort_edges(store, n_req, max_len, k_in, f_in, o, k_out, f_out, p_out if with_perm else None)
+    torch.cuda.synchronize()
+    assert (k_buf[:guard] == -7).all() and (k_buf[guard + E:] == -7).all()
+    assert (f_buf[:guard] == 7).all() and (f_buf[guard + E:] == 7).all()
+    assert (p_buf[:guard] == -7).all() and (p_buf[guard + E:] == -7).all()
+    return k_out, f_out, p_out
+
+
+@pytest.mark.parametrize("dups", [False, True])
+def test_sort_matches_oracle_on_config1_and_the_join_accepts_it(B, dups):
+    wl = W.config1(n_docs=100_000, n_req=24, n_cand=3_000)
+    b = wl.batch
+    keys_u, feats_u = _shuffle_records(b, 1, duplicate_keys=dups)
+    want_k, want_f, want_p = oracle.sort_edges(keys_u, feats_u, b.edge_offsets)
+    store = B.store_from_workload(wl)
+    k, f, p = _gpu_sort(B, store, keys_u, feats_u, b.edge_offsets)
+    assert np.array_equal(k.cpu().numpy(), want_k)
+    assert np.array_equal(p.cpu().numpy(), want_p)
+    assert np.array_equal(f.cpu().numpy().view(np.uint16), want_f.view(np.uint16))
+    if not dups:
+        # sorted on the device, joined on the device == oracle join of the originally sorted records
+        db = B.DeviceBatch(b)
+        db.edge_keys, db.edge_feats = k.contiguous(), f.contiguous()
+        rows, mask = gpu_join(store, db)
+        want_rows, want_mask = oracle.join_workload(wl)
+        assert np.array_equal(rows, want_rows) and np.array_equal(mask, want_mask)
+    store.free()
+
+
+@pytest.mark.parametrize("lens", [[0, 1, 2, 3, 31, 32, 33, 1023, 1024, 1025, 4097], [18_999, 19_000, 7], [19_001, 40_000, 5, 0, 65_537]])
+def test_sort_lengths_around_the_block_and_shared_memory_limits(B, lens):
+    rng = np.random.default_rng(sum(lens))
+    keys = np.concatenate([rng.integers(0, 10 * max(n, 1), size=n) for n in lens] + [np.empty(0, np.int64)]).astype(np.int64)
+    feats = rng.standard_normal((len(keys), 64)).astype(np.float16)
+    eo = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    want_k, want_f, want_p = oracle.sort_edges(keys, feats, eo)
+    wl = W.config3(n_docs=1000, n_req=1, n_cand=10, gen_doc_feats=True, extra_pools=0)  # a store with 128-byte edge rows
+    store = B.store_from_workload(wl)
+    k, f, p = _gpu_sort(B, store, keys, feats, eo)
+    assert np.array_equal(k.cpu().numpy(), want_k) and np.array_equal(p.cpu().numpy(), want_p)
+    assert np.array_equal(f.cpu().numpy().view(np.uint16), want_f.view(np.uint16))
+    if max(lens) <= 19_000:
+        k2, f2, _ = _gpu_sort(B, store, keys, feats, eo, with_perm=False)
+        assert np.array_equal(k2.cpu().numpy(), want_k) and np.array_equal(f2.cpu().numpy().view(np.uint16), want_f.view(np.uint16))
+    else:
+        with pytest.raises(B.CcrError) as e:
+            _gpu_sort(B, store, keys, feats, eo, with_perm=False)
+        assert e.value.status == B.CCR_ERR_INVALID_ARG
+    store.free()
+
+
+def test_sort_with_keys_that_cannot_share_a_word_with_the_index(B):
+    """Keys near INT64_MAX (and negative ones, outside the join's contract but legal for the sort) force the
+    two-array network; mixed with small-key requests in one launch."""
+    rng = np.random.default_rng(9)
+    imax = np.iinfo(np.int64).max
+    lens = [700, 5000, 64, 3000]
+    parts = [imax - rng.integers(0, 10_000, size=lens[0]), rng.integers(0, 1 << 40, size=lens[1]),
+             rng.integers(-50, 50, size=lens[2]), rng.integers(0, 1 << 62, size=lens[3])]
+    keys = np.concatenate(parts).astype(np.int64)
+    feats = rng.standard_normal((len(keys), 64)).astype(np.float16)
+    eo = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    want_k, want_f, want_p = oracle.sort_edges(keys, feats, eo)
+    wl = W.config3(n_docs=1000, n_req=1, n_cand=10, gen_doc_feats=True, extra_pools=0)
+    store = B.store_from_workload(wl)
+    k, f, p = _gpu_sort(B, store, keys, feats, eo)
+    assert np.array_equal(k.cpu().numpy(), want_k) and np.array_equal(p.cpu().numpy(), want_p)
+    assert np.array_equal(f.cpu().numpy().view(np.uint16), want_f.view(np.uint16))
+    store.free()

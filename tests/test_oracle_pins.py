@@ -331,3 +331,52 @@ def test_generators_are_deterministic():
     for r in range(3):
         k = a.batch.edge_keys[a.batch.edge_offsets[r]:a.batch.edge_offsets[r + 1]]
         assert np.all(np.diff(k) > 0)
+
+
+# ---------------------------------------------------------------- Algorithm 1 step 1 (sort of the affinity records)
+def _unsorted_batch(seed, n_req, kmax, alphabet, dup=False):
+    rng = np.random.default_rng(seed)
+    keys_l, feats_l = [], []
+    for _ in range(n_req):
+        k = int(rng.integers(0, kmax + 1))
+        keys = rng.integers(0, alphabet, size=k) if dup else rng.permutation(alphabet)[:k]
+        keys_l.append(keys.astype(np.int64))
+        feats_l.append(rng.standard_normal((k, 8)).astype(np.float16))
+    eo = np.concatenate([[0], np.cumsum([len(k) for k in keys_l])]).astype(np.int64)
+    return np.concatenate(keys_l + [np.empty(0, np.int64)]), np.concatenate(feats_l + [np.empty((0, 8), np.float16)]), eo
+
+
+@pytest.mark.parametrize("dup", [False, True])
+def test_sort_step_matches_library_sort_and_gather(dup):
+    keys, feats, eo = _unsorted_batch(3 + dup, n_req=9, kmax=300, alphabet=200 if dup else 5000, dup=dup)
+    ks, fs, perm = oracle.sort_edges(keys, feats, eo)
+    for r in range(len(eo) - 1):
+        a, z = int(eo[r]), int(eo[r + 1])
+        # numpy's stable argsort, and Algorithm 1 step 1 restated with torch.sort(stable=True) + gather
+        order = np.argsort(keys[a:z], kind="stable")
+        assert np.array_equal(perm[a:z], order)
+        assert np.array_equal(ks[a:z], keys[a:z][order])
+        assert np.array_equal(fs[a:z].view(np.uint16), feats[a:z][order].view(np.uint16))
+        tk, tidx = torch.sort(torch.from_numpy(keys[a:z]), stable=True)
+        assert np.array_equal(tk.numpy(), ks[a:z]) and np.array_equal(tidx.numpy(), perm[a:z])
+        assert np.all(np.diff(ks[a:z]) >= 0)
+        assert sorted(perm[a:z].tolist()) == list(range(z - a))
+
+
+def test_join_after_sort_equals_naive_scan_on_unsorted_records():
+    """Eq. 1 does not ask for sorted records: the naive scan on the *unsorted* (a, F) must equal the join of
+    the records sorted by Algorithm 1 step 1 (unique keys)."""
+    wl = tiny_workload(21, n_docs=60, alphabet=40, n_req=4, kmax=25, nmax=50, second=False, req_dim=4)
+    b, s = wl.batch, wl.store
+    rng = np.random.default_rng(2)
+    keys_u, feats_u = b.edge_keys.copy(), b.edge_feats.copy()
+    for r in range(b.n_req):
+        a, z = int(b.edge_offsets[r]), int(b.edge_offsets[r + 1])
+        p = rng.permutation(z - a)
+        keys_u[a:z], feats_u[a:z] = b.edge_keys[a:z][p], b.edge_feats[a:z][p]
+    ks, fs, _ = oracle.sort_edges(keys_u, feats_u, b.edge_offsets)
+    assert np.array_equal(ks, b.edge_keys) and np.array_equal(fs.view(np.uint16), b.edge_feats.view(np.uint16))
+    rows, mask = oracle.join(s.doc_feats, s.author_ids, ks, fs, b.edge_offsets, b.cand_idx, b.cand_offsets, req_feats=b.req_feats)
+    brows, bmask = brute_force.join(s.doc_feats, s.author_ids, keys_u, feats_u, b.edge_offsets, b.cand_idx, b.cand_offsets,
+                                    req_feats=b.req_feats)
+    assert np.array_equal(mask, bmask) and np.array_equal(rows, brows)
