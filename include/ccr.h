@@ -29,6 +29,7 @@ extern "C" {
 
 typedef struct ccr_docstore ccr_docstore;   /* opaque; owns its device memory */
 typedef struct ccr_workspace ccr_workspace; /* opaque; device staging for the host-buffer entry */
+typedef struct ccr_idindex ccr_idindex;     /* opaque; sorted document ids + sampled search levels on the device */
 
 typedef enum {
   CCR_OK = 0,
@@ -152,6 +153,22 @@ ccr_status ccr_join_batch(const ccr_docstore* store,
 ccr_status ccr_sort_edges(const ccr_docstore* store, int32_t n_req, int64_t max_edge_len,
                           const int64_t* edge_keys_in, const void* edge_feats_in, const int64_t* edge_offsets,
                           int64_t* edge_keys_out, void* edge_feats_out, int32_t* perm_out, void* stream);
+
+/* Document-id resolution on the GPU (Section 6.3.1 "Document ID Resolution", Eq. 6): pos(q) = position of
+ * document id q in the index, or -1 when q is not indexed.
+ *
+ * ccr_idindex_create copies n_ids ascending, unique ids (HOST or DEVICE source per src_on_device) into device
+ * memory and builds the sampled search levels above them (every 32nd key, repeatedly, until at most 16,384
+ * keys remain).  `positions` (optional, int32[n_ids], same source side) gives the store position of each id;
+ * NULL means the position of an id is its rank.  Synchronous; allocates 8.3 bytes per id (+4 with positions).
+ * ccr_resolve_ids writes out_pos[i] = position of query_ids[i] or -1 for n_queries DEVICE queries: one kernel
+ * on `stream`, no allocation, no sync.  Ids that break the ascending order give unspecified positions but
+ * every access stays in bounds.  The output is what ccr_join_batch takes as cand_idx (-1 = unresolved).      */
+ccr_status ccr_idindex_create(int32_t device, int64_t n_ids, const int64_t* sorted_ids, const int32_t* positions,
+                              int src_on_device, ccr_idindex** out);
+ccr_status ccr_idindex_free(ccr_idindex* index);
+ccr_status ccr_resolve_ids(const ccr_idindex* index, int64_t n_queries, const int64_t* query_ids,
+                           int32_t* out_pos, void* stream);
 
 /* Device staging buffers for ccr_join_batch_host, sized for the largest batch the caller will pass.
  * HOST calls; allocation happens here, never inside the join.                                      */

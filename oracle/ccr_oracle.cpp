@@ -28,6 +28,9 @@
 //   * Algorithm 1 step 1 (ccr_oracle_sort_edges): a_sorted, idx = sort(a); F_sorted = gather(F, idx), per
 //     request, as std::stable_sort of the record indices by key followed by a row-by-row copy.
 //
+//   * Eq. 6 (Section 6.3.1, ccr_oracle_resolve_ids): pos(q) = H[q] if q is indexed, else -1, evaluated with
+//     std::lower_bound on the ascending id array (the paper's own first design).
+//
 // Plain, slow and unblocked on purpose; single-threaded unless n_threads > 1, in which case the flat
 // candidate range is cut into contiguous chunks, one std::thread each.
 #include <algorithm>
@@ -282,6 +285,17 @@ int ccr_oracle_sort_edges(int32_t n_req, const int64_t* keys_in, const void* fea
       std::memcpy(fout + (e0 + i) * row_bytes, fin + (e0 + src) * row_bytes, static_cast<size_t>(row_bytes));
       if (perm_out) perm_out[e0 + i] = src;
     }
+  }
+  return 0;
+}
+
+// Eq. 6: out_pos[i] = position of query i in the index (positions[rank] when given, else the rank), or -1.
+int ccr_oracle_resolve_ids(int64_t n_ids, const int64_t* sorted_ids, const int32_t* positions, int64_t n_queries,
+                           const int64_t* queries, int32_t* out_pos) {
+  for (int64_t i = 0; i < n_queries; ++i) {
+    const int64_t* it = std::lower_bound(sorted_ids, sorted_ids + n_ids, queries[i]);
+    const int64_t rank = it - sorted_ids;
+    out_pos[i] = (rank < n_ids && *it == queries[i]) ? (positions ? positions[rank] : static_cast<int32_t>(rank)) : -1;
   }
   return 0;
 }

@@ -46,6 +46,8 @@ def _load():
             i64, vp, i64, vp, i32, vp, vp, i32, i32, u64,
             i32, vp, vp, vp, vp, vp, vp, i64, i32, vp, vp, i32,
         ]
+        lib.ccr_oracle_resolve_ids.restype = ctypes.c_int
+        lib.ccr_oracle_resolve_ids.argtypes = [i64, vp, vp, i64, vp, vp]
         lib.ccr_oracle_sort_edges.restype = ctypes.c_int
         lib.ccr_oracle_sort_edges.argtypes = [i32, vp, vp, vp, i64, vp, vp, vp]
         lib.ccr_oracle_half_to_float_bits.restype = ctypes.c_uint32
@@ -149,6 +151,17 @@ def sort_edges(edge_keys: np.ndarray, edge_feats: np.ndarray, edge_offsets: np.n
     if rc != 0:
         raise ValueError("malformed offsets")
     return keys_out, feats_out, perm
+
+
+def resolve_ids(sorted_ids: np.ndarray, queries: np.ndarray, positions: Optional[np.ndarray] = None) -> np.ndarray:
+    """Eq. 6: position of each query id in the ascending id array (positions[rank] if given), or -1."""
+    lib = _load()
+    sorted_ids = _c(sorted_ids, np.int64)
+    queries = _c(queries, np.int64)
+    positions = _c(positions, np.int32)
+    out = np.full(len(queries), -77, dtype=np.int32)
+    lib.ccr_oracle_resolve_ids(len(sorted_ids), _ptr(sorted_ids), _ptr(positions), len(queries), _ptr(queries), _ptr(out))
+    return out
 
 
 def join_workload(wl, first_degree_only: bool = False, n_threads: int = 1):

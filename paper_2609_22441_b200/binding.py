@@ -42,7 +42,7 @@ EXPORTS = (
     "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
     "ccr_static_payload_capacity", "ccr_join_payload_static", "ccr_docstore_selftest_wait",
-    "ccr_sort_edges",
+    "ccr_sort_edges", "ccr_idindex_create", "ccr_idindex_free", "ccr_resolve_ids",
 )
 
 
@@ -103,6 +103,12 @@ def lib() -> ctypes.CDLL:
     L.ccr_static_payload_capacity.argtypes = []
     L.ccr_join_payload_static.restype = ctypes.c_int
     L.ccr_join_payload_static.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
+    L.ccr_idindex_create.restype = ctypes.c_int
+    L.ccr_idindex_create.argtypes = [i32, i64, vp, vp, ctypes.c_int, ctypes.POINTER(vp)]
+    L.ccr_idindex_free.restype = ctypes.c_int
+    L.ccr_idindex_free.argtypes = [vp]
+    L.ccr_resolve_ids.restype = ctypes.c_int
+    L.ccr_resolve_ids.argtypes = [vp, i64, vp, vp, vp]
     L.ccr_sort_edges.restype = ctypes.c_int
     L.ccr_sort_edges.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, vp, vp]
     L.ccr_docstore_selftest_wait.restype = ctypes.c_int
@@ -318,6 +324,43 @@ def ccr_join_payload_static(store: Docstore, n_req: int, total_cands: int, max_e
                                        _ptr(out_mask), int(flags), _stream_ptr(stream))
     _check(st, "ccr_join_payload_static")
     return st
+
+
+class IdIndex:
+    """ccr_idindex handle: sorted document ids (+ optional positions) with sampled search levels on the device."""
+
+    def __init__(self, sorted_ids, positions=None, device: int = 0):
+        self._h = ctypes.c_void_p()
+        on_dev = isinstance(sorted_ids, torch.Tensor) and sorted_ids.is_cuda
+        if positions is not None and (isinstance(positions, torch.Tensor) and positions.is_cuda) != on_dev:
+            raise ValueError("ids and positions must be on the same side")
+        self.n_ids = int(sorted_ids.shape[0])
+        self.device = int(device)
+        _check(lib().ccr_idindex_create(int(device), self.n_ids, _ptr(sorted_ids), _ptr(positions), 1 if on_dev else 0,
+                                        ctypes.byref(self._h)), "ccr_idindex_create")
+
+    @property
+    def handle(self):
+        return self._h
+
+    def resolve(self, query_ids: torch.Tensor, out_pos: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """ccr_resolve_ids on a device tensor of int64 queries; returns int32 positions (-1 = not indexed)."""
+        if out_pos is None:
+            out_pos = torch.empty(query_ids.shape, dtype=torch.int32, device=query_ids.device)
+        _check(lib().ccr_resolve_ids(self._h, int(query_ids.numel()), _ptr(query_ids), _ptr(out_pos), _stream_ptr(stream)),
+               "ccr_resolve_ids")
+        return out_pos
+
+    def free(self) -> None:
+        if self._h:
+            _check(lib().ccr_idindex_free(self._h), "ccr_idindex_free")
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
 
 
 def ccr_sort_edges(store: Docstore, n_req: int, max_edge_len: int, edge_keys_in, edge_feats_in, edge_offsets,

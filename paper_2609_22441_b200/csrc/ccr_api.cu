@@ -12,6 +12,7 @@
 #include <new>
 
 #include "ccr_join.cuh"
+#include "ccr_resolve.cuh"
 #include "ccr_sort.cuh"
 #include "ccr_ws.cuh"
 
@@ -19,6 +20,7 @@ namespace {
 
 constexpr uint64_t kStoreMagic = 0x43435253544f5245ull;  // "CCRSTORE"
 constexpr uint64_t kWsMagic = 0x4343525753504143ull;     // "CCRWSPAC"
+constexpr uint64_t kIxMagic = 0x4343524944494e44ull;     // "CCRIDIND"
 constexpr int kMaxSmemBytes = 227 * 1024;
 constexpr int kDefaultTileWs = 256;        // candidates per ring slot of the warp-specialised kernel
 constexpr int kDefaultTileTwoPhase = 1024; // candidates per search/copy phase pair of the two-phase kernel
@@ -80,6 +82,18 @@ struct ccr_workspace {
   uint8_t* req_feats;
   uint8_t* out_rows;
   uint8_t* out_mask;
+};
+
+struct ccr_idindex {
+  uint64_t magic;
+  int device;
+  int n_sms;
+  int64_t n_ids;
+  int n_levels;
+  int64_t* level[ccr::kResolveMaxLevels];  // level[0] = sorted ids (owned copy)
+  long long count[ccr::kResolveMaxLevels];
+  int32_t* positions;                      // owned copy, or null
+  int64_t launches;
 };
 
 namespace {
@@ -422,6 +436,116 @@ ccr_status ccr_docstore_device_status(ccr_docstore* s, void* stream) {
     return CCR_ERR_CUDA;
   }
   return s->status_host[0] == ccr::kDevWaitExpired ? CCR_ERR_DEVICE_WAIT : CCR_OK;
+}
+
+ccr_status ccr_idindex_free(ccr_idindex* ix) {
+  if (ix == nullptr || ix->magic != kIxMagic) return CCR_ERR_BAD_HANDLE;
+  DeviceScope scope(ix->device);
+  ix->magic = 0;
+  for (int l = 0; l < ccr::kResolveMaxLevels; ++l) cudaFree(ix->level[l]);
+  cudaFree(ix->positions);
+  delete ix;
+  return CCR_OK;
+}
+
+ccr_status ccr_idindex_create(int32_t device, int64_t n_ids, const int64_t* sorted_ids, const int32_t* positions,
+                              int src_on_device, ccr_idindex** out) {
+  if (out == nullptr) return CCR_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (device < 0 || n_ids < 0 || (n_ids > 0 && sorted_ids == nullptr)) return CCR_ERR_INVALID_ARG;
+  if (n_ids > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;  // positions are int32
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) {
+    cudaGetLastError();
+    return CCR_ERR_CUDA;
+  }
+  DeviceScope scope(device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  // level sizes: sample every 32nd key until the top fits shared memory
+  long long count[ccr::kResolveMaxLevels];
+  int n_levels = 1;
+  count[0] = n_ids;
+  while (count[n_levels - 1] > ccr::kResolveTopMax) {
+    if (n_levels == ccr::kResolveMaxLevels) return CCR_ERR_UNSUPPORTED;
+    count[n_levels] = count[n_levels - 1] >> ccr::kResolveFanLog2;
+    ++n_levels;
+  }
+  if (n_levels == 1) {  // a tiny index still gets a (possibly empty) top level of its own
+    count[1] = count[0] >> ccr::kResolveFanLog2;
+    n_levels = 2;
+  }
+  size_t need = 4096 + (positions ? static_cast<size_t>(n_ids) * 4 : 0);
+  for (int l = 0; l < n_levels; ++l) need += static_cast<size_t>(count[l]) * 8 + 256;
+  size_t free_b = 0, total_b = 0;
+  if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return CCR_ERR_CUDA;
+  if (need > free_b) return CCR_ERR_OOM;
+  ccr_idindex* ix = new (std::nothrow) ccr_idindex();
+  if (ix == nullptr) return CCR_ERR_OOM;
+  std::memset(ix, 0, sizeof(*ix));
+  ix->device = device;
+  ix->n_ids = n_ids;
+  ix->n_levels = n_levels;
+  bool ok = cudaDeviceGetAttribute(&ix->n_sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess;
+  for (int l = 0; l < n_levels && ok; ++l) {
+    ix->count[l] = count[l];
+    ok = cudaMalloc(&ix->level[l], static_cast<size_t>(count[l]) * 8 + 256) == cudaSuccess;
+  }
+  const cudaMemcpyKind kind = src_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  if (ok && n_ids > 0) ok = cudaMemcpy(ix->level[0], sorted_ids, static_cast<size_t>(n_ids) * 8, kind) == cudaSuccess;
+  if (ok && positions && n_ids > 0) {
+    ok = cudaMalloc(&ix->positions, static_cast<size_t>(n_ids) * 4) == cudaSuccess;
+    ok = ok && cudaMemcpy(ix->positions, positions, static_cast<size_t>(n_ids) * 4, kind) == cudaSuccess;
+  }
+  for (int l = 1; l < n_levels && ok; ++l) {
+    if (count[l] == 0) continue;
+    const unsigned blocks = static_cast<unsigned>((count[l] + 255) / 256 < 8192 ? (count[l] + 255) / 256 : 8192);
+    ccr::build_level_kernel<<<blocks, 256>>>(ix->level[l - 1], count[l - 1], ix->level[l], count[l]);
+    ix->launches++;
+    ok = cudaGetLastError() == cudaSuccess;
+  }
+  ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(ccr::resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  ccr::kResolveTopMax * 8 + 256) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    ix->magic = kIxMagic;
+    ccr_idindex_free(ix);
+    return CCR_ERR_CUDA;
+  }
+  ix->magic = kIxMagic;
+  *out = ix;
+  return CCR_OK;
+}
+
+ccr_status ccr_resolve_ids(const ccr_idindex* cix, int64_t n_queries, const int64_t* query_ids, int32_t* out_pos,
+                           void* stream) {
+  if (cix == nullptr || cix->magic != kIxMagic) return CCR_ERR_BAD_HANDLE;
+  ccr_idindex* ix = const_cast<ccr_idindex*>(cix);  // only the launch counter changes
+  if (n_queries < 0) return CCR_ERR_INVALID_ARG;
+  if (n_queries == 0) return CCR_OK;
+  if (!query_ids || !out_pos) return CCR_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(query_ids) & 7u) || (reinterpret_cast<uintptr_t>(out_pos) & 3u)) return CCR_ERR_INVALID_ARG;
+  DeviceScope scope(ix->device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  ccr::ResolveArgs a;
+  for (int l = 0; l < ccr::kResolveMaxLevels; ++l) {
+    a.level[l] = ix->level[l];
+    a.count[l] = ix->count[l];
+  }
+  a.n_levels = ix->n_levels;
+  a.positions = ix->positions;
+  a.n_queries = n_queries;
+  a.queries = query_ids;
+  a.out_pos = out_pos;
+  const long long per_block = static_cast<long long>(ccr::kResolveThreads) * ccr::kResolveUnroll;
+  long long blocks = (n_queries + per_block - 1) / per_block;
+  const long long cap = static_cast<long long>(ix->n_sms) * 4;  // the top level is re-read by every block
+  if (blocks > cap) blocks = cap;
+  const size_t smem = static_cast<size_t>(ix->count[ix->n_levels - 1]) * 8 + 16;
+  ccr::resolve_kernel<<<static_cast<unsigned>(blocks), ccr::kResolveThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  ix->launches++;
+  if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+  return CCR_OK;
 }
 
 ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edge_len, const int64_t* keys_in,

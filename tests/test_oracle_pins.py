@@ -380,3 +380,21 @@ def test_join_after_sort_equals_naive_scan_on_unsorted_records():
     brows, bmask = brute_force.join(s.doc_feats, s.author_ids, keys_u, feats_u, b.edge_offsets, b.cand_idx, b.cand_offsets,
                                     req_feats=b.req_feats)
     assert np.array_equal(mask, bmask) and np.array_equal(rows, brows)
+
+
+# ---------------------------------------------------------------- Eq. 6 (document id -> position)
+def test_id_resolution_matches_a_hash_map_and_searchsorted():
+    rng = np.random.default_rng(8)
+    ids = np.cumsum(rng.integers(1, 9, size=5000)).astype(np.int64) * 2  # ascending, unique, even
+    positions = rng.permutation(len(ids)).astype(np.int32)
+    present = ids[rng.integers(0, len(ids), size=3000)]
+    absent = np.concatenate([present[:500] + 1, [ids[0] - 2, ids[-1] + 2, -5, np.iinfo(np.int64).max]])
+    q = np.concatenate([present, absent])
+    rng.shuffle(q)
+    H = {int(k): int(p) for k, p in zip(ids, positions)}  # the paper's CPU design: a hash map
+    want = np.array([H.get(int(x), -1) for x in q], dtype=np.int32)
+    assert np.array_equal(oracle.resolve_ids(ids, q, positions), want)
+    rank = np.searchsorted(ids, q)
+    hit = (rank < len(ids)) & (ids[np.minimum(rank, len(ids) - 1)] == q)
+    assert np.array_equal(oracle.resolve_ids(ids, q), np.where(hit, rank, -1).astype(np.int32))
+    assert np.array_equal(oracle.resolve_ids(ids[:0], q), np.full(len(q), -1, np.int32))
