@@ -19,7 +19,7 @@ constexpr int kResolveFanLog2 = 5;                 // 32 keys = one 256-byte win
 constexpr int kResolveMaxLevels = 8;
 constexpr int kResolveTopMax = 16384;              // keys of the top level (128 KB of shared memory)
 constexpr int kResolveThreads = 256;
-constexpr int kResolveUnroll = 4;                 // queries a lane keeps in flight
+constexpr int kResolveUnroll = 8;                 // queries a lane keeps in flight
 
 struct ResolveArgs {
   const int64_t* level[kResolveMaxLevels];         // level[0] = the sorted ids, level[n_levels-1] = top
@@ -65,12 +65,34 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
     for (int l = top_l - 1; l >= 0; --l) {
       const int64_t* lev = a.level[l];
       const long long n = a.count[l];
+      // the searches of the lane's queries advance in lock step, one probe of each per step, so that their
+      // memory accesses are independent and in flight together (a window has at most 32 keys: 5 halvings + 1)
+      long long lo[kResolveUnroll];
+      int w[kResolveUnroll];
 #pragma unroll
       for (int u = 0; u < kResolveUnroll; ++u) {
-        const long long lo = c[u] << kResolveFanLog2;
-        const long long rest = n - lo;
-        const int w = rest < (1 << kResolveFanLog2) ? static_cast<int>(rest > 0 ? rest : 0) : (1 << kResolveFanLog2);
-        c[u] = lo + lower_bound_global(lev + lo, w, q[u]);
+        lo[u] = c[u] << kResolveFanLog2;
+        const long long rest = n - lo[u];
+        w[u] = rest < (1 << kResolveFanLog2) ? static_cast<int>(rest > 0 ? rest : 0) : (1 << kResolveFanLog2);
+      }
+#pragma unroll
+      for (int step = 0; step < kResolveFanLog2; ++step) {
+        int64_t probe[kResolveUnroll];
+#pragma unroll
+        for (int u = 0; u < kResolveUnroll; ++u) probe[u] = w[u] > 1 ? __ldg(lev + lo[u] + (w[u] >> 1) - 1) : 0;
+#pragma unroll
+        for (int u = 0; u < kResolveUnroll; ++u) {
+          if (w[u] > 1) {
+            const int half = w[u] >> 1;
+            if (probe[u] < q[u]) lo[u] += half;
+            w[u] -= half;
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kResolveUnroll; ++u) {
+        if (w[u] == 1 && __ldg(lev + lo[u]) < q[u]) ++lo[u];
+        c[u] = lo[u];
       }
     }
 #pragma unroll
