@@ -537,7 +537,7 @@ ccr_status ccr_resolve_ids(const ccr_idindex* cix, int64_t n_queries, const int6
   a.n_queries = n_queries;
   a.queries = query_ids;
   a.out_pos = out_pos;
-  const long long per_block = static_cast<long long>(ccr::kResolveThreads) * ccr::kResolveUnroll;
+  const long long per_block = static_cast<long long>(ccr::kResolveThreads);
   long long blocks = (n_queries + per_block - 1) / per_block;
   const long long cap = static_cast<long long>(ix->n_sms) * 4;  // the top level is re-read by every block
   if (blocks > cap) blocks = cap;

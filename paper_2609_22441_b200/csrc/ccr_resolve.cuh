@@ -50,14 +50,15 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
   // (whole window per coalesced access, __ballot_sync rank) was measured and is slower at every batch size:
   // 886 vs 743 us for 1.92M queries, the extra shuffles and the lower number of independent accesses in
   // flight outweigh the saved sector fetches.
-  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x * kResolveUnroll;
-  for (long long base = (blockIdx.x * static_cast<long long>(blockDim.x)) * kResolveUnroll + threadIdx.x; base < a.n_queries;
-       base += stride) {
+  // query u of a lane is `threads` apart from query u-1, so that a small launch still spreads over all blocks
+  const long long threads = static_cast<long long>(gridDim.x) * blockDim.x;
+  for (long long base = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; base < a.n_queries;
+       base += threads * kResolveUnroll) {
     int64_t q[kResolveUnroll];
     long long c[kResolveUnroll];  // number of keys of the current level that are below q
 #pragma unroll
     for (int u = 0; u < kResolveUnroll; ++u) {
-      const long long j = base + static_cast<long long>(u) * blockDim.x;
+      const long long j = base + static_cast<long long>(u) * threads;
       q[u] = j < a.n_queries ? __ldg(a.queries + j) : 0;
       c[u] = lower_bound_smem(top, n_top, q[u]);
     }
@@ -97,7 +98,7 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
     }
 #pragma unroll
     for (int u = 0; u < kResolveUnroll; ++u) {
-      const long long j = base + static_cast<long long>(u) * blockDim.x;
+      const long long j = base + static_cast<long long>(u) * threads;
       if (j >= a.n_queries) continue;
       int pos = -1;
       if (c[u] < a.count[0] && __ldg(a.level[0] + c[u]) == q[u])
