@@ -63,6 +63,8 @@ def parse_args():
     p.add_argument("--key-cap", type=int, default=0, help="keys staged per request (0 = library default)")
     p.add_argument("--streamers", type=int, default=0)
     p.add_argument("--resolvers", type=int, default=0)
+    p.add_argument("--padded", action="store_true",
+                   help="time the padded batch layout: ccr_compact_valid + ccr_join_batch_padded into T[n_req, n_max]")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--timed-only", action="store_true",
                    help="only warm-up and the timed region (for profiler captures): no sustain loop, e2e, latency or CPU legs")
@@ -552,11 +554,21 @@ def main():
     out_b = store.out_row_bytes(flags)
     C = b.total_cands
     n_buf = 2  # outputs rotate so that consecutive steps do not rewrite lines still in L2
-    outs = [(torch.empty((C, out_b), dtype=torch.uint8, device=dev), torch.empty((C,), dtype=torch.uint8, device=dev))
+    n_out = db.n_req * db.n_max_cands if args.padded else C
+    outs = [(torch.empty((n_out, out_b), dtype=torch.uint8, device=dev), torch.empty((n_out,), dtype=torch.uint8, device=dev))
             for _ in range(n_buf)]
+    if args.padded:
+        c_idx = torch.empty((C,), dtype=torch.int32, device=dev)
+        c_src = torch.empty((C,), dtype=torch.int32, device=dev)
+        c_off = torch.empty((db.n_req + 1,), dtype=torch.int64, device=dev)
 
     def step(i: int):
         rows, mask = outs[i % n_buf]
+        if args.padded:
+            B.ccr_compact_valid(store, db.n_req, C, db.cand_idx, db.cand_offsets, c_idx, c_off, c_src)
+            B.ccr_join_batch_padded(store, db.n_req, C, db.max_edge_len, db.n_max_cands, db.edge_keys, db.edge_feats,
+                                    db.edge_offsets, c_idx, c_off, db.req_feats, rows, mask, flags)
+            return
         B.ccr_join_batch(store, db.n_req, C, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets, db.cand_idx,
                          db.cand_offsets, db.req_feats, rows, mask, flags)
 
@@ -580,6 +592,14 @@ def main():
             step(i)
         torch.cuda.synchronize(dev)
     t_wall1 = time.time()
+    compact_us = None
+    if args.padded:
+        ev0.record()
+        for i in range(200):
+            B.ccr_compact_valid(store, db.n_req, C, db.cand_idx, db.cand_offsets, c_idx, c_off, c_src)
+        ev1.record()
+        torch.cuda.synchronize(dev)
+        compact_us = ev0.elapsed_time(ev1) * 1e3 / 200
     total_cands_job = sum_over_ranks(float(C))
     if store.device_status() != B.CCR_OK:
         raise SystemExit("device status not clean after the timed region")
@@ -673,6 +693,10 @@ def main():
                            "p50": pct(lat, 0.50), "p99": pct(lat, 0.99), "n": len(lat)},
             "clocks": sampler.summary(t_wall0, t_wall1) if sampler is not None else None,
         }
+        if args.padded:
+            line["config"]["layout"] = ("padded T[%d, %d]: a step is ccr_compact_valid (3 launches, %.1f us alone, L2-warm) + "
+                                        "pad fill + join; the roofline figure divides the join's bytes by the whole step"
+                                        % (db.n_req, db.n_max_cands, compact_us))
         if world == 1 and not args.no_cpu_baseline and not args.timed_only:
             from oracle import oracle
 

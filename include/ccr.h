@@ -142,6 +142,52 @@ ccr_status ccr_join_batch(const ccr_docstore* store,
                           uint32_t       flags,
                           void*          stream);
 
+/* Batching and padding of variable-length requests (Section 6.3.1, "Batching and Padding for Variable-Length
+ * Requests").  The section pads a batch of b requests with n_i valid candidates each to n_max = max n_i in
+ * three steps: scatter indices (batch_idx, pos_idx) from the valid-position masks; the valid positions
+ * flattened across the batch for a single gather; a scatter of the gathered rows into T[b, n_max, features].
+ * The two entries below are those steps.
+ *
+ * ccr_compact_valid is the first two: a candidate is valid when 0 <= cand_idx[j] < n_docs (the resolver writes
+ * -1 for an unknown id).  For every request r its valid positions are copied, in their input order, to
+ * idx_out[offsets_out[r] .. offsets_out[r+1]); offsets_out[0] = 0 and offsets_out[r+1] - offsets_out[r] = n_r.
+ * The scatter index of kept candidate k of request r is therefore (r, k - offsets_out[r]).  src_out (optional,
+ * int32[>= number of valid candidates]) receives the flat input index j of every kept candidate, so that
+ * scores can be carried back to the caller's candidate order.  idx_out needs room for cand_offsets[n_req]
+ * entries (all candidates may be valid); idx_out / offsets_out must not alias the inputs.  All pointers are
+ * DEVICE pointers; three small kernels on `stream`, nothing allocated, no synchronisation.  total_cands only
+ * chooses how many blocks share a request (from the mean request length); the count pass uses one block per
+ * request, so the cost grows with the longest request rather than with the batch.
+ *
+ * ccr_join_batch_padded is the gather and the scatter in one kernel: the join of ccr_join_batch with the
+ * same arguments, flags and kernels, except that the row and mask of candidate j of request r are written at
+ * slot r * n_max + (j - cand_offsets[r]) of out_rows [n_req * n_max, out_row_bytes] / out_mask
+ * [n_req * n_max] instead of at j, so every gathered row is written once, at its place in T.  Slots behind a
+ * request's last candidate (pads) are all-zero rows — request section included — with mask 0; the caller
+ * masks their scores using n_r from the offsets.  n_max (HOST scalar, > 0) is normally the longest request;
+ * with a smaller n_max the candidates of a request behind its n_max-th are dropped.  Because the compacted
+ * offsets live on the device, total_cands may here be any upper bound of cand_offsets[n_req] (for instance
+ * the candidate count before compaction): flat indices at or above cand_offsets[n_req] belong to no request
+ * and are skipped.  CCR_FLAG_VALIDATE is not supported (CCR_ERR_UNSUPPORTED): validate with ccr_join_batch
+ * semantics first.  Two kernels on `stream` (pad fill, join); nothing allocated.                          */
+ccr_status ccr_compact_valid(const ccr_docstore* store, int32_t n_req,
+                             int64_t        total_cands,  /* HOST: cand_offsets[n_req] (sizes the launch only) */
+                             const int32_t* cand_idx,     /* DEVICE [cand_offsets[n_req]]               */
+                             const int64_t* cand_offsets, /* DEVICE [n_req + 1]                         */
+                             int32_t*       idx_out,      /* DEVICE [cand_offsets[n_req]]               */
+                             int64_t*       offsets_out,  /* DEVICE [n_req + 1]                         */
+                             int32_t*       src_out,      /* DEVICE [cand_offsets[n_req]] or NULL       */
+                             void*          stream);
+
+ccr_status ccr_join_batch_padded(const ccr_docstore* store,
+                                 int32_t n_req, int64_t total_cands, int64_t max_edge_len, int64_t n_max,
+                                 const int64_t* edge_keys, const void* edge_feats, const int64_t* edge_offsets,
+                                 const int32_t* cand_idx, const int64_t* cand_offsets, const void* req_feats,
+                                 void*          out_rows,  /* DEVICE [n_req * n_max, out_row_bytes]       */
+                                 uint8_t*       out_mask,  /* DEVICE [n_req * n_max]                      */
+                                 uint32_t       flags,
+                                 void*          stream);
+
 /* Algorithm 1 step 1 for request payloads whose affinity records arrive unsorted: for every request r the
  * records [edge_offsets[r], edge_offsets[r+1]) — key int64 + feature row of the store's edge width — are put
  * in ascending key order (records with equal keys keep their input order) into keys_out / feats_out, which

@@ -164,6 +164,51 @@ def resolve_ids(sorted_ids: np.ndarray, queries: np.ndarray, positions: Optional
     return out
 
 
+def scatter_indices(cand_idx: np.ndarray, cand_offsets: np.ndarray, n_docs: int):
+    """Section 6.3.1, batching and padding, step 1: from the valid-position mask (0 <= position < n_docs) the
+    scatter index (batch_idx, pos_idx) of every valid candidate, pos_idx counting the request's valid
+    candidates in their input order.  Returns (valid bool[C], batch_idx int64[V], pos_idx int64[V])."""
+    cand_idx = np.asarray(cand_idx, dtype=np.int64)
+    valid = (cand_idx >= 0) & (cand_idx < n_docs)
+    batch_idx, pos_idx = [], []
+    for r in range(len(cand_offsets) - 1):
+        k = 0
+        for j in range(int(cand_offsets[r]), int(cand_offsets[r + 1])):
+            if valid[j]:
+                batch_idx.append(r)
+                pos_idx.append(k)
+                k += 1
+    return valid, np.asarray(batch_idx, dtype=np.int64), np.asarray(pos_idx, dtype=np.int64)
+
+
+def join_padded(doc_feats, author_ids, edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets, n_max=None, **kw):
+    """Section 6.3.1, batching and padding: T[b, n_max, row] and its mask [b, n_max].
+    Step 1: scatter indices from the valid masks.  Step 2: the valid positions flattened across the batch and
+    gathered in one pass (the join of `join`, per request over its valid candidates).  Step 3: scatter
+    T[batch_idx, pos_idx] = gathered row.  Pads are zero rows with mask 0.  n_max defaults to max n_i.
+    Returns (T uint8[b, n_max, out_b], M uint8[b, n_max], n_valid int64[b], src int64[V] flat input index of
+    every kept candidate)."""
+    cand_idx = np.asarray(cand_idx)
+    b = len(cand_offsets) - 1
+    valid, batch_idx, pos_idx = scatter_indices(cand_idx, cand_offsets, int(doc_feats.shape[0]))
+    n_valid = np.bincount(batch_idx, minlength=b).astype(np.int64) if b else np.zeros(0, np.int64)
+    if n_max is None:
+        n_max = int(n_valid.max()) if b else 0
+    flat = cand_idx[valid]                                    # step 2: flattened valid positions
+    flat_offsets = np.concatenate([[0], np.cumsum(n_valid)]).astype(np.int64)
+    gathered, gmask = join(doc_feats, author_ids, edge_keys, edge_feats, edge_offsets, flat, flat_offsets, **kw)
+    out_b = gathered.shape[1] if gathered.ndim == 2 and gathered.shape[0] else out_row_bytes(
+        doc_feats, edge_feats, kw.get("req_feats"), 0 if kw.get("actor_ids") is None else kw["actor_ids"].shape[1],
+        kw.get("first_degree_only", False))
+    T = np.zeros((b, n_max, out_b), dtype=np.uint8)
+    M = np.zeros((b, n_max), dtype=np.uint8)
+    for v in range(len(batch_idx)):                           # step 3: scatter
+        if pos_idx[v] < n_max:
+            T[batch_idx[v], pos_idx[v]] = gathered[v]
+            M[batch_idx[v], pos_idx[v]] = gmask[v]
+    return T, M, n_valid, np.nonzero(valid)[0].astype(np.int64)
+
+
 def join_workload(wl, first_degree_only: bool = False, n_threads: int = 1):
     """Convenience for objects with `.store` and `.batch` attributes (duck-typed, nothing imported)."""
     s, b = wl.store, wl.batch

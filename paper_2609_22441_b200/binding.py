@@ -39,6 +39,7 @@ CCR_FLAG_TWO_PHASE = 1 << 7
 
 EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
+    "ccr_compact_valid", "ccr_join_batch_padded",
     "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
     "ccr_static_payload_capacity", "ccr_join_payload_static", "ccr_docstore_selftest_wait",
@@ -97,6 +98,10 @@ def lib() -> ctypes.CDLL:
     L.ccr_workspace_create.argtypes = [vp, i32, i64, i64, ctypes.POINTER(vp)]
     L.ccr_workspace_free.restype = ctypes.c_int
     L.ccr_workspace_free.argtypes = [vp]
+    L.ccr_compact_valid.restype = ctypes.c_int
+    L.ccr_compact_valid.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, vp]
+    L.ccr_join_batch_padded.restype = ctypes.c_int
+    L.ccr_join_batch_padded.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
     L.ccr_join_batch_host.restype = ctypes.c_int
     L.ccr_join_batch_host.argtypes = [vp, vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
     L.ccr_static_payload_capacity.restype = ctypes.c_size_t
@@ -238,6 +243,27 @@ def ccr_join_batch(store: Docstore, n_req: int, total_cands: int, max_edge_len: 
     return st
 
 
+def ccr_compact_valid(store: Docstore, n_req: int, total_cands: int, cand_idx, cand_offsets, idx_out, offsets_out,
+                      src_out=None, stream=None) -> int:
+    """Raw call: per-request stable compaction of the valid positions (device tensors in and out)."""
+    st = lib().ccr_compact_valid(store.handle, int(n_req), int(total_cands), _ptr(cand_idx), _ptr(cand_offsets), _ptr(idx_out),
+                                 _ptr(offsets_out), _ptr(src_out), _stream_ptr(stream))
+    _check(st, "ccr_compact_valid")
+    return st
+
+
+def ccr_join_batch_padded(store: Docstore, n_req: int, total_cands: int, max_edge_len: int, n_max: int,
+                          edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets, req_feats,
+                          out_rows, out_mask, flags: int = 0, stream=None) -> int:
+    """Raw call: the join written straight into the padded [n_req, n_max] layout."""
+    st = lib().ccr_join_batch_padded(store.handle, int(n_req), int(total_cands), int(max_edge_len), int(n_max),
+                                     _ptr(edge_keys), _ptr(edge_feats), _ptr(edge_offsets), _ptr(cand_idx),
+                                     _ptr(cand_offsets), _ptr(req_feats), _ptr(out_rows), _ptr(out_mask), int(flags),
+                                     _stream_ptr(stream))
+    _check(st, "ccr_join_batch_padded")
+    return st
+
+
 class DeviceBatch:
     """A ragged batch resident on the device (torch tensors), plus the host scalars the call needs."""
 
@@ -247,6 +273,7 @@ class DeviceBatch:
         self.total_cands = int(batch.total_cands)
         self.max_edge_len = int(batch.max_edge_len)
         self.total_edges = int(len(batch.edge_keys))
+        self.n_max_cands = int(np.diff(np.asarray(batch.cand_offsets)).max()) if self.n_req > 0 else 0
 
         def up(a):
             if a is None:
@@ -274,6 +301,27 @@ def join_batch(store: Docstore, db: DeviceBatch, flags: int = 0, out_rows: Optio
     ccr_join_batch(store, db.n_req, db.total_cands, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets,
                    db.cand_idx, db.cand_offsets, db.req_feats, out_rows, out_mask, flags, stream)
     return out_rows, out_mask
+
+
+def join_batch_padded(store: Docstore, db: DeviceBatch, n_max: Optional[int] = None, flags: int = 0, stream=None):
+    """Section 6.3.1 batching and padding in two calls: ccr_compact_valid, then ccr_join_batch_padded over the
+    compacted candidates.  Returns (T uint8[n_req, n_max, out_b], mask uint8[n_req, n_max],
+    offsets int64[n_req + 1] of the compacted batch, src int32[total_cands] flat input index per kept
+    candidate; entries behind offsets[n_req] are unwritten).  n_max defaults to the longest request of the
+    input, an upper bound of the longest compacted one, known on the host without a synchronisation."""
+    dev = torch.device("cuda", store.device)
+    if n_max is None:
+        n_max = max(1, int(db.n_max_cands))
+    out_b = store.out_row_bytes(flags)
+    idx = torch.empty((db.total_cands,), dtype=torch.int32, device=dev)
+    src = torch.empty((db.total_cands,), dtype=torch.int32, device=dev)
+    offs = torch.empty((db.n_req + 1,), dtype=torch.int64, device=dev)
+    T = torch.empty((db.n_req, n_max, out_b), dtype=torch.uint8, device=dev)
+    M = torch.empty((db.n_req, n_max), dtype=torch.uint8, device=dev)
+    ccr_compact_valid(store, db.n_req, db.total_cands, db.cand_idx, db.cand_offsets, idx, offs, src, stream)
+    ccr_join_batch_padded(store, db.n_req, db.total_cands, db.max_edge_len, n_max, db.edge_keys, db.edge_feats,
+                          db.edge_offsets, idx, offs, db.req_feats, T, M, flags, stream)
+    return T, M, offs, src
 
 
 class Workspace:

@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
 #include <cstdio>
 #include <cstdlib>
@@ -12,6 +13,7 @@
 #include <new>
 
 #include "ccr_join.cuh"
+#include "ccr_pad.cuh"
 #include "ccr_resolve.cuh"
 #include "ccr_sort.cuh"
 #include "ccr_ws.cuh"
@@ -592,10 +594,15 @@ ccr_status ccr_docstore_selftest_wait(ccr_docstore* s, void* stream) {
   return CCR_OK;
 }
 
-ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
-                          const int64_t* edge_keys, const void* edge_feats, const int64_t* edge_offsets,
-                          const int32_t* cand_idx, const int64_t* cand_offsets, const void* req_feats,
-                          void* out_rows, uint8_t* out_mask, uint32_t flags, void* stream) {
+}  // extern "C"
+
+namespace {
+// ccr_join_batch (n_max == 0, ragged output) and ccr_join_batch_padded (n_max > 0) share everything but the
+// output addressing.
+ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                     const int64_t* edge_keys, const void* edge_feats, const int64_t* edge_offsets,
+                     const int32_t* cand_idx, const int64_t* cand_offsets, const void* req_feats,
+                     void* out_rows, uint8_t* out_mask, uint32_t flags, void* stream, int64_t n_max) {
   if (!good(cs)) return CCR_ERR_BAD_HANDLE;
   ccr_docstore* s = const_cast<ccr_docstore*>(cs);  // only the launch counter and status words change
   if (n_req < 0 || total_cands < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
@@ -672,6 +679,7 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
   a.req_feats = static_cast<const uint8_t*>(req_feats);
   a.out_rows = static_cast<uint8_t*>(out_rows);
   a.out_mask = out_mask;
+  a.n_max = n_max;
   a.tile = tile;
   a.key_cap = key_cap;
   a.min_stride_log2 = (flags & CCR_FLAG_FORCE_SAMPLED) ? 2 : 0;
@@ -727,6 +735,76 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
     fn<<<static_cast<unsigned>(blocks), ccr::kThreads, smem, st>>>(a);
   }
   s->launches++;
+  if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+  return CCR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                          const int64_t* edge_keys, const void* edge_feats, const int64_t* edge_offsets,
+                          const int32_t* cand_idx, const int64_t* cand_offsets, const void* req_feats,
+                          void* out_rows, uint8_t* out_mask, uint32_t flags, void* stream) {
+  return join_impl(cs, n_req, total_cands, max_edge_len, edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets,
+                   req_feats, out_rows, out_mask, flags, stream, 0);
+}
+
+ccr_status ccr_join_batch_padded(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                                 int64_t n_max, const int64_t* edge_keys, const void* edge_feats,
+                                 const int64_t* edge_offsets, const int32_t* cand_idx, const int64_t* cand_offsets,
+                                 const void* req_feats, void* out_rows, uint8_t* out_mask, uint32_t flags,
+                                 void* stream) {
+  if (!good(cs)) return CCR_ERR_BAD_HANDLE;
+  if (n_max <= 0 || n_req < 0) return CCR_ERR_INVALID_ARG;
+  if (flags & CCR_FLAG_VALIDATE) return CCR_ERR_UNSUPPORTED;  // validate with ccr_join_batch semantics first
+  if (n_req == 0) return CCR_OK;
+  if (!cand_offsets || !out_rows || !out_mask) return CCR_ERR_INVALID_ARG;
+  ccr_docstore* s = const_cast<ccr_docstore*>(cs);
+  {
+    DeviceScope scope(s->desc.device);
+    if (!scope.ok) return CCR_ERR_CUDA;
+    // enough blocks to fill the device however few requests there are
+    const unsigned slices = static_cast<unsigned>(std::max(1, std::min(64, (2 * s->n_sms + n_req - 1) / n_req)));
+    ccr::pad_fill_kernel<<<dim3(static_cast<unsigned>(n_req), slices), ccr::kPadThreads, 0,
+                           static_cast<cudaStream_t>(stream)>>>(
+        cand_offsets, n_max, static_cast<long long>(out_row_bytes(s, flags)), static_cast<uint8_t*>(out_rows), out_mask);
+    s->launches++;
+    if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+  }
+  if (total_cands == 0) return CCR_OK;
+  return join_impl(cs, n_req, total_cands, max_edge_len, edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets,
+                   req_feats, out_rows, out_mask, flags, stream, n_max);
+}
+
+ccr_status ccr_compact_valid(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, const int32_t* cand_idx, const int64_t* cand_offsets,
+                             int32_t* idx_out, int64_t* offsets_out, int32_t* src_out, void* stream) {
+  if (!good(cs)) return CCR_ERR_BAD_HANDLE;
+  ccr_docstore* s = const_cast<ccr_docstore*>(cs);  // only the launch counter changes
+  if (n_req < 0 || total_cands < 0) return CCR_ERR_INVALID_ARG;
+  if (n_req == 0) return CCR_OK;
+  if (!cand_offsets || !offsets_out || (total_cands > 0 && (!cand_idx || !idx_out))) return CCR_ERR_INVALID_ARG;
+  if (cand_idx == idx_out || static_cast<const void*>(cand_offsets) == static_cast<const void*>(offsets_out))
+    return CCR_ERR_INVALID_ARG;  // not in place
+  if ((reinterpret_cast<uintptr_t>(cand_idx) & 3u) || (reinterpret_cast<uintptr_t>(idx_out) & 3u) ||
+      (reinterpret_cast<uintptr_t>(src_out) & 3u) || (reinterpret_cast<uintptr_t>(cand_offsets) & 7u) ||
+      (reinterpret_cast<uintptr_t>(offsets_out) & 7u))
+    return CCR_ERR_INVALID_ARG;
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const long long n_docs = s->desc.n_docs;
+  ccr::count_valid_kernel<<<static_cast<unsigned>(n_req), ccr::kPadThreads, 0, st>>>(cand_idx, cand_offsets, n_docs,
+                                                                                      offsets_out);
+  ccr::scan_counts_kernel<<<1, ccr::kPadThreads, 0, st>>>(offsets_out, n_req);
+  // slices per request: about one round of the compaction each, bounded so that the re-count stays small
+  const long long per_round = static_cast<long long>(ccr::kPadThreads) * ccr::kPadItems;
+  const long long avg = (total_cands + n_req - 1) / n_req;
+  const unsigned slices = static_cast<unsigned>(std::max(1LL, std::min(8LL, (avg + per_round - 1) / per_round)));
+  ccr::compact_valid_kernel<<<dim3(static_cast<unsigned>(n_req), slices), ccr::kPadThreads, 0, st>>>(
+      cand_idx, cand_offsets, n_docs, offsets_out, idx_out, src_out);
+  s->launches += 3;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
   return CCR_OK;
 }

@@ -52,6 +52,7 @@ struct JoinArgs {
   const uint8_t* req_feats;
   uint8_t* out_rows;
   uint8_t* out_mask;
+  long long n_max;            // 0: ragged output (row j); > 0: padded output, row r * n_max + (j - cand_offsets[r])
   // launch shape
   int tile;                   // candidates per block
   int key_cap;                // keys (or sampled keys) a block may stage per request; 0 = search global memory

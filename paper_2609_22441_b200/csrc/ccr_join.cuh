@@ -305,8 +305,12 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
       }
     }
 
-    for (long long sub = seg; sub < seg_end; sub += a.tile) {
-      const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_end - sub));
+    // padded output: a request's candidates behind its n_max-th have no slot and are dropped
+    const long long r_first = __ldg(a.cand_offsets + r);
+    const long long seg_lim = a.n_max > 0 ? min(seg_end, r_first + a.n_max) : seg_end;
+    for (long long sub = seg; sub < seg_lim; sub += a.tile) {
+      const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_lim - sub));
+      const long long out0 = a.n_max > 0 ? r * a.n_max + (sub - r_first) : sub;
 
       // ================= phase A: resolve every candidate of the sub-tile =================
       if (!MERGE) {
@@ -368,7 +372,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
             }
             s_idx[i] = idx[u];
             s_pos[i] = found[u] ? pos[u] : -1;
-            a.out_mask[sub + i] = static_cast<uint8_t>(m);
+            a.out_mask[out0 + i] = static_cast<uint8_t>(m);
           }
         }
       } else {
@@ -430,14 +434,14 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
             int p = s_pos[i];
             if (p >= K) p = -1;
             s_pos[i] = p;
-            a.out_mask[sub + i] = p >= 0 ? 1 : 0;
+            a.out_mask[out0 + i] = p >= 0 ? 1 : 0;
           }
         } else {
           for (int i = tid; i < n; i += kThreads) {
             int pos = 0;
             const bool found = s_idx[i] >= 0 && keys.find(s_auth[i], pos);
             s_pos[i] = found ? pos : -1;
-            a.out_mask[sub + i] = found ? 1 : 0;
+            a.out_mask[out0 + i] = found ? 1 : 0;
           }
         }
       }
@@ -446,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
       // ================= phase B: stream the rows =================
       for (int g = warp * 32; g < n; g += kWarps * 32) {
         emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND>(a, sh, s_idx + g, s_pos + g, s_apos + g, edge_base, req_src,
-                                                    a.out_rows + (sub + g) * sh.out_b, min(32, n - g), lane);
+                                                    a.out_rows + (out0 + g) * sh.out_b, min(32, n - g), lane);
       }
       __syncthreads();  // phase A of the next sub-tile overwrites the resolved arrays (and, in merge mode, the keys)
     }

@@ -39,11 +39,13 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 struct WsSlot {          // descriptor of one ring slot
   long long sub;         // first flat candidate of the sub-tile
+  long long out0;        // output row of that candidate (= sub for the ragged layout)
   long long kb;          // first key / edge row of its request
   int n;                 // candidates in the sub-tile (0 = stop)
   int r;                 // request index
   int next;              // next 32-row group a streamer warp may take (reset by the resolvers)
   int pad;
+  long long pad2;
 };
 
 struct WsLayout {
@@ -137,7 +139,7 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
         g = __shfl_sync(kFull, g, 0) * 32;
         if (g >= d.n) break;
         emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND>(a, sh, idx + g, pos + g, apos + g, edge_base, req_src,
-                                                    a.out_rows + (d.sub + g) * sh.out_b, min(32, d.n - g), lane);
+                                                    a.out_rows + (d.out0 + g) * sh.out_b, min(32, d.n - g), lane);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
@@ -210,15 +212,18 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
         }
         staged_r = r;
       }
-      for (long long sub = seg; sub < seg_end; sub += a.tile, ++it) {
+      // padded output: a request's candidates behind its n_max-th have no slot and are dropped
+      const long long seg_lim = a.n_max > 0 ? min(seg_end, co[r] + a.n_max) : seg_end;
+      for (long long sub = seg; sub < seg_lim; sub += a.tile, ++it) {
         if (static_cast<int>(it % n_resolvers) != rwarp || dead) continue;
-        const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_end - sub));
+        const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_lim - sub));
         const int s = it % kWsSlots;
         if (it >= static_cast<unsigned>(kWsSlots) && !mbar_wait_bounded(empty0 + 8 * s, (it / kWsSlots - 1) & 1u)) {
           if (lane == 0) atomicExch(a.status, kDevWaitExpired);
           dead = true;  // the streamers are gone
           continue;
         }
+        const long long out0 = a.n_max > 0 ? r * a.n_max + (sub - co[r]) : sub;
         int* out_idx = s_idx + s * a.tile;
         int* out_pos = s_pos + s * a.tile;
         int4* out_apos = s_apos + s * a.tile;
@@ -296,7 +301,7 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
                 out_apos[i] = make_int4(ap[u][0], ap[u][1], ap[u][2], ap[u][3]);
                 out_idx[i] = idx[u];
                 out_pos[i] = found[u] ? pos[u] : -1;
-                a.out_mask[sub + i] = static_cast<uint8_t>(m);
+                a.out_mask[out0 + i] = static_cast<uint8_t>(m);
               }
             }
           } else {
@@ -306,7 +311,7 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
               if (i < n) {
                 out_idx[i] = idx[u];
                 out_pos[i] = found[u] ? pos[u] : -1;
-                a.out_mask[sub + i] = found[u] ? 1 : 0;
+                a.out_mask[out0 + i] = found[u] ? 1 : 0;
               }
             }
           }
@@ -315,11 +320,13 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
         if (lane == 0) {
           WsSlot d;
           d.sub = sub;
+          d.out0 = out0;
           d.kb = kb;
           d.n = n;
           d.r = r;
           d.next = 0;
           d.pad = 0;
+          d.pad2 = 0;
           slots[s] = d;
           mbar_arrive(full0 + 8 * s);
         }
@@ -338,11 +345,13 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
       if (!ok) atomicExch(a.status, kDevWaitExpired);
       WsSlot d;
       d.sub = 0;
+      d.out0 = 0;
       d.kb = 0;
       d.n = 0;
       d.r = 0;
       d.next = 0;
       d.pad = 0;
+      d.pad2 = 0;
       if (ok) {
         slots[s] = d;
         mbar_arrive(full0 + 8 * s);

@@ -162,6 +162,103 @@ def test_worked_batching_example_from_the_paper():
         assert rows[k, :4].copy().view(np.float32)[0] == (p * 8) % 2048
 
 
+def _read_golden_example():
+    req, flat, scatter, T = [], None, None, []
+    for line in open(os.path.join(GOLDEN, "batching_example.txt")):
+        if line.startswith("request"):
+            req.append([int(x) for x in line.split(":")[1].split()])
+        elif line.startswith("flattened"):
+            flat = [int(x) for x in line.split(":")[1].split()]
+        elif line.startswith("scatter"):
+            scatter = [tuple(int(v) for v in x.split(",")) for x in line.split(":")[1].split()]
+        elif line.startswith("T "):
+            T.append([None if x == "pad" else int(x) for x in line.split(":")[1].split()])
+    return req, flat, scatter, T
+
+
+def _example_workload(cands, n_docs=100):
+    rng = np.random.default_rng(1)
+    store = W.make_store(rng, n_docs, 50, 8, np.float32, tagged=True)
+    keys, feats = W.make_viewer(rng, 50, 5, 8, np.float16)
+    batch = W.assemble_batch([keys] * len(cands), [feats] * len(cands), [np.array(x, np.int32) for x in cands], None,
+                             8, np.float16, 0, np.float32)
+    return W.Workload("example", 1, store, batch)
+
+
+def _padded(wl, n_max=None, **kw):
+    s, b = wl.store, wl.batch
+    return oracle.join_padded(
+        s.doc_feats, s.author_ids, b.edge_keys, b.edge_feats, b.edge_offsets, b.cand_idx, b.cand_offsets, n_max=n_max,
+        req_feats=b.req_feats, actor_ids=s.actor_ids, actor_types=s.actor_types, reduce_sum_mask=s.reduce_sum_mask, **kw)
+
+
+def test_padded_layout_of_the_worked_example():
+    """The scatter indices and the padded tensor T the paper prints for its b = 2 example."""
+    req, flat, scatter, T = _read_golden_example()
+    wl = _example_workload(req)
+    s, b = wl.store, wl.batch
+    valid, batch_idx, pos_idx = oracle.scatter_indices(b.cand_idx, b.cand_offsets, s.n_docs)
+    assert valid.all() and list(zip(batch_idx.tolist(), pos_idx.tolist())) == scatter
+    out, mask, n_valid, src = _padded(wl)
+    assert out.shape[:2] == (2, 3) and list(n_valid) == [3, 2] and list(src) == [0, 1, 2, 3, 4]
+    doc_b = s.doc_row_bytes
+    for r, line in enumerate(T):
+        for k, p in enumerate(line):
+            if p is None:  # the pad
+                assert not out[r, k].any() and mask[r, k] == 0
+            else:
+                assert np.array_equal(out[r, k, :doc_b], s.doc_feats[p].view(np.uint8))
+                assert out[r, k, :4].copy().view(np.float32)[0] == (p * 8) % 2048  # tagged store: row p starts with p * 8
+
+
+def test_padded_layout_drops_unresolved_positions_by_hand():
+    """Same example with unresolved (-1) and out-of-range positions mixed in: they get no scatter index, the
+    valid ones close ranks in their input order.  Expected values written out by hand."""
+    wl = _example_workload([[-1, 10, 42, -1, 87], [100, 5, -1, 63], [-1, -1], []])
+    s, b = wl.store, wl.batch
+    valid, batch_idx, pos_idx = oracle.scatter_indices(b.cand_idx, b.cand_offsets, s.n_docs)
+    assert valid.tolist() == [False, True, True, False, True, False, True, False, True, False, False]
+    assert list(zip(batch_idx.tolist(), pos_idx.tolist())) == [(0, 0), (0, 1), (0, 2), (1, 0), (1, 1)]
+    out, mask, n_valid, src = _padded(wl)
+    assert out.shape[:2] == (4, 3) and list(n_valid) == [3, 2, 0, 0] and list(src) == [1, 2, 4, 6, 8]
+    want = [[10, 42, 87], [5, 63, None], [None] * 3, [None] * 3]
+    for r in range(4):
+        for k in range(3):
+            if want[r][k] is None:
+                assert not out[r, k].any() and mask[r, k] == 0
+            else:
+                assert out[r, k, :4].copy().view(np.float32)[0] == (want[r][k] * 8) % 2048
+    # a wider n_max only adds pads; a narrower one drops the tail of the longer requests
+    wide, wmask, _, _ = _padded(wl, n_max=5)
+    assert np.array_equal(wide[:, :3], out) and not wide[:, 3:].any() and not wmask[:, 3:].any()
+    narrow, nmask, _, _ = _padded(wl, n_max=2)
+    assert np.array_equal(narrow, out[:, :2]) and np.array_equal(nmask, mask[:, :2])
+
+
+@settings(max_examples=40, deadline=None, suppress_health_check=list(HealthCheck))
+@given(seed=st.integers(0, 2**31), n_docs=st.integers(1, 40), alphabet=st.integers(1, 24),
+       n_req=st.integers(0, 4), second=st.booleans(), req_dim=st.sampled_from([0, 4]))
+def test_padded_equals_naive_scan_rows_placed_one_by_one(seed, n_docs, alphabet, n_req, second, req_dim):
+    """Compaction before the join (the oracle's route) against the naive scan over the uncompacted batch whose
+    valid rows are then placed one at a time."""
+    wl = _tiny(seed, n_docs, alphabet, n_req, 16, 48, second, req_dim)
+    s, b = wl.store, wl.batch
+    out, mask, n_valid, src = _padded(wl)
+    brows, bmask = _brute(wl)
+    assert out.shape[0] == b.n_req
+    kept = []
+    for r in range(b.n_req):
+        k = 0
+        for j in range(int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])):
+            if 0 <= int(b.cand_idx[j]) < s.n_docs:
+                assert np.array_equal(out[r, k], brows[j]) and mask[r, k] == bmask[j]
+                kept.append(j)
+                k += 1
+        assert k == n_valid[r]
+        assert not out[r, k:].any() and not mask[r, k:].any()
+    assert kept == list(src)
+
+
 # ---------------------------------------------------------------- invariants at realistic shapes
 def _check_invariants(wl):
     s, b = wl.store, wl.batch
