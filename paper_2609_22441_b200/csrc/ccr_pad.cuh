@@ -95,36 +95,50 @@ __global__ void __launch_bounds__(kPadThreads) scan_counts_kernel(int64_t* count
 // src_out[k] (optional) is the flat input index of kept candidate k, so scores can be carried back.
 // Blocks (r, 0 .. gridDim.y) each take one slice of request r; a block first counts the valid candidates in
 // the slices before its own (a re-read of at most the request's positions, which sit in L2), then walks its
-// slice in rounds of kPadThreads * kPadItems candidates, thread t holding the kPadItems consecutive ones
-// from t * kPadItems, which keeps the order without a second pass.
+// slice in rounds of kPadThreads * kPadItems candidates.  In a round warp w owns the kPadItems consecutive
+// groups of 32 candidates from w * 32 * kPadItems: a ballot per group ranks its valid lanes, so loads and
+// stores are both contiguous per warp instruction and the order is kept without a second pass.
 __global__ void __launch_bounds__(kPadThreads)
 compact_valid_kernel(const int32_t* cand_idx, const int64_t* cand_offsets, long long n_docs, const int64_t* offsets_out,
                      int32_t* idx_out, int32_t* src_out) {
   __shared__ int warp_sums[kPadThreads / 32];
   const int r = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long j0 = cand_offsets[r], j1 = cand_offsets[r + 1];
-  const long long slice = (((j1 - j0) + gridDim.y - 1) / gridDim.y + kPadItems - 1) / kPadItems * kPadItems;
+  const long long slice = (((j1 - j0) + gridDim.y - 1) / gridDim.y + 31) / 32 * 32;
   const long long s0 = min(j1, j0 + blockIdx.y * slice), s1 = min(j1, s0 + slice);
   if (s0 >= s1) return;
   long long out = offsets_out[r] + block_count_valid(cand_idx, j0, s0, n_docs, warp_sums);
   for (long long base = s0; base < s1; base += kPadThreads * kPadItems) {
-    const long long jt = base + static_cast<long long>(threadIdx.x) * kPadItems;
+    const long long jw = base + static_cast<long long>(warp) * (32 * kPadItems) + lane;
     int p[kPadItems];
-    int keep = 0;
+#pragma unroll
+    for (int k = 0; k < kPadItems; ++k) p[k] = jw + 32 * k < s1 ? __ldg(cand_idx + jw + 32 * k) : -1;
+    unsigned votes[kPadItems];
+    int warp_total = 0;
 #pragma unroll
     for (int k = 0; k < kPadItems; ++k) {
-      p[k] = jt + k < s1 ? __ldg(cand_idx + jt + k) : -1;
-      keep += position_valid(p[k], n_docs) ? 1 : 0;
+      votes[k] = __ballot_sync(0xffffffffu, position_valid(p[k], n_docs));
+      warp_total += __popc(votes[k]);
     }
-    int total;
-    long long w = out + block_scan_inclusive(keep, warp_sums, total) - keep;
+    if (lane == 0) warp_sums[warp] = warp_total;
+    __syncthreads();
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < kPadThreads / 32; ++w) {
+      const int c = warp_sums[w];
+      if (w < warp) before += c;
+      total += c;
+    }
+    long long w0 = out + before;
 #pragma unroll
     for (int k = 0; k < kPadItems; ++k) {
-      if (position_valid(p[k], n_docs)) {
+      if ((votes[k] >> lane) & 1u) {
+        const long long w = w0 + __popc(votes[k] & ((1u << lane) - 1u));
         idx_out[w] = p[k];
-        if (src_out != nullptr) src_out[w] = static_cast<int32_t>(jt + k);
-        ++w;
+        if (src_out != nullptr) src_out[w] = static_cast<int32_t>(jw + 32 * k);
       }
+      w0 += __popc(votes[k]);
     }
     out += total;
     __syncthreads();  // warp_sums is rewritten by the next round
