@@ -98,6 +98,28 @@ ccr_status ccr_docstore_upload(ccr_docstore* store, int64_t first_doc, int64_t n
                                const int64_t* actor_ids, const uint8_t* actor_types,
                                int src_on_device, void* stream);
 
+/* Write a batch of rows by position (Section 6.2, "Scaling ingestion": bootstrap step 3, "GPU scatter features to
+ * assigned positions", and the steady-state updates).  Row i of the batch replaces row positions[i] of the store:
+ * doc_feats [n, doc_dim], author_ids int64[n], and for second-degree stores actor_ids int64[n, max_actors] /
+ * actor_types uint8[n, max_actors], with the meaning they have in ccr_docstore_upload.  A NULL source leaves that
+ * array untouched (an engagement update that only rewrites the engager slots passes only those).  A position
+ * outside [0, n_docs) skips its row.  The positions of one call must be distinct: rows are written by many
+ * threads, so two batch rows aimed at one position would leave a mixture (the paper's host-side hash map hands
+ * out one position per document; coalescing repeated updates of a document inside a batch is the caller's job).
+ * All pointers are DEVICE pointers (the caller brings the batch over on its ingestion stream).  One kernel on
+ * `stream`, nothing allocated, no synchronisation.
+ * Concurrency: a join may run at the same time on another stream as long as none of its candidates points at
+ * a row this call writes — new documents go to positions no request can name before the host publishes their
+ * ids, which is the order the paper's protocol prescribes (step 4 after step 3); rewriting rows that in-flight
+ * requests may read needs the paper's index-level read-write lock, which stays with the caller.            */
+ccr_status ccr_docstore_upsert(ccr_docstore* store, int64_t n,
+                               const int32_t* positions,   /* DEVICE [n]                                  */
+                               const void*    doc_feats,   /* DEVICE [n, doc_dim] or NULL                 */
+                               const int64_t* author_ids,  /* DEVICE [n] or NULL                          */
+                               const int64_t* actor_ids,   /* DEVICE [n, max_actors] or NULL              */
+                               const uint8_t* actor_types, /* DEVICE [n, max_actors] or NULL              */
+                               void* stream);
+
 /* Free the store and its device memory.  A second free of the same handle returns
  * CCR_ERR_BAD_HANDLE as long as the freed block has not been reused by the allocator.              */
 ccr_status ccr_docstore_free(ccr_docstore* store);

@@ -164,6 +164,35 @@ def resolve_ids(sorted_ids: np.ndarray, queries: np.ndarray, positions: Optional
     return out
 
 
+def upsert(doc_feats, author_ids, positions, new_doc_feats=None, new_author_ids=None, actor_ids=None, actor_types=None,
+           new_actor_ids=None, new_actor_types=None):
+    """Section 6.2, ingestion, step 3 of the per-batch protocol: batch row i is written to row positions[i] of the
+    index (features and the ids stored beside them); a position outside [0, n_docs) writes nothing; an array
+    for which no new values are given stays as it was.  Positions of one batch are distinct.  Returns copies
+    (doc_feats, author_ids, actor_ids, actor_types)."""
+    doc_feats, author_ids = np.array(doc_feats), np.array(author_ids)
+    actor_ids = None if actor_ids is None else np.array(actor_ids)
+    actor_types = None if actor_types is None else np.array(actor_types)
+    n_docs = doc_feats.shape[0]
+    seen = set()
+    for i in range(len(positions)):
+        p = int(positions[i])
+        if p < 0 or p >= n_docs:
+            continue
+        if p in seen:
+            raise ValueError("the oracle does not define a batch with repeated positions")
+        seen.add(p)
+        if new_doc_feats is not None:
+            doc_feats[p] = new_doc_feats[i]
+        if new_author_ids is not None:
+            author_ids[p] = new_author_ids[i]
+        if new_actor_ids is not None:
+            actor_ids[p] = new_actor_ids[i]
+        if new_actor_types is not None:
+            actor_types[p] = new_actor_types[i]
+    return doc_feats, author_ids, actor_ids, actor_types
+
+
 def scatter_indices(cand_idx: np.ndarray, cand_offsets: np.ndarray, n_docs: int):
     """Section 6.3.1, batching and padding, step 1: from the valid-position mask (0 <= position < n_docs) the
     scatter index (batch_idx, pos_idx) of every valid candidate, pos_idx counting the request's valid

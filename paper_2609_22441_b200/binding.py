@@ -38,7 +38,7 @@ CCR_FLAG_STATIC_SPLIT = 1 << 6
 CCR_FLAG_TWO_PHASE = 1 << 7
 
 EXPORTS = (
-    "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
+    "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_upsert", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
     "ccr_compact_valid", "ccr_join_batch_padded",
     "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
@@ -98,6 +98,8 @@ def lib() -> ctypes.CDLL:
     L.ccr_workspace_create.argtypes = [vp, i32, i64, i64, ctypes.POINTER(vp)]
     L.ccr_workspace_free.restype = ctypes.c_int
     L.ccr_workspace_free.argtypes = [vp]
+    L.ccr_docstore_upsert.restype = ctypes.c_int
+    L.ccr_docstore_upsert.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp]
     L.ccr_compact_valid.restype = ctypes.c_int
     L.ccr_compact_valid.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, vp]
     L.ccr_join_batch_padded.restype = ctypes.c_int
@@ -200,6 +202,12 @@ class Docstore:
         _check(lib().ccr_docstore_upload(self._h, int(first_doc), n, _ptr(doc_feats), _ptr(author_ids),
                                          _ptr(actor_ids), _ptr(actor_types), 1 if all(on_dev) else 0,
                                          _stream_ptr(stream)), "ccr_docstore_upload")
+
+    def upsert(self, positions, doc_feats=None, author_ids=None, actor_ids=None, actor_types=None, stream=None) -> None:
+        """ccr_docstore_upsert: batch row i replaces row positions[i]; every argument is a device tensor."""
+        _check(lib().ccr_docstore_upsert(self._h, int(positions.shape[0]), _ptr(positions), _ptr(doc_feats),
+                                         _ptr(author_ids), _ptr(actor_ids), _ptr(actor_types), _stream_ptr(stream)),
+               "ccr_docstore_upsert")
 
     def out_row_bytes(self, flags: int = 0) -> int:
         return int(lib().ccr_out_row_bytes(self._h, int(flags)))

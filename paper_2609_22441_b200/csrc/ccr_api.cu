@@ -16,6 +16,7 @@
 #include "ccr_pad.cuh"
 #include "ccr_resolve.cuh"
 #include "ccr_sort.cuh"
+#include "ccr_upsert.cuh"
 #include "ccr_ws.cuh"
 
 namespace {
@@ -396,6 +397,45 @@ ccr_status ccr_docstore_upload(ccr_docstore* s, int64_t first_doc, int64_t n, co
     cudaGetLastError();
     return CCR_ERR_CUDA;
   }
+  return CCR_OK;
+}
+
+ccr_status ccr_docstore_upsert(ccr_docstore* s, int64_t n, const int32_t* positions, const void* doc_feats,
+                               const int64_t* author_ids, const int64_t* actor_ids, const uint8_t* actor_types,
+                               void* stream) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  if (n < 0) return CCR_ERR_INVALID_ARG;
+  if (n == 0) return CCR_OK;
+  if (!positions) return CCR_ERR_INVALID_ARG;
+  if (!aligned16(doc_feats) || (reinterpret_cast<uintptr_t>(positions) & 3u) ||
+      (reinterpret_cast<uintptr_t>(author_ids) & 7u) || (reinterpret_cast<uintptr_t>(actor_ids) & 7u))
+    return CCR_ERR_INVALID_ARG;
+  const int ma = s->desc.max_actors;
+  if (ma == 0 && (actor_ids || actor_types)) return CCR_ERR_INVALID_ARG;  // a first-degree store has no engager slots
+  if (!doc_feats && !author_ids && !actor_ids && !actor_types) return CCR_OK;
+  DeviceScope scope(s->desc.device);
+  if (!scope.ok) return CCR_ERR_CUDA;
+  ccr::UpsertArgs a;
+  a.n = n;
+  a.n_docs = s->desc.n_docs;
+  a.positions = positions;
+  a.src_rows = static_cast<const uint8_t*>(doc_feats);
+  a.dst_rows = s->doc_feats;
+  a.row_ch = s->doc_b / 16;
+  a.src_author = author_ids;
+  a.src_actor = actor_ids;
+  a.src_type = actor_types;
+  a.dst_author = s->author_ids;
+  a.dst_recs = ma > 0 ? s->id_recs : nullptr;
+  a.max_actors = ma;
+  const long long work = doc_feats ? n * a.row_ch : n;
+  const long long per_block = static_cast<long long>(ccr::kUpsertThreads) * ccr::kUpsertUnroll;
+  long long blocks = (work + per_block - 1) / per_block;
+  const long long cap = static_cast<long long>(s->n_sms) * 8;
+  blocks = blocks < 1 ? 1 : (blocks > cap ? cap : blocks);
+  ccr::upsert_kernel<<<static_cast<unsigned>(blocks), ccr::kUpsertThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  s->launches++;
+  if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
   return CCR_OK;
 }
 

@@ -495,3 +495,69 @@ def test_id_resolution_matches_a_hash_map_and_searchsorted():
     hit = (rank < len(ids)) & (ids[np.minimum(rank, len(ids) - 1)] == q)
     assert np.array_equal(oracle.resolve_ids(ids, q), np.where(hit, rank, -1).astype(np.int32))
     assert np.array_equal(oracle.resolve_ids(ids[:0], q), np.full(len(q), -1, np.int32))
+
+
+# ---------------------------------------------------------------- store write path (Section 6.2, ingestion step 3)
+def test_upsert_closed_forms():
+    rng = np.random.default_rng(3)
+    n, d = 57, 6
+    X = rng.standard_normal((n, d)).astype(np.float32)
+    ids = rng.integers(0, 1000, size=n, dtype=np.int64)
+    act = rng.integers(-1, 50, size=(n, 4), dtype=np.int64)
+    typ = rng.integers(0, 3, size=(n, 4)).astype(np.uint8)
+    # a batch that names every row once, positions = a permutation pi: the result is the batch read through pi^-1
+    pi = rng.permutation(n)
+    newX = rng.standard_normal((n, d)).astype(np.float32)
+    newids = rng.integers(0, 1000, size=n, dtype=np.int64)
+    newact = rng.integers(-1, 50, size=(n, 4), dtype=np.int64)
+    newtyp = rng.integers(0, 3, size=(n, 4)).astype(np.uint8)
+    X0, ids0 = X.copy(), ids.copy()
+    Y, yid, yact, ytyp = oracle.upsert(X, ids, pi, newX, newids, act, typ, newact, newtyp)
+    inv = np.argsort(pi)
+    assert np.array_equal(Y, newX[inv]) and np.array_equal(yid, newids[inv])
+    assert np.array_equal(yact, newact[inv]) and np.array_equal(ytyp, newtyp[inv])
+    assert np.array_equal(X, X0) and np.array_equal(ids, ids0) and not np.shares_memory(Y, X)  # inputs are not modified
+    # a partial batch: named rows change, all others keep their old content; out-of-range positions write nothing
+    pos = np.array([5, -1, 56, n, 0, 2**31 - 1, 17], dtype=np.int64)
+    Z, zid, zact, ztyp = oracle.upsert(X, ids, pos, newX[:7], newids[:7], act, typ, newact[:7], None)
+    keep = np.ones(n, dtype=bool)
+    for i, p in [(0, 5), (2, 56), (4, 0), (6, 17)]:
+        assert np.array_equal(Z[p], newX[i]) and zid[p] == newids[i] and np.array_equal(zact[p], newact[i])
+        keep[p] = False
+    assert np.array_equal(Z[keep], X[keep]) and np.array_equal(zid[keep], ids[keep]) and np.array_equal(zact[keep], act[keep])
+    assert np.array_equal(ztyp, typ)  # no new types given: untouched everywhere
+    # the same batch twice = once; batches over disjoint rows commute; the empty batch is the identity
+    Z2 = oracle.upsert(Z, zid, pos, newX[:7], newids[:7], zact, ztyp, newact[:7], None)
+    assert all(np.array_equal(a, b) for a, b in zip(Z2, (Z, zid, zact, ztyp)))
+    a_pos, b_pos = np.array([1, 2, 3]), np.array([40, 41])
+    ab = oracle.upsert(*oracle.upsert(X, ids, a_pos, newX[:3], newids[:3])[:2], b_pos, newX[3:5], newids[3:5])
+    ba = oracle.upsert(*oracle.upsert(X, ids, b_pos, newX[3:5], newids[3:5])[:2], a_pos, newX[:3], newids[:3])
+    assert np.array_equal(ab[0], ba[0]) and np.array_equal(ab[1], ba[1])
+    E = oracle.upsert(X, ids, np.empty(0, np.int64), newX[:0], newids[:0])
+    assert np.array_equal(E[0], X) and np.array_equal(E[1], ids)
+    with pytest.raises(ValueError):
+        oracle.upsert(X, ids, np.array([4, 4]), newX[:2], newids[:2])
+
+
+def test_join_sees_upserted_rows_like_a_store_built_directly():
+    """Join after an upsert = naive scan over a store that was generated with the final contents."""
+    wl = _tiny(77, 30, 12, 3, 10, 40, True, 4)
+    s = wl.store
+    rng = np.random.default_rng(8)
+    pos = rng.permutation(s.n_docs)[:11]
+    donor = W.make_store(np.random.default_rng(99), s.n_docs, 12, 4, np.float32, max_actors=4, reduce_sum_mask=s.reduce_sum_mask)
+    doc, auth, act, typ = oracle.upsert(s.doc_feats, s.author_ids, pos, donor.doc_feats[pos], donor.author_ids[pos],
+                                        s.actor_ids, s.actor_types, donor.actor_ids[pos], donor.actor_types[pos])
+    # built directly: donor rows where named, original rows elsewhere, chosen row by row
+    named = set(int(p) for p in pos)
+    for arr_new, arr_old, arr_don in ((doc, s.doc_feats, donor.doc_feats), (auth, s.author_ids, donor.author_ids),
+                                      (act, s.actor_ids, donor.actor_ids), (typ, s.actor_types, donor.actor_types)):
+        for p in range(s.n_docs):
+            assert np.array_equal(arr_new[p], arr_don[p] if p in named else arr_old[p])
+    b = wl.batch
+    rows, mask = oracle.join(doc, auth, b.edge_keys, b.edge_feats, b.edge_offsets, b.cand_idx, b.cand_offsets,
+                             req_feats=b.req_feats, actor_ids=act, actor_types=typ, reduce_sum_mask=s.reduce_sum_mask)
+    brows, bmask = brute_force.join(doc, auth, b.edge_keys, b.edge_feats, b.edge_offsets, b.cand_idx, b.cand_offsets,
+                                    req_feats=b.req_feats, actor_ids=act, actor_types=typ,
+                                    reduce_sum_mask=s.reduce_sum_mask)
+    assert np.array_equal(rows, brows) and np.array_equal(mask, bmask)
