@@ -48,7 +48,7 @@ def parse_args():
     p.add_argument("--steps", type=int, default=2000)
     p.add_argument("--warmup", type=int, default=10)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--config", default="1", choices=["1", "2b", "3", "3b", "3s", "4", "sort", "resolve"],
+    p.add_argument("--config", default="1", choices=["1", "2b", "3", "3b", "3s", "4", "sort", "resolve", "ingest"],
                    help="1 batched first-degree (default, the headline); 2b second-degree on the same shape; 3 production-scale "
                         "store, first-degree; 3b the same on candidates sorted by author (merge path); 3s production scale, "
                         "second-degree; 4 single-request latency sweep on the production-scale store; sort: Algorithm 1 step 1 "
@@ -382,6 +382,107 @@ def resolve_bench(args, B, device: int):
     ix.free()
 
 
+def ingest_bench(args, B, device: int):
+    """Store write path (Section 6.2, ingestion step 3) and its effect on the join: a config-1 store with spare
+    rows; batches of 300,000 rows (the bootstrap size, "hundreds of thousands") and of 100,000 rows (the
+    steady-state size, a third of it) are scattered to new positions on an ingestion stream while the
+    config-1 join runs back to back on the serving stream.  In-flight requests name live rows only, new rows go
+    to positions nobody can name yet (the paper publishes ids after the write)."""
+    import torch
+
+    from paper_2609_22441_b200 import workloads as W
+
+    dev = torch.device("cuda", device)
+    wl = W.config1()
+    s, b = wl.store, wl.batch
+    n_live, spare = s.n_docs, 600_000
+    store = B.Docstore(n_live + spare, s.doc_dim, s.doc_dtype, b.edge_dim, b.edge_dtype, b.req_dim, b.req_dtype, 0, 0, device)
+    store.upload(0, s.doc_feats, s.author_ids)
+    db = B.DeviceBatch(b, device=device)
+    C, out_b = b.total_cands, store.out_row_bytes(0)
+    outs = [(torch.empty((C, out_b), dtype=torch.uint8, device=dev), torch.empty((C,), dtype=torch.uint8, device=dev))
+            for _ in range(2)]
+    g = torch.Generator(device=dev)
+    g.manual_seed(W.config_seed(6))
+    doc_t = torch.float16 if np.dtype(s.doc_dtype) == np.float16 else torch.float32
+    s_join, s_ing = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    peak, peak_kind = measured_peak_gbs()
+
+    def join(i):
+        B.ccr_join_batch(store, db.n_req, C, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets, db.cand_idx,
+                         db.cand_offsets, db.req_feats, outs[i % 2][0], outs[i % 2][1], 0, s_join)
+
+    def timed(fn, n, stream):
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(n):
+            fn(i)
+        z.record(stream)
+        return a, z
+
+    quick = args.timed_only  # profiler captures: a handful of launches per cell
+    n_join = 3 if quick else 300
+    for i in range(1 if quick else 5):
+        join(i)
+    torch.cuda.synchronize(dev)
+    a, z = timed(join, n_join, s_join)
+    torch.cuda.synchronize(dev)
+    join_alone_us = a.elapsed_time(z) * 1e3 / n_join
+    cells = []
+    for rows, order in ((300_000, "random"), (300_000, "consecutive"), (100_000, "random"), (100_000, "consecutive")):
+        # several source batches (2 x 154 MB at 300k rows) so that consecutive launches do not re-read L2 lines
+        srcs = []
+        for k in range(2):
+            pos = n_live + (torch.randperm(spare, generator=g, device=dev)[:rows] if order == "random"
+                            else torch.arange(rows, device=dev) + k * rows)
+            srcs.append((pos.to(torch.int32), torch.randn((rows, s.doc_dim), generator=g, device=dev, dtype=torch.float32).to(doc_t),
+                         torch.randint(0, 5 * n_live, (rows,), generator=g, device=dev, dtype=torch.int64)))
+
+        def upsert(i):
+            p, d, au = srcs[i % 2]
+            store.upsert(p, d, au, stream=s_ing)
+
+        for i in range(1 if quick else 5):
+            upsert(i)
+        torch.cuda.synchronize(dev)
+        n_up = 3 if quick else 400
+        a, z = timed(upsert, n_up, s_ing)
+        torch.cuda.synchronize(dev)
+        up_alone_us = a.elapsed_time(z) * 1e3 / n_up
+        bytes_per_batch = rows * (2 * s.doc_row_bytes + 4 + 8 + 8)
+        # both at once: enough upserts queued to cover the whole join window
+        n_cover = 3 if quick else int(1.3 * n_join * join_alone_us / up_alone_us) + 20
+        torch.cuda.synchronize(dev)
+        ua, uz = timed(upsert, n_cover, s_ing)
+        ja, jz = timed(join, n_join, s_join)
+        torch.cuda.synchronize(dev)
+        join_busy_us = ja.elapsed_time(jz) * 1e3 / n_join
+        up_busy_us = ua.elapsed_time(uz) * 1e3 / n_cover
+        # the paper's regime: tens of thousands of updates per second = one steady-state batch every few seconds;
+        # here one batch per 10 ms (10M rows/s at 100k rows), far above it
+        cells.append({"rows_per_batch": rows, "positions": order, "upsert_alone_us": up_alone_us,
+                      "upsert_alone_rows_per_s": rows / (up_alone_us * 1e-6),
+                      "upsert_alone_gbs": bytes_per_batch / (up_alone_us * 1e-6) / 1e9,
+                      "upsert_alone_frac_of_hbm_peak": bytes_per_batch / (up_alone_us * 1e-6) / 1e9 / peak,
+                      "bytes_per_batch": bytes_per_batch,
+                      "join_us_with_back_to_back_upserts": join_busy_us, "join_slowdown": join_busy_us / join_alone_us,
+                      "upsert_us_with_back_to_back_joins": up_busy_us})
+    if store.device_status() != B.CCR_OK:
+        raise SystemExit("device status not clean")
+    head = cells[0]
+    print(json.dumps({
+        "metric": "rows_upserted_per_sec", "value": head["upsert_alone_rows_per_s"], "unit": "rows/s", "n_gpus": 1, "steps": 400,
+        "warmup": 5, "ms_per_step": head["upsert_alone_us"] * 1e-3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "ccr_docstore_upsert into a config-1 store (1,000,000 live rows x 256 B + 600,000 spare); batches of "
+                   "300,000 / 100,000 new rows (features + author id) from device memory; join = config 1 on a second stream"},
+        "roofline": {"bound": "hbm", "achieved": head["upsert_alone_gbs"], "peak": peak, "unit": "GB/s",
+                     "frac": head["upsert_alone_frac_of_hbm_peak"], "traffic": None, "peak_kind": "of " + peak_kind},
+        "join_alone_us": join_alone_us, "cells": cells, "gpu_launches": 400,
+    }))
+    store.free()
+
+
 def sort_bench(args, B, device: int):
     """Algorithm 1 step 1 on the device: the affinity records of every request of a batch, shuffled, are put
     back in key order by ccr_sort_edges.  Timed on the payloads of config 1 (64 lists of 50..5000 records,
@@ -534,6 +635,10 @@ def main():
     if args.config == "sort":
         if rank == 0:
             sort_bench(args, B, local_rank)
+        return
+    if args.config == "ingest":
+        if rank == 0:
+            ingest_bench(args, B, local_rank)
         return
     wl, cfg_flags = make_workload(args.config, rank, args.c3_docs, args.c3_requests)
     b = wl.batch
