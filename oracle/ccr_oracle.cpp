@@ -31,9 +31,18 @@
 //   * Eq. 6 (Section 6.3.1, ccr_oracle_resolve_ids): pos(q) = H[q] if q is indexed, else -1, evaluated with
 //     std::lower_bound on the ascending id array (the paper's own first design).
 //
+//   * Section 4.1.2 "Derived Features" (ccr_oracle_cosine): the member representation is n_chunks medoid
+//     embeddings of `dim` values each, the item embedding has `dim` values; per chunk k the cosine similarity
+//     cos_k = <m_k, x> / (|m_k| |x|) is computed in float32 and stored as float16.  The paper fixes the
+//     precision, not the order or the guard; this build's reading: the three sums (dot, |m|^2, |x|^2) are
+//     float32 fused-multiply-add chains from +0 over the elements in ascending order, the denominator is
+//     sqrtf(|x|^2) * sqrtf(|m|^2) (one rounded product), a denominator below 1e-8 (or NaN) is replaced by 1e-8
+//     (so a zero vector gives 0), the quotient is rounded once to float16 (ties to even), NaN is stored as 0x7fff.
+//
 // Plain, slow and unblocked on purpose; single-threaded unless n_threads > 1, in which case the flat
 // candidate range is cut into contiguous chunks, one std::thread each.
 #include <algorithm>
+#include <cmath>
 #include <cstdint>
 #include <cstring>
 #include <thread>
@@ -296,6 +305,44 @@ int ccr_oracle_resolve_ids(int64_t n_ids, const int64_t* sorted_ids, const int32
     const int64_t* it = std::lower_bound(sorted_ids, sorted_ids + n_ids, queries[i]);
     const int64_t rank = it - sorted_ids;
     out_pos[i] = (rank < n_ids && *it == queries[i]) ? (positions ? positions[rank] : static_cast<int32_t>(rank)) : -1;
+  }
+  return 0;
+}
+
+// Section 4.1.2, derived features: for candidate j of request r with position p = cand_idx[j], x = elements
+// [item_first, item_first + dim) of document row p (float16; a position outside [0, n_docs) gives x = 0) and
+// m_k = member_emb[r][k * dim .. (k + 1) * dim) (float16): out[j * 8 + k] = float16(cos_k), k < n_chunks <= 8;
+// the other entries of the 8-value block are +0.
+int ccr_oracle_cosine(int64_t n_docs, const void* doc_feats, int64_t doc_row_bytes, int32_t item_first, int32_t dim,
+                      int32_t n_chunks, int32_t n_req, const uint16_t* member_emb, const int32_t* cand_idx,
+                      const int64_t* cand_offsets, uint16_t* out) {
+  if (dim <= 0 || n_chunks <= 0 || n_chunks > 8 || item_first < 0) return -1;
+  if (static_cast<int64_t>(item_first + dim) * 2 > doc_row_bytes) return -2;
+  std::vector<float> x(dim);
+  for (int32_t r = 0; r < n_req; ++r) {
+    for (int64_t j = cand_offsets[r]; j < cand_offsets[r + 1]; ++j) {
+      const int64_t p = cand_idx[j];
+      const bool in_range = p >= 0 && p < n_docs;
+      const uint16_t* row = reinterpret_cast<const uint16_t*>(static_cast<const uint8_t*>(doc_feats) + (in_range ? p : 0) * doc_row_bytes);
+      float nx = 0.0f;
+      for (int32_t e = 0; e < dim; ++e) {
+        x[e] = in_range ? half_bits_to_float(row[item_first + e]) : 0.0f;
+        nx = std::fmaf(x[e], x[e], nx);
+      }
+      for (int32_t k = 0; k < 8; ++k) out[j * 8 + k] = 0;
+      for (int32_t k = 0; k < n_chunks; ++k) {
+        const uint16_t* m = member_emb + (static_cast<int64_t>(r) * n_chunks + k) * dim;
+        float dot = 0.0f, nm = 0.0f;
+        for (int32_t e = 0; e < dim; ++e) {
+          const float me = half_bits_to_float(m[e]);
+          dot = std::fmaf(x[e], me, dot);
+          nm = std::fmaf(me, me, nm);
+        }
+        float den = std::sqrt(nx) * std::sqrt(nm);
+        if (!(den > 1e-8f)) den = 1e-8f;
+        out[j * 8 + k] = float_to_half_bits(dot / den);
+      }
+    }
   }
   return 0;
 }

@@ -50,6 +50,8 @@ def _load():
         lib.ccr_oracle_resolve_ids.argtypes = [i64, vp, vp, i64, vp, vp]
         lib.ccr_oracle_sort_edges.restype = ctypes.c_int
         lib.ccr_oracle_sort_edges.argtypes = [i32, vp, vp, vp, i64, vp, vp, vp]
+        lib.ccr_oracle_cosine.restype = ctypes.c_int
+        lib.ccr_oracle_cosine.argtypes = [i64, vp, i64, i32, i32, i32, i32, vp, vp, vp, vp]
         lib.ccr_oracle_half_to_float_bits.restype = ctypes.c_uint32
         lib.ccr_oracle_half_to_float_bits.argtypes = [ctypes.c_uint16]
         lib.ccr_oracle_float_bits_to_half.restype = ctypes.c_uint16
@@ -162,6 +164,30 @@ def resolve_ids(sorted_ids: np.ndarray, queries: np.ndarray, positions: Optional
     out = np.full(len(queries), -77, dtype=np.int32)
     lib.ccr_oracle_resolve_ids(len(sorted_ids), _ptr(sorted_ids), _ptr(positions), len(queries), _ptr(queries), _ptr(out))
     return out
+
+
+def cosine_features(doc_feats, member_emb, cand_idx, cand_offsets, item_first: int, dim: int, n_chunks: int) -> np.ndarray:
+    """Section 4.1.2, derived features: per-chunk cosine similarity between the request's medoid embeddings
+    (member_emb float16 [n_req, n_chunks * dim]) and the candidate's item embedding (float16 elements
+    [item_first, item_first + dim) of its document row), float32 arithmetic, float16 result.
+    Returns uint8[C, 16]: n_chunks float16 values followed by zeros (the row's derived section)."""
+    lib = _load()
+    doc_feats = _c(doc_feats)
+    if doc_feats.dtype != np.float16:
+        raise ValueError("the item embedding is float16")
+    member_emb = _c(member_emb, np.float16)
+    cand_idx = _c(cand_idx, np.int32)
+    cand_offsets = _c(cand_offsets, np.int64)
+    n_req = len(cand_offsets) - 1
+    if member_emb.shape != (n_req, n_chunks * dim):
+        raise ValueError("member_emb is [n_req, n_chunks * dim]")
+    total = int(cand_offsets[-1]) if n_req > 0 else 0
+    out = np.full((total, 8), 0xCDCD, dtype=np.uint16)
+    rc = lib.ccr_oracle_cosine(doc_feats.shape[0], _ptr(doc_feats), doc_feats.shape[1] * 2, int(item_first), int(dim),
+                               int(n_chunks), n_req, _ptr(member_emb), _ptr(cand_idx), _ptr(cand_offsets), _ptr(out))
+    if rc != 0:
+        raise ValueError("the oracle does not define this case (code %d)" % rc)
+    return out.view(np.uint8).reshape(total, 16)
 
 
 def upsert(doc_feats, author_ids, positions, new_doc_feats=None, new_author_ids=None, actor_ids=None, actor_types=None,

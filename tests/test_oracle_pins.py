@@ -561,3 +561,94 @@ def test_join_sees_upserted_rows_like_a_store_built_directly():
                                     req_feats=b.req_feats, actor_ids=act, actor_types=typ,
                                     reduce_sum_mask=s.reduce_sum_mask)
     assert np.array_equal(rows, brows) and np.array_equal(mask, bmask)
+
+
+# ---------------------------------------------------------------- derived features (Section 4.1.2): chunked cosine
+def _f16_ulp(v):
+    """Spacing of float16 at |v| (subnormal spacing below the smallest normal)."""
+    a = np.maximum(np.abs(np.asarray(v, dtype=np.float64)), 2.0 ** -14)
+    return 2.0 ** (np.floor(np.log2(a)) - 10)
+
+
+def _cos_case(seed, n_docs=200, doc_dim=64, item_first=8, dim=50, n_chunks=3, n_req=3, n_cand=40, scale=1.0):
+    rng = np.random.default_rng(seed)
+    docs = (scale * rng.standard_normal((n_docs, doc_dim))).astype(np.float16)
+    member = (scale * rng.standard_normal((n_req, n_chunks * dim))).astype(np.float16)
+    cands = [rng.integers(-1, n_docs + 1, size=int(rng.integers(0, n_cand + 1))).astype(np.int32) for _ in range(n_req)]
+    co = np.concatenate([[0], np.cumsum([len(c) for c in cands])]).astype(np.int64)
+    return docs, member, np.concatenate(cands).astype(np.int32), co
+
+
+@pytest.mark.parametrize("seed,dim,n_chunks,item_first,scale", [(0, 50, 3, 8, 1.0), (1, 50, 3, 0, 30.0), (2, 7, 1, 16, 0.01),
+                                                                (3, 64, 4, 0, 1.0), (4, 1, 8, 56, 1.0)])
+def test_cosine_against_float64_and_a_numpy_float32_restatement(seed, dim, n_chunks, item_first, scale):
+    docs, member, ci, co = _cos_case(seed, dim=dim, n_chunks=n_chunks, item_first=item_first, scale=scale)
+    got = oracle.cosine_features(docs, member, ci, co, item_first, dim, n_chunks)
+    assert got.shape == (len(ci), 16)
+    vals = got.copy().view(np.float16).astype(np.float64)  # [C, 8]
+    assert not vals[:, n_chunks:].any()
+    req_of = np.searchsorted(co, np.arange(len(ci)), side="right") - 1
+    ok = (ci >= 0) & (ci < docs.shape[0])
+    x = np.where(ok[:, None], docs[np.where(ok, ci, 0), item_first:item_first + dim], 0)
+    # (a) the mathematical definition in float64: within one float16 spacing + the float32 accumulation error
+    x64 = x.astype(np.float64)
+    for k in range(n_chunks):
+        m64 = member[req_of, k * dim:(k + 1) * dim].astype(np.float64)
+        den = np.linalg.norm(x64, axis=1) * np.linalg.norm(m64, axis=1)
+        want = np.where(den > 1e-8, (x64 * m64).sum(axis=1) / np.maximum(den, 1e-8), 0.0)
+        assert np.all(np.abs(vals[:, k] - want) <= _f16_ulp(want) * 0.5001 + 1e-5), k
+    # (b) bit for bit: float16 x float16 products are exact in float32, so the fused chain equals a plain float32
+    #     multiply-add chain, written here with numpy float32 ops over all candidates at once
+    x32 = x.astype(np.float32)
+    nx = np.zeros(len(ci), np.float32)
+    for e in range(dim):
+        nx = nx + x32[:, e] * x32[:, e]
+    for k in range(n_chunks):
+        m32 = member[req_of, k * dim:(k + 1) * dim].astype(np.float32)
+        dot, nm = np.zeros(len(ci), np.float32), np.zeros(len(ci), np.float32)
+        for e in range(dim):
+            dot = dot + x32[:, e] * m32[:, e]
+            nm = nm + m32[:, e] * m32[:, e]
+        den = np.sqrt(nx) * np.sqrt(nm)
+        den = np.where(den > np.float32(1e-8), den, np.float32(1e-8)).astype(np.float32)
+        with np.errstate(over="ignore"):
+            want16 = (dot / den).astype(np.float16)
+        assert np.array_equal(got[:, 2 * k:2 * k + 2].copy().view(np.uint16)[:, 0], want16.view(np.uint16)), k
+
+
+def test_cosine_closed_forms():
+    dim, n_chunks, first = 50, 3, 8
+    rng = np.random.default_rng(9)
+    base = rng.standard_normal(dim).astype(np.float16)
+    base[base == 0] = np.float16(0.5)
+    ortho_a = np.zeros(dim, np.float16); ortho_a[3] = 2.0
+    ortho_b = np.zeros(dim, np.float16); ortho_b[4] = -7.0
+    docs = np.zeros((6, 64), np.float16)
+    docs[:, :first] = 9.0          # other document features around the embedding must not leak in
+    docs[:, first + dim:] = -9.0
+    docs[0, first:first + dim] = base                  # same direction as medoid 0
+    docs[1, first:first + dim] = -base                 # opposite
+    docs[2, first:first + dim] = base * np.float16(2)  # scaled (exact in float16)
+    docs[3, first:first + dim] = ortho_a               # orthogonal to medoid 1
+    docs[4, first:first + dim] = 0                     # zero item embedding
+    docs[5, first:first + dim] = base
+    member = np.zeros((2, n_chunks * dim), np.float16)
+    member[0, 0:dim] = base
+    member[0, dim:2 * dim] = ortho_b
+    member[0, 2 * dim:] = base * np.float16(-0.5)
+    member[1] = 0                                      # a request with an all-zero member representation
+    ci = np.array([0, 1, 2, 3, 4, -1, 6, 5], np.int32)
+    co = np.array([0, 7, 8], np.int64)
+    v = oracle.cosine_features(docs, member, ci, co, first, dim, n_chunks).copy().view(np.float16).reshape(-1, 8)
+    one, minus = np.float16(1.0), np.float16(-1.0)
+    assert v[0, 0] == one and v[0, 2] == minus           # parallel / anti-parallel
+    assert v[1, 0] == minus and v[1, 2] == one
+    assert v[2, 0] == one and v[2, 2] == minus           # scale invariance
+    assert v[3, 1] == 0 and v[0, 1] != 0                 # orthogonal unit directions
+    assert not v[4].any() and not v[5].any() and not v[6].any()  # zero item, unresolved (-1) and out-of-range position
+    assert not v[7].any()                                # zero member representation
+    assert not v[:, n_chunks:].any()
+    # NaN is stored as 0x7fff: an infinite component makes |x| infinite and the quotient inf / inf
+    docs[0, first] = np.float16(np.inf)
+    w = oracle.cosine_features(docs, member, ci[:1], np.array([0, 1, 1], np.int64), first, dim, n_chunks)
+    assert w.copy().view(np.uint16)[0, 0] == 0x7FFF
