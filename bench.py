@@ -65,6 +65,8 @@ def parse_args():
     p.add_argument("--resolvers", type=int, default=0)
     p.add_argument("--padded", action="store_true",
                    help="time the padded batch layout: ccr_compact_valid + ccr_join_batch_padded into T[n_req, n_max]")
+    p.add_argument("--cosine", action="store_true",
+                   help="add the derived cosine section (3 medoids x 50 values against elements 8..57 of the document row)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--timed-only", action="store_true",
                    help="only warm-up and the timed region (for profiler captures): no sustain loop, e2e, latency or CPU legs")
@@ -656,6 +658,13 @@ def main():
                          ws_resolvers=args.resolvers)
     db = B.DeviceBatch(b, device=local_rank)
     flags = args.flags | cfg_flags
+    member = None
+    if args.cosine:
+        store.set_cosine(8, 50, 3)
+        flags |= B.CCR_FLAG_COSINE
+        gm = torch.Generator(device=dev)
+        gm.manual_seed(wl.seed + 7)
+        member = torch.randn((db.n_req, 150), generator=gm, device=dev, dtype=torch.float32).to(torch.float16)
     out_b = store.out_row_bytes(flags)
     C = b.total_cands
     n_buf = 2  # outputs rotate so that consecutive steps do not rewrite lines still in L2
@@ -671,8 +680,12 @@ def main():
         rows, mask = outs[i % n_buf]
         if args.padded:
             B.ccr_compact_valid(store, db.n_req, C, db.cand_idx, db.cand_offsets, c_idx, c_off, c_src)
-            B.ccr_join_batch_padded(store, db.n_req, C, db.max_edge_len, db.n_max_cands, db.edge_keys, db.edge_feats,
-                                    db.edge_offsets, c_idx, c_off, db.req_feats, rows, mask, flags)
+            B.ccr_join_batch_ex(store, db.n_req, C, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets, c_idx,
+                                c_off, db.req_feats, rows, mask, flags, None, db.n_max_cands, member)
+            return
+        if args.cosine:
+            B.ccr_join_batch_ex(store, db.n_req, C, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets,
+                                db.cand_idx, db.cand_offsets, db.req_feats, rows, mask, flags, None, 0, member)
             return
         B.ccr_join_batch(store, db.n_req, C, db.max_edge_len, db.edge_keys, db.edge_feats, db.edge_offsets, db.cand_idx,
                          db.cand_offsets, db.req_feats, rows, mask, flags)
@@ -714,13 +727,15 @@ def main():
     pin = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
     h_in = [pin(b.edge_keys), pin(b.edge_feats.view(np.uint8)), pin(b.edge_offsets), pin(b.cand_idx), pin(b.cand_offsets),
             pin(None if b.req_feats is None else b.req_feats.view(np.uint8))]
-    h_rows = torch.empty((C, out_b), dtype=torch.uint8).pin_memory()
+    flags_plain = flags & ~B.CCR_FLAG_COSINE  # the host-buffer and single-request legs run without the derived section
+    out_b_plain = store.out_row_bytes(flags_plain)
+    h_rows = torch.empty((C, out_b_plain), dtype=torch.uint8).pin_memory()
     h_mask = torch.empty((C,), dtype=torch.uint8).pin_memory()
     h2d = int(sum(t.numel() * t.element_size() for t in h_in if t is not None))
     d2h = int(h_rows.numel() + h_mask.numel())
 
     def e2e_step():
-        B.ccr_join_batch_host(store, ws, b.n_req, C, b.max_edge_len, len(b.edge_keys), *h_in, h_rows, h_mask, flags)
+        B.ccr_join_batch_host(store, ws, b.n_req, C, b.max_edge_len, len(b.edge_keys), *h_in, h_rows, h_mask, flags_plain)
 
     e2e_steps = args.e2e_steps or max(1, min(args.steps, 10 if C < 4_000_000 else 2))
     if args.timed_only:
@@ -760,7 +775,7 @@ def main():
                 a.record()
                 B.ccr_join_batch(store, 1, c1 - c0, e1 - e0a, db.edge_keys[e0a:], db.edge_feats[e0a:], one_eo,
                                  db.cand_idx[c0:], one_co, None if db.req_feats is None else db.req_feats[r:],
-                                 rows0, mask0, flags)
+                                 rows0, mask0, flags_plain)
                 z.record()
                 evs.append((a, z))
         torch.cuda.synchronize(dev)
@@ -798,6 +813,10 @@ def main():
                            "p50": pct(lat, 0.50), "p99": pct(lat, 0.99), "n": len(lat)},
             "clocks": sampler.summary(t_wall0, t_wall1) if sampler is not None else None,
         }
+        if args.cosine:
+            line["config"]["derived"] = ("cosine section: 3 medoids x 50 values (per-request float16 member embeddings) against "
+                                         "elements 8..57 of the document row, 32 more bytes per output row; e2e and latency legs "
+                                         "run without it")
         if args.padded:
             line["config"]["layout"] = ("padded T[%d, %d]: a step is ccr_compact_valid (3 launches, %.1f us alone, L2-warm) + "
                                         "pad fill + join; the roofline figure divides the join's bytes by the whole step"

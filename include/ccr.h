@@ -75,8 +75,10 @@ enum {
                                            tree) even when the list would fit; testing aid          */
   CCR_FLAG_STATIC_SPLIT      = 1u << 6, /* warp-specialised kernel: give every block one equal contiguous
                                            slice instead of drawing chunks from a device-side counter */
-  CCR_FLAG_TWO_PHASE         = 1u << 7  /* use the two-phase kernel (every warp alternates search and
+  CCR_FLAG_TWO_PHASE         = 1u << 7, /* use the two-phase kernel (every warp alternates search and
                                            row streaming) instead of the warp-specialised kernel      */
+  CCR_FLAG_COSINE            = 1u << 8  /* append the derived cosine section (ccr_docstore_set_cosine,
+                                           ccr_join_batch_ex); adds 32 bytes to the row                */
 };
 
 /* Create an empty store on desc->device.  Allocates doc_feats [n_docs, doc_dim] and author ids
@@ -209,6 +211,51 @@ ccr_status ccr_join_batch_padded(const ccr_docstore* store,
                                  uint8_t*       out_mask,  /* DEVICE [n_req * n_max]                      */
                                  uint32_t       flags,
                                  void*          stream);
+
+/* Derived features (Section 4.1.2 "Derived Features"): the member representation is n_chunks medoid embeddings
+ * of `dim` values each (3 x 50 in the paper), the item embedding has `dim` values; per chunk the cosine
+ * similarity is computed in float32 and stored as float16.  Here the item embedding is elements
+ * [item_first, item_first + dim) of the document row (float16 stores only; item_first a multiple of 8; the
+ * 16-byte piece holding the last element must lie inside the row), and the member embeddings arrive per
+ * request through ccr_join_io::member_emb.  With CCR_FLAG_COSINE every output row gets a last 32-byte section
+ * [cos_0 .. cos_{n_chunks-1}, 0 ...] of float16 values (one whole 32-byte sector, so that rows whose other
+ * sections are multiples of 32 bytes stay sector-aligned), computed by the join kernel from the row it streams:
+ *     dot_k = sum_e x[e] m_k[e],  |x|^2 = sum_e x[e]^2,  |m_k|^2 = sum_e m_k[e]^2
+ *             each a float32 fused-multiply-add chain from +0 over e = 0 .. dim-1 in ascending order;
+ *     den_k = sqrtf(|x|^2) * sqrtf(|m_k|^2), replaced by 1e-8 unless den_k > 1e-8 (zero vectors give 0);
+ *     cos_k = float16(dot_k / den_k), round to nearest even; NaN is stored as 0x7fff.
+ * A candidate whose position is outside [0, n_docs) has x = 0.  dim <= 64, n_chunks <= 4
+ * (CCR_ERR_UNSUPPORTED above).  spec == NULL switches the section off.  HOST call, no device work.      */
+typedef struct {
+  int32_t item_first; /* first element of the item embedding in a document row            */
+  int32_t dim;        /* elements per chunk                                                 */
+  int32_t n_chunks;   /* medoid chunks of the member representation                         */
+  int32_t reserved;   /* 0                                                                  */
+} ccr_cosine_spec;
+ccr_status ccr_docstore_set_cosine(ccr_docstore* store, const ccr_cosine_spec* spec);
+
+/* The join with every optional input in one argument block: ccr_join_batch (n_max == 0) or
+ * ccr_join_batch_padded (n_max > 0) with the same meaning of every field, plus member_emb for
+ * CCR_FLAG_COSINE: DEVICE float16 [n_req, n_chunks * dim], chunk k of request r at
+ * member_emb[(r * n_chunks + k) * dim], 2-byte aligned; ignored without the flag.  struct_bytes must be
+ * sizeof(ccr_join_io).  The derived section is computed by the warp-specialised kernel only: with
+ * CCR_FLAG_TWO_PHASE or a first-degree CCR_FLAG_CANDS_SORTED the call returns CCR_ERR_UNSUPPORTED.        */
+typedef struct {
+  uint32_t       struct_bytes;
+  int32_t        n_req;
+  int64_t        total_cands, max_edge_len;
+  int64_t        n_max;          /* 0 = ragged output                                       */
+  const int64_t* edge_keys;
+  const void*    edge_feats;
+  const int64_t* edge_offsets;
+  const int32_t* cand_idx;
+  const int64_t* cand_offsets;
+  const void*    req_feats;
+  const void*    member_emb;     /* DEVICE float16 [n_req, n_chunks * dim] or NULL          */
+  void*          out_rows;
+  uint8_t*       out_mask;
+} ccr_join_io;
+ccr_status ccr_join_batch_ex(const ccr_docstore* store, const ccr_join_io* io, uint32_t flags, void* stream);
 
 /* Algorithm 1 step 1 for request payloads whose affinity records arrive unsorted: for every request r the
  * records [edge_offsets[r], edge_offsets[r+1]) — key int64 + feature row of the store's edge width — are put

@@ -311,8 +311,8 @@ int ccr_oracle_resolve_ids(int64_t n_ids, const int64_t* sorted_ids, const int32
 
 // Section 4.1.2, derived features: for candidate j of request r with position p = cand_idx[j], x = elements
 // [item_first, item_first + dim) of document row p (float16; a position outside [0, n_docs) gives x = 0) and
-// m_k = member_emb[r][k * dim .. (k + 1) * dim) (float16): out[j * 8 + k] = float16(cos_k), k < n_chunks <= 8;
-// the other entries of the 8-value block are +0.
+// m_k = member_emb[r][k * dim .. (k + 1) * dim) (float16): out[j * 16 + k] = float16(cos_k), k < n_chunks <= 8;
+// the other entries of the 16-value (32-byte) block are +0.
 int ccr_oracle_cosine(int64_t n_docs, const void* doc_feats, int64_t doc_row_bytes, int32_t item_first, int32_t dim,
                       int32_t n_chunks, int32_t n_req, const uint16_t* member_emb, const int32_t* cand_idx,
                       const int64_t* cand_offsets, uint16_t* out) {
@@ -329,7 +329,7 @@ int ccr_oracle_cosine(int64_t n_docs, const void* doc_feats, int64_t doc_row_byt
         x[e] = in_range ? half_bits_to_float(row[item_first + e]) : 0.0f;
         nx = std::fmaf(x[e], x[e], nx);
       }
-      for (int32_t k = 0; k < 8; ++k) out[j * 8 + k] = 0;
+      for (int32_t k = 0; k < 16; ++k) out[j * 16 + k] = 0;
       for (int32_t k = 0; k < n_chunks; ++k) {
         const uint16_t* m = member_emb + (static_cast<int64_t>(r) * n_chunks + k) * dim;
         float dot = 0.0f, nm = 0.0f;
@@ -340,7 +340,7 @@ int ccr_oracle_cosine(int64_t n_docs, const void* doc_feats, int64_t doc_row_byt
         }
         float den = std::sqrt(nx) * std::sqrt(nm);
         if (!(den > 1e-8f)) den = 1e-8f;
-        out[j * 8 + k] = float_to_half_bits(dot / den);
+        out[j * 16 + k] = float_to_half_bits(dot / den);
       }
     }
   }

@@ -170,7 +170,7 @@ def cosine_features(doc_feats, member_emb, cand_idx, cand_offsets, item_first: i
     """Section 4.1.2, derived features: per-chunk cosine similarity between the request's medoid embeddings
     (member_emb float16 [n_req, n_chunks * dim]) and the candidate's item embedding (float16 elements
     [item_first, item_first + dim) of its document row), float32 arithmetic, float16 result.
-    Returns uint8[C, 16]: n_chunks float16 values followed by zeros (the row's derived section)."""
+    Returns uint8[C, 32]: n_chunks float16 values followed by zeros (the row's derived section, one 32-byte sector)."""
     lib = _load()
     doc_feats = _c(doc_feats)
     if doc_feats.dtype != np.float16:
@@ -182,12 +182,12 @@ def cosine_features(doc_feats, member_emb, cand_idx, cand_offsets, item_first: i
     if member_emb.shape != (n_req, n_chunks * dim):
         raise ValueError("member_emb is [n_req, n_chunks * dim]")
     total = int(cand_offsets[-1]) if n_req > 0 else 0
-    out = np.full((total, 8), 0xCDCD, dtype=np.uint16)
+    out = np.full((total, 16), 0xCDCD, dtype=np.uint16)
     rc = lib.ccr_oracle_cosine(doc_feats.shape[0], _ptr(doc_feats), doc_feats.shape[1] * 2, int(item_first), int(dim),
                                int(n_chunks), n_req, _ptr(member_emb), _ptr(cand_idx), _ptr(cand_offsets), _ptr(out))
     if rc != 0:
         raise ValueError("the oracle does not define this case (code %d)" % rc)
-    return out.view(np.uint8).reshape(total, 16)
+    return out.view(np.uint8).reshape(total, 32)
 
 
 def upsert(doc_feats, author_ids, positions, new_doc_feats=None, new_author_ids=None, actor_ids=None, actor_types=None,

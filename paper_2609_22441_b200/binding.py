@@ -36,15 +36,29 @@ CCR_FLAG_FIRST_DEGREE_ONLY = 1 << 4
 CCR_FLAG_FORCE_SAMPLED = 1 << 5
 CCR_FLAG_STATIC_SPLIT = 1 << 6
 CCR_FLAG_TWO_PHASE = 1 << 7
+CCR_FLAG_COSINE = 1 << 8
 
 EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_upsert", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
-    "ccr_compact_valid", "ccr_join_batch_padded",
+    "ccr_compact_valid", "ccr_join_batch_padded", "ccr_join_batch_ex", "ccr_docstore_set_cosine",
     "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
     "ccr_static_payload_capacity", "ccr_join_payload_static", "ccr_docstore_selftest_wait",
     "ccr_sort_edges", "ccr_idindex_create", "ccr_idindex_free", "ccr_resolve_ids",
 )
+
+
+class ccr_cosine_spec(ctypes.Structure):
+    _fields_ = [("item_first", ctypes.c_int32), ("dim", ctypes.c_int32), ("n_chunks", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+class ccr_join_io(ctypes.Structure):
+    _fields_ = [("struct_bytes", ctypes.c_uint32), ("n_req", ctypes.c_int32), ("total_cands", ctypes.c_int64),
+                ("max_edge_len", ctypes.c_int64), ("n_max", ctypes.c_int64), ("edge_keys", ctypes.c_void_p),
+                ("edge_feats", ctypes.c_void_p), ("edge_offsets", ctypes.c_void_p), ("cand_idx", ctypes.c_void_p),
+                ("cand_offsets", ctypes.c_void_p), ("req_feats", ctypes.c_void_p), ("member_emb", ctypes.c_void_p),
+                ("out_rows", ctypes.c_void_p), ("out_mask", ctypes.c_void_p)]
 
 
 class ccr_docstore_desc(ctypes.Structure):
@@ -100,6 +114,10 @@ def lib() -> ctypes.CDLL:
     L.ccr_workspace_free.argtypes = [vp]
     L.ccr_docstore_upsert.restype = ctypes.c_int
     L.ccr_docstore_upsert.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp]
+    L.ccr_join_batch_ex.restype = ctypes.c_int
+    L.ccr_join_batch_ex.argtypes = [vp, ctypes.POINTER(ccr_join_io), u32, vp]
+    L.ccr_docstore_set_cosine.restype = ctypes.c_int
+    L.ccr_docstore_set_cosine.argtypes = [vp, ctypes.POINTER(ccr_cosine_spec)]
     L.ccr_compact_valid.restype = ctypes.c_int
     L.ccr_compact_valid.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, vp]
     L.ccr_join_batch_padded.restype = ctypes.c_int
@@ -209,6 +227,14 @@ class Docstore:
                                          _ptr(author_ids), _ptr(actor_ids), _ptr(actor_types), _stream_ptr(stream)),
                "ccr_docstore_upsert")
 
+    def set_cosine(self, item_first: int, dim: int, n_chunks: int) -> None:
+        """ccr_docstore_set_cosine: where the item embedding sits in a document row (n_chunks == 0 switches off)."""
+        if n_chunks == 0:
+            _check(lib().ccr_docstore_set_cosine(self._h, None), "ccr_docstore_set_cosine")
+            return
+        spec = ccr_cosine_spec(int(item_first), int(dim), int(n_chunks), 0)
+        _check(lib().ccr_docstore_set_cosine(self._h, ctypes.byref(spec)), "ccr_docstore_set_cosine")
+
     def out_row_bytes(self, flags: int = 0) -> int:
         return int(lib().ccr_out_row_bytes(self._h, int(flags)))
 
@@ -248,6 +274,19 @@ def ccr_join_batch(store: Docstore, n_req: int, total_cands: int, max_edge_len: 
                               _ptr(edge_feats), _ptr(edge_offsets), _ptr(cand_idx), _ptr(cand_offsets),
                               _ptr(req_feats), _ptr(out_rows), _ptr(out_mask), int(flags), _stream_ptr(stream))
     _check(st, "ccr_join_batch")
+    return st
+
+
+def ccr_join_batch_ex(store: Docstore, n_req: int, total_cands: int, max_edge_len: int, edge_keys, edge_feats,
+                      edge_offsets, cand_idx, cand_offsets, req_feats, out_rows, out_mask, flags: int = 0, stream=None,
+                      n_max: int = 0, member_emb=None) -> int:
+    """Raw call: the join with every optional input (padded layout, member embeddings for the cosine section)."""
+    p = _ptr
+    io = ccr_join_io(ctypes.sizeof(ccr_join_io), int(n_req), int(total_cands), int(max_edge_len), int(n_max),
+                     p(edge_keys), p(edge_feats), p(edge_offsets), p(cand_idx), p(cand_offsets), p(req_feats),
+                     p(member_emb), p(out_rows), p(out_mask))
+    st = lib().ccr_join_batch_ex(store.handle, ctypes.byref(io), int(flags), _stream_ptr(stream))
+    _check(st, "ccr_join_batch_ex")
     return st
 
 

@@ -68,6 +68,7 @@ struct ccr_docstore {
   int blocks_per_sm;  // cap on resident blocks per SM of the two-phase kernel (0 = as many as fit)
   int ws_streamers, ws_resolvers;  // warp split of the warp-specialised kernel
   int n_sms;
+  int cos_first, cos_dim, cos_chunks;  // derived cosine section (cos_chunks == 0: not configured)
   int64_t launches;
 };
 
@@ -176,17 +177,23 @@ __global__ void pack_ids_kernel(ccr::IdRec* recs, long long n, int max_actors, c
 using KernelFn = void (*)(const ccr::JoinArgs);
 using WsKernelFn = void (*)(const ccr::JoinArgs, int);
 
+// The tuned variants compute the derived cosine section for an item embedding of exactly this many 16-byte
+// pieces (the paper's 50 values span 7); any other shape runs on the generic variant.
+constexpr int kTunedCosPieces = 7;
+
 struct Variant {
   int doc_ch, edge_ch, req_ch;
   KernelFn first, second, merge;
-  WsKernelFn ws_first, ws_second;
+  WsKernelFn ws_first, ws_second, ws_first_cos, ws_second_cos;
 };
 
 #define CCR_VARIANT(D, E, R)                                                                                      \
   Variant {                                                                                                       \
     D, E, R, ccr::join_kernel<D, E, R, false, false>, ccr::join_kernel<D, E, R, true, false>,                     \
         ccr::join_kernel<D, E, R, false, true>,                                                                   \
-        ccr::join_ws_kernel<D, E, R, false>, ccr::join_ws_kernel<D, E, R, true>                                   \
+        ccr::join_ws_kernel<D, E, R, false>, ccr::join_ws_kernel<D, E, R, true>,                                  \
+        ccr::join_ws_kernel<D, E, R, false, (D > 0 ? kTunedCosPieces : -1)>,                                      \
+        ccr::join_ws_kernel<D, E, R, true, (D > 0 ? kTunedCosPieces : -1)>                                        \
   }
 
 const Variant kVariants[] = {
@@ -220,7 +227,8 @@ ccr_status allow_large_smem() {
       cudaGetLastError();
       return CCR_ERR_CUDA;
     }
-    const WsKernelFn ws[2] = {kVariants[i].ws_first, kVariants[i].ws_second};
+    const WsKernelFn ws[4] = {kVariants[i].ws_first, kVariants[i].ws_second, kVariants[i].ws_first_cos,
+                              kVariants[i].ws_second_cos};
     for (WsKernelFn f : ws) {
       if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemBytes) != cudaSuccess) {
         cudaGetLastError();
@@ -233,7 +241,7 @@ ccr_status allow_large_smem() {
 
 size_t out_row_bytes(const ccr_docstore* s, uint32_t flags) {
   const bool second = s->desc.max_actors > 0 && !(flags & CCR_FLAG_FIRST_DEGREE_ONLY);
-  return static_cast<size_t>(s->doc_b) + s->edge_b * (second ? 2 : 1) + s->req_b;
+  return static_cast<size_t>(s->doc_b) + s->edge_b * (second ? 2 : 1) + s->req_b + ((flags & CCR_FLAG_COSINE) ? ccr::kCosSectionBytes : 0);
 }
 
 }  // namespace
@@ -642,7 +650,8 @@ namespace {
 ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
                      const int64_t* edge_keys, const void* edge_feats, const int64_t* edge_offsets,
                      const int32_t* cand_idx, const int64_t* cand_offsets, const void* req_feats,
-                     void* out_rows, uint8_t* out_mask, uint32_t flags, void* stream, int64_t n_max) {
+                     void* out_rows, uint8_t* out_mask, uint32_t flags, void* stream, int64_t n_max,
+                     const void* member_emb) {
   if (!good(cs)) return CCR_ERR_BAD_HANDLE;
   ccr_docstore* s = const_cast<ccr_docstore*>(cs);  // only the launch counter and status words change
   if (n_req < 0 || total_cands < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
@@ -667,8 +676,18 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   // which kernel: the merge path and CCR_FLAG_TWO_PHASE take the two-phase kernel, everything else the
   // warp-specialised kernel
   const bool use_ws = !merge && !(flags & CCR_FLAG_TWO_PHASE);
+  const bool cos = (flags & CCR_FLAG_COSINE) != 0;
+  if (cos) {
+    if (s->cos_chunks == 0 || !member_emb) return CCR_ERR_INVALID_ARG;  // not configured / no member embeddings
+    if (!use_ws) return CCR_ERR_UNSUPPORTED;  // the derived section is computed by the warp-specialised kernel only
+    if (reinterpret_cast<uintptr_t>(member_emb) & 1u) return CCR_ERR_INVALID_ARG;
+  }
+  const int n_str = s->ws_streamers > 0 ? s->ws_streamers : (second ? 11 : 12);
+  const int n_res = s->ws_resolvers > 0 ? s->ws_resolvers : (second ? 5 : 4);
+  const int cos_stage = cos ? 32 * (((s->cos_dim + 7) / 8) | 1) * 16 : 0;
+  const int cos_bytes = cos ? ccr::ws_cos_bytes(n_str, cos_stage) : 0;
   auto smem_for = [&](int t, int cap) -> size_t {
-    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, cap, n_req <= ccr::kWsMaxCachedReq ? n_req : 0).bytes)
+    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, cap, n_req <= ccr::kWsMaxCachedReq ? n_req : 0, cos_bytes).bytes)
                   : static_cast<size_t>(ccr::TileLayout(t, second, merge, cap).bytes);
   };
   // Keys staged per request.  The warp-specialised kernel runs one block per SM, so by default it stages
@@ -720,6 +739,11 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   a.out_rows = static_cast<uint8_t*>(out_rows);
   a.out_mask = out_mask;
   a.n_max = n_max;
+  a.member_emb = static_cast<const uint16_t*>(member_emb);
+  a.cos_first = s->cos_first;
+  a.cos_dim = s->cos_dim;
+  a.cos_chunks = cos ? s->cos_chunks : 0;
+  a.cos_stage = cos_stage;
   a.tile = tile;
   a.key_cap = key_cap;
   a.min_stride_log2 = (flags & CCR_FLAG_FORCE_SAMPLED) ? 2 : 0;
@@ -743,13 +767,14 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     if (s->status_host[1] != 0) return CCR_ERR_VALIDATION;
   }
 
-  const Variant& v = pick_variant(a.doc_ch, a.edge_ch, a.req_ch);
+  const bool cos_tuned = cos && (s->cos_dim + 7) / 8 == kTunedCosPieces;
+  const Variant& v = (cos && !cos_tuned) ? kVariants[kNumVariants - 1] : pick_variant(a.doc_ch, a.edge_ch, a.req_ch);
   const long long groups = (total_cands + 31) / 32;
   if (use_ws) {
     // one persistent warp-specialised block per SM (fewer when there are fewer 32-row groups than SMs)
     long long blocks = s->n_sms;
     if (blocks > groups) blocks = groups;
-    const WsKernelFn fn = second ? v.ws_second : v.ws_first;
+    const WsKernelFn fn = cos ? (second ? v.ws_second_cos : v.ws_first_cos) : (second ? v.ws_second : v.ws_first);
     // dynamic chunk scheduling through a pair of device words; each launch takes the next pair in turn, so
     // up to kSchedRegions launches of one store may be in flight at once (on any streams)
     // Small launches (fewer tiles than two rounds per block) are split evenly instead: drawing whole rounds
@@ -758,8 +783,6 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     const long long n_tiles = (total_cands + a.tile - 1) / a.tile;
     const bool dynamic = !(flags & CCR_FLAG_STATIC_SPLIT) && n_tiles >= 2LL * blocks * n_res_auto;
     if (dynamic) a.sched = s->status + 4 + 2 * static_cast<int>(s->launches % kSchedRegions);
-    const int n_str = s->ws_streamers > 0 ? s->ws_streamers : (second ? 11 : 12);
-    const int n_res = s->ws_resolvers > 0 ? s->ws_resolvers : (second ? 5 : 4);
     fn<<<static_cast<unsigned>(blocks), (n_str + n_res) * 32, smem, st>>>(a, n_str);
   } else {
     // persistent two-phase kernel: as many blocks as stay resident, each with at least 256 candidates
@@ -787,15 +810,19 @@ ccr_status ccr_join_batch(const ccr_docstore* cs, int32_t n_req, int64_t total_c
                           const int64_t* edge_keys, const void* edge_feats, const int64_t* edge_offsets,
                           const int32_t* cand_idx, const int64_t* cand_offsets, const void* req_feats,
                           void* out_rows, uint8_t* out_mask, uint32_t flags, void* stream) {
+  if (flags & CCR_FLAG_COSINE) return CCR_ERR_INVALID_ARG;  // the member embeddings come through ccr_join_batch_ex
   return join_impl(cs, n_req, total_cands, max_edge_len, edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets,
-                   req_feats, out_rows, out_mask, flags, stream, 0);
+                   req_feats, out_rows, out_mask, flags, stream, 0, nullptr);
 }
 
-ccr_status ccr_join_batch_padded(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
-                                 int64_t n_max, const int64_t* edge_keys, const void* edge_feats,
-                                 const int64_t* edge_offsets, const int32_t* cand_idx, const int64_t* cand_offsets,
-                                 const void* req_feats, void* out_rows, uint8_t* out_mask, uint32_t flags,
-                                 void* stream) {
+}  // extern "C"
+
+namespace {
+ccr_status padded_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                       int64_t n_max, const int64_t* edge_keys, const void* edge_feats,
+                       const int64_t* edge_offsets, const int32_t* cand_idx, const int64_t* cand_offsets,
+                       const void* req_feats, void* out_rows, uint8_t* out_mask, uint32_t flags,
+                       void* stream, const void* member_emb) {
   if (!good(cs)) return CCR_ERR_BAD_HANDLE;
   if (n_max <= 0 || n_req < 0) return CCR_ERR_INVALID_ARG;
   if (flags & CCR_FLAG_VALIDATE) return CCR_ERR_UNSUPPORTED;  // validate with ccr_join_batch semantics first
@@ -815,7 +842,49 @@ ccr_status ccr_join_batch_padded(const ccr_docstore* cs, int32_t n_req, int64_t 
   }
   if (total_cands == 0) return CCR_OK;
   return join_impl(cs, n_req, total_cands, max_edge_len, edge_keys, edge_feats, edge_offsets, cand_idx, cand_offsets,
-                   req_feats, out_rows, out_mask, flags, stream, n_max);
+                   req_feats, out_rows, out_mask, flags, stream, n_max, member_emb);
+}
+}  // namespace
+
+extern "C" {
+
+ccr_status ccr_join_batch_padded(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, int64_t max_edge_len,
+                                 int64_t n_max, const int64_t* edge_keys, const void* edge_feats,
+                                 const int64_t* edge_offsets, const int32_t* cand_idx, const int64_t* cand_offsets,
+                                 const void* req_feats, void* out_rows, uint8_t* out_mask, uint32_t flags,
+                                 void* stream) {
+  if (flags & CCR_FLAG_COSINE) return CCR_ERR_INVALID_ARG;  // the member embeddings come through ccr_join_batch_ex
+  return padded_impl(cs, n_req, total_cands, max_edge_len, n_max, edge_keys, edge_feats, edge_offsets, cand_idx,
+                     cand_offsets, req_feats, out_rows, out_mask, flags, stream, nullptr);
+}
+
+ccr_status ccr_join_batch_ex(const ccr_docstore* cs, const ccr_join_io* io, uint32_t flags, void* stream) {
+  if (!good(cs)) return CCR_ERR_BAD_HANDLE;
+  if (io == nullptr || io->struct_bytes != sizeof(ccr_join_io) || io->n_max < 0) return CCR_ERR_INVALID_ARG;
+  if (io->n_max > 0)
+    return padded_impl(cs, io->n_req, io->total_cands, io->max_edge_len, io->n_max, io->edge_keys, io->edge_feats,
+                       io->edge_offsets, io->cand_idx, io->cand_offsets, io->req_feats, io->out_rows, io->out_mask,
+                       flags, stream, io->member_emb);
+  return join_impl(cs, io->n_req, io->total_cands, io->max_edge_len, io->edge_keys, io->edge_feats, io->edge_offsets,
+                   io->cand_idx, io->cand_offsets, io->req_feats, io->out_rows, io->out_mask, flags, stream, 0,
+                   io->member_emb);
+}
+
+ccr_status ccr_docstore_set_cosine(ccr_docstore* s, const ccr_cosine_spec* spec) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  if (spec == nullptr) {
+    s->cos_first = s->cos_dim = s->cos_chunks = 0;
+    return CCR_OK;
+  }
+  if (spec->item_first < 0 || spec->dim <= 0 || spec->n_chunks <= 0 || (spec->item_first & 7)) return CCR_ERR_INVALID_ARG;
+  if (s->desc.doc_dtype != CCR_F16) return CCR_ERR_UNSUPPORTED;  // the item embedding is float16
+  if (spec->dim > ccr::kCosMaxDim || spec->n_chunks > ccr::kCosMaxChunks) return CCR_ERR_UNSUPPORTED;
+  // the embedding is read in 16-byte pieces: the last piece must end inside the row
+  if ((spec->item_first + ((spec->dim + 7) & ~7)) * 2 > s->doc_b) return CCR_ERR_INVALID_ARG;
+  s->cos_first = spec->item_first;
+  s->cos_dim = spec->dim;
+  s->cos_chunks = spec->n_chunks;
+  return CCR_OK;
 }
 
 ccr_status ccr_compact_valid(const ccr_docstore* cs, int32_t n_req, int64_t total_cands, const int32_t* cand_idx, const int64_t* cand_offsets,

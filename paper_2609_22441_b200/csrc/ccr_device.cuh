@@ -30,6 +30,11 @@ struct __align__(64) IdRec {
 static_assert(sizeof(IdRec) == 64, "one record per 64-byte line");
 
 // Everything a join launch needs, passed by value as the kernel argument.
+constexpr int kCosMaxDim = 64;     // most elements per medoid chunk
+constexpr int kCosMaxChunks = 4;   // most medoid chunks
+constexpr int kCosSectionBytes = 32;  // derived section of a row: fp16 cosines, zero-filled to one 32-byte sector
+constexpr int kCosSlotFloat4 = kCosMaxDim + 1;  // per ring slot: element e -> (m_0[e] .. m_3[e]), then the squared norms
+
 struct JoinArgs {
   // store
   const uint8_t* doc_feats;
@@ -52,6 +57,13 @@ struct JoinArgs {
   const uint8_t* req_feats;
   uint8_t* out_rows;
   uint8_t* out_mask;
+  // derived features (Section 4.1.2): per-chunk cosine of the request's medoid embeddings and the candidate's
+  // item embedding, appended to the row as a 32-byte section of fp16 values (zero-filled)
+  const uint16_t* member_emb;  // fp16 [n_req, cos_chunks * cos_dim]; unused when cos_chunks == 0
+  int cos_first;               // first element of the item embedding inside a document row (multiple of 8)
+  int cos_dim;                 // elements per chunk (<= kCosMaxDim)
+  int cos_chunks;              // chunks (<= kCosMaxChunks); 0 = no derived section
+  int cos_stage;               // bytes of embedding staging per streamer warp: 32 rows x (pieces | 1) x 16
   long long n_max;            // 0: ragged output (row j); > 0: padded output, row r * n_max + (j - cand_offsets[r])
   // launch shape
   int tile;                   // candidates per block

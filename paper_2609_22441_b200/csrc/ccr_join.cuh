@@ -88,7 +88,7 @@ __device__ __forceinline__ uint4 edge2_reduce(unsigned long long reduce_sum_mask
 }
 
 // Section widths of a launch, in 16-byte chunks and bytes (compile-time where the variant fixes them).
-template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND>
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, bool COS = false>
 struct RowShape {
   int doc_ch, edge_ch, req_ch, doc_b, edge_b, req_b;
   long long out_b;
@@ -99,7 +99,7 @@ struct RowShape {
     doc_b = doc_ch * 16;
     edge_b = edge_ch * 16;
     req_b = req_ch * 16;
-    out_b = doc_b + edge_b * (SECOND ? 2 : 1) + req_b;
+    out_b = doc_b + edge_b * (SECOND ? 2 : 1) + req_b + (COS ? kCosSectionBytes : 0);
   }
 };
 
@@ -167,12 +167,74 @@ struct TileLayout {
 };
 
 // ---- phase B: 32 rows of one warp, everything already resolved in shared memory -------------------
-template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND>
-__device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND>& sh,
+// Derived section (Section 4.1.2) of the row held by this lane.  xv: the 16-byte pieces of the document row that
+// hold the item embedding (element e of the embedding is half e of the pieces taken in order).  Dot product and
+// squared norms are float32 fused-multiply-add chains over the elements in ascending order, exactly the order
+// of the definition, so the result does not depend on how rows are spread over lanes.  cosM: element e ->
+// (m_0[e], m_1[e], m_2[e], m_3[e]) as float32, cosM[kCosMaxDim] = the chunks' squared norms.
+// TUNED: the embedding spans exactly NP pieces (cos_dim > 8 * (NP - 1)), so only the last piece needs the
+// element bound; otherwise every piece is checked against the run-time width.  xrow: this lane's row in the
+// warp's staging block.
+template <int NP, bool TUNED>
+__device__ __forceinline__ uint4 cosine_section(const JoinArgs& a, const uint4* xrow, const float4* cosM) {
+  const int pieces = TUNED ? NP : (a.cos_dim + 7) >> 3;
+  float nx = 0.0f, d[kCosMaxChunks] = {0.0f, 0.0f, 0.0f, 0.0f};
+  auto element = [&](float x, int e) {
+    const float4 m = cosM[e];
+    nx = fmaf(x, x, nx);
+    d[0] = fmaf(x, m.x, d[0]);
+    d[1] = fmaf(x, m.y, d[1]);
+    d[2] = fmaf(x, m.z, d[2]);
+    d[3] = fmaf(x, m.w, d[3]);
+  };
+  uint4 xq[NP];  // the whole embedding is requested before the first element is used
+#pragma unroll
+  for (int q = 0; q < NP; ++q) xq[q] = q < pieces ? xrow[q] : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+  for (int q = 0; q < NP; ++q) {
+    if (q >= pieces) break;  // warp-uniform
+    const uint4 xv = xq[q];
+    const unsigned w[4] = {xv.x, xv.y, xv.z, xv.w};
+    const bool whole = TUNED && q < NP - 1;  // every element of the piece belongs to the embedding
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[t]));
+      const int e = q * 8 + t * 2;
+      if (whole || e < a.cos_dim) element(f.x, e);
+      if (whole || e + 1 < a.cos_dim) element(f.y, e + 1);
+    }
+  }
+  const float4 nm4 = cosM[kCosMaxDim];
+  const float nm[kCosMaxChunks] = {nm4.x, nm4.y, nm4.z, nm4.w};
+  const float sx = sqrtf(nx);
+  unsigned h[kCosMaxChunks];
+#pragma unroll
+  for (int k = 0; k < kCosMaxChunks; ++k) {
+    float den = sx * sqrtf(nm[k]);
+    if (!(den > 1e-8f)) den = 1e-8f;
+    const float c = d[k] / den;
+    h[k] = __half_as_ushort(__float2half_rn(c));
+    if (c != c) h[k] = 0x7fffu;
+    if (k >= a.cos_chunks) h[k] = 0u;
+  }
+  return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), 0u, 0u);
+}
+
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0>
+__device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND, CNP != 0>& sh,
                                            const int* s_idx, const int* s_pos, const int4* s_apos,
                                            const uint8_t* edge_base, const uint8_t* req_src, uint8_t* out, int cnt,
-                                           int lane) {
+                                           int lane, const float4* cosM = nullptr, uint4* stage = nullptr) {
   const long long out_b = sh.out_b;
+  // Derived section: the row streaming below is unchanged; the lanes that hold a piece of the item embedding
+  // also drop it into this warp's staging block in shared memory (row-major, an odd number of 16-byte units
+  // per row so that the read-back by lane = row is conflict-free), and once the group's stores are issued
+  // every lane reads its row's embedding back and computes the cosines.
+  constexpr bool kCos = CNP != 0;
+  [[maybe_unused]] const int p0 = a.cos_first >> 3;
+  [[maybe_unused]] const int np = CNP > 0 ? CNP : (a.cos_dim + 7) >> 3;
+  [[maybe_unused]] const int sstride = np | 1;
+  if constexpr (kCos) __syncwarp();  // the previous group's read-back is done before the block is rewritten
   if constexpr (DOC_CH > 0 && EDGE_CH > 0) {
     // every load of the group is issued before its first store
     uint4 dv[DOC_CH], ev[EDGE_CH];
@@ -194,6 +256,10 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
     for (int i = 0; i < DOC_CH; ++i) {
       const int c = i * 32 + lane, row = c / DOC_CH, piece = c % DOC_CH;
       if (row < cnt) st128_stream(out + row * out_b + piece * 16, dv[i]);
+      if constexpr (kCos) {
+        const int q = piece - p0;
+        if (q >= 0 && q < np) stage[row * sstride + q] = dv[i];
+      }
     }
 #pragma unroll
     for (int i = 0; i < EDGE_CH; ++i) {
@@ -207,6 +273,10 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (ridx >= 0) v = ldg128(a.doc_feats + static_cast<long long>(ridx) * sh.doc_b + piece * 16);
       if (row < cnt) st128_stream(out + row * out_b + piece * 16, v);
+      if constexpr (kCos) {
+        const int q = piece - p0;
+        if (q >= 0 && q < np) stage[row * sstride + q] = v;
+      }
     }
     for (int i = 0; i < sh.edge_ch; ++i) {
       const int c = i * 32 + lane, row = c / sh.edge_ch, piece = c - row * sh.edge_ch;
@@ -245,6 +315,15 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       const int c = i * 32 + lane, row = c / sh.req_ch, piece = c - row * sh.req_ch;
       const uint4 v = ldg128(req_src + piece * 16);
       if (row < cnt) st128_stream(out + row * out_b + off + piece * 16, v);
+    }
+  }
+  if constexpr (kCos) {
+    constexpr int kPieces = CNP > 0 ? CNP : kCosMaxDim / 8;
+    __syncwarp();
+    const uint4 sec = cosine_section<kPieces, (CNP > 0)>(a, stage + lane * sstride, cosM);
+    if (lane < cnt) {  // the section is one whole 32-byte sector: values, then zeros
+      st128_stream(out + lane * out_b + out_b - kCosSectionBytes, sec);
+      st128_stream(out + lane * out_b + out_b - kCosSectionBytes + 16, make_uint4(0u, 0u, 0u, 0u));
     }
   }
 }

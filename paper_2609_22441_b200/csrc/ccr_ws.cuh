@@ -45,13 +45,20 @@ struct WsSlot {          // descriptor of one ring slot
   int r;                 // request index
   int next;              // next 32-row group a streamer warp may take (reset by the resolvers)
   int pad;
-  long long pad2;
+  int cos_r;             // request whose member block the slot's cosine buffer holds (-1 = none)
+  int pad2;
 };
 
+__host__ __device__ inline int ws_cos_bytes(int n_streamers, int stage_per_warp) {
+  return kWsSlots * kCosSlotFloat4 * 16 + n_streamers * stage_per_warp;
+}
+
 struct WsLayout {
-  int off_full, off_empty, off_slots, off_grab, off_offs, off_idx, off_pos, off_apos, off_keys, bytes;
+  int off_full, off_empty, off_slots, off_grab, off_offs, off_idx, off_pos, off_apos, off_cos, off_keys, bytes;
   // n_req_cached: requests whose offsets are mirrored in shared memory (0 = read them from global memory)
-  __host__ __device__ WsLayout(int tile, bool second, int key_cap, int n_req_cached) {
+  // cos_bytes: shared memory of the derived cosine section (0 = off): a block of member-embedding floats per
+  // ring slot, then one embedding staging block per streamer warp
+  __host__ __device__ WsLayout(int tile, bool second, int key_cap, int n_req_cached, int cos_bytes) {
     off_full = kSmemHeader;                 // after the key-staging mbarrier
     off_empty = off_full + kWsSlots * 8;
     off_slots = off_empty + kWsSlots * 8;
@@ -61,27 +68,31 @@ struct WsLayout {
     off_idx = (off_idx + 15) & ~15;
     off_pos = off_idx + kWsSlots * tile * 4;
     off_apos = off_pos + kWsSlots * tile * 4;
-    off_keys = off_apos + (second ? kWsSlots * tile * 16 : 0);
+    off_cos = off_apos + (second ? kWsSlots * tile * 16 : 0);
+    off_keys = off_cos + cos_bytes;
     bytes = off_keys + search_bytes(key_cap, true);
   }
 };
 
-template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND>
+// CNP: 0 = no derived section; > 0 = the item embedding spans exactly CNP 16-byte pieces (tuned); < 0 = any shape
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0>
 __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArgs a, int n_streamers) {
   extern __shared__ __align__(16) unsigned char smem_ws[];
   unsigned char* smem = smem_ws;
+  constexpr bool COS = CNP != 0;
   const int n_req_cached = a.n_req <= kWsMaxCachedReq ? a.n_req : 0;
-  const WsLayout lay(a.tile, SECOND, a.key_cap, n_req_cached);
+  const WsLayout lay(a.tile, SECOND, a.key_cap, n_req_cached, COS ? ws_cos_bytes(n_streamers, a.cos_stage) : 0);
   WsSlot* slots = reinterpret_cast<WsSlot*>(smem + lay.off_slots);
   int* grab = reinterpret_cast<int*>(smem + lay.off_grab);
   int* s_idx = reinterpret_cast<int*>(smem + lay.off_idx);
   int* s_pos = reinterpret_cast<int*>(smem + lay.off_pos);
   int4* s_apos = reinterpret_cast<int4*>(smem + lay.off_apos);
+  float4* s_cos = reinterpret_cast<float4*>(smem + lay.off_cos);
   const SearchSmem ssm = carve_search(smem + lay.off_keys, a.key_cap, true);
   const uint32_t bar = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_threads = blockDim.x;
-  const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND> sh(a);
+  const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND, COS> sh(a);
   const uint32_t full0 = smem_u32(smem + lay.off_full), empty0 = smem_u32(smem + lay.off_empty);
   const int kBarGroup = 1;  // named barrier of the resolver group
 
@@ -101,6 +112,7 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   if (tid == 0) {
     mbar_init(bar, 1);
     for (int s = 0; s < kWsSlots; ++s) {
+      slots[s].cos_r = -1;
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, static_cast<uint32_t>(n_streamers));
     }
@@ -119,6 +131,9 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   const int role_rank = (n_threads >> 5) - 1 - warp;  // resolvers are the last n_res warps
   if (role_rank >= n_res) {
     // ============================ streamers ============================
+    // this warp's embedding staging block (derived cosine section), behind the per-slot member blocks
+    [[maybe_unused]] uint4* cos_stage = reinterpret_cast<uint4*>(
+        smem + lay.off_cos + kWsSlots * kCosSlotFloat4 * 16 + (role_rank - n_res) * (COS ? a.cos_stage : 0));
     for (unsigned it = 0;; ++it) {
       const int s = it % kWsSlots;
       if (!mbar_wait_bounded(full0 + 8 * s, (it / kWsSlots) & 1u)) {
@@ -138,8 +153,10 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
         if (lane == 0) g = atomicAdd(&slots[s].next, 1);
         g = __shfl_sync(kFull, g, 0) * 32;
         if (g >= d.n) break;
-        emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND>(a, sh, idx + g, pos + g, apos + g, edge_base, req_src,
-                                                    a.out_rows + (d.out0 + g) * sh.out_b, min(32, d.n - g), lane);
+        emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND, CNP>(a, sh, idx + g, pos + g, apos + g, edge_base, req_src,
+                                                         a.out_rows + (d.out0 + g) * sh.out_b, min(32, d.n - g), lane,
+                                                         COS ? s_cos + s * kCosSlotFloat4 : nullptr,
+                                                         COS ? cos_stage : nullptr);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
@@ -162,6 +179,8 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   bool dead = false;     // this warp's wait for a free slot expired: keep walking (barriers!), fill nothing
   int staged_r = -1;     // request whose keys are in shared memory
   StagedKeys keys;
+  int cos_r = -1;        // request whose squared member norms lane k < kCosMaxChunks holds in cos_nm
+  float cos_nm = 0.0f;
   const long long n_tiles = (a.total + a.tile - 1) / a.tile;
   constexpr int U = SECOND ? 4 : 8;  // candidates a lane keeps in flight
 
@@ -316,6 +335,36 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
             }
           }
         }
+        if constexpr (COS) {
+          // the request's medoid embeddings as float32, element-major, for the streamers of this slot; a slot
+          // that already holds this request's block (tiles of one request follow each other) keeps it
+          float4* M = s_cos + s * kCosSlotFloat4;
+          if (slots[s].cos_r != r) {
+            const uint16_t* mem = a.member_emb + static_cast<long long>(r) * a.cos_chunks * a.cos_dim;
+            for (int e = lane; e < kCosMaxDim; e += 32) {
+              float m[kCosMaxChunks] = {0.0f, 0.0f, 0.0f, 0.0f};
+              if (e < a.cos_dim) {
+#pragma unroll
+                for (int k = 0; k < kCosMaxChunks; ++k)
+                  if (k < a.cos_chunks) m[k] = __half2float(__ushort_as_half(__ldg(mem + k * a.cos_dim + e)));
+              }
+              M[e] = make_float4(m[0], m[1], m[2], m[3]);
+            }
+            if (r != cos_r) {  // squared norms: lane k sums chunk k in element order, once per request and warp
+              cos_nm = 0.0f;
+              if (lane < a.cos_chunks) {
+                for (int e = 0; e < a.cos_dim; ++e) {
+                  const float v = __half2float(__ushort_as_half(__ldg(mem + lane * a.cos_dim + e)));
+                  cos_nm = fmaf(v, v, cos_nm);
+                }
+              }
+              cos_r = r;
+            }
+            const float n0 = __shfl_sync(kFull, cos_nm, 0), n1 = __shfl_sync(kFull, cos_nm, 1);
+            const float n2 = __shfl_sync(kFull, cos_nm, 2), n3 = __shfl_sync(kFull, cos_nm, 3);
+            if (lane == 0) M[kCosMaxDim] = make_float4(n0, n1, n2, n3);
+          }
+        }
         __syncwarp();  // the whole warp's part of the slot is written
         if (lane == 0) {
           WsSlot d;
@@ -326,6 +375,7 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
           d.r = r;
           d.next = 0;
           d.pad = 0;
+          d.cos_r = COS ? r : -1;
           d.pad2 = 0;
           slots[s] = d;
           mbar_arrive(full0 + 8 * s);
@@ -351,6 +401,7 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
       d.r = 0;
       d.next = 0;
       d.pad = 0;
+      d.cos_r = -1;
       d.pad2 = 0;
       if (ok) {
         slots[s] = d;

@@ -584,8 +584,8 @@ def _cos_case(seed, n_docs=200, doc_dim=64, item_first=8, dim=50, n_chunks=3, n_
 def test_cosine_against_float64_and_a_numpy_float32_restatement(seed, dim, n_chunks, item_first, scale):
     docs, member, ci, co = _cos_case(seed, dim=dim, n_chunks=n_chunks, item_first=item_first, scale=scale)
     got = oracle.cosine_features(docs, member, ci, co, item_first, dim, n_chunks)
-    assert got.shape == (len(ci), 16)
-    vals = got.copy().view(np.float16).astype(np.float64)  # [C, 8]
+    assert got.shape == (len(ci), 32)
+    vals = got.copy().view(np.float16).astype(np.float64)  # [C, 16]
     assert not vals[:, n_chunks:].any()
     req_of = np.searchsorted(co, np.arange(len(ci)), side="right") - 1
     ok = (ci >= 0) & (ci < docs.shape[0])
@@ -639,7 +639,7 @@ def test_cosine_closed_forms():
     member[1] = 0                                      # a request with an all-zero member representation
     ci = np.array([0, 1, 2, 3, 4, -1, 6, 5], np.int32)
     co = np.array([0, 7, 8], np.int64)
-    v = oracle.cosine_features(docs, member, ci, co, first, dim, n_chunks).copy().view(np.float16).reshape(-1, 8)
+    v = oracle.cosine_features(docs, member, ci, co, first, dim, n_chunks).copy().view(np.float16).reshape(-1, 16)
     one, minus = np.float16(1.0), np.float16(-1.0)
     assert v[0, 0] == one and v[0, 2] == minus           # parallel / anti-parallel
     assert v[1, 0] == minus and v[1, 2] == one
