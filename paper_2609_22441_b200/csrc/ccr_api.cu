@@ -687,7 +687,7 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   const int cos_stage = cos ? 32 * (((s->cos_dim + 7) / 8) | 1) * 16 : 0;
   const int cos_bytes = cos ? ccr::ws_cos_bytes(n_str, cos_stage) : 0;
   auto smem_for = [&](int t, int cap) -> size_t {
-    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, cap, n_req <= ccr::kWsMaxCachedReq ? n_req : 0, cos_bytes).bytes)
+    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, cap, n_req <= ccr::kWsMaxCachedReq ? n_req : 0, cos_bytes, n_res).bytes)
                   : static_cast<size_t>(ccr::TileLayout(t, second, merge, cap).bytes);
   };
   // Keys staged per request.  The warp-specialised kernel runs one block per SM, so by default it stages

@@ -32,6 +32,8 @@ constexpr int kWsSlots = 8;        // ring depth
 constexpr int kWsMaxThreads = 512;
 constexpr int kWsMaxCachedReq = 1024;  // batches up to this many requests keep their offsets in shared memory
 constexpr int kMaxRounds = 4;      // most tiles per resolver warp a block draws at once
+constexpr int kWsWorkItems = 4 * 32 * 4;  // engager slots of one resolver batch: 4 candidates per lane x 4 slots
+constexpr int kWsWorkListBytes = kWsWorkItems * (8 + 2);  // ids (int64) + tags (uint16) per resolver warp
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -54,11 +56,12 @@ __host__ __device__ inline int ws_cos_bytes(int n_streamers, int stage_per_warp)
 }
 
 struct WsLayout {
-  int off_full, off_empty, off_slots, off_grab, off_offs, off_idx, off_pos, off_apos, off_cos, off_keys, bytes;
+  int off_full, off_empty, off_slots, off_grab, off_offs, off_idx, off_pos, off_apos, off_cos, off_wl, off_keys, bytes;
   // n_req_cached: requests whose offsets are mirrored in shared memory (0 = read them from global memory)
   // cos_bytes: shared memory of the derived cosine section (0 = off): a block of member-embedding floats per
   // ring slot, then one embedding staging block per streamer warp
-  __host__ __device__ WsLayout(int tile, bool second, int key_cap, int n_req_cached, int cos_bytes) {
+  // n_res: resolver warps (second-degree joins give each a work list of engager lookups)
+  __host__ __device__ WsLayout(int tile, bool second, int key_cap, int n_req_cached, int cos_bytes, int n_res) {
     off_full = kSmemHeader;                 // after the key-staging mbarrier
     off_empty = off_full + kWsSlots * 8;
     off_slots = off_empty + kWsSlots * 8;
@@ -69,7 +72,8 @@ struct WsLayout {
     off_pos = off_idx + kWsSlots * tile * 4;
     off_apos = off_pos + kWsSlots * tile * 4;
     off_cos = off_apos + (second ? kWsSlots * tile * 16 : 0);
-    off_keys = off_cos + cos_bytes;
+    off_wl = off_cos + cos_bytes;
+    off_keys = off_wl + (second ? n_res * kWsWorkListBytes : 0);
     bytes = off_keys + search_bytes(key_cap, true);
   }
 };
@@ -81,7 +85,8 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   unsigned char* smem = smem_ws;
   constexpr bool COS = CNP != 0;
   const int n_req_cached = a.n_req <= kWsMaxCachedReq ? a.n_req : 0;
-  const WsLayout lay(a.tile, SECOND, a.key_cap, n_req_cached, COS ? ws_cos_bytes(n_streamers, a.cos_stage) : 0);
+  const WsLayout lay(a.tile, SECOND, a.key_cap, n_req_cached, COS ? ws_cos_bytes(n_streamers, a.cos_stage) : 0,
+                     (static_cast<int>(blockDim.x) >> 5) - n_streamers);
   WsSlot* slots = reinterpret_cast<WsSlot*>(smem + lay.off_slots);
   int* grab = reinterpret_cast<int*>(smem + lay.off_grab);
   int* s_idx = reinterpret_cast<int*>(smem + lay.off_idx);
@@ -179,6 +184,9 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   bool dead = false;     // this warp's wait for a free slot expired: keep walking (barriers!), fill nothing
   int staged_r = -1;     // request whose keys are in shared memory
   StagedKeys keys;
+  // this warp's work list of engager lookups (second-degree joins)
+  [[maybe_unused]] int64_t* wl_id = reinterpret_cast<int64_t*>(smem + lay.off_wl + (SECOND ? rwarp * kWsWorkListBytes : 0));
+  [[maybe_unused]] uint16_t* wl_tag = reinterpret_cast<uint16_t*>(wl_id + kWsWorkItems);
   int cos_r = -1;        // request whose squared member norms lane k < kCosMaxChunks holds in cos_nm
   float cos_nm = 0.0f;
   const long long n_tiles = (a.total + a.tile - 1) / a.tile;
@@ -287,37 +295,72 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
             }
           }
           if constexpr (SECOND) {
-            // engager lookups, the slots of two candidates (8 ids) interleaved per batch
-            bool af[U][4];
-            int ap[U][4];
-#pragma unroll
-            for (int h = 0; h < U; h += 2) {
-              const int64_t id8[8] = {act[h][0], act[h][1], act[h][2], act[h][3],
-                                      act[h + 1][0], act[h + 1][1], act[h + 1][2], act[h + 1][3]};
-              bool f8[8];
-              int p8[8];
-              keys.find_batch<8, 2>(id8, f8, p8);
-#pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                af[h + (q >> 2)][q & 3] = f8[q];
-                ap[h + (q >> 2)][q & 3] = p8[q];
-              }
-            }
+            // Engager lookups.  Most slots are empty, and which ones differs from lane to lane, so looking up
+            // "slot s of candidate u" in lock step would spend most of the warp's instructions on empty
+            // slots.  The non-empty (candidate, slot) pairs of the batch are compacted into a work list in
+            // shared memory (lane-major, so workers read consecutive entries) and the lanes share them out,
+            // four interleaved lookups at a time; a hit writes its key index straight into the slot's
+            // position array, which the owner lane has preset to -1.
+            int* apos_i = reinterpret_cast<int*>(out_apos);
+            int mine = 0;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
               const int i = base + u * 32 + lane;
-              unsigned m = found[u] ? 1u : 0u;
+              if (i < n) out_apos[i] = make_int4(-1, -1, -1, -1);
+#pragma unroll
+              for (int sl = 0; sl < 4; ++sl) mine += act[u][sl] >= 0 ? 1 : 0;
+            }
+            int incl = mine;
+#pragma unroll
+            for (int dlt = 1; dlt < 32; dlt <<= 1) {
+              const int t = __shfl_up_sync(kFull, incl, dlt);
+              if (lane >= dlt) incl += t;
+            }
+            const int total = __shfl_sync(kFull, incl, 31);
+            int w = incl - mine;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
 #pragma unroll
               for (int sl = 0; sl < 4; ++sl) {
-                if (af[u][sl]) {
-                  m |= 1u << (1 + sl);
-                  m |= 1u << (5 + ((types[u] >> (8 * sl)) & 0xffu) % 3u);
-                } else {
-                  ap[u][sl] = -1;
+                if (act[u][sl] >= 0) {
+                  wl_id[w] = act[u][sl];
+                  wl_tag[w] = static_cast<uint16_t>(((base + u * 32 + lane) << 2) | sl);
+                  ++w;
                 }
               }
+            }
+            __syncwarp();
+            for (int w0 = 0; w0 < total; w0 += 4 * 32) {
+              int64_t id4[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const int wi = w0 + q * 32 + lane;
+                id4[q] = wi < total ? wl_id[wi] : -1;
+              }
+              bool f4[4];
+              int p4[4];
+              keys.find_batch<4>(id4, f4, p4);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const int wi = w0 + q * 32 + lane;
+                if (wi < total && f4[q]) apos_i[wl_tag[wi]] = p4[q];
+              }
+            }
+            __syncwarp();
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+              const int i = base + u * 32 + lane;
               if (i < n) {
-                out_apos[i] = make_int4(ap[u][0], ap[u][1], ap[u][2], ap[u][3]);
+                const int4 ap4 = out_apos[i];
+                const int ap[4] = {ap4.x, ap4.y, ap4.z, ap4.w};
+                unsigned m = found[u] ? 1u : 0u;
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) {
+                  if (ap[sl] >= 0) {
+                    m |= 1u << (1 + sl);
+                    m |= 1u << (5 + ((types[u] >> (8 * sl)) & 0xffu) % 3u);
+                  }
+                }
                 out_idx[i] = idx[u];
                 out_pos[i] = found[u] ? pos[u] : -1;
                 a.out_mask[out0 + i] = static_cast<uint8_t>(m);
