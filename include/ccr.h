@@ -364,7 +364,7 @@ typedef struct {
                                  unset = as many as fit (warp-specialised kernel) or 4096 (the others)       */
   int32_t ws_streamers;       /* warp-specialised kernel: row-streaming warps per block (1..14)              */
   int32_t ws_resolvers;       /* warp-specialised kernel: search warps per block (1..8); sum <= 16; set both
-                                 or neither (unset = 12 + 4, or 11 + 5 for second-degree joins)              */
+                                 or neither (unset = 12 + 4)              */
   int32_t blocks_per_sm;      /* two-phase kernel: cap on resident blocks per SM (1..8)                      */
 } ccr_tuning;
 ccr_status ccr_docstore_set_tuning(ccr_docstore* store, const ccr_tuning* tuning);

@@ -302,7 +302,7 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   s->req_b = static_cast<int>(req_b);
   s->tile = 0;  // automatic: kDefaultTileWs / kDefaultTileTwoPhase
   s->key_cap = 0;  // automatic
-  s->ws_streamers = 0;  // automatic: 12 + 4 (first-degree joins), 11 + 5 (second-degree joins)
+  s->ws_streamers = 0;  // automatic: 12 streamer + 4 resolver warps
   s->ws_resolvers = 0;
   if (cudaDeviceGetAttribute(&s->n_sms, cudaDevAttrMultiProcessorCount, d->device) != cudaSuccess || s->n_sms <= 0) {
     cudaGetLastError();
@@ -682,8 +682,8 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     if (!use_ws) return CCR_ERR_UNSUPPORTED;  // the derived section is computed by the warp-specialised kernel only
     if (reinterpret_cast<uintptr_t>(member_emb) & 1u) return CCR_ERR_INVALID_ARG;
   }
-  const int n_str = s->ws_streamers > 0 ? s->ws_streamers : (second ? 11 : 12);
-  const int n_res = s->ws_resolvers > 0 ? s->ws_resolvers : (second ? 5 : 4);
+  const int n_str = s->ws_streamers > 0 ? s->ws_streamers : 12;
+  const int n_res = s->ws_resolvers > 0 ? s->ws_resolvers : 4;
   const int cos_stage = cos ? 32 * (((s->cos_dim + 7) / 8) | 1) * 16 : 0;
   const int cos_bytes = cos ? ccr::ws_cos_bytes(n_str, cos_stage) : 0;
   auto smem_for = [&](int t, int cap) -> size_t {
@@ -779,7 +779,7 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     // up to kSchedRegions launches of one store may be in flight at once (on any streams)
     // Small launches (fewer tiles than two rounds per block) are split evenly instead: drawing whole rounds
     // from the counter would leave most SMs without work, and a single request is the latency-critical case.
-    const int n_res_auto = s->ws_resolvers > 0 ? s->ws_resolvers : (second ? 5 : 4);
+    const int n_res_auto = s->ws_resolvers > 0 ? s->ws_resolvers : 4;
     const long long n_tiles = (total_cands + a.tile - 1) / a.tile;
     const bool dynamic = !(flags & CCR_FLAG_STATIC_SPLIT) && n_tiles >= 2LL * blocks * n_res_auto;
     if (dynamic) a.sched = s->status + 4 + 2 * static_cast<int>(s->launches % kSchedRegions);
