@@ -177,7 +177,8 @@ ccr_status ccr_join_batch(const ccr_docstore* store,
  * idx_out[offsets_out[r] .. offsets_out[r+1]); offsets_out[0] = 0 and offsets_out[r+1] - offsets_out[r] = n_r.
  * The scatter index of kept candidate k of request r is therefore (r, k - offsets_out[r]).  src_out (optional,
  * int32[>= number of valid candidates]) receives the flat input index j of every kept candidate, so that
- * scores can be carried back to the caller's candidate order.  idx_out needs room for cand_offsets[n_req]
+ * scores can be carried back to the caller's candidate order (CCR_ERR_UNSUPPORTED when total_cands exceeds
+ * 2^31 - 1, the range of those indices).  idx_out needs room for cand_offsets[n_req]
  * entries (all candidates may be valid); idx_out / offsets_out must not alias the inputs.  All pointers are
  * DEVICE pointers; three small kernels on `stream`, nothing allocated, no synchronisation.  total_cands only
  * chooses how many blocks share a request (from the mean request length); the count pass uses one block per

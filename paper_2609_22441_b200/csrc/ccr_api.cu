@@ -205,6 +205,11 @@ const Variant kVariants[] = {
 };
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
 
+// The padded output layout on the two-phase kernels (CCR_FLAG_TWO_PHASE, merge path): generic widths only.
+const KernelFn kPaddedFirst = ccr::join_kernel<0, 0, 0, false, false, true>;
+const KernelFn kPaddedSecond = ccr::join_kernel<0, 0, 0, true, false, true>;
+const KernelFn kPaddedMerge = ccr::join_kernel<0, 0, 0, false, true, true>;
+
 const Variant& pick_variant(int doc_ch, int edge_ch, int req_ch) {
   for (int i = 0; i < kNumVariants - 1; ++i) {
     const Variant& v = kVariants[i];
@@ -215,7 +220,8 @@ const Variant& pick_variant(int doc_ch, int edge_ch, int req_ch) {
 
 ccr_status allow_large_smem() {
   for (int i = 0; i < kNumVariants; ++i) {
-    const KernelFn fns[3] = {kVariants[i].first, kVariants[i].second, kVariants[i].merge};
+    const KernelFn fns[6] = {kVariants[i].first, kVariants[i].second, kVariants[i].merge,
+                             kPaddedFirst,       kPaddedSecond,      kPaddedMerge};
     for (KernelFn f : fns) {
       if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemBytes) != cudaSuccess) {
         cudaGetLastError();
@@ -786,7 +792,8 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     fn<<<static_cast<unsigned>(blocks), (n_str + n_res) * 32, smem, st>>>(a, n_str);
   } else {
     // persistent two-phase kernel: as many blocks as stay resident, each with at least 256 candidates
-    const KernelFn fn = merge ? v.merge : (second ? v.second : v.first);
+    const KernelFn fn = n_max > 0 ? (merge ? kPaddedMerge : (second ? kPaddedSecond : kPaddedFirst))
+                                  : (merge ? v.merge : (second ? v.second : v.first));
     const int by_regs = ccr::kJoinMinBlocks;  // matches the kernel's __launch_bounds__
     int per_sm = static_cast<int>(kSmemPerSm / (smem + 1024));
     if (per_sm > by_regs) per_sm = by_regs;
@@ -894,6 +901,7 @@ ccr_status ccr_compact_valid(const ccr_docstore* cs, int32_t n_req, int64_t tota
   if (n_req < 0 || total_cands < 0) return CCR_ERR_INVALID_ARG;
   if (n_req == 0) return CCR_OK;
   if (!cand_offsets || !offsets_out || (total_cands > 0 && (!cand_idx || !idx_out))) return CCR_ERR_INVALID_ARG;
+  if (src_out != nullptr && total_cands > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;  // source indices are int32
   if (cand_idx == idx_out || static_cast<const void*>(cand_offsets) == static_cast<const void*>(offsets_out))
     return CCR_ERR_INVALID_ARG;  // not in place
   if ((reinterpret_cast<uintptr_t>(cand_idx) & 3u) || (reinterpret_cast<uintptr_t>(idx_out) & 3u) ||

@@ -334,7 +334,9 @@ constexpr int kUnroll = 8;  // candidates a thread keeps in flight in phase A
 #endif
 constexpr int kJoinMinBlocks = CCR_JOIN_MIN_BLOCKS;  // resident blocks per SM the register budget is set for
 
-template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, bool MERGE>
+// PADDED: rows go to slot r * n_max + (j - cand_offsets[r]) (JoinArgs::n_max > 0); a separate instantiation so
+// that the ragged kernels carry no register for it.
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, bool MERGE, bool PADDED = false>
 __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const JoinArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
   const TileLayout lay(a.tile, SECOND, MERGE, a.key_cap);
@@ -385,11 +387,11 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
     }
 
     // padded output: a request's candidates behind its n_max-th have no slot and are dropped
-    const long long r_first = __ldg(a.cand_offsets + r);
-    const long long seg_lim = a.n_max > 0 ? min(seg_end, r_first + a.n_max) : seg_end;
+    const long long r_first = PADDED ? __ldg(a.cand_offsets + r) : 0;
+    const long long seg_lim = PADDED ? min(seg_end, r_first + a.n_max) : seg_end;
     for (long long sub = seg; sub < seg_lim; sub += a.tile) {
       const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_lim - sub));
-      const long long out0 = a.n_max > 0 ? r * a.n_max + (sub - r_first) : sub;
+      const long long out0 = PADDED ? r * a.n_max + (sub - r_first) : sub;
 
       // ================= phase A: resolve every candidate of the sub-tile =================
       if (!MERGE) {
