@@ -362,7 +362,8 @@ typedef struct {
   int32_t tile_cands;         /* candidates per ring slot / search-copy phase pair: multiple of 256, <= 4096;
                                  unset = 256 (warp-specialised kernel) / 1024 (two-phase kernel)               */
   int32_t key_capacity;       /* most keys (or sampled keys) a block stages in shared memory per request;
-                                 unset = as many as fit (warp-specialised kernel) or 4096 (the others)       */
+                                 unset = whole lists up to a 160 KB shared-memory budget per block
+                                 (warp-specialised kernel) or 4096 (the others)                              */
   int32_t ws_streamers;       /* warp-specialised kernel: row-streaming warps per block (1..14)              */
   int32_t ws_resolvers;       /* warp-specialised kernel: search warps per block (1..8); sum <= 16; set both
                                  or neither (unset = 12 + 4)              */

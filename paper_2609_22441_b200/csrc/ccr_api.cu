@@ -29,6 +29,7 @@ constexpr int kDefaultTileWs = 256;        // candidates per ring slot of the wa
 constexpr int kDefaultTileTwoPhase = 1024; // candidates per search/copy phase pair of the two-phase kernel
 constexpr int kSmemPerSm = 228 * 1024;
 constexpr int kDefaultKeyCap = 4096;
+constexpr int kAutoSmemBudget = 160 * 1024;  // shared memory the warp-specialised kernel takes by default
 constexpr int kMaxTile = 4096;
 constexpr size_t kStageBytes = 16u << 20;  // staging block of second-degree stores (ids uploaded from the host)
 constexpr int kSchedRegions = 64;                    // launches of one store that may be in flight at once
@@ -697,8 +698,8 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
                   : static_cast<size_t>(ccr::TileLayout(t, second, merge, cap).bytes);
   };
   // Keys staged per request.  The warp-specialised kernel runs one block per SM, so by default it stages
-  // as many keys as fit next to its ring (whole lists of up to ~20,000 ids); the kernels that keep several
-  // blocks per SM default to kDefaultKeyCap.  A configured key_capacity overrides both.
+  // whole lists up to a shared-memory budget (about 13,000 ids for a first-degree join); the kernels that keep
+  // several blocks per SM default to kDefaultKeyCap.  A configured key_capacity overrides both.
   const int tile_cfg = s->tile > 0 ? s->tile : (use_ws ? kDefaultTileWs : kDefaultTileTwoPhase);
   int tile = tile_cfg;
   int key_cap;
@@ -710,13 +711,13 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     const long long cap = s->key_cap > 0 ? s->key_cap : kDefaultKeyCap;
     key_cap = static_cast<int>(max_edge_len < cap ? max_edge_len : cap);
   } else {
+    // Whole lists are staged as long as the block's shared memory stays within kAutoSmemBudget.  What the
+    // block takes from the SM's 228 KB is taken from the L1 that the streamers' loads pass through: the
+    // production-scale join (lists up to 20,000 keys) ran a third slower with every list staged (~205 KB per
+    // block) than with 100-150 KB, while 140 KB with every list staged beats sampling for second-degree joins.  Longer lists get a sampled top of the tree instead.
     key_cap = static_cast<int>(max_edge_len);
-    // shrink the ring first; if the longest list still does not fit, stage a sampled top of the tree
-    while (tile > 256 && smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) tile -= 256;
-    if (smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) {
-      tile = tile_cfg;
-      key_cap = kDefaultKeyCap;
-    }
+    while (key_cap > kDefaultKeyCap && smem_for(tile, key_cap) > static_cast<size_t>(kAutoSmemBudget))
+      key_cap = std::max(kDefaultKeyCap, key_cap - 1024);
   }
   // sub-tile size: the configured one, shrunk (in steps of 256) until the kernel's arrays fit next to the keys
   while (tile > 256 && smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) tile -= 256;
