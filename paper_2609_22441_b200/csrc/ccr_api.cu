@@ -715,9 +715,13 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     // block takes from the SM's 228 KB is taken from the L1 that the streamers' loads pass through: the
     // production-scale join (lists up to 20,000 keys) ran a third slower with every list staged (~205 KB per
     // block) than with 100-150 KB, while 140 KB with every list staged beats sampling for second-degree joins.  Longer lists get a sampled top of the tree instead.
+    // A launch of a few tiles per block (a single request: the latency case) is bound by the searches, not by
+    // streaming, and keeps every list staged that fits (55.9 us against 70.3 us for 100,000 candidates x 20,000 keys).
     key_cap = static_cast<int>(max_edge_len);
-    while (key_cap > kDefaultKeyCap && smem_for(tile, key_cap) > static_cast<size_t>(kAutoSmemBudget))
-      key_cap = std::max(kDefaultKeyCap, key_cap - 1024);
+    const long long tiles = (total_cands + tile - 1) / tile;
+    const bool streaming_bound = tiles >= 2LL * s->n_sms * n_res;
+    const size_t budget = streaming_bound ? static_cast<size_t>(kAutoSmemBudget) : static_cast<size_t>(kMaxSmemBytes);
+    while (key_cap > kDefaultKeyCap && smem_for(tile, key_cap) > budget) key_cap = std::max(kDefaultKeyCap, key_cap - 1024);
   }
   // sub-tile size: the configured one, shrunk (in steps of 256) until the kernel's arrays fit next to the keys
   while (tile > 256 && smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) tile -= 256;
