@@ -59,6 +59,7 @@ def parse_args():
     p.add_argument("--c3-requests", type=int, default=256, help="requests of configs 3/3b/3s (smaller for profiler captures)")
     p.add_argument("--e2e-steps", type=int, default=0, help="0 = min(steps, 10)")
     p.add_argument("--flags", type=int, default=0, help="extra CCR_FLAG_* bits (experiments)")
+    p.add_argument("--drop-flags", type=int, default=0, help="CCR_FLAG_* bits of the configuration to clear (experiments)")
     p.add_argument("--tile", type=int, default=0, help="candidates per ring slot (0 = library default)")
     p.add_argument("--key-cap", type=int, default=0, help="keys staged per request (0 = library default)")
     p.add_argument("--streamers", type=int, default=0)
@@ -87,7 +88,7 @@ def make_workload(config: str, rank: int, c3_docs: int = 50_000_000, c3_requests
                    extra_pools=160 if c3_docs >= 50_000_000 else 0)
     if config == "3":
         return wl, B.CCR_FLAG_FIRST_DEGREE_ONLY
-    if config == "3b":
+    if config == "3b":  # sorted candidates: default kernel; add --flags 128 for the merge-path kernel
         return W.sort_candidates_by_author(wl), B.CCR_FLAG_FIRST_DEGREE_ONLY | B.CCR_FLAG_CANDS_SORTED
     return wl, 0
 
@@ -657,7 +658,7 @@ def main():
         store.set_tuning(tile_cands=args.tile, key_capacity=args.key_cap, ws_streamers=args.streamers,
                          ws_resolvers=args.resolvers)
     db = B.DeviceBatch(b, device=local_rank)
-    flags = args.flags | cfg_flags
+    flags = (args.flags | cfg_flags) & ~args.drop_flags
     member = None
     if args.cosine:
         store.set_cosine(8, 50, 3)

@@ -66,7 +66,9 @@ enum {
                                            (CCR_ERR_UNSUPPORTED if max_edge_len does not fit)       */
   CCR_FLAG_FORCE_GLOBAL      = 1u << 1, /* never stage keys: search them in global memory / L2      */
   CCR_FLAG_CANDS_SORTED      = 1u << 2, /* caller promises that, inside each request, the candidates'
-                                           author ids are non-decreasing: use the merge-path kernel  */
+                                           author ids are non-decreasing.  Together with CCR_FLAG_TWO_PHASE
+                                           this selects the merge-path kernel; the default kernel does not
+                                           need the promise (sorted candidates still help its locality)    */
   CCR_FLAG_VALIDATE          = 1u << 3, /* check offsets, key order (and candidate order) on the
                                            device first; synchronises the stream                     */
   CCR_FLAG_FIRST_DEGREE_ONLY = 1u << 4, /* ignore engager slots of a second-degree store: no edge2
@@ -240,7 +242,7 @@ ccr_status ccr_docstore_set_cosine(ccr_docstore* store, const ccr_cosine_spec* s
  * CCR_FLAG_COSINE: DEVICE float16 [n_req, n_chunks * dim], chunk k of request r at
  * member_emb[(r * n_chunks + k) * dim], 2-byte aligned; ignored without the flag.  struct_bytes must be
  * sizeof(ccr_join_io).  The derived section is computed by the warp-specialised kernel only: with
- * CCR_FLAG_TWO_PHASE or a first-degree CCR_FLAG_CANDS_SORTED the call returns CCR_ERR_UNSUPPORTED.        */
+ * CCR_FLAG_TWO_PHASE the call returns CCR_ERR_UNSUPPORTED.                                                 */
 typedef struct {
   uint32_t       struct_bytes;
   int32_t        n_req;

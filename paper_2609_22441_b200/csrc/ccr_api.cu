@@ -678,7 +678,9 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   const bool second = s->desc.max_actors > 0 && !(flags & CCR_FLAG_FIRST_DEGREE_ONLY);
   // engager ids are not sorted, so the merge path serves first-degree joins only; a second-degree join
   // on sorted candidates takes the binary-search kernel (same result by definition)
-  const bool merge = (flags & CCR_FLAG_CANDS_SORTED) && !second;
+  // (and only when the two-phase kernel is asked for: the warp-specialised kernel is the faster one on sorted
+  // candidates too — 212 against 262 us on the batched configuration, 1631 against 1780 us at production scale)
+  const bool merge = (flags & CCR_FLAG_CANDS_SORTED) && (flags & CCR_FLAG_TWO_PHASE) && !second;
 
   // which kernel: the merge path and CCR_FLAG_TWO_PHASE take the two-phase kernel, everything else the
   // warp-specialised kernel

@@ -172,7 +172,7 @@ def test_argument_errors(B):
         assert L.ccr_docstore_set_cosine(store.handle, spec(8, 50, 3, 0)) == B.CCR_OK
         assert ex(B.CCR_FLAG_COSINE, member_emb=None) == B.CCR_ERR_INVALID_ARG
         assert ex(B.CCR_FLAG_COSINE | B.CCR_FLAG_TWO_PHASE) == B.CCR_ERR_UNSUPPORTED
-        assert ex(B.CCR_FLAG_COSINE | B.CCR_FLAG_CANDS_SORTED) == B.CCR_ERR_UNSUPPORTED
+        assert ex(B.CCR_FLAG_COSINE | B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE) == B.CCR_ERR_UNSUPPORTED
         assert ex(B.CCR_FLAG_COSINE, struct_bytes=8) == B.CCR_ERR_INVALID_ARG
         assert ex(B.CCR_FLAG_COSINE) == B.CCR_OK
         assert ex(0) == B.CCR_OK                                                    # same entry without the section

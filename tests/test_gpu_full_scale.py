@@ -104,11 +104,14 @@ def test_config3_first_degree_headline(env):
 def test_config3_merge_path_on_sorted_candidates(env):
     B, wl, store, kept, full, J = env
     ws = W.sort_candidates_by_author(wl)
-    flags = B.CCR_FLAG_FIRST_DEGREE_ONLY | B.CCR_FLAG_CANDS_SORTED
+    flags = B.CCR_FLAG_FIRST_DEGREE_ONLY | B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE  # the merge-path kernel
     rows, mask, db = _run(B, store, ws, flags)
     member = _membership(ws, ws.batch.cand_idx)
     m = _check_full(ws, full, rows, mask, ws.batch.cand_idx, member)
-    # sorted input through the binary-search kernel must give the same bytes as the merge path
+    # sorted input through the default kernel (with and without the promise) must give the same bytes as the merge path
+    rows2, mask2, _ = _run(B, store, ws, B.CCR_FLAG_FIRST_DEGREE_ONLY | B.CCR_FLAG_CANDS_SORTED)
+    assert torch.equal(rows2, rows) and torch.equal(mask2, mask)
+    del rows2, mask2
     rows2, mask2, _ = _run(B, store, ws, B.CCR_FLAG_FIRST_DEGREE_ONLY)
     assert torch.equal(rows2, rows) and torch.equal(mask2, mask)
     # the kept rows cover the same docs; sample the sorted list at the positions of those docs

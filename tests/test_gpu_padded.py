@@ -158,7 +158,7 @@ def test_ragged_multi_tile_batch(B):
 def test_sorted_candidates_take_the_merge_path(B):
     """Compaction keeps the input order, so candidates sorted by author id stay sorted."""
     wl = W.sort_candidates_by_author(W.config1(n_docs=50_000, n_req=5, n_cand=4_000))
-    _check(B, wl, [("merge", B.CCR_FLAG_CANDS_SORTED)])
+    _check(B, wl, [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)])
 
 
 def test_second_degree_scaled(B):

@@ -66,14 +66,14 @@ def _check(B, wl, flag_sets, first_degree_only=False, tunings=((0, 0),)):
 def test_config0_single_tiny_request_all_search_paths(B):
     wl = W.config0()
     _check(B, wl, _variants(B))
-    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)])
 
 
 def test_config1_batched_first_degree_full_size(B):
     wl = W.config1()
     assert wl.batch.total_cands == 64 * 30_000 and wl.out_row_bytes() == 384
     _check(B, wl, _variants(B), tunings=((0, 0), (512, 0, 1, 1, 1), (2048, 0, 14, 2, 3), (768, 0, 5, 8, 2), (256, 0, 3, 1, 0)))
-    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)])
 
 
 def test_config2a_second_degree_on_config0_shape(B):
@@ -84,7 +84,7 @@ def test_config2a_second_degree_on_config0_shape(B):
     _check(B, wl, [("auto", 0)], first_degree_only=True)
     ws = W.sort_candidates_by_author(wl)
     _check(B, ws, [("sorted-second", B.CCR_FLAG_CANDS_SORTED)])
-    _check(B, ws, [("merge", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=True)
+    _check(B, ws, [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=True)
 
 
 def test_config2b_second_degree_on_config1_shape_full_size(B):
@@ -100,7 +100,7 @@ def test_config3_scaled_store_long_edge_lists(B):
     wl = W.config3(n_docs=2_000_000, n_req=12, n_cand=20_000, gen_doc_feats=True, extra_pools=0)
     assert wl.batch.max_edge_len > 4096
     _check(B, wl, _variants(B), first_degree_only=True, tunings=((0, 0), (512, 1000), (2048, 20_000), (256, 7)))
-    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=True,
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=True,
            tunings=((0, 0), (256, 64)))
     _check(B, wl, [("auto", 0)])
 
@@ -114,7 +114,7 @@ def test_tiny_random_batches(B, seed):
     _check(B, wl, _variants(B), tunings=((256, 0), (0, 0)))
     if second:
         _check(B, wl, [("auto", 0)], first_degree_only=True)
-    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=second,
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)], first_degree_only=second,
            tunings=((256, 3),))
 
 
@@ -174,7 +174,7 @@ def test_edge_list_lengths_around_every_path_threshold(B, k):
     wl = _manual([keys1, keys2], cand, authors, edge_dim=8)
     fits_smem = k <= 20_000
     _check(B, wl, _variants(B, include_smem=fits_smem))
-    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)])
     if not fits_smem:
         store = B.store_from_workload(wl)
         db = B.DeviceBatch(wl.batch)
@@ -189,7 +189,7 @@ def test_many_small_requests_in_one_launch(B):
     wl = tiny_workload(7, n_docs=3000, alphabet=900, n_req=700, kmax=300, nmax=40, second=False, req_dim=4,
                        doc_dim=64, edge_dim=32)
     _check(B, wl, _variants(B))
-    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED)])
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)])
 
 
 def test_batch_equals_single_request_launches(B):
