@@ -30,7 +30,7 @@ constexpr int kDefaultTileTwoPhase = 1024; // candidates per search/copy phase p
 constexpr int kSmemPerSm = 228 * 1024;
 constexpr int kDefaultKeyCap = 4096;
 constexpr int kAutoSmemBudget = 160 * 1024;  // shared memory the warp-specialised kernel takes by default
-constexpr int kMaxTile = 4096;
+constexpr int kMaxTile = ccr::kMaxTileCands;
 constexpr size_t kStageBytes = 16u << 20;  // staging block of second-degree stores (ids uploaded from the host)
 constexpr int kSchedRegions = 64;                    // launches of one store that may be in flight at once
 constexpr int kStatusInts = 4 + 2 * kSchedRegions;   // [0] wait expiry, [1] validation code, [4..] scheduling words

@@ -32,6 +32,7 @@ constexpr int kWsSlots = 8;        // ring depth
 constexpr int kWsMaxThreads = 512;
 constexpr int kWsMaxCachedReq = 1024;  // batches up to this many requests keep their offsets in shared memory
 constexpr int kMaxRounds = 4;      // most tiles per resolver warp a block draws at once
+constexpr int kMaxTileCands = 4096;  // largest sub-tile the host accepts
 constexpr int kWsWorkItems = 4 * 32 * 4;  // engager slots of one resolver batch: 4 candidates per lane x 4 slots
 constexpr int kWsWorkListBytes = kWsWorkItems * (8 + 2);  // ids (int64) + tags (uint16) per resolver warp
 
@@ -191,6 +192,8 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   float cos_nm = 0.0f;
   const long long n_tiles = (a.total + a.tile - 1) / a.tile;
   constexpr int U = SECOND ? 4 : 8;  // candidates a lane keeps in flight
+  static_assert(!SECOND || U * 32 * 4 == kWsWorkItems, "the work list holds every engager slot of one batch");
+  static_assert(kMaxTileCands * 4 <= 65536, "work-list tags are 16 bits: candidate index in the tile x 4 + slot");
 
   for (bool more = true; more && !failed;) {
     long long j0, j1;

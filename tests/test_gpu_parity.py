@@ -90,7 +90,9 @@ def test_config2a_second_degree_on_config0_shape(B):
 def test_config2b_second_degree_on_config1_shape_full_size(B):
     wl = W.config1(second_degree=True)
     assert wl.out_row_bytes() == 448
-    _check(B, wl, [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL)])
+    # large sub-tiles and other warp splits: the engager work lists address candidates by their index in the sub-tile
+    _check(B, wl, [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL)],
+           tunings=((0, 0), (4096, 0, 12, 4, 0), (2048, 0, 8, 8, 0), (768, 0, 14, 1, 0)))
 
 
 def test_config3_scaled_store_long_edge_lists(B):
