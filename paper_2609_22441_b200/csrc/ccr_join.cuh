@@ -179,29 +179,35 @@ template <int NP, bool TUNED>
 __device__ __forceinline__ uint4 cosine_section(const JoinArgs& a, const uint4* xrow, const float4* cosM) {
   const int pieces = TUNED ? NP : (a.cos_dim + 7) >> 3;
   float nx = 0.0f, d[kCosMaxChunks] = {0.0f, 0.0f, 0.0f, 0.0f};
-  auto element = [&](float x, int e) {
-    const float4 m = cosM[e];
-    nx = fmaf(x, x, nx);
-    d[0] = fmaf(x, m.x, d[0]);
-    d[1] = fmaf(x, m.y, d[1]);
-    d[2] = fmaf(x, m.z, d[2]);
-    d[3] = fmaf(x, m.w, d[3]);
-  };
   uint4 xq[NP];  // the whole embedding is requested before the first element is used
 #pragma unroll
   for (int q = 0; q < NP; ++q) xq[q] = q < pieces ? xrow[q] : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
   for (int q = 0; q < NP; ++q) {
     if (q >= pieces) break;  // warp-uniform
-    const uint4 xv = xq[q];
-    const unsigned w[4] = {xv.x, xv.y, xv.z, xv.w};
-    const bool whole = TUNED && q < NP - 1;  // every element of the piece belongs to the embedding
+    // the eight medoid operands of the piece are requested together: one shared-memory latency per piece
+    // instead of one per element in front of each group of dependent FMAs
+    float4 m[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) m[t] = cosM[q * 8 + t];
+    const unsigned w[4] = {xq[q].x, xq[q].y, xq[q].z, xq[q].w};
+    float x[8];
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
       const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[t]));
-      const int e = q * 8 + t * 2;
-      if (whole || e < a.cos_dim) element(f.x, e);
-      if (whole || e + 1 < a.cos_dim) element(f.y, e + 1);
+      x[2 * t] = f.x;
+      x[2 * t + 1] = f.y;
+    }
+    const bool whole = TUNED && q < NP - 1;  // every element of the piece belongs to the embedding
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      if (whole || q * 8 + t < a.cos_dim) {
+        nx = fmaf(x[t], x[t], nx);
+        d[0] = fmaf(x[t], m[t].x, d[0]);
+        d[1] = fmaf(x[t], m[t].y, d[1]);
+        d[2] = fmaf(x[t], m[t].z, d[2]);
+        d[3] = fmaf(x[t], m[t].w, d[3]);
+      }
     }
   }
   const float4 nm4 = cosM[kCosMaxDim];
