@@ -633,6 +633,7 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   a.smem_keys = static_cast<int>(max_edge_len < ccr::kSortSmemMaxKeys ? max_edge_len : ccr::kSortSmemMaxKeys);
   a.smem_keys = (a.smem_keys + 1) & ~1;  // keeps the index array 8-byte aligned behind the keys
   const size_t smem = static_cast<size_t>(a.smem_keys) * 12;
+  a.smem_words = static_cast<int>(smem / 8);  // packed key|index words fit half as many bytes again
   ccr::sort_edges_kernel<<<static_cast<unsigned>(n_req), ccr::kSortThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
   s->launches++;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;

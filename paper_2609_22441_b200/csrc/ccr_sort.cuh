@@ -4,8 +4,9 @@
 // One 1024-thread block per request.  Keys and record indices are sorted together in shared memory with a
 // bitonic network written for arbitrary n (flip + disperse steps, every compare-exchange ascending, partners
 // beyond n skipped — equivalent to padding with +infinity); the order is on (key, index), which makes the
-// result the stable sort.  Lists that do not fit shared memory are sorted by the same network directly on the
-// output arrays in global memory (L2).  The rows then follow their keys in 16-byte chunks.
+// result the stable sort.  Keys that leave room for the index in the same 64-bit word (the usual case) take 8
+// bytes per record, so lists of up to ~29,000 records are sorted in shared memory; other keys take 12 bytes
+// (~19,000 records).  Longer lists are sorted by the same network directly on the output arrays in global memory (L2).  The rows then follow their keys in 16-byte chunks.
 #pragma once
 
 #include "ccr_device.cuh"
@@ -85,7 +86,8 @@ struct SortArgs {
   int64_t* keys_out;
   uint8_t* feats_out;
   int* perm_out;         // may be null when every list fits shared memory
-  int smem_keys;         // records the dynamic shared memory can hold
+  int smem_keys;         // (key, index) records the dynamic shared memory can hold: 12 bytes each
+  int smem_words;        // packed key|index words it can hold: 8 bytes each
 };
 
 __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortArgs a) {
@@ -95,12 +97,9 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
   const long long Kl = __ldg(a.edge_offsets + r + 1) - e0;
   if (Kl <= 0) return;
   const int K = static_cast<int>(Kl);
-  const bool in_smem = K <= a.smem_keys;
-  if (!in_smem && a.perm_out == nullptr) return;  // refused on the host; never reached
-  long long* keys = in_smem ? reinterpret_cast<long long*>(smem_sort) : reinterpret_cast<long long*>(a.keys_out + e0);
-  int* idx = in_smem ? reinterpret_cast<int*>(smem_sort + static_cast<size_t>(a.smem_keys) * 8) : a.perm_out + e0;
   // keys that leave room for the record index in one 64-bit word (non-negative, below 2^(63 - index bits)) are
-  // sorted as single words: key << shift | index orders like (key, index)
+  // sorted as single words: key << shift | index orders like (key, index), needs 8 bytes per record and no
+  // index array at all (the word's low bits are the index)
   int idx_bits = 1;
   while ((1 << idx_bits) < K) ++idx_bits;
   long long kmax = 0;
@@ -111,7 +110,34 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
     negative |= (k < 0);
   }
   const bool packable = __syncthreads_or(negative || (kmax >> (63 - idx_bits)) != 0) == 0;
-  if (packable) {
+  const long long chunks = static_cast<long long>(K) * a.row_ch;
+  const uint4* src = reinterpret_cast<const uint4*>(a.feats_in) + e0 * a.row_ch;
+  uint4* dst = reinterpret_cast<uint4*>(a.feats_out) + e0 * a.row_ch;
+
+  if (packable && K <= a.smem_words) {
+    unsigned long long* w = reinterpret_cast<unsigned long long*>(smem_sort);
+    for (int i = threadIdx.x; i < K; i += blockDim.x)
+      w[i] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
+    __syncthreads();
+    sort_words_bitonic(w, K);
+    const unsigned long long low = (1ull << idx_bits) - 1;
+    for (int i = threadIdx.x; i < K; i += blockDim.x) {
+      const unsigned long long v = w[i];
+      a.keys_out[e0 + i] = static_cast<long long>(v >> idx_bits);
+      if (a.perm_out) a.perm_out[e0 + i] = static_cast<int>(v & low);
+    }
+    for (long long c = threadIdx.x; c < chunks; c += blockDim.x) {  // rows follow their keys
+      const int row = static_cast<int>(c / a.row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * a.row_ch);
+      dst[c] = __ldg(src + static_cast<long long>(w[row] & low) * a.row_ch + piece);
+    }
+    return;
+  }
+
+  const bool in_smem = K <= a.smem_keys;
+  if (!in_smem && a.perm_out == nullptr) return;  // refused on the host; never reached
+  long long* keys = in_smem ? reinterpret_cast<long long*>(smem_sort) : reinterpret_cast<long long*>(a.keys_out + e0);
+  int* idx = in_smem ? reinterpret_cast<int*>(smem_sort + static_cast<size_t>(a.smem_keys) * 8) : a.perm_out + e0;
+  if (packable) {  // only reached by lists too long for shared memory: the words live in the key output array
     unsigned long long* w = reinterpret_cast<unsigned long long*>(keys);
     for (int i = threadIdx.x; i < K; i += blockDim.x)
       w[i] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
@@ -138,11 +164,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
       if (a.perm_out) a.perm_out[e0 + i] = idx[i];
     }
   }
-  // rows follow their keys
-  const long long chunks = static_cast<long long>(K) * a.row_ch;
-  const uint4* src = reinterpret_cast<const uint4*>(a.feats_in) + e0 * a.row_ch;
-  uint4* dst = reinterpret_cast<uint4*>(a.feats_out) + e0 * a.row_ch;
-  for (long long c = threadIdx.x; c < chunks; c += blockDim.x) {
+  for (long long c = threadIdx.x; c < chunks; c += blockDim.x) {  // rows follow their keys
     const int row = static_cast<int>(c / a.row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * a.row_ch);
     dst[c] = __ldg(src + static_cast<long long>(idx[row]) * a.row_ch + piece);
   }
