@@ -52,12 +52,85 @@ __device__ __forceinline__ void sort_pairs_bitonic(long long* keys, int* idx, in
   }
 }
 
-// The same network on single 64-bit words (key << shift | index): half the shared-memory traffic.
+// M consecutive disperse steps of the network (partner distances 2^b, 2^(b-1), ..., 2^(b-M+1)) in one pass:
+// the 2^M elements whose indices differ only in those M bits form a closed group, so a thread loads the group,
+// runs the M rounds of compare-exchanges in registers and stores it — one barrier and one trip through shared
+// memory instead of M.  Elements at or beyond n count as +infinity (every real word is below 2^63).
+template <int M>
+__device__ __forceinline__ void disperse_fused(unsigned long long* w, int n, int b) {
+  const int sh = b - M + 1;
+  for (int g = threadIdx.x;; g += blockDim.x) {
+    const int base = ((g >> sh) << (b + 1)) | (g & ((1 << sh) - 1));
+    if (base >= n) break;  // base grows with g
+    unsigned long long v[1 << M];
+#pragma unroll
+    for (int m = 0; m < (1 << M); ++m) {
+      const int i = base + (m << sh);
+      v[m] = i < n ? w[i] : ~0ull;
+    }
+#pragma unroll
+    for (int s = M - 1; s >= 0; --s) {
+#pragma unroll
+      for (int m = 0; m < (1 << M); ++m) {
+        if ((m & (1 << s)) == 0) {
+          const int p = m | (1 << s);
+          const unsigned long long lo = min(v[m], v[p]), hi = max(v[m], v[p]);
+          v[m] = lo;
+          v[p] = hi;
+        }
+      }
+    }
+#pragma unroll
+    for (int m = 0; m < (1 << M); ++m) {
+      const int i = base + (m << sh);
+      if (i < n) w[i] = v[m];
+    }
+  }
+  __syncthreads();
+}
+
+// Every step whose partner distance is below 32 stays inside 32 consecutive elements, so a warp holding one
+// element per lane runs those steps with shuffles: no shared-memory traffic, no bank conflicts, no barriers.
+// FIRST: the whole network up to blocks of 32 (flip and disperse steps of k = 2 .. 32); otherwise the last five
+// disperse steps (distances 16 .. 1) of a larger block.  The lane with the lower index keeps the minimum.
+template <bool FIRST>
+__device__ __forceinline__ void warp_steps(unsigned long long* w, int n) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  for (int c = warp; c * 32 < n; c += n_warps) {
+    const int i = c * 32 + lane;
+    unsigned long long v = i < n ? w[i] : ~0ull;
+    if (FIRST) {
+#pragma unroll
+      for (int L = 1; L <= 5; ++L) {
+        const unsigned long long pf = __shfl_xor_sync(0xffffffffu, v, (1 << L) - 1);  // flip: mirror inside the block
+        v = (lane & (1 << (L - 1))) == 0 ? min(v, pf) : max(v, pf);
+#pragma unroll
+        for (int d = (1 << L) >> 2; d >= 1; d >>= 1) {
+          const unsigned long long pv = __shfl_xor_sync(0xffffffffu, v, d);
+          v = (lane & d) == 0 ? min(v, pv) : max(v, pv);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) {
+        const unsigned long long pv = __shfl_xor_sync(0xffffffffu, v, d);
+        v = (lane & d) == 0 ? min(v, pv) : max(v, pv);
+      }
+    }
+    if (i < n) w[i] = v;
+  }
+  __syncthreads();
+}
+
+// The same network on single 64-bit words (key << shift | index): half the shared-memory traffic; steps at
+// distances below 32 run in registers (warp_steps), the others are fused up to three at a time
+// (disperse_fused, always at strides of 32 words or more, which keeps them free of bank conflicts).
 __device__ __forceinline__ void sort_words_bitonic(unsigned long long* w, int n) {
   if (n < 2) return;
-  for (int k = 2;; k <<= 1) {
-    for (int j = k - 1;;) {
-      const int top = 31 - __clz(j);
+  warp_steps<true>(w, n);  // blocks of 32 are sorted
+  for (int k = 64, log_k = 6; (k >> 1) < n; k <<= 1, ++log_k) {
+    {  // flip: i pairs with its mirror inside the block of k
+      const int j = k - 1, top = log_k - 1;
       for (int p = threadIdx.x;; p += blockDim.x) {
         const int i = pair_low_index(p, top), l = i ^ j;
         if (i >= n) break;  // i grows with p
@@ -70,10 +143,39 @@ __device__ __forceinline__ void sort_words_bitonic(unsigned long long* w, int n)
         }
       }
       __syncthreads();
-      if (j == k - 1) j = k >> 2; else j >>= 1;
-      if (j == 0) break;
     }
-    if (k >= n) break;
+    // disperse at distances k/4 ... 32 in shared memory, 16 ... 1 in registers
+    for (int b = log_k - 2; b >= 5;) {
+      const int m = b - 4 >= 3 ? 3 : b - 4;
+      if (m == 3) disperse_fused<3>(w, n, b);
+      else if (m == 2) disperse_fused<2>(w, n, b);
+      else disperse_fused<1>(w, n, b);
+      b -= m;
+    }
+    warp_steps<false>(w, n);
+  }
+}
+
+// Rows follow their keys: output chunk c (16 bytes) comes from row source_of(c / row_ch) of the input.  One block
+// moves a whole list, so every thread keeps kSortGatherUnroll loads in flight.
+constexpr int kSortGatherUnroll = 8;
+template <typename SourceOf>
+__device__ __forceinline__ void gather_rows(const uint4* src, uint4* dst, long long chunks, int row_ch, SourceOf source_of) {
+  for (long long c0 = threadIdx.x; c0 < chunks; c0 += static_cast<long long>(blockDim.x) * kSortGatherUnroll) {
+    uint4 v[kSortGatherUnroll];
+#pragma unroll
+    for (int u = 0; u < kSortGatherUnroll; ++u) {
+      const long long c = c0 + static_cast<long long>(u) * blockDim.x;
+      if (c < chunks) {
+        const int row = static_cast<int>(c / row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * row_ch);
+        v[u] = __ldg(src + source_of(row) * row_ch + piece);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kSortGatherUnroll; ++u) {
+      const long long c = c0 + static_cast<long long>(u) * blockDim.x;
+      if (c < chunks) dst[c] = v[u];
+    }
   }
 }
 
@@ -126,10 +228,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
       a.keys_out[e0 + i] = static_cast<long long>(v >> idx_bits);
       if (a.perm_out) a.perm_out[e0 + i] = static_cast<int>(v & low);
     }
-    for (long long c = threadIdx.x; c < chunks; c += blockDim.x) {  // rows follow their keys
-      const int row = static_cast<int>(c / a.row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * a.row_ch);
-      dst[c] = __ldg(src + static_cast<long long>(w[row] & low) * a.row_ch + piece);
-    }
+    gather_rows(src, dst, chunks, a.row_ch, [&](int row) { return static_cast<long long>(w[row] & low); });
     return;
   }
 
@@ -164,10 +263,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
       if (a.perm_out) a.perm_out[e0 + i] = idx[i];
     }
   }
-  for (long long c = threadIdx.x; c < chunks; c += blockDim.x) {  // rows follow their keys
-    const int row = static_cast<int>(c / a.row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * a.row_ch);
-    dst[c] = __ldg(src + static_cast<long long>(idx[row]) * a.row_ch + piece);
-  }
+  gather_rows(src, dst, chunks, a.row_ch, [&](int row) { return static_cast<long long>(idx[row]); });
 }
 
 }  // namespace ccr
