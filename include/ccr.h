@@ -264,9 +264,15 @@ ccr_status ccr_join_batch_ex(const ccr_docstore* store, const ccr_join_io* io, u
  * records [edge_offsets[r], edge_offsets[r+1]) — key int64 + feature row of the store's edge width — are put
  * in ascending key order (records with equal keys keep their input order) into keys_out / feats_out, which
  * use the same offsets and must not alias the inputs.  perm_out (optional, int32[E]) receives for every
- * output record the index of its source record inside the request; it is required when max_edge_len exceeds
- * 19,000, because longer lists are sorted in place in keys_out / perm_out instead of in shared memory.
- * All pointers DEVICE; one kernel on `stream` (one 1024-thread block per request), no allocation, no sync.
+ * output record the index of its source record inside the request.  Without perm_out every list is sorted by
+ * one 1024-thread block in shared memory (one kernel); lists of more than 19,000 records then have no place to
+ * be sorted in and the call returns CCR_ERR_INVALID_ARG.  With perm_out, and max_edge_len above 4,096, lists
+ * whose keys leave room for the record index in one 64-bit word (non-negative, below 2^(63 - index bits): every
+ * realistic id) are sorted in chunks of 4,096 records by one block each and merged by grid-wide passes of the
+ * same sorting network over the key output array, so that a single long list is spread over many SMs instead
+ * of one (a batch whose long lists would keep the SMs busy one list each stays on the one-block path), and the
+ * rows of all lists are moved by one grid-wide gather: up to ~14 small kernels on `stream`.
+ * All pointers DEVICE; no allocation, no synchronisation.
  * The output is what ccr_join_batch expects as edge_keys / edge_feats.                                    */
 ccr_status ccr_sort_edges(const ccr_docstore* store, int32_t n_req, int64_t max_edge_len,
                           const int64_t* edge_keys_in, const void* edge_feats_in, const int64_t* edge_offsets,

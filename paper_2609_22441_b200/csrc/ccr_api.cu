@@ -634,8 +634,41 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   a.smem_keys = (a.smem_keys + 1) & ~1;  // keeps the index array 8-byte aligned behind the keys
   const size_t smem = static_cast<size_t>(a.smem_keys) * 12;
   a.smem_words = static_cast<int>(smem / 8);  // packed key|index words fit half as many bytes again
-  ccr::sort_edges_kernel<<<static_cast<unsigned>(n_req), ccr::kSortThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // Lists longer than one chunk are spread over many blocks when the caller provides perm_out (the row gather
+  // of that path reads the source indices from it).
+  a.multi = (perm_out != nullptr && max_edge_len > ccr::kSortChunk) ? 1 : 0;
+  if (a.multi) {
+    const unsigned n_chunks = static_cast<unsigned>((max_edge_len + ccr::kSortChunk - 1) / ccr::kSortChunk);
+    const long long pairs_per_block = static_cast<long long>(ccr::kSortThreads) * ccr::kSortPairsPerThread;
+    // pair number p maps to a lower partner i >= p, so p < max_edge_len covers every pair (in the flip of the
+    // largest block most partners lie beyond the list, which is why half as many would not do)
+    const unsigned pair_blocks = static_cast<unsigned>((n_chunks * static_cast<long long>(ccr::kSortChunk) + pairs_per_block - 1) / pairs_per_block);
+    const dim3 per_chunk(static_cast<unsigned>(n_req), n_chunks), per_pairs(static_cast<unsigned>(n_req), pair_blocks);
+    ccr::sort_chunks_kernel<<<per_chunk, ccr::kSortThreads, 0, st>>>(a);
+    s->launches++;
+    for (long long k = 2LL * ccr::kSortChunk; (k >> 1) < max_edge_len; k <<= 1) {
+      ccr::sort_global_step_kernel<<<per_pairs, ccr::kSortThreads, 0, st>>>(a, static_cast<int>(k), static_cast<int>(k - 1));
+      s->launches++;
+      for (long long d = k >> 2; d >= ccr::kSortChunk; d >>= 1) {
+        ccr::sort_global_step_kernel<<<per_pairs, ccr::kSortThreads, 0, st>>>(a, static_cast<int>(k), static_cast<int>(d));
+        s->launches++;
+      }
+      ccr::sort_chunk_finish_kernel<<<per_chunk, ccr::kSortThreads, 0, st>>>(a, static_cast<int>(k));
+      s->launches++;
+    }
+    ccr::sort_unpack_kernel<<<per_chunk, ccr::kSortThreads, 0, st>>>(a);
+    s->launches++;
+  }
+  // short or unpackable lists (all lists without perm_out): one block per list
+  ccr::sort_edges_kernel<<<static_cast<unsigned>(n_req), ccr::kSortThreads, smem, st>>>(a);
   s->launches++;
+  if (a.multi) {
+    const long long per_block = static_cast<long long>(ccr::kSortThreads) * ccr::kSortGatherUnroll;
+    const unsigned row_blocks = static_cast<unsigned>((max_edge_len * a.row_ch + per_block - 1) / per_block);
+    ccr::gather_all_kernel<<<dim3(static_cast<unsigned>(n_req), row_blocks), ccr::kSortThreads, 0, st>>>(a);
+    s->launches++;
+  }
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
   return CCR_OK;
 }

@@ -190,7 +190,33 @@ struct SortArgs {
   int* perm_out;         // may be null when every list fits shared memory
   int smem_keys;         // (key, index) records the dynamic shared memory can hold: 12 bytes each
   int smem_words;        // packed key|index words it can hold: 8 bytes each
+  int multi;             // 1: packable lists longer than kSortChunk are sorted by the multi-block kernels, and the
+                         //    rows of every list are moved by gather_all_kernel (perm_out is then required)
 };
+
+constexpr int kSortChunkLog = 12;
+constexpr int kSortChunk = 1 << kSortChunkLog;  // records one block of the multi-block path sorts in shared memory
+constexpr int kSortMultiBalance = 64;  // long lists are spread over blocks while their total length is at most this many times the longest
+constexpr int kSortMultiFlag = 0x5a17ed01;      // "this list is on the multi-block path", kept in the list's first output row
+
+__device__ __forceinline__ int sort_index_bits(int K) {
+  int idx_bits = 1;
+  while ((1 << idx_bits) < K) ++idx_bits;
+  return idx_bits;
+}
+
+// Block-wide: do the K keys leave room for the record index in one 64-bit word (non-negative, below
+// 2^(63 - idx_bits))?  All threads of the block must call.
+__device__ __forceinline__ bool list_is_packable(const int64_t* keys, int K, int idx_bits) {
+  long long kmax = 0;
+  int negative = 0;
+  for (int i = threadIdx.x; i < K; i += blockDim.x) {
+    const long long k = __ldg(keys + i);
+    kmax = max(kmax, k);
+    negative |= (k < 0);
+  }
+  return __syncthreads_or(negative || (kmax >> (63 - idx_bits)) != 0) == 0;
+}
 
 __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortArgs a) {
   extern __shared__ __align__(16) unsigned char smem_sort[];
@@ -202,17 +228,11 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
   // keys that leave room for the record index in one 64-bit word (non-negative, below 2^(63 - index bits)) are
   // sorted as single words: key << shift | index orders like (key, index), needs 8 bytes per record and no
   // index array at all (the word's low bits are the index)
-  int idx_bits = 1;
-  while ((1 << idx_bits) < K) ++idx_bits;
-  long long kmax = 0;
-  int negative = 0;
-  for (int i = threadIdx.x; i < K; i += blockDim.x) {
-    const long long k = __ldg(a.keys_in + e0 + i);
-    kmax = max(kmax, k);
-    negative |= (k < 0);
-  }
-  const bool packable = __syncthreads_or(negative || (kmax >> (63 - idx_bits)) != 0) == 0;
-  const long long chunks = static_cast<long long>(K) * a.row_ch;
+  if (a.multi && *reinterpret_cast<const volatile int*>(a.feats_out + e0 * a.row_ch * 16) == kSortMultiFlag)
+    return;  // the chunked kernels have sorted this list
+  const int idx_bits = sort_index_bits(K);
+  const bool packable = list_is_packable(a.keys_in + e0, K, idx_bits);
+  const long long chunks = a.multi ? 0 : static_cast<long long>(K) * a.row_ch;  // multi: rows move in gather_all_kernel
   const uint4* src = reinterpret_cast<const uint4*>(a.feats_in) + e0 * a.row_ch;
   uint4* dst = reinterpret_cast<uint4*>(a.feats_out) + e0 * a.row_ch;
 
@@ -264,6 +284,165 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
     }
   }
   gather_rows(src, dst, chunks, a.row_ch, [&](int row) { return static_cast<long long>(idx[row]); });
+}
+
+
+// ---------------------------------------------------------------------------------------------------
+// Multi-block path for long lists.  One block per list leaves a 19,000-record list to a single SM (264 us,
+// instruction-bound) while the others idle.  Here the same network runs over the packed words in global
+// memory (the key output array): chunks of kSortChunk records are sorted in shared memory by one block each;
+// then, for every larger block size k, the steps whose partner distance reaches across chunks (the flip, and
+// disperse steps at distances >= kSortChunk) run as grid-wide passes, one launch each, and the remaining steps
+// of the phase run per chunk in shared memory again.  A flag in the list's first output row (written by the
+// chunk kernel, overwritten by the final row gather) tells the later kernels that the list is packable.
+
+__device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, long long& e0, int& K) {
+  e0 = __ldg(a.edge_offsets + r);
+  const long long Kl = __ldg(a.edge_offsets + r + 1) - e0;
+  K = Kl > 0 ? static_cast<int>(Kl) : 0;
+  if (K == 0) return false;
+  return *reinterpret_cast<const volatile int*>(a.feats_out + e0 * a.row_ch * 16) == kSortMultiFlag;
+}
+
+// grid (n_req, chunks of the longest list): sort chunk blockIdx.y of list blockIdx.x
+__global__ void __launch_bounds__(kSortThreads, 1) sort_chunks_kernel(const SortArgs a) {
+  __shared__ unsigned long long w[kSortChunk];
+  const int r = blockIdx.x;
+  const long long e0 = __ldg(a.edge_offsets + r);
+  const long long Kl = __ldg(a.edge_offsets + r + 1) - e0;
+  const int K = Kl > 0x7fffffffLL ? 0x7fffffff : static_cast<int>(Kl);
+  const int c0 = blockIdx.y * kSortChunk;
+  if (c0 >= K) return;  // also K <= 0
+  const int idx_bits = sort_index_bits(K);
+  bool take = list_is_packable(a.keys_in + e0, K, idx_bits);
+  if (K > kSortChunk) {
+    // Spreading a long list over many blocks costs more SM time than sorting it in one block, so it pays only
+    // while the batch's long lists would not keep the SMs busy one list each.
+    // every block sizes up the batch's long lists for itself (the same numbers in all of them): their total
+    // length against the longest one — one block per list takes about 14 ns per record of the longest list,
+    // the chunked path about 0.2 ns per record of all long lists (measured)
+    __shared__ unsigned long long sum_long_s;
+    __shared__ int max_long_s;
+    if (threadIdx.x == 0) {
+      sum_long_s = 0;
+      max_long_s = 0;
+    }
+    __syncthreads();
+    unsigned long long sum = 0;
+    int longest = 0;
+    for (int q = threadIdx.x; q < a.n_req; q += blockDim.x) {
+      const long long len = __ldg(a.edge_offsets + q + 1) - __ldg(a.edge_offsets + q);
+      if (len > kSortChunk) {
+        sum += static_cast<unsigned long long>(len);
+        longest = max(longest, static_cast<int>(min(len, 0x7fffffffLL)));
+      }
+    }
+    if (sum) {
+      atomicAdd(&sum_long_s, sum);
+      atomicMax(&max_long_s, longest);
+    }
+    __syncthreads();
+    take = take && sum_long_s <= static_cast<unsigned long long>(kSortMultiBalance) * max_long_s;
+  }
+  if (blockIdx.y == 0 && threadIdx.x == 0)
+    *reinterpret_cast<int*>(a.feats_out + e0 * a.row_ch * 16) = take ? kSortMultiFlag : 0;
+  if (!take) return;
+  const int n = min(kSortChunk, K - c0);
+  for (int t = threadIdx.x; t < n; t += blockDim.x)
+    w[t] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + c0 + t)) << idx_bits) | static_cast<unsigned>(c0 + t);
+  __syncthreads();
+  sort_words_bitonic(w, n);
+  unsigned long long* W = reinterpret_cast<unsigned long long*>(a.keys_out + e0);
+  for (int t = threadIdx.x; t < n; t += blockDim.x) W[c0 + t] = w[t];
+}
+
+// grid (n_req, pair blocks): one step of the network across chunks — partner mask j = k - 1 (flip) or a
+// power of two >= kSortChunk (disperse) — for the lists that have a block of size k to sort.
+constexpr int kSortPairsPerThread = 4;
+__global__ void __launch_bounds__(kSortThreads) sort_global_step_kernel(const SortArgs a, int k, int j) {
+  long long e0;
+  int K;
+  if (!list_on_multi_path(a, blockIdx.x, e0, K) || (k >> 1) >= K) return;
+  unsigned long long* W = reinterpret_cast<unsigned long long*>(a.keys_out + e0);
+  const int top = 31 - __clz(j);
+#pragma unroll
+  for (int u = 0; u < kSortPairsPerThread; ++u) {
+    const int p = (blockIdx.y * kSortPairsPerThread + u) * kSortThreads + threadIdx.x;
+    const int i = pair_low_index(p, top), l = i ^ j;
+    if (i < K && l < K) {
+      const unsigned long long wi = W[i], wl = W[l];
+      if (wi > wl) {
+        W[i] = wl;
+        W[l] = wi;
+      }
+    }
+  }
+}
+
+// grid (n_req, chunks): the disperse steps at distances kSortChunk / 2 ... 1 of phase k, per chunk in shared memory
+__global__ void __launch_bounds__(kSortThreads, 1) sort_chunk_finish_kernel(const SortArgs a, int k) {
+  __shared__ unsigned long long w[kSortChunk];
+  long long e0;
+  int K;
+  const int c0 = blockIdx.y * kSortChunk;
+  if (!list_on_multi_path(a, blockIdx.x, e0, K) || (k >> 1) >= K || c0 >= K) return;
+  unsigned long long* W = reinterpret_cast<unsigned long long*>(a.keys_out + e0);
+  const int n = min(kSortChunk, K - c0);
+  for (int t = threadIdx.x; t < n; t += blockDim.x) w[t] = W[c0 + t];
+  __syncthreads();
+  for (int b = kSortChunkLog - 1; b >= 5;) {
+    const int m = b - 4 >= 3 ? 3 : b - 4;
+    if (m == 3) disperse_fused<3>(w, n, b);
+    else if (m == 2) disperse_fused<2>(w, n, b);
+    else disperse_fused<1>(w, n, b);
+    b -= m;
+  }
+  warp_steps<false>(w, n);
+  for (int t = threadIdx.x; t < n; t += blockDim.x) W[c0 + t] = w[t];
+}
+
+// grid (n_req, chunks): words -> keys (in place) and source indices
+__global__ void __launch_bounds__(kSortThreads) sort_unpack_kernel(const SortArgs a) {
+  long long e0;
+  int K;
+  const int c0 = blockIdx.y * kSortChunk;
+  if (!list_on_multi_path(a, blockIdx.x, e0, K) || c0 >= K) return;
+  const int idx_bits = sort_index_bits(K);
+  const unsigned long long low = (1ull << idx_bits) - 1;
+  const int n = min(kSortChunk, K - c0);
+  for (int t = threadIdx.x; t < n; t += blockDim.x) {
+    const unsigned long long v = reinterpret_cast<const unsigned long long*>(a.keys_out + e0)[c0 + t];
+    a.keys_out[e0 + c0 + t] = static_cast<long long>(v >> idx_bits);
+    a.perm_out[e0 + c0 + t] = static_cast<int>(v & low);
+  }
+}
+
+// grid (n_req, row blocks): rows follow their keys, for every list of the batch, kSortGatherUnroll 16-byte chunks
+// per thread in flight
+__global__ void __launch_bounds__(kSortThreads) gather_all_kernel(const SortArgs a) {
+  const int r = blockIdx.x;
+  const long long e0 = __ldg(a.edge_offsets + r);
+  const long long K = __ldg(a.edge_offsets + r + 1) - e0;
+  const long long chunks = K * a.row_ch;
+  const long long first = static_cast<long long>(blockIdx.y) * kSortThreads * kSortGatherUnroll;
+  if (first >= chunks) return;
+  const uint4* src = reinterpret_cast<const uint4*>(a.feats_in) + e0 * a.row_ch;
+  uint4* dst = reinterpret_cast<uint4*>(a.feats_out) + e0 * a.row_ch;
+  const int* perm = a.perm_out + e0;
+  uint4 v[kSortGatherUnroll];
+#pragma unroll
+  for (int u = 0; u < kSortGatherUnroll; ++u) {
+    const long long c = first + static_cast<long long>(u) * kSortThreads + threadIdx.x;
+    if (c < chunks) {
+      const int row = static_cast<int>(c / a.row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * a.row_ch);
+      v[u] = __ldg(src + static_cast<long long>(__ldg(perm + row)) * a.row_ch + piece);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < kSortGatherUnroll; ++u) {
+    const long long c = first + static_cast<long long>(u) * kSortThreads + threadIdx.x;
+    if (c < chunks) dst[c] = v[u];
+  }
 }
 
 }  // namespace ccr
