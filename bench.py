@@ -547,7 +547,7 @@ def sort_bench(args, B, device: int):
                    "peak_kind": "of " + peak_kind},
         "roofline": {"bound": "hbm", "achieved": head["algorithmic_gbs"], "peak": peak, "unit": "GB/s",
                      "frac": head["frac_of_hbm_peak"], "traffic": None,
-                     "note": "latency-bound: one block per request, the longest list sets the launch time"},
+                     "note": "bound by the sorting network of the longest lists (instruction issue), not by HBM"},
         "payloads": results, "gpu_launches": max(args.steps // 20, 20),
     }))
 

@@ -112,3 +112,39 @@ def test_sort_with_keys_that_cannot_share_a_word_with_the_index(B):
     assert np.array_equal(k.cpu().numpy(), want_k) and np.array_equal(p.cpu().numpy(), want_p)
     assert np.array_equal(f.cpu().numpy().view(np.uint16), want_f.view(np.uint16))
     store.free()
+
+
+@pytest.mark.parametrize("case", ["few_long", "many_long", "mixed_unpackable", "powers_of_two"])
+def test_sort_chunked_path_and_its_policy(B, case):
+    """With perm_out, lists longer than 4,096 records are sorted in chunks by many blocks and merged by grid-wide
+    passes — unless the batch's long lists add up to more than 64 times the longest, or a list's keys cannot
+    share a word with the index; those stay on the one-block path inside the same launch sequence."""
+    rng = np.random.default_rng({"few_long": 1, "many_long": 2, "mixed_unpackable": 3, "powers_of_two": 4}[case])
+    imax = np.iinfo(np.int64).max
+    if case == "few_long":
+        lens = [4097, 9000, 20_000, 3, 0, 12_288, 4096, 16_385]
+        keyf = [lambda n: rng.integers(0, 50 * max(n, 1), size=n)] * len(lens)
+    elif case == "many_long":
+        lens = [5000] * 70 + [100, 8191]
+        keyf = [lambda n: rng.integers(0, 1 << 30, size=n)] * len(lens)
+    elif case == "mixed_unpackable":
+        lens = [6000, 10_000, 5000, 7000, 50]
+        keyf = [lambda n: rng.integers(0, 1 << 40, size=n), lambda n: imax - rng.integers(0, 1 << 20, size=n),
+                lambda n: rng.integers(-1000, 1000, size=n), lambda n: rng.integers(0, 1000, size=n),  # many ties
+                lambda n: rng.integers(0, 1 << 40, size=n)]
+    else:
+        lens = [8192, 16_384, 32_768, 8193, 16_383]
+        keyf = [lambda n: rng.integers(0, 1 << 45, size=n)] * len(lens)
+    keys = np.concatenate([f(n) for f, n in zip(keyf, lens)] + [np.empty(0, np.int64)]).astype(np.int64)
+    feats = rng.standard_normal((len(keys), 64)).astype(np.float16)
+    eo = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    want_k, want_f, want_p = oracle.sort_edges(keys, feats, eo)
+    wl = W.config3(n_docs=1000, n_req=1, n_cand=10, gen_doc_feats=True, extra_pools=0)
+    store = B.store_from_workload(wl)
+    try:
+        for _ in range(2):  # twice: the flag left in the output rows by the first call must not confuse the second
+            k, f, p = _gpu_sort(B, store, keys, feats, eo)
+            assert np.array_equal(k.cpu().numpy(), want_k) and np.array_equal(p.cpu().numpy(), want_p)
+            assert np.array_equal(f.cpu().numpy().view(np.uint16), want_f.view(np.uint16))
+    finally:
+        store.free()
