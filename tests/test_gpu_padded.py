@@ -155,6 +155,12 @@ def test_ragged_multi_tile_batch(B):
     _check(B, wl, _kernels(B), n_max_list=(None, 6_000, 1_000), tunings=((0, 0), (512, 0, 5, 3, 2)))
 
 
+def test_many_small_requests(B):
+    """1500 requests (more than the kernels mirror in shared memory, several rounds of the offset scan)."""
+    wl = _with_unresolved(W.config1(n_docs=30_000, n_req=1500, n_cand=150, edge_lo=3, edge_hi=80), 0.2, 4)
+    _check(B, wl, [("ws", 0), ("2phase", B.CCR_FLAG_TWO_PHASE)], n_max_list=(None, 40))
+
+
 def test_sorted_candidates_take_the_merge_path(B):
     """Compaction keeps the input order, so candidates sorted by author id stay sorted."""
     wl = W.sort_candidates_by_author(W.config1(n_docs=50_000, n_req=5, n_cand=4_000))

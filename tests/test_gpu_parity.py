@@ -107,6 +107,16 @@ def test_config3_scaled_store_long_edge_lists(B):
     _check(B, wl, [("auto", 0)])
 
 
+def test_more_requests_than_the_kernel_mirrors_in_shared_memory(B):
+    """Batches of up to 1024 requests keep their offsets in shared memory; larger ones read them from global
+    memory.  1500 small requests, first and second degree, every kernel."""
+    for second in (False, True):
+        wl = W.config1(n_docs=30_000, n_req=1500, n_cand=150, second_degree=second, edge_lo=3, edge_hi=80)
+        assert wl.batch.n_req == 1500
+        _check(B, wl, [("auto", 0), ("static", B.CCR_FLAG_STATIC_SPLIT), ("2phase", B.CCR_FLAG_TWO_PHASE),
+                       ("global", B.CCR_FLAG_FORCE_GLOBAL)])
+
+
 # ------------------------------------------------------------------ ragged / degenerate inputs
 @pytest.mark.parametrize("seed", range(12))
 def test_tiny_random_batches(B, seed):
