@@ -15,6 +15,11 @@ request features).  Rank 0 prints ONE JSON line:
 With N > 1 (torchrun, one rank per GPU) every rank joins its own batch against its own replica of the
 store: the path has no exchange step, so there is no collective in the data path (weak scaling).
 `--impl reference` times the CPU oracle alone on a bounded sample of the same workload.
+
+Other workloads (`--config`): 2b second-degree; 3 / 3b / 3s production scale; 4 single-request latency sweep; and
+the steps around the join — sort (Algorithm 1 step 1), resolve (Eq. 6), ingest (Section 6.2 scatter, alone and
+beside the join), flow (ids -> positions -> compaction -> sort -> padded join with the cosine section, chained).
+`--padded` and `--cosine` time the padded layout and the derived cosine section on the chosen workload.
 """
 from __future__ import annotations
 
@@ -50,7 +55,7 @@ def parse_args():
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--config", default="1", choices=["1", "2b", "3", "3b", "3s", "4", "sort", "resolve", "ingest", "flow"],
                    help="1 batched first-degree (default, the headline); 2b second-degree on the same shape; 3 production-scale "
-                        "store, first-degree; 3b the same on candidates sorted by author (merge path); 3s production scale, "
+                        "store, first-degree; 3b the same on candidates sorted by author (add --flags 128 for the merge-path kernel); 3s production scale, "
                         "second-degree; 4 single-request latency sweep on the production-scale store; sort: Algorithm 1 step 1 "
                         "(per-request sort of unsorted affinity records) on the payloads of configs 1 and 3; resolve: document id -> "
                         "position over a 300M-id index (Eq. 6), batches of 1, 8 and 64 requests of 30,000 ids")
