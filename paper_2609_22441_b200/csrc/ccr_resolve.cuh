@@ -6,9 +6,9 @@
 // Here the sorted array gets a static search tree of sampled levels, fan-out 32: level l+1 holds the last
 // key of every full block of 32 keys of level l.  The top level (<= 16,384 keys) is staged in shared
 // memory; below it a query touches one 256-byte window (two cache lines) per level, inside which a lane
-// finishes its 5-step search: the ~2 MB level stays in L2, the larger ones come from HBM.  A query over 300M
-// ids walks 3 windows instead of 29 dependent probes across the whole array; four queries per lane are in
-// flight at once.
+// needs two dependent rounds of loads (octant, then position): the ~2 MB level stays in L2, the larger ones come
+// from HBM.  A query over 300M ids makes 6 dependent rounds instead of 29 dependent probes across the whole
+// array; eight queries per lane are in flight at once.
 #pragma once
 
 #include "ccr_device.cuh"
@@ -20,6 +20,11 @@ constexpr int kResolveMaxLevels = 8;
 constexpr int kResolveTopMax = 16384;              // keys of the top level (128 KB of shared memory)
 constexpr int kResolveThreads = 256;
 constexpr int kResolveUnroll = 8;                 // queries a lane keeps in flight
+#ifndef CCR_RESOLVE_ROUND2
+#define CCR_RESOLVE_ROUND2 2
+#endif
+constexpr int kResolveRound2 = CCR_RESOLVE_ROUND2;  // queries of a lane whose octants are in flight together
+constexpr long long kResolveInf = 0x7fffffffffffffffLL;  // stands for the keys beyond the end of a level
 
 struct ResolveArgs {
   const int64_t* level[kResolveMaxLevels];         // level[0] = the sorted ids, level[n_levels-1] = top
@@ -66,34 +71,49 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
     for (int l = top_l - 1; l >= 0; --l) {
       const int64_t* lev = a.level[l];
       const long long n = a.count[l];
-      // the searches of the lane's queries advance in lock step, one probe of each per step, so that their
-      // memory accesses are independent and in flight together (a window has at most 32 keys: 5 halvings + 1)
+      // Inside the 32-key window a query needs two dependent rounds instead of a six-probe binary search:
+      // round 1 reads the last key of the first three octants (three independent loads; the fourth octant's last
+      // key is not below q by construction of the level above) and picks the octant, round 2 reads the octant's
+      // eight keys as four 16-byte loads and counts the ones below q.  Keys beyond the end of the level count as
+      // +infinity.  All queries of the lane do round 1 together; round 2 runs for kResolveRound2 of them at a time, which
+      // keeps the keys in flight within the register budget.
       long long lo[kResolveUnroll];
-      int w[kResolveUnroll];
+      int64_t r1[kResolveUnroll][3];
 #pragma unroll
       for (int u = 0; u < kResolveUnroll; ++u) {
         lo[u] = c[u] << kResolveFanLog2;
-        const long long rest = n - lo[u];
-        w[u] = rest < (1 << kResolveFanLog2) ? static_cast<int>(rest > 0 ? rest : 0) : (1 << kResolveFanLog2);
-      }
 #pragma unroll
-      for (int step = 0; step < kResolveFanLog2; ++step) {
-        int64_t probe[kResolveUnroll];
-#pragma unroll
-        for (int u = 0; u < kResolveUnroll; ++u) probe[u] = w[u] > 1 ? __ldg(lev + lo[u] + (w[u] >> 1) - 1) : 0;
-#pragma unroll
-        for (int u = 0; u < kResolveUnroll; ++u) {
-          if (w[u] > 1) {
-            const int half = w[u] >> 1;
-            if (probe[u] < q[u]) lo[u] += half;
-            w[u] -= half;
-          }
+        for (int o = 0; o < 3; ++o) {
+          const long long i = lo[u] + 8 * o + 7;
+          r1[u][o] = i < n ? __ldg(lev + i) : kResolveInf;
         }
       }
 #pragma unroll
-      for (int u = 0; u < kResolveUnroll; ++u) {
-        if (w[u] == 1 && __ldg(lev + lo[u]) < q[u]) ++lo[u];
-        c[u] = lo[u];
+      for (int u = 0; u < kResolveUnroll; ++u)
+        lo[u] += 8 * ((r1[u][0] < q[u] ? 1 : 0) + (r1[u][1] < q[u] ? 1 : 0) + (r1[u][2] < q[u] ? 1 : 0));
+#pragma unroll
+      for (int h = 0; h < kResolveUnroll; h += kResolveRound2) {
+        longlong2 r2[kResolveRound2][4];
+#pragma unroll
+        for (int v = 0; v < kResolveRound2; ++v) {
+#pragma unroll
+          for (int p = 0; p < 4; ++p) {
+            const long long i = lo[h + v] + 2 * p;  // even, and the level's base is 16-byte aligned
+            if (i + 1 < n) {
+              r2[v][p] = __ldg(reinterpret_cast<const longlong2*>(lev + i));
+            } else {
+              r2[v][p].x = i < n ? __ldg(lev + i) : kResolveInf;
+              r2[v][p].y = kResolveInf;
+            }
+          }
+        }
+#pragma unroll
+        for (int v = 0; v < kResolveRound2; ++v) {
+          int below = 0;
+#pragma unroll
+          for (int p = 0; p < 4; ++p) below += (r2[v][p].x < q[h + v] ? 1 : 0) + (r2[v][p].y < q[h + v] ? 1 : 0);
+          c[h + v] = lo[h + v] + below;
+        }
       }
     }
 #pragma unroll
