@@ -92,7 +92,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 
 // 1-D bulk copy global -> this block's shared memory through the TMA engine; completion is signalled
 // on `bar` as `bytes` of transaction count.  Both addresses 16-B aligned, bytes a multiple of 16.
-// No multicast: one block, one destination.
+// The copy has a single destination: the issuing block.
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
