@@ -872,6 +872,19 @@ def main():
     barrier()
     e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
     e2e_value = total_cands_job / (e2e_ms * 1e-3)
+    # the serving case: the rows stay on the device for the ranking model, only the mask travels back
+    def e2e_step_rows_on_device():
+        B.ccr_join_batch_host(store, ws, b.n_req, C, b.max_edge_len, len(b.edge_keys), *h_in, None, h_mask, flags_plain)
+
+    for _ in range(0 if args.timed_only else 3):
+        e2e_step_rows_on_device()
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step_rows_on_device()
+    ev1.record()
+    barrier()
+    e2e_dev_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_steps
     mask_host = h_mask.numpy().copy()
     ws.free()
 
@@ -930,6 +943,8 @@ def main():
                          "logical_gbs": bc["logical"] / launch_s / 1e9},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "e2e_rows_stay_on_device": {"value": total_cands_job / (e2e_dev_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                                        "d2h_bytes_per_step": int(h_mask.numel()), "ms_per_step": e2e_dev_ms, "steps": e2e_steps},
             "gpu_launches": int(launches),
             "latency_ms": {"what": "one request (%d candidates) per launch, CUDA events" % (C // max(b.n_req, 1)),
                            "p50": pct(lat, 0.50), "p99": pct(lat, 0.99), "n": len(lat)},

@@ -299,11 +299,16 @@ ccr_status ccr_resolve_ids(const ccr_idindex* index, int64_t n_queries, const in
 ccr_status ccr_workspace_create(const ccr_docstore* store, int32_t max_req, int64_t max_cands,
                                 int64_t max_edges, ccr_workspace** out);
 ccr_status ccr_workspace_free(ccr_workspace* ws);
+/* DEVICE pointers of the workspace's output buffers: rows [max_cands, out_row_bytes], mask [max_cands]. */
+ccr_status ccr_workspace_outputs(const ccr_workspace* ws, void** rows, uint8_t** mask);
 
 /* The same join with HOST buffers (the request payload of Section 6.1.3 arrives in host memory):
  * copies the inputs to the workspace, runs ccr_join_batch, copies rows and mask back — all enqueued
  * on `stream`, nothing synchronised.  Pinned host memory makes the copies asynchronous.
- * total_edges = edge_offsets[n_req].  Sizes beyond the workspace give CCR_ERR_INVALID_ARG.          */
+ * total_edges = edge_offsets[n_req].  Sizes beyond the workspace give CCR_ERR_INVALID_ARG.
+ * out_rows may be NULL: the rows then stay in the workspace's device buffer, where the ranking model reads them
+ * (ccr_workspace_outputs gives the DEVICE pointers; valid until the next call on this workspace), and only the
+ * mask travels back — the serving case, in which the rows never leave the GPU.                      */
 ccr_status ccr_join_batch_host(const ccr_docstore* store, ccr_workspace* ws,
                                int32_t n_req, int64_t total_cands, int64_t max_edge_len,
                                int64_t total_edges,

@@ -41,7 +41,7 @@ CCR_FLAG_COSINE = 1 << 8
 EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_upsert", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
     "ccr_compact_valid", "ccr_join_batch_padded", "ccr_join_batch_ex", "ccr_docstore_set_cosine",
-    "ccr_workspace_create", "ccr_workspace_free", "ccr_join_batch_host", "ccr_docstore_device_status",
+    "ccr_workspace_create", "ccr_workspace_free", "ccr_workspace_outputs", "ccr_join_batch_host", "ccr_docstore_device_status",
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
     "ccr_static_payload_capacity", "ccr_join_payload_static", "ccr_docstore_selftest_wait",
     "ccr_sort_edges", "ccr_idindex_create", "ccr_idindex_free", "ccr_resolve_ids",
@@ -122,6 +122,8 @@ def lib() -> ctypes.CDLL:
     L.ccr_compact_valid.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, vp]
     L.ccr_join_batch_padded.restype = ctypes.c_int
     L.ccr_join_batch_padded.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
+    L.ccr_workspace_outputs.restype = ctypes.c_int
+    L.ccr_workspace_outputs.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
     L.ccr_join_batch_host.restype = ctypes.c_int
     L.ccr_join_batch_host.argtypes = [vp, vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
     L.ccr_static_payload_capacity.restype = ctypes.c_size_t
@@ -383,6 +385,12 @@ class Workspace:
     @property
     def handle(self):
         return self._h
+
+    def outputs(self):
+        """ccr_workspace_outputs: device addresses (rows, mask) of the workspace's output buffers."""
+        rows, mask = ctypes.c_void_p(), ctypes.c_void_p()
+        _check(lib().ccr_workspace_outputs(self._h, ctypes.byref(rows), ctypes.byref(mask)), "ccr_workspace_outputs")
+        return rows.value, mask.value
 
     def free(self) -> None:
         if self._h:

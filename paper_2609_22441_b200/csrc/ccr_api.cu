@@ -1028,6 +1028,13 @@ ccr_status ccr_workspace_free(ccr_workspace* w) {
   return CCR_OK;
 }
 
+ccr_status ccr_workspace_outputs(const ccr_workspace* w, void** rows, uint8_t** mask) {
+  if (w == nullptr || w->magic != kWsMagic) return CCR_ERR_BAD_HANDLE;
+  if (rows) *rows = w->out_rows;
+  if (mask) *mask = w->out_mask;
+  return CCR_OK;
+}
+
 ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t n_req, int64_t total_cands,
                                int64_t max_edge_len, int64_t total_edges, const int64_t* edge_keys,
                                const void* edge_feats, const int64_t* edge_offsets, const int32_t* cand_idx,
@@ -1038,7 +1045,7 @@ ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t 
   if (n_req < 0 || total_cands < 0 || total_edges < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
   if (n_req > w->max_req || total_cands > w->max_cands || total_edges > w->max_edges) return CCR_ERR_INVALID_ARG;
   if (n_req == 0 || total_cands == 0) return (n_req == 0 && total_cands != 0) ? CCR_ERR_INVALID_ARG : CCR_OK;
-  if (!edge_offsets || !cand_offsets || !cand_idx || !out_rows || !out_mask) return CCR_ERR_INVALID_ARG;
+  if (!edge_offsets || !cand_offsets || !cand_idx || !out_mask) return CCR_ERR_INVALID_ARG;  // out_rows may be NULL
   if (total_edges > 0 && (!edge_keys || !edge_feats)) return CCR_ERR_INVALID_ARG;
   if (s->req_b > 0 && !req_feats) return CCR_ERR_INVALID_ARG;
   DeviceScope scope(s->desc.device);
@@ -1063,7 +1070,8 @@ ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t 
                                        w->cand_idx, w->cand_offsets, s->req_b ? w->req_feats : nullptr, w->out_rows,
                                        w->out_mask, flags, stream);
   if (js != CCR_OK) return js;
-  ok = ok && cudaMemcpyAsync(out_rows, w->out_rows, total_cands * out_b, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (out_rows != nullptr)  // NULL: the rows stay in the workspace for a consumer on the device (ccr_workspace_outputs)
+    ok = ok && cudaMemcpyAsync(out_rows, w->out_rows, total_cands * out_b, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(out_mask, w->out_mask, total_cands, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();

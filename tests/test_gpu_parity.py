@@ -237,6 +237,16 @@ def test_host_buffer_entry_matches_device_entry(B):
                               out_rows, out_mask)
         torch.cuda.synchronize()
         assert np.array_equal(out_rows.numpy(), want_rows) and np.array_equal(out_mask.numpy(), want_mask)
+    # the serving case: no host buffer for the rows, they stay in the workspace on the device; only the mask returns
+    out_mask.fill_(9)
+    B.ccr_join_batch_host(store, ws, b.n_req, b.total_cands, b.max_edge_len, len(b.edge_keys), *args, None, out_mask)
+    torch.cuda.synchronize()
+    rows_ptr, mask_ptr = ws.outputs()
+    class _View:  # the workspace's device buffer seen as a tensor (CUDA array interface)
+        __cuda_array_interface__ = {"shape": (b.total_cands * store.out_row_bytes(),), "typestr": "|u1",
+                                    "data": (rows_ptr, False), "version": 2}
+    dev_rows = torch.as_tensor(_View(), device="cuda").view(b.total_cands, store.out_row_bytes())
+    assert np.array_equal(dev_rows.cpu().numpy(), want_rows) and np.array_equal(out_mask.numpy(), want_mask)
     with pytest.raises(B.CcrError) as e:
         B.ccr_join_batch_host(store, ws, b.n_req, b.total_cands + 1, b.max_edge_len, len(b.edge_keys), *args,
                               out_rows, out_mask)
