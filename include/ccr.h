@@ -272,6 +272,8 @@ ccr_status ccr_join_batch_ex(const ccr_docstore* store, const ccr_join_io* io, u
  * same sorting network over the key output array, so that a single long list is spread over many SMs instead
  * of one (a batch whose long lists would keep the SMs busy one list each stays on the one-block path), and the
  * rows of all lists are moved by one grid-wide gather: up to ~14 small kernels on `stream`.
+ * max_edge_len (HOST) must be at least the longest list; a longer list is cut there (its first max_edge_len
+ * records are sorted among themselves, the rest of its output is left unwritten) and no access leaves the arrays.
  * All pointers DEVICE; no allocation, no synchronisation.
  * The output is what ccr_join_batch expects as edge_keys / edge_feats.                                    */
 ccr_status ccr_sort_edges(const ccr_docstore* store, int32_t n_req, int64_t max_edge_len,

@@ -630,6 +630,7 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   a.keys_out = keys_out;
   a.feats_out = static_cast<uint8_t*>(feats_out);
   a.perm_out = perm_out;
+  a.max_len = static_cast<int>(max_edge_len);
   a.smem_keys = static_cast<int>(max_edge_len < ccr::kSortSmemMaxKeys ? max_edge_len : ccr::kSortSmemMaxKeys);
   a.smem_keys = (a.smem_keys + 1) & ~1;  // keeps the index array 8-byte aligned behind the keys
   const size_t smem = static_cast<size_t>(a.smem_keys) * 12;

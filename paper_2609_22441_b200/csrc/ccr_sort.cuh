@@ -190,6 +190,7 @@ struct SortArgs {
   int* perm_out;         // may be null when every list fits shared memory
   int smem_keys;         // (key, index) records the dynamic shared memory can hold: 12 bytes each
   int smem_words;        // packed key|index words it can hold: 8 bytes each
+  int max_len;           // the host's bound on the list length: longer lists are cut there (their tail is left alone)
   int multi;             // 1: packable lists longer than kSortChunk are sorted by the multi-block kernels, and the
                          //    rows of every list are moved by gather_all_kernel (perm_out is then required)
 };
@@ -222,7 +223,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
   extern __shared__ __align__(16) unsigned char smem_sort[];
   const int r = blockIdx.x;
   const long long e0 = __ldg(a.edge_offsets + r);
-  const long long Kl = __ldg(a.edge_offsets + r + 1) - e0;
+  const long long Kl = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   if (Kl <= 0) return;
   const int K = static_cast<int>(Kl);
   // keys that leave room for the record index in one 64-bit word (non-negative, below 2^(63 - index bits)) are
@@ -298,7 +299,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
 
 __device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, long long& e0, int& K) {
   e0 = __ldg(a.edge_offsets + r);
-  const long long Kl = __ldg(a.edge_offsets + r + 1) - e0;
+  const long long Kl = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   K = Kl > 0 ? static_cast<int>(Kl) : 0;
   if (K == 0) return false;
   return *reinterpret_cast<const volatile int*>(a.feats_out + e0 * a.row_ch * 16) == kSortMultiFlag;
@@ -309,8 +310,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_chunks_kernel(const Sort
   __shared__ unsigned long long w[kSortChunk];
   const int r = blockIdx.x;
   const long long e0 = __ldg(a.edge_offsets + r);
-  const long long Kl = __ldg(a.edge_offsets + r + 1) - e0;
-  const int K = Kl > 0x7fffffffLL ? 0x7fffffff : static_cast<int>(Kl);
+  const int K = static_cast<int>(min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len)));
   const int c0 = blockIdx.y * kSortChunk;
   if (c0 >= K) return;  // also K <= 0
   const int idx_bits = sort_index_bits(K);
@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_chunks_kernel(const Sort
     unsigned long long sum = 0;
     int longest = 0;
     for (int q = threadIdx.x; q < a.n_req; q += blockDim.x) {
-      const long long len = __ldg(a.edge_offsets + q + 1) - __ldg(a.edge_offsets + q);
+      const long long len = min(static_cast<long long>(__ldg(a.edge_offsets + q + 1) - __ldg(a.edge_offsets + q)), static_cast<long long>(a.max_len));
       if (len > kSortChunk) {
         sum += static_cast<unsigned long long>(len);
         longest = max(longest, static_cast<int>(min(len, 0x7fffffffLL)));
@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(kSortThreads) sort_unpack_kernel(const SortArg
 __global__ void __launch_bounds__(kSortThreads) gather_all_kernel(const SortArgs a) {
   const int r = blockIdx.x;
   const long long e0 = __ldg(a.edge_offsets + r);
-  const long long K = __ldg(a.edge_offsets + r + 1) - e0;
+  const long long K = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   const long long chunks = K * a.row_ch;
   const long long first = static_cast<long long>(blockIdx.y) * kSortThreads * kSortGatherUnroll;
   if (first >= chunks) return;

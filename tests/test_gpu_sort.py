@@ -148,3 +148,32 @@ def test_sort_chunked_path_and_its_policy(B, case):
             assert np.array_equal(f.cpu().numpy().view(np.uint16), want_f.view(np.uint16))
     finally:
         store.free()
+
+
+def test_sort_with_an_untruthful_length_bound_stays_in_bounds(B):
+    """max_edge_len below the longest list (a broken promise): lists are cut at the bound — their first
+    max_edge_len records sorted among themselves, nothing written behind, no access outside the arrays."""
+    rng = np.random.default_rng(12)
+    lens = [9000, 300, 12_000]
+    keys = np.concatenate([rng.integers(0, 1 << 30, size=n) for n in lens]).astype(np.int64)
+    feats = rng.standard_normal((len(keys), 64)).astype(np.float16)
+    eo = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    wl = W.config3(n_docs=1000, n_req=1, n_cand=10, gen_doc_feats=True, extra_pools=0)
+    store = B.store_from_workload(wl)
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    try:
+        for bound in (5000, 200):
+            k_out = torch.full((len(keys),), -7, dtype=torch.int64, device="cuda")
+            f_out = torch.full(feats.shape, 7.0, dtype=torch.float16, device="cuda")
+            p_out = torch.full((len(keys),), -7, dtype=torch.int32, device="cuda")
+            B.ccr_sort_edges(store, len(lens), bound, dev(keys), dev(feats), dev(eo), k_out, f_out, p_out)
+            torch.cuda.synchronize()
+            k, f, p = k_out.cpu().numpy(), f_out.cpu().numpy(), p_out.cpu().numpy()
+            for r, n in enumerate(lens):
+                a, m = int(eo[r]), min(n, bound)
+                order = np.argsort(keys[a:a + m], kind="stable")
+                assert np.array_equal(k[a:a + m], keys[a:a + m][order]) and np.array_equal(p[a:a + m], order)
+                assert np.array_equal(f[a:a + m].view(np.uint16), feats[a:a + m][order].view(np.uint16))
+                assert (k[a + m:a + n] == -7).all() and (p[a + m:a + n] == -7).all() and (f[a + m:a + n] == 7).all()
+    finally:
+        store.free()
