@@ -37,6 +37,7 @@ CCR_FLAG_FORCE_SAMPLED = 1 << 5
 CCR_FLAG_STATIC_SPLIT = 1 << 6
 CCR_FLAG_TWO_PHASE = 1 << 7
 CCR_FLAG_COSINE = 1 << 8
+CCR_FLAG_WARP_SPECIALISED = 1 << 9
 
 EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_upsert", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",

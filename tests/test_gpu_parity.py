@@ -33,7 +33,9 @@ def _variants(B, include_smem=True):
     v = [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL), ("sampled", B.CCR_FLAG_FORCE_SAMPLED)]
     if include_smem:
         v.append(("smem", B.CCR_FLAG_FORCE_SMEM))
+    # without a kernel flag a small launch takes the two-phase kernel and a large one the warp-specialised kernel
     return (v + [(n + "+2phase", f | B.CCR_FLAG_TWO_PHASE) for n, f in v] +
+            [(n + "+ws", f | B.CCR_FLAG_WARP_SPECIALISED) for n, f in v] +
             [(n + "+static", f | B.CCR_FLAG_STATIC_SPLIT) for n, f in v])
 
 
@@ -92,7 +94,7 @@ def test_config2b_second_degree_on_config1_shape_full_size(B):
     assert wl.out_row_bytes() == 448
     # large sub-tiles and other warp splits: the engager work lists address candidates by their index in the sub-tile
     _check(B, wl, [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL)],
-           tunings=((0, 0), (4096, 0, 12, 4, 0), (2048, 0, 8, 8, 0), (768, 0, 14, 1, 0)))
+           tunings=((0, 0), (4096, 0, 12, 4, 0), (2048, 0, 8, 8, 0), (768, 0, 14, 1, 0)))  # second degree: always warp-specialised
 
 
 def test_config3_scaled_store_long_edge_lists(B):
@@ -113,8 +115,8 @@ def test_more_requests_than_the_kernel_mirrors_in_shared_memory(B):
     for second in (False, True):
         wl = W.config1(n_docs=30_000, n_req=1500, n_cand=150, second_degree=second, edge_lo=3, edge_hi=80)
         assert wl.batch.n_req == 1500
-        _check(B, wl, [("auto", 0), ("static", B.CCR_FLAG_STATIC_SPLIT), ("2phase", B.CCR_FLAG_TWO_PHASE),
-                       ("global", B.CCR_FLAG_FORCE_GLOBAL)])
+        _check(B, wl, [("auto", 0), ("ws", B.CCR_FLAG_WARP_SPECIALISED), ("static", B.CCR_FLAG_STATIC_SPLIT),
+                       ("2phase", B.CCR_FLAG_TWO_PHASE), ("global+ws", B.CCR_FLAG_FORCE_GLOBAL | B.CCR_FLAG_WARP_SPECIALISED)])
 
 
 # ------------------------------------------------------------------ ragged / degenerate inputs

@@ -75,7 +75,7 @@ def test_tiny_stores_every_combination_of_sources(B, seed):
                          reduce_sum_mask=s.reduce_sum_mask)
     store = B.store_from_workload(wl)
     state = _host_state(s)
-    kernels = [("ws", 0), ("2phase", B.CCR_FLAG_TWO_PHASE)]
+    kernels = [("auto", 0), ("ws", B.CCR_FLAG_WARP_SPECIALISED), ("2phase", B.CCR_FLAG_TWO_PHASE)]
     try:
         _compare(B, store, state, batch, s, kernels)  # before any write
         used = 0
@@ -127,7 +127,7 @@ def test_scaled_config1_batches_of_new_and_updated_documents(B, second):
             else:
                 _apply(B, store, state, pos, donor.doc_feats[src], donor.author_ids[src],
                        donor.actor_ids[src] if second else None, donor.actor_types[src] if second else None)
-        _compare(B, store, state, b, s, [("ws", 0), ("2phase", B.CCR_FLAG_TWO_PHASE)])
+        _compare(B, store, state, b, s, [("auto", 0), ("ws", B.CCR_FLAG_WARP_SPECIALISED), ("2phase", B.CCR_FLAG_TWO_PHASE)])
     finally:
         store.free()
 
