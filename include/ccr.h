@@ -82,8 +82,8 @@ enum {
   CCR_FLAG_COSINE            = 1u << 8, /* append the derived cosine section (ccr_docstore_set_cosine,
                                            ccr_join_batch_ex); adds 32 bytes to the row                */
   CCR_FLAG_WARP_SPECIALISED  = 1u << 9  /* take the warp-specialised kernel whatever the launch size (by default a
-                                           first-degree ragged launch of at most 131,072 candidates — a single
-                                           request — runs on the two-phase kernel, which has the shorter start-up) */
+                                           ragged launch of at most 131,072 candidates — a single request —
+                                           runs on the two-phase kernel, which has the shorter start-up)      */
 };
 
 /* Create an empty store on desc->device.  Allocates doc_feats [n_docs, doc_dim] and author ids

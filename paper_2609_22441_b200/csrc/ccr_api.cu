@@ -721,9 +721,10 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   // which kernel: the merge path and CCR_FLAG_TWO_PHASE take the two-phase kernel, and so does a small plain
   // launch (a single request: the latency case), where the two-phase kernel's shorter start-up wins — measured
   // on one request of 30,000 candidates 16.4 against 18.4 us, 100,000 candidates x 20,000 keys 38 against 56 us;
-  // from about 200,000 candidates on the warp-specialised kernel is ahead (240,000: 43 against 48 us).
+  // from about 200,000 candidates on the warp-specialised kernel is ahead (240,000: 43 against 48 us).  The
+  // same holds for second-degree joins (one request: 20.5 against 28.7 us; 240,000 candidates: equal).
   const bool cos = (flags & CCR_FLAG_COSINE) != 0;
-  const bool small = total_cands <= kSmallLaunchCands && !second && !cos && n_max == 0 &&
+  const bool small = total_cands <= kSmallLaunchCands && !cos && n_max == 0 &&
                      !(flags & (CCR_FLAG_WARP_SPECIALISED | CCR_FLAG_STATIC_SPLIT));
   const bool use_ws = !merge && !(flags & CCR_FLAG_TWO_PHASE) && !small;
   if (cos) {

@@ -93,8 +93,8 @@ def test_config2b_second_degree_on_config1_shape_full_size(B):
     wl = W.config1(second_degree=True)
     assert wl.out_row_bytes() == 448
     # large sub-tiles and other warp splits: the engager work lists address candidates by their index in the sub-tile
-    _check(B, wl, [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL)],
-           tunings=((0, 0), (4096, 0, 12, 4, 0), (2048, 0, 8, 8, 0), (768, 0, 14, 1, 0)))  # second degree: always warp-specialised
+    _check(B, wl, [("auto", 0), ("global", B.CCR_FLAG_FORCE_GLOBAL), ("ws", B.CCR_FLAG_WARP_SPECIALISED)],
+           tunings=((0, 0), (4096, 0, 12, 4, 0), (2048, 0, 8, 8, 0), (768, 0, 14, 1, 0)))
 
 
 def test_config3_scaled_store_long_edge_lists(B):
