@@ -154,11 +154,17 @@ def distinct_sample_excluding(rng: np.random.Generator, high: int, k: int, exclu
     if k == 0:
         return np.empty(0, dtype=np.int64)
     got = np.empty(0, dtype=np.int64)
+    rounds = 0
     while len(got) < k:
         need = k - len(got)
         draw = rng.integers(0, high, size=need + need // 4 + 16, dtype=np.int64)
         draw = draw[~excluded_mark[draw]]
         got = np.union1d(got, draw)
+        rounds += 1
+        if rounds == 64:  # far more rounds than a satisfiable request needs: is it satisfiable at all?
+            available = int(high) - int(np.count_nonzero(excluded_mark[:high]))
+            if k > available:
+                raise ValueError("asked for %d distinct values but only %d are available" % (k, available))
     return got[rng.permutation(len(got))[:k]]
 
 

@@ -430,6 +430,13 @@ def test_generators_are_deterministic():
         assert np.all(np.diff(k) > 0)
 
 
+@pytest.mark.timeout(60)
+def test_generator_refuses_more_distinct_candidates_than_documents():
+    # a request cannot draw more distinct documents than the store holds: an error, not an endless rejection loop
+    with pytest.raises(ValueError):
+        W.config1(n_docs=5_754, n_req=3, n_cand=8_134, second_degree=True, edge_lo=37, edge_hi=5_164)
+
+
 # ---------------------------------------------------------------- Algorithm 1 step 1 (sort of the affinity records)
 def _unsorted_batch(seed, n_req, kmax, alphabet, dup=False):
     rng = np.random.default_rng(seed)
