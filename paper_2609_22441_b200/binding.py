@@ -14,6 +14,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
+# CCR_LIB_OVERRIDE names another build of the same library (kernel A/B comparisons); unset = the in-tree build
 LIB_PATH = os.environ.get("CCR_LIB_OVERRIDE") or os.path.join(_HERE, "libccr.so")
 
 CCR_OK = 0
