@@ -287,9 +287,9 @@ ccr_status ccr_sort_edges(const ccr_docstore* store, int32_t n_req, int64_t max_
  * document id q in the index, or -1 when q is not indexed.
  *
  * ccr_idindex_create copies n_ids ascending, unique ids (HOST or DEVICE source per src_on_device) into device
- * memory and builds the sampled search levels above them (every 32nd key, repeatedly, until at most 16,384
+ * memory and builds the sampled search levels above them (every 8th key, repeatedly, until at most 2,048
  * keys remain).  `positions` (optional, int32[n_ids], same source side) gives the store position of each id;
- * NULL means the position of an id is its rank.  Synchronous; allocates 8.3 bytes per id (+4 with positions).
+ * NULL means the position of an id is its rank.  Synchronous; allocates 9.2 bytes per id (+4 with positions).
  * ccr_resolve_ids writes out_pos[i] = position of query_ids[i] or -1 for n_queries DEVICE queries: one kernel
  * on `stream`, no allocation, no sync.  Ids that break the ascending order give unspecified positions but
  * every access stays in bounds.  The output is what ccr_join_batch takes as cand_idx (-1 = unresolved).      */

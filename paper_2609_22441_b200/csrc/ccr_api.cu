@@ -519,7 +519,7 @@ ccr_status ccr_idindex_create(int32_t device, int64_t n_ids, const int64_t* sort
   }
   DeviceScope scope(device);
   if (!scope.ok) return CCR_ERR_CUDA;
-  // level sizes: sample every 32nd key until the top fits shared memory
+  // level sizes: sample every 8th key until the top level is small enough to stage per block
   long long count[ccr::kResolveMaxLevels];
   int n_levels = 1;
   count[0] = n_ids;
@@ -561,6 +561,11 @@ ccr_status ccr_idindex_create(int32_t device, int64_t n_ids, const int64_t* sort
     ix->launches++;
     ok = cudaGetLastError() == cudaSuccess;
   }
+  for (int l = 0; l < n_levels && ok; ++l) {  // the +infinity keys behind every level (the allocation has room)
+    ccr::pad_level_kernel<<<1, 32>>>(ix->level[l], count[l]);
+    ix->launches++;
+    ok = cudaGetLastError() == cudaSuccess;
+  }
   ok = ok && cudaDeviceSynchronize() == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(ccr::resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   ccr::kResolveTopMax * 8 + 256) == cudaSuccess;
@@ -596,8 +601,9 @@ ccr_status ccr_resolve_ids(const ccr_idindex* cix, int64_t n_queries, const int6
   a.queries = query_ids;
   a.out_pos = out_pos;
   const long long per_block = static_cast<long long>(ccr::kResolveThreads);
-  long long blocks = (n_queries + per_block - 1) / per_block;
-  const long long cap = static_cast<long long>(ix->n_sms) * 4;  // the top level is re-read by every block
+  const long long lanes = 1LL << (ccr::kResolveFanLog2 - 1);  // lanes that share a query
+  long long blocks = (n_queries * lanes + per_block - 1) / per_block;
+  const long long cap = static_cast<long long>(ix->n_sms) * ccr::kResolveBlocksPerSm;  // the top level is re-read by every block
   if (blocks > cap) blocks = cap;
   const size_t smem = static_cast<size_t>(ix->count[ix->n_levels - 1]) * 8 + 16;
   ccr::resolve_kernel<<<static_cast<unsigned>(blocks), ccr::kResolveThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);

@@ -3,27 +3,29 @@
 // in HBM, resolved queries with a binary-search kernel (~5 ms per request over a few hundred million ids,
 // ~47 ms at batch 8, every probe a dependent HBM access) and then moved the step to a CPU hash map.
 //
-// Here the sorted array gets a static search tree of sampled levels, fan-out 32: level l+1 holds the last
-// key of every full block of 32 keys of level l.  The top level (<= 16,384 keys) is staged in shared
-// memory; below it a query touches one 256-byte window (two cache lines) per level, inside which a lane
-// needs two dependent rounds of loads (octant, then position): the ~2 MB level stays in L2, the larger ones come
-// from HBM.  A query over 300M ids makes 6 dependent rounds instead of 29 dependent probes across the whole
-// array; eight queries per lane are in flight at once.
+// Here the sorted array gets a static search tree of sampled levels, fan-out 8: level l+1 holds the last
+// key of every full block of 8 keys of level l.  The top level (<= 2,048 keys, 16 KB) is staged in shared
+// memory; below it a query reads one 64-byte window per level in one dependent round: the four lanes that share
+// the query load 16 bytes each (one access for the load unit instead of four, which is what bounded the
+// lane-per-query form: every scattered 16-byte load of a lane is a pass of its own through the L1), count the
+// keys below the id and add the counts up with two shuffles; the leaf round also says whether the id is
+// present.  The small levels stay in L2, the large ones come from HBM 64 bytes at a time.  A query over 300M ids
+// makes 6 dependent rounds instead of 29 dependent probes across the whole array.  Two queries per group of
+// lanes in flight, up to 2,048 threads per SM.  Measured and slower: wider windows (128 bytes with eight lanes
+// per query; 256 bytes in two rounds), a lane per query with 1-8 queries in flight, and a larger staged top
+// level (it takes shared memory from the L1 and start-up time from every block).
 #pragma once
 
 #include "ccr_device.cuh"
 
 namespace ccr {
 
-constexpr int kResolveFanLog2 = 5;                 // 32 keys = one 256-byte window per level
-constexpr int kResolveMaxLevels = 8;
-constexpr int kResolveTopMax = 16384;              // keys of the top level (128 KB of shared memory)
+constexpr int kResolveFanLog2 = 3;                 // 8 keys = one 64-byte window per level
+constexpr int kResolveMaxLevels = 8;               // 2,048 x 8^7 ids: more than int32 positions can name
+constexpr int kResolveTopMax = 2048;               // keys of the top level (16 KB of shared memory)
 constexpr int kResolveThreads = 256;
-constexpr int kResolveUnroll = 8;                 // queries a lane keeps in flight
-#ifndef CCR_RESOLVE_ROUND2
-#define CCR_RESOLVE_ROUND2 2
-#endif
-constexpr int kResolveRound2 = CCR_RESOLVE_ROUND2;  // queries of a lane whose octants are in flight together
+constexpr int kResolveBlocksPerSm = 8;             // grid cap: the top level is staged by every block
+constexpr int kResolveUnroll = 2;                  // queries a group of lanes keeps in flight
 constexpr long long kResolveInf = 0x7fffffffffffffffLL;  // stands for the keys beyond the end of a level
 
 struct ResolveArgs {
@@ -42,6 +44,14 @@ __global__ void build_level_kernel(const int64_t* below, long long n_below, int6
     above[i] = below[((i + 1) << kResolveFanLog2) - 1];
 }
 
+// Every level is followed by kResolvePad keys of +infinity, so that the window a query reads (window c of a level
+// with n keys, c <= n / 8) needs no bounds checks; the allocation of a level leaves room for them.
+constexpr int kResolvePad = 2 << kResolveFanLog2;
+static_assert(kResolvePad <= 32 && kResolvePad * 8 <= 256, "one warp writes the padding; a level is allocated with 256 spare bytes");
+__global__ void pad_level_kernel(int64_t* level, long long n) {
+  if (threadIdx.x < kResolvePad) level[n + threadIdx.x] = kResolveInf;
+}
+
 __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveArgs a) {
   extern __shared__ __align__(16) unsigned char smem_res[];
   int64_t* top = reinterpret_cast<int64_t*>(smem_res);
@@ -49,81 +59,66 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
   const int n_top = static_cast<int>(a.count[top_l]);
   for (int i = threadIdx.x; i < n_top; i += blockDim.x) top[i] = __ldg(a.level[top_l] + i);
   __syncthreads();
-
-  // lane-per-query, kResolveUnroll queries of a lane in flight; inside a 32-key window the lane runs a
-  // 5-step branch-free search (its sectors come from L2 / HBM on demand).  A warp-cooperative variant
-  // (whole window per coalesced access, __ballot_sync rank) was measured and is slower at every batch size:
-  // 886 vs 743 us for 1.92M queries, the extra shuffles and the lower number of independent accesses in
-  // flight outweigh the saved sector fetches.
-  // query u of a lane is `threads` apart from query u-1, so that a small launch still spreads over all blocks
-  const long long threads = static_cast<long long>(gridDim.x) * blockDim.x;
-  for (long long base = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; base < a.n_queries;
-       base += threads * kResolveUnroll) {
+  constexpr int G = 1 << (kResolveFanLog2 - 1);  // lanes that share a query: one 16-byte load each per window
+  const unsigned sub = threadIdx.x & (G - 1);
+  const long long groups = (static_cast<long long>(gridDim.x) * blockDim.x) / G;
+  const long long gid = (blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x) / G;
+  const long long rounds = (a.n_queries + groups * kResolveUnroll - 1) / (groups * kResolveUnroll);
+  for (long long it = 0; it < rounds; ++it) {  // warp-uniform trip count: the shuffles below need every lane
+    const long long base = it * groups * kResolveUnroll + gid;
     int64_t q[kResolveUnroll];
-    long long c[kResolveUnroll];  // number of keys of the current level that are below q
+    unsigned c[kResolveUnroll];  // number of keys of the current level that are below q (an index has < 2^31 ids)
 #pragma unroll
     for (int u = 0; u < kResolveUnroll; ++u) {
-      const long long j = base + static_cast<long long>(u) * threads;
+      const long long j = base + static_cast<long long>(u) * groups;
       q[u] = j < a.n_queries ? __ldg(a.queries + j) : 0;
-      c[u] = lower_bound_smem(top, n_top, q[u]);
+      c[u] = 0;
     }
-    // descend: c keys of level l+1 below q  =>  blocks 0..c-1 of level l are below q, the answer is in block c
-    for (int l = top_l - 1; l >= 0; --l) {
-      const int64_t* lev = a.level[l];
-      const long long n = a.count[l];
-      // Inside the 32-key window a query needs two dependent rounds instead of a six-probe binary search:
-      // round 1 reads the last key of the first three octants (three independent loads; the fourth octant's last
-      // key is not below q by construction of the level above) and picks the octant, round 2 reads the octant's
-      // eight keys as four 16-byte loads and counts the ones below q.  Keys beyond the end of the level count as
-      // +infinity.  All queries of the lane do round 1 together; round 2 runs for kResolveRound2 of them at a time, which
-      // keeps the keys in flight within the register budget.
-      long long lo[kResolveUnroll];
-      int64_t r1[kResolveUnroll][3];
+    {  // the group's searches of the top level step together, so their shared-memory reads overlap
+      int n = n_top;
+      while (n > 1) {
+        const int half = n >> 1;
+#pragma unroll
+        for (int u = 0; u < kResolveUnroll; ++u) c[u] = (top[c[u] + half - 1] < q[u]) ? c[u] + half : c[u];
+        n -= half;
+      }
+      if (n == 1) {
+#pragma unroll
+        for (int u = 0; u < kResolveUnroll; ++u) c[u] += (top[c[u]] < q[u]) ? 1 : 0;
+      }
+    }
+    // descend: c keys of level l+1 below q  =>  windows 0..c-1 of level l are below q, the answer is in window c
+    for (int l = top_l - 1; l >= 1; --l) {
+      const longlong2* lev = reinterpret_cast<const longlong2*>(a.level[l]);
+      longlong2 k[kResolveUnroll];
+#pragma unroll
+      for (int u = 0; u < kResolveUnroll; ++u) k[u] = __ldg(lev + (static_cast<size_t>(c[u]) * G + sub));
 #pragma unroll
       for (int u = 0; u < kResolveUnroll; ++u) {
-        lo[u] = c[u] << kResolveFanLog2;
+        unsigned v = (k[u].x < q[u] ? 1u : 0u) + (k[u].y < q[u] ? 1u : 0u);
 #pragma unroll
-        for (int o = 0; o < 3; ++o) {
-          const long long i = lo[u] + 8 * o + 7;
-          r1[u][o] = i < n ? __ldg(lev + i) : kResolveInf;
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < kResolveUnroll; ++u)
-        lo[u] += 8 * ((r1[u][0] < q[u] ? 1 : 0) + (r1[u][1] < q[u] ? 1 : 0) + (r1[u][2] < q[u] ? 1 : 0));
-#pragma unroll
-      for (int h = 0; h < kResolveUnroll; h += kResolveRound2) {
-        longlong2 r2[kResolveRound2][4];
-#pragma unroll
-        for (int v = 0; v < kResolveRound2; ++v) {
-#pragma unroll
-          for (int p = 0; p < 4; ++p) {
-            const long long i = lo[h + v] + 2 * p;  // even, and the level's base is 16-byte aligned
-            if (i + 1 < n) {
-              r2[v][p] = __ldg(reinterpret_cast<const longlong2*>(lev + i));
-            } else {
-              r2[v][p].x = i < n ? __ldg(lev + i) : kResolveInf;
-              r2[v][p].y = kResolveInf;
-            }
-          }
-        }
-#pragma unroll
-        for (int v = 0; v < kResolveRound2; ++v) {
-          int below = 0;
-#pragma unroll
-          for (int p = 0; p < 4; ++p) below += (r2[v][p].x < q[h + v] ? 1 : 0) + (r2[v][p].y < q[h + v] ? 1 : 0);
-          c[h + v] = lo[h + v] + below;
-        }
+        for (int d = 1; d < G; d <<= 1) v += __shfl_xor_sync(kFull, v, d);
+        c[u] = (c[u] << kResolveFanLog2) + v;
       }
     }
+    {  // the leaf round also tells whether the id is present (a match with the padding lands at c >= count[0])
+      const longlong2* lev = reinterpret_cast<const longlong2*>(a.level[0]);
+      longlong2 k[kResolveUnroll];
 #pragma unroll
-    for (int u = 0; u < kResolveUnroll; ++u) {
-      const long long j = base + static_cast<long long>(u) * threads;
-      if (j >= a.n_queries) continue;
-      int pos = -1;
-      if (c[u] < a.count[0] && __ldg(a.level[0] + c[u]) == q[u])
-        pos = a.positions ? __ldg(a.positions + c[u]) : static_cast<int>(c[u]);
-      a.out_pos[j] = pos;
+      for (int u = 0; u < kResolveUnroll; ++u) k[u] = __ldg(lev + (static_cast<size_t>(c[u]) * G + sub));
+#pragma unroll
+      for (int u = 0; u < kResolveUnroll; ++u) {
+        unsigned v = (k[u].x < q[u] ? 1u : 0u) + (k[u].y < q[u] ? 1u : 0u) + ((k[u].x == q[u] || k[u].y == q[u]) ? 256u : 0u);
+#pragma unroll
+        for (int d = 1; d < G; d <<= 1) v += __shfl_xor_sync(kFull, v, d);
+        c[u] = (c[u] << kResolveFanLog2) + (v & 255u);
+        const long long j = base + static_cast<long long>(u) * groups;
+        if (sub == 0 && j < a.n_queries) {
+          int pos = -1;
+          if (v >= 256u && c[u] < a.count[0]) pos = a.positions ? __ldg(a.positions + c[u]) : static_cast<int>(c[u]);
+          a.out_pos[j] = pos;
+        }
+      }
     }
   }
 }

@@ -28,7 +28,9 @@ def _queries(rng, ids, n):
     return q.astype(np.int64)
 
 
-@pytest.mark.parametrize("n_ids", [0, 1, 2, 31, 32, 33, 1023, 1024, 1025, 16384, 16385, 32 * 16384 + 5, 3_000_000])
+# sizes around every boundary of the search tree (windows of 8 keys, a top level of at most 2,048 keys)
+@pytest.mark.parametrize("n_ids", [0, 1, 2, 7, 8, 9, 31, 32, 33, 1023, 1024, 1025, 2047, 2048, 2049, 2055, 2056, 16383, 16384,
+                                   16385, 8 * 16384 - 1, 8 * 16384, 8 * 16384 + 5, 32 * 16384 + 5, 3_000_000])
 @pytest.mark.parametrize("with_positions", [False, True])
 def test_resolve_matches_oracle(B, n_ids, with_positions):
     rng = np.random.default_rng(n_ids + with_positions)
@@ -46,6 +48,27 @@ def test_resolve_matches_oracle(B, n_ids, with_positions):
     if n_ids:
         assert (want >= 0).mean() > 0.5
     ix.free()
+
+
+@pytest.mark.parametrize("n_ids", [5, 8, 13, 2048, 2051, 40_001])
+def test_resolve_with_the_largest_int64_as_an_id(B, n_ids):
+    """Keys beyond the end of a level count as +infinity inside the kernel; an id equal to that value is still
+    found when it is indexed and not found when it is not."""
+    rng = np.random.default_rng(n_ids)
+    top = np.iinfo(np.int64).max
+    ids = (np.cumsum(rng.integers(1, 6, size=n_ids)) * 2).astype(np.int64)
+    for with_top in (False, True):
+        if with_top:
+            ids[-1] = top
+        q = np.concatenate([ids, ids + 1, [top, top - 1, -1, 0]]).astype(np.int64)  # ids + 1 wraps for the top id
+        want = oracle.resolve_ids(ids, q)
+        assert (want[-4] >= 0) == with_top
+        ix = B.IdIndex(ids)
+        out = torch.full((len(q),), -7, dtype=torch.int32, device="cuda")
+        ix.resolve(torch.from_numpy(q).cuda(), out)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.cpu().numpy(), want)
+        ix.free()
 
 
 def test_resolve_a_few_hundred_million_ids(B):
