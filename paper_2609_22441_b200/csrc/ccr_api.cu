@@ -845,7 +845,8 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     if (dynamic) a.sched = s->status + 4 + 2 * static_cast<int>(s->launches % kSchedRegions);
     fn<<<static_cast<unsigned>(blocks), (n_str + n_res) * 32, smem, st>>>(a, n_str);
   } else {
-    // persistent two-phase kernel: as many blocks as stay resident, each with at least 256 candidates
+    // persistent two-phase kernel: as many blocks as stay resident, each with at least 64 candidates (a single
+    // small request is spread over many SMs: 21.6 against 23.4 us for 1,000 candidates with 256 per block)
     const KernelFn fn = n_max > 0 ? (merge ? kPaddedMerge : (second ? kPaddedSecond : kPaddedFirst))
                                   : (merge ? v.merge : (second ? v.second : v.first));
     const int by_regs = ccr::kJoinMinBlocks;  // matches the kernel's __launch_bounds__
@@ -854,7 +855,7 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     if (s->blocks_per_sm > 0 && per_sm > s->blocks_per_sm) per_sm = s->blocks_per_sm;
     if (per_sm < 1) per_sm = 1;
     long long blocks = static_cast<long long>(s->n_sms) * per_sm;
-    const long long most = (groups + ccr::kWarps - 1) / ccr::kWarps;
+    const long long most = (groups + 1) / 2;
     if (blocks > most) blocks = most;
     fn<<<static_cast<unsigned>(blocks), ccr::kThreads, smem, st>>>(a);
   }
