@@ -16,6 +16,13 @@
  *   - Feature, key and output buffers must be 16-byte aligned; section widths (dim * element size)
  *     must be multiples of 16 bytes.
  *   - There is no CPU fallback: without a CUDA device every compute entry returns CCR_ERR_CUDA.
+ *   - Host threads: the join entries (ccr_join_batch, _padded, _ex, _host with a workspace of its own) may be
+ *     called on one store from several host threads at once, each on its own stream: the launch counter is
+ *     atomic and every launch draws its own pair of scheduling words.  Everything that changes a store or reads
+ *     its status (upload, upsert, set_tuning, set_cosine, CCR_FLAG_VALIDATE, device_status, selftest_wait, free)
+ *     and ccr_join_payload_static (one shared block) must be serialised by the caller.
+ *   - Handles are looked up in a table of live handles before they are used: a freed, NULL or foreign pointer
+ *     gives CCR_ERR_BAD_HANDLE without being dereferenced.
  */
 #ifndef CCR_H_
 #define CCR_H_
@@ -65,8 +72,10 @@ enum {
   CCR_FLAG_FORCE_SMEM        = 1u << 0, /* stage every request's full key list in shared memory
                                            (CCR_ERR_UNSUPPORTED if max_edge_len does not fit)       */
   CCR_FLAG_FORCE_GLOBAL      = 1u << 1, /* never stage keys: search them in global memory / L2      */
-  CCR_FLAG_CANDS_SORTED      = 1u << 2, /* caller promises that, inside each request, the candidates'
-                                           author ids are non-decreasing.  Together with CCR_FLAG_TWO_PHASE
+  CCR_FLAG_CANDS_SORTED      = 1u << 2, /* caller promises that, inside each request, the author ids of the
+                                           resolved candidates are non-decreasing (a position outside
+                                           [0, n_docs) has no author and may sit anywhere: a sub-tile that holds
+                                           one is searched candidate by candidate).  Together with CCR_FLAG_TWO_PHASE
                                            this selects the merge-path kernel; the default kernel does not
                                            need the promise (sorted candidates still help its locality)    */
   CCR_FLAG_VALIDATE          = 1u << 3, /* check offsets, key order (and candidate order) on the
@@ -105,8 +114,9 @@ ccr_status ccr_docstore_upload(ccr_docstore* store, int64_t first_doc, int64_t n
                                const int64_t* actor_ids, const uint8_t* actor_types,
                                int src_on_device, void* stream);
 
-/* Write a batch of rows by position (Section 6.2, "Scaling ingestion": bootstrap step 3, "GPU scatter features to
- * assigned positions", and the steady-state updates).  Row i of the batch replaces row positions[i] of the store:
+/* Write a batch of rows by position: the device-side write of step 3 of the per-batch bootstrap protocol of
+ * Section 6.2 (features go to the positions the host assigned in step 2), also used for the steady-state
+ * updates.  Row i of the batch replaces row positions[i] of the store:
  * doc_feats [n, doc_dim], author_ids int64[n], and for second-degree stores actor_ids int64[n, max_actors] /
  * actor_types uint8[n, max_actors], with the meaning they have in ccr_docstore_upload.  A NULL source leaves that
  * array untouched (an engagement update that only rewrites the engager slots passes only those).  A position
@@ -127,8 +137,8 @@ ccr_status ccr_docstore_upsert(ccr_docstore* store, int64_t n,
                                const uint8_t* actor_types, /* DEVICE [n, max_actors] or NULL              */
                                void* stream);
 
-/* Free the store and its device memory.  A second free of the same handle returns
- * CCR_ERR_BAD_HANDLE as long as the freed block has not been reused by the allocator.              */
+/* Free the store and its device memory.  A second free of the same handle returns CCR_ERR_BAD_HANDLE
+ * (the handle is no longer in the table of live handles; the freed memory is not read).              */
 ccr_status ccr_docstore_free(ccr_docstore* store);
 
 /* Bytes of one output row for this store and these flags:
@@ -139,7 +149,8 @@ size_t ccr_out_row_bytes(const ccr_docstore* store, uint32_t flags);
 /* The join (Eq. 1 / Algorithm 1 steps 2-4, fused with the document gather and request broadcast).
  *
  * For request r = 0 .. n_req-1, with keys = edge_keys[edge_offsets[r] .. edge_offsets[r+1]) (K of
- * them, ascending and unique) and candidates j in [cand_offsets[r], cand_offsets[r+1]):
+ * them, ascending, unique and non-negative: ids are signed 64-bit and a negative id means "no id" — an empty
+ * engager slot — so a negative key can never be matched) and candidates j in [cand_offsets[r], cand_offsets[r+1]):
  *     p   = cand_idx[j]                       position in the store
  *     d   = author_id[p]                      Algorithm 1's d_j
  *     pos = lower bound of d in keys;  found = pos < K and keys[pos] == d
@@ -336,11 +347,15 @@ ccr_status ccr_join_batch_host(const ccr_docstore* store, ccr_workspace* ws,
  * cudaFree nor any allocating library routine.
  *
  * What it uses instead: one fixed 16 MiB block of device memory that belongs to the library image (every GPU
- * that loads the library holds it until the process exits).  The block carries the kernel's status and
+ * that loads the library holds it until the process exits).  The block carries the kernel's
  * scheduling words and the device copy of the payload (keys, edge rows, offsets, candidate positions, request
  * rows, each rounded up to 256 bytes).  ccr_static_payload_capacity() returns the bytes available to the
  * payload; a batch that needs more is refused with CCR_ERR_UNSUPPORTED before anything is enqueued.
- * CCR_FLAG_VALIDATE is not accepted here (CCR_ERR_UNSUPPORTED).
+ * CCR_FLAG_VALIDATE is not accepted here (CCR_ERR_UNSUPPORTED).  Because the offsets are host-readable in this
+ * entry, they are checked before anything is enqueued (CCR_ERR_INVALID_ARG): cand_offsets[0] == 0, both arrays
+ * non-decreasing, no request longer than max_edge_len, edge_offsets[n_req] <= total_edges and
+ * cand_offsets[n_req] == total_cands.  Only the scheduling words live in the block; a bounded device-side wait
+ * that runs out is recorded in the store's own status word and reported by ccr_docstore_device_status as usual.
  *
  * Sharing: all calls in a process use the same block on a device and it keeps the previous call's contents.
  * Each call re-clears the control words on `stream` before use and overwrites the payload area, so calls on

@@ -5,12 +5,14 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdint>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <unordered_set>
 
 #include "ccr_join.cuh"
 #include "ccr_pad.cuh"
@@ -71,7 +73,7 @@ struct ccr_docstore {
   int ws_streamers, ws_resolvers;  // warp split of the warp-specialised kernel
   int n_sms;
   int cos_first, cos_dim, cos_chunks;  // derived cosine section (cos_chunks == 0: not configured)
-  int64_t launches;
+  std::atomic<int64_t> launches;  // kernels launched for this store; also hands out the scheduling-word pairs
 };
 
 struct ccr_workspace {
@@ -104,7 +106,30 @@ struct ccr_idindex {
 
 namespace {
 
-inline bool good(const ccr_docstore* s) { return s != nullptr && s->magic == kStoreMagic; }
+// Live handles of every kind.  A handle is looked up here before it is dereferenced, so a freed (or never
+// created) pointer is refused without reading the memory behind it.
+std::mutex g_handles_mutex;
+std::unordered_set<const void*>& live_handles() {
+  static std::unordered_set<const void*>* h = new std::unordered_set<const void*>();  // never destroyed: no exit-order hazard
+  return *h;
+}
+inline void handle_add(const void* p) {
+  std::lock_guard<std::mutex> lock(g_handles_mutex);
+  live_handles().insert(p);
+}
+inline bool handle_remove(const void* p) {  // true if it was live
+  std::lock_guard<std::mutex> lock(g_handles_mutex);
+  return live_handles().erase(p) != 0;
+}
+inline bool handle_live(const void* p) {
+  if (p == nullptr) return false;
+  std::lock_guard<std::mutex> lock(g_handles_mutex);
+  return live_handles().count(p) != 0;
+}
+
+inline bool good(const ccr_docstore* s) { return handle_live(s) && s->magic == kStoreMagic; }
+inline bool good(const ccr_workspace* w) { return handle_live(w) && w->magic == kWsMagic; }
+inline bool good(const ccr_idindex* ix) { return handle_live(ix) && ix->magic == kIxMagic; }
 
 // ---------------------------------------------------------------------------------------------------
 // Precondition check behind CCR_FLAG_VALIDATE: one block per request.
@@ -129,12 +154,14 @@ __global__ void validate_kernel(const ccr::JoinArgs a, int check_sorted, int* co
     if (k < 0 || (i > e0 && a.edge_keys[i - 1] >= k)) atomicCAS(code, 0, 3);
   }
   if (check_sorted) {
+    // the promise is over author ids, so it binds resolved candidates only: each one is compared with the
+    // nearest resolved candidate before it (unresolved / out-of-range positions may sit anywhere)
     for (int64_t j = c0 + 1 + threadIdx.x; j < c1; j += blockDim.x) {
-      const int p = a.cand_idx[j - 1], q = a.cand_idx[j];
-      const bool pin = p >= 0 && p < a.n_docs, qin = q >= 0 && q < a.n_docs;
-      const long long ap = pin ? ccr::load_author(a, p) : ccr::kNoAuthor;
-      const long long aq = qin ? ccr::load_author(a, q) : ccr::kNoAuthor;
-      if (ap > aq) atomicCAS(code, 0, 4);
+      const int q = a.cand_idx[j];
+      if (q < 0 || q >= a.n_docs) continue;
+      int64_t i = j - 1;
+      while (i >= c0 && (a.cand_idx[i] < 0 || a.cand_idx[i] >= a.n_docs)) --i;
+      if (i >= c0 && ccr::load_author(a, a.cand_idx[i]) > ccr::load_author(a, q)) atomicCAS(code, 0, 4);
     }
   }
 }
@@ -301,9 +328,9 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return CCR_ERR_CUDA;
   if (need > free_b) return CCR_ERR_OOM;
 
-  ccr_docstore* s = new (std::nothrow) ccr_docstore();
+  ccr_docstore* s = new (std::nothrow) ccr_docstore();  // value-initialised: every field zero
   if (s == nullptr) return CCR_ERR_OOM;
-  std::memset(s, 0, sizeof(*s));
+  s->launches.store(0);
   s->desc = *d;
   s->doc_b = static_cast<int>(doc_b);
   s->edge_b = static_cast<int>(edge_b);
@@ -342,12 +369,13 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
     return st;
   }
   s->magic = kStoreMagic;
+  handle_add(s);
   *out = s;
   return CCR_OK;
 }
 
 ccr_status ccr_docstore_free(ccr_docstore* s) {
-  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  if (!good(s) || !handle_remove(s)) return CCR_ERR_BAD_HANDLE;  // of two racing frees only one gets past this
   DeviceScope scope(s->desc.device);
   s->magic = 0;
   cudaFree(s->doc_feats);
@@ -479,7 +507,7 @@ ccr_status ccr_docstore_set_tuning(ccr_docstore* s, const ccr_tuning* t) {
   return CCR_OK;
 }
 
-int64_t ccr_docstore_launch_count(const ccr_docstore* s) { return good(s) ? s->launches : -1; }
+int64_t ccr_docstore_launch_count(const ccr_docstore* s) { return good(s) ? s->launches.load() : -1; }
 
 ccr_status ccr_docstore_device_status(ccr_docstore* s, void* stream) {
   if (!good(s)) return CCR_ERR_BAD_HANDLE;
@@ -497,7 +525,7 @@ ccr_status ccr_docstore_device_status(ccr_docstore* s, void* stream) {
 }
 
 ccr_status ccr_idindex_free(ccr_idindex* ix) {
-  if (ix == nullptr || ix->magic != kIxMagic) return CCR_ERR_BAD_HANDLE;
+  if (!good(ix) || !handle_remove(ix)) return CCR_ERR_BAD_HANDLE;
   DeviceScope scope(ix->device);
   ix->magic = 0;
   for (int l = 0; l < ccr::kResolveMaxLevels; ++l) cudaFree(ix->level[l]);
@@ -569,20 +597,20 @@ ccr_status ccr_idindex_create(int32_t device, int64_t n_ids, const int64_t* sort
   ok = ok && cudaDeviceSynchronize() == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(ccr::resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   ccr::kResolveTopMax * 8 + 256) == cudaSuccess;
+  ix->magic = kIxMagic;
+  handle_add(ix);
   if (!ok) {
     cudaGetLastError();
-    ix->magic = kIxMagic;
     ccr_idindex_free(ix);
     return CCR_ERR_CUDA;
   }
-  ix->magic = kIxMagic;
   *out = ix;
   return CCR_OK;
 }
 
 ccr_status ccr_resolve_ids(const ccr_idindex* cix, int64_t n_queries, const int64_t* query_ids, int32_t* out_pos,
                            void* stream) {
-  if (cix == nullptr || cix->magic != kIxMagic) return CCR_ERR_BAD_HANDLE;
+  if (!good(cix)) return CCR_ERR_BAD_HANDLE;
   ccr_idindex* ix = const_cast<ccr_idindex*>(cix);  // only the launch counter changes
   if (n_queries < 0) return CCR_ERR_INVALID_ARG;
   if (n_queries == 0) return CCR_OK;
@@ -700,7 +728,7 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
                      const int64_t* edge_keys, const void* edge_feats, const int64_t* edge_offsets,
                      const int32_t* cand_idx, const int64_t* cand_offsets, const void* req_feats,
                      void* out_rows, uint8_t* out_mask, uint32_t flags, void* stream, int64_t n_max,
-                     const void* member_emb) {
+                     const void* member_emb, int* sched_override = nullptr) {
   if (!good(cs)) return CCR_ERR_BAD_HANDLE;
   ccr_docstore* s = const_cast<ccr_docstore*>(cs);  // only the launch counter and status words change
   if (n_req < 0 || total_cands < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
@@ -842,7 +870,10 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     const int n_res_auto = s->ws_resolvers > 0 ? s->ws_resolvers : 4;
     const long long n_tiles = (total_cands + a.tile - 1) / a.tile;
     const bool dynamic = !(flags & CCR_FLAG_STATIC_SPLIT) && n_tiles >= 2LL * blocks * n_res_auto;
-    if (dynamic) a.sched = s->status + 4 + 2 * static_cast<int>(s->launches % kSchedRegions);
+    // (the pair is drawn from the atomic launch counter, so host threads that join against one store at the
+    // same time never share a pair)
+    const int64_t seq = s->launches.fetch_add(1);
+    if (dynamic) a.sched = sched_override ? sched_override : s->status + 4 + 2 * static_cast<int>(seq % kSchedRegions);
     fn<<<static_cast<unsigned>(blocks), (n_str + n_res) * 32, smem, st>>>(a, n_str);
   } else {
     // persistent two-phase kernel: as many blocks as stay resident, each with at least 64 candidates (a single
@@ -858,8 +889,8 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     const long long most = (groups + 1) / 2;
     if (blocks > most) blocks = most;
     fn<<<static_cast<unsigned>(blocks), ccr::kThreads, smem, st>>>(a);
+    s->launches++;
   }
-  s->launches++;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
   return CCR_OK;
 }
@@ -1015,19 +1046,19 @@ ccr_status ccr_workspace_create(const ccr_docstore* s, int32_t max_req, int64_t 
   ok = ok && cudaMalloc(&w->req_feats, (max_req + 1) * (w->req_b ? w->req_b : 16)) == cudaSuccess;
   ok = ok && cudaMalloc(&w->out_rows, max_cands * w->out_b_max) == cudaSuccess;
   ok = ok && cudaMalloc(&w->out_mask, max_cands) == cudaSuccess;
+  w->magic = kWsMagic;
+  handle_add(w);
   if (!ok) {
     cudaGetLastError();
-    w->magic = kWsMagic;
     ccr_workspace_free(w);
     return CCR_ERR_OOM;
   }
-  w->magic = kWsMagic;
   *out = w;
   return CCR_OK;
 }
 
 ccr_status ccr_workspace_free(ccr_workspace* w) {
-  if (w == nullptr || w->magic != kWsMagic) return CCR_ERR_BAD_HANDLE;
+  if (!good(w) || !handle_remove(w)) return CCR_ERR_BAD_HANDLE;
   DeviceScope scope(w->device);
   w->magic = 0;
   cudaFree(w->edge_keys);
@@ -1043,7 +1074,7 @@ ccr_status ccr_workspace_free(ccr_workspace* w) {
 }
 
 ccr_status ccr_workspace_outputs(const ccr_workspace* w, void** rows, uint8_t** mask) {
-  if (w == nullptr || w->magic != kWsMagic) return CCR_ERR_BAD_HANDLE;
+  if (!good(w)) return CCR_ERR_BAD_HANDLE;
   if (rows) *rows = w->out_rows;
   if (mask) *mask = w->out_mask;
   return CCR_OK;
@@ -1055,7 +1086,7 @@ ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t 
                                const int64_t* cand_offsets, const void* req_feats, void* out_rows,
                                uint8_t* out_mask, uint32_t flags, void* stream) {
   if (!good(s)) return CCR_ERR_BAD_HANDLE;
-  if (w == nullptr || w->magic != kWsMagic || w->device != s->desc.device) return CCR_ERR_BAD_HANDLE;
+  if (!good(w) || w->device != s->desc.device) return CCR_ERR_BAD_HANDLE;
   if (n_req < 0 || total_cands < 0 || total_edges < 0 || max_edge_len < 0) return CCR_ERR_INVALID_ARG;
   if (n_req > w->max_req || total_cands > w->max_cands || total_edges > w->max_edges) return CCR_ERR_INVALID_ARG;
   if (n_req == 0 || total_cands == 0) return (n_req == 0 && total_cands != 0) ? CCR_ERR_INVALID_ARG : CCR_OK;
@@ -1142,7 +1173,15 @@ ccr_status ccr_join_payload_static(const ccr_docstore* s, int32_t n_req, int64_t
   if (!edge_offsets || !cand_offsets || !cand_idx || !out_rows || !out_mask) return CCR_ERR_INVALID_ARG;
   if (total_edges > 0 && (!edge_keys || !edge_feats)) return CCR_ERR_INVALID_ARG;
   if (s->req_b > 0 && !req_feats) return CCR_ERR_INVALID_ARG;
-  if (flags & CCR_FLAG_VALIDATE) return CCR_ERR_UNSUPPORTED;  // validation synchronises and uses the store's own words
+  if (flags & CCR_FLAG_VALIDATE) return CCR_ERR_UNSUPPORTED;  // validation synchronises the stream
+  if (flags & CCR_FLAG_COSINE) return CCR_ERR_INVALID_ARG;    // the member embeddings come through ccr_join_batch_ex
+  // the offsets are host-readable here, so the scalars that size the copies are checked against them
+  if (edge_offsets[0] < 0 || cand_offsets[0] != 0) return CCR_ERR_INVALID_ARG;
+  for (int32_t r = 0; r < n_req; ++r) {
+    if (edge_offsets[r + 1] < edge_offsets[r] || cand_offsets[r + 1] < cand_offsets[r]) return CCR_ERR_INVALID_ARG;
+    if (edge_offsets[r + 1] - edge_offsets[r] > max_edge_len) return CCR_ERR_INVALID_ARG;
+  }
+  if (edge_offsets[n_req] > total_edges || cand_offsets[n_req] != total_cands) return CCR_ERR_INVALID_ARG;
 
   // device copy of the payload, every piece on a 256-byte boundary behind the control words
   const size_t n_off = static_cast<size_t>(n_req) + 1;
@@ -1173,17 +1212,14 @@ ccr_status ccr_join_payload_static(const ccr_docstore* s, int32_t n_req, int64_t
     cudaGetLastError();
     return CCR_ERR_CUDA;
   }
-  // a view of the store whose status / scheduling words are the ones in the fixed block
-  ccr_docstore view = *s;
-  view.status = reinterpret_cast<int*>(base);
-  view.launches = 0;  // always the first pair of scheduling words
-  const ccr_status js = ccr_join_batch(&view, n_req, total_cands, max_edge_len,
-                                       reinterpret_cast<const int64_t*>(base + o_keys), base + o_feats,
-                                       reinterpret_cast<const int64_t*>(base + o_eo),
-                                       reinterpret_cast<const int32_t*>(base + o_idx),
-                                       reinterpret_cast<const int64_t*>(base + o_co),
-                                       s->req_b > 0 ? base + o_req : nullptr, out_rows, out_mask, flags, stream);
-  const_cast<ccr_docstore*>(s)->launches += view.launches;
+  // The kernel's scheduling words are the ones at the head of the fixed block; its status word stays the store's
+  // own (allocated when the store was created), so a bounded wait that runs out in this launch is reported by
+  // ccr_docstore_device_status like any other.
+  const ccr_status js = join_impl(s, n_req, total_cands, max_edge_len, reinterpret_cast<const int64_t*>(base + o_keys),
+                                  base + o_feats, reinterpret_cast<const int64_t*>(base + o_eo),
+                                  reinterpret_cast<const int32_t*>(base + o_idx),
+                                  reinterpret_cast<const int64_t*>(base + o_co), s->req_b > 0 ? base + o_req : nullptr,
+                                  out_rows, out_mask, flags, stream, 0, nullptr, reinterpret_cast<int*>(base));
   return js;
 }
 

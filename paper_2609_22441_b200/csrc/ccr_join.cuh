@@ -464,6 +464,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
         }
       } else {
         // 1. author ids of the sub-tile
+        int bad = 0;
         for (int base = 0; base < n; base += kThreads * kUnroll) {
           int idx[kUnroll];
 #pragma unroll
@@ -476,18 +477,21 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
             const int i = base + u * kThreads + tid;
             if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;
             if (i < n) {
+              bad |= idx[u] < 0;
               s_idx[i] = idx[u];
               s_auth[i] = idx[u] >= 0 ? load_author(a, idx[u]) : kNoAuthor;
             }
           }
         }
-        __syncthreads();
+        // An unresolved / out-of-range position has no author, so a sub-tile that holds one is not a sorted run
+        // (the sortedness promise is over author ids): it takes the per-candidate search below instead of the merge.
+        const bool any_invalid = __syncthreads_or(bad);
         // 2. the only keys this sub-tile can touch: window [lo, hi)
         const int64_t* gk = a.edge_keys + kb;
         const int lo = block_lower_bound(gk, K, s_auth[0]);
         const int hi = min(K, block_lower_bound(gk, K, s_auth[n - 1]) + 1);
         const int w = max(hi - lo, 0);
-        const bool windowed = (a.key_cap > 0) && (w <= a.key_cap) && (a.min_stride_log2 == 0);
+        const bool windowed = (a.key_cap > 0) && (w <= a.key_cap) && (a.min_stride_log2 == 0) && !any_invalid;
         // 3. stage the window (or, if it is too long, the request's keys as the binary-search mode does)
         if (!stage_keys(a, ssm, bar, phase, windowed ? kb + lo : kb, windowed ? w : K, false, keys, grp)) {
           give_up_wait(a, bar, phase);

@@ -162,6 +162,10 @@ struct NamedGroup {
 template <typename G>
 __device__ __forceinline__ bool stage_keys(const JoinArgs& a, const SearchSmem& sm, uint32_t bar, uint32_t& phase,
                                            long long kb, int K, bool index, StagedKeys& st, const G& g) {
+  // The key area may hold ordinary (generic-proxy) stores of an earlier staging — sampled keys, the unaligned
+  // head / tail key — at addresses the bulk copy below writes through the async proxy: every thread orders its
+  // own earlier stores against the async proxy before the barrier that precedes the copy.
+  fence_proxy_async_smem();
   g.sync();
   int64_t* skeys = sm.keys;
   st.gk = a.edge_keys + kb;

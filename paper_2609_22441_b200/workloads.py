@@ -246,8 +246,33 @@ def _normal_block(rng: np.random.Generator, rows: int, dim: int, dtype) -> np.nd
     return out
 
 
-def make_viewer(rng: np.random.Generator, n_authors: int, k: int, edge_dim: int, edge_dtype):
-    keys = sorted_unique_sample(rng, n_authors, k)
+KEY_DISTRIBUTIONS = ("uniform", "clustered", "pareto")
+KEY_OUTLIER_BASE = np.iinfo(np.int64).max - (1 << 20)  # the far outlier of a "clustered" list lies above this
+
+
+def make_keys(rng: np.random.Generator, n_authors: int, k: int, key_dist: str = "uniform") -> np.ndarray:
+    """k ascending unique non-negative ids.
+    uniform   : a sorted unique sample of [0, n_authors) — what the benchmark configurations describe.
+    clustered : member ids handed out in blocks: k - 1 consecutive ids from a random base plus one id near the top of
+                the int64 range (an old or foreign account), so a linear map of the key range to buckets puts
+                the whole block into one bucket.
+    pareto    : heavy-tailed gaps (1 + floor of Pareto(0.5) draws scaled by 8, capped at 2^40): dense runs
+                separated by a few huge jumps, so nearly every key shares a linear bucket with hundreds of others."""
+    k = int(k)
+    if key_dist == "uniform" or k < 2:
+        return sorted_unique_sample(rng, n_authors, k)
+    if key_dist == "clustered":
+        base = int(rng.integers(0, max(1, n_authors - k)))
+        far = KEY_OUTLIER_BASE + int(rng.integers(0, 1 << 20))
+        return np.concatenate([base + np.arange(k - 1, dtype=np.int64), np.array([far], dtype=np.int64)])
+    if key_dist == "pareto":
+        gaps = 1 + np.minimum(np.floor(rng.pareto(0.5, size=k) * 8.0), float(1 << 40)).astype(np.int64)
+        return int(rng.integers(0, max(1, n_authors))) + np.cumsum(gaps)
+    raise ValueError("key_dist must be one of %s" % (KEY_DISTRIBUTIONS,))
+
+
+def make_viewer(rng: np.random.Generator, n_authors: int, k: int, edge_dim: int, edge_dtype, key_dist: str = "uniform"):
+    keys = make_keys(rng, n_authors, k, key_dist)
     feats = rng.random(size=(len(keys), edge_dim), dtype=np.float32).astype(edge_dtype)
     return keys, feats
 
@@ -323,6 +348,7 @@ def make_workload(
     gen_doc_feats: bool = True,
     edge_dtype=np.float16,
     req_dtype=np.float32,
+    key_dist: str = "uniform",
 ) -> Workload:
     """One store and one ragged batch of `n_req` requests (draw order in the module docstring)."""
     rng = np.random.default_rng(seed)
@@ -333,7 +359,7 @@ def make_workload(
     keys_l: List[np.ndarray] = []
     feats_l: List[np.ndarray] = []
     for r in range(n_req):
-        k, f = make_viewer(rng, n_authors, int(ks[r]), edge_dim, edge_dtype)
+        k, f = make_viewer(rng, n_authors, int(ks[r]), edge_dim, edge_dtype, key_dist)
         keys_l.append(k)
         feats_l.append(f)
     req_feats = None
@@ -358,6 +384,7 @@ def make_workload(
         "edge_len_min": int(ks.min()) if n_req else 0,
         "edge_len_max": int(ks.max()) if n_req else 0,
         "edge_len_mean": float(ks.mean()) if n_req else 0.0,
+        "key_dist": key_dist,
     }
     return Workload(name=name, seed=int(seed), store=store, batch=batch, meta=meta)
 
@@ -423,7 +450,7 @@ def config0(seed: Optional[int] = None, n_docs: int = 100_000, n_cand: int = 20_
 
 
 def config1(seed: Optional[int] = None, n_docs: int = 1_000_000, n_req: int = 64, n_cand: int = 30_000,
-            second_degree: bool = False, edge_lo: int = 50, edge_hi: int = 5000) -> Workload:
+            second_degree: bool = False, edge_lo: int = 50, edge_hi: int = 5000, key_dist: str = "uniform") -> Workload:
     """Batched first-degree join: 1M docs x 128 fp16, A = 5M, 64 requests, K ~ clip(Zipf(1.2), 50, 5000)
     x 32 fp16, N = 30k unsorted, 16 fp32 request features; match 0.5 (limited by the pool size)."""
     return make_workload(
@@ -432,13 +459,13 @@ def config1(seed: Optional[int] = None, n_docs: int = 1_000_000, n_req: int = 64
         n_docs=n_docs, n_authors=5 * n_docs, doc_dim=128, doc_dtype=np.float16, edge_dim=32, req_dim=16,
         n_req=n_req, edge_len=zipf_clipped_lengths(edge_lo, edge_hi, 1.2), n_cand=n_cand, match=0.5,
         max_actors=MAX_ACTOR_SLOTS if second_degree else 0,
-        reduce_sum_mask=SUM_DIMS_16_31 if second_degree else 0, n_pools=n_req,
+        reduce_sum_mask=SUM_DIMS_16_31 if second_degree else 0, n_pools=n_req, key_dist=key_dist,
     )
 
 
 def config3(seed: Optional[int] = None, n_docs: int = 50_000_000, n_req: int = 256, n_cand: int = 50_000,
             edge_lo: int = 10, edge_hi: int = 20_000, gen_doc_feats: bool = False,
-            extra_pools: int = 160) -> Workload:
+            extra_pools: int = 160, key_dist: str = "uniform") -> Workload:
     """Production-scale store: 50M docs x 128 fp16 (+ author and engager ids), 256 requests,
     K log-uniform in [10, 20000] x 64 fp16, N = 50k, match 0.7, no request features.  The doc
     feature matrix (12.8 GB) is normally produced in chunks by `doc_feats_chunk`."""
@@ -447,7 +474,7 @@ def config3(seed: Optional[int] = None, n_docs: int = 50_000_000, n_req: int = 2
         n_docs=n_docs, n_authors=n_docs, doc_dim=128, doc_dtype=np.float16, edge_dim=64, req_dim=0,
         n_req=n_req, edge_len=log_uniform_lengths(edge_lo, edge_hi), n_cand=n_cand, match=0.7,
         max_actors=MAX_ACTOR_SLOTS, reduce_sum_mask=SUM_DIMS_16_31 | (SUM_DIMS_16_31 << 32),
-        n_pools=n_req + extra_pools, gen_doc_feats=gen_doc_feats,
+        n_pools=n_req + extra_pools, gen_doc_feats=gen_doc_feats, key_dist=key_dist,
     )
 
 

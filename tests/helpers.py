@@ -79,3 +79,30 @@ def sampled_oracle_rows(wl, kept, J, first_degree_only):
         actor_ids=None if s.actor_ids is None else s.actor_ids[safe],
         actor_types=None if s.actor_types is None else s.actor_types[safe],
         reduce_sum_mask=s.reduce_sum_mask, first_degree_only=first_degree_only, n_threads=4)
+
+
+def request_oracle_rows(wl, full, r, first_degree_only, cand_idx=None):
+    """Oracle rows and mask of ALL candidates of request r of a production-scale workload whose feature matrix
+    lives on the device only (`full`: the generator's output, i.e. an input, as a device tensor).  The rows of
+    the request's docs are gathered from that input matrix to the host and the request is re-expressed as a
+    compact single-request problem (store = those rows, candidates = 0..n-1) for the unmodified oracle."""
+    import torch
+
+    from oracle import oracle
+
+    s, b = wl.store, wl.batch
+    cand_idx = b.cand_idx if cand_idx is None else cand_idx
+    c0, c1 = int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])
+    e0, e1 = int(b.edge_offsets[r]), int(b.edge_offsets[r + 1])
+    docs = cand_idx[c0:c1].astype(np.int64)
+    ok = (docs >= 0) & (docs < s.n_docs)
+    safe = np.where(ok, docs, 0)
+    feats = full.index_select(0, torch.from_numpy(safe).to(full.device)).cpu().numpy()
+    n = c1 - c0
+    return oracle.join(
+        feats, s.author_ids[safe], b.edge_keys[e0:e1], b.edge_feats[e0:e1], np.array([0, e1 - e0], np.int64),
+        np.where(ok, np.arange(n), -1).astype(np.int32), np.array([0, n], np.int64),
+        req_feats=None if b.req_feats is None else b.req_feats[r:r + 1],
+        actor_ids=None if s.actor_ids is None else s.actor_ids[safe],
+        actor_types=None if s.actor_types is None else s.actor_types[safe],
+        reduce_sum_mask=s.reduce_sum_mask, first_degree_only=first_degree_only, n_threads=4)

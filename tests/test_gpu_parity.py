@@ -198,6 +198,57 @@ def test_edge_list_lengths_around_every_path_threshold(B, k):
         store.free()
 
 
+@pytest.mark.parametrize("key_dist", ["clustered", "pareto"])
+@pytest.mark.parametrize("k", [37, 4096, 13_000, 20_000])
+def test_clustered_and_heavy_tailed_keys_through_every_search_path(B, key_dist, k):
+    """Ids that a linear map of the key range cannot spread: a block of consecutive ids plus one id near the top
+    of the int64 range (the whole block shares one bucket of such a map), and heavy-tailed gaps (dense runs
+    separated by huge jumps).  Candidates hit the block's first and last keys, the far key, ids just outside
+    the block and inside the gaps; two requests, so the second key list starts at an odd offset when k is odd."""
+    rng = np.random.default_rng(1000 + k)
+    n_docs = 40_000
+    keys1 = W.make_keys(rng, 5_000_000, k, key_dist)
+    keys2 = W.make_keys(rng, 5_000_000, k - 1, key_dist)
+    near = np.concatenate([keys1, keys1 + 1, keys1 - 1, keys2, keys2[-1:] + 1, keys1[:1] - 1])
+    authors = np.where(rng.random(n_docs) < 0.8, near[rng.integers(0, len(near), size=n_docs)],
+                       rng.integers(0, 5_000_000, size=n_docs)).astype(np.int64)
+    authors[:4] = [keys1[0], keys1[-1], keys1[-2], max(int(keys1[0]) - 1, 0)]
+    cand = [np.concatenate([np.arange(4), rng.integers(0, n_docs, size=6000)]), rng.integers(0, n_docs, size=3500)]
+    wl = _manual([keys1, keys2], cand, authors, edge_dim=32)
+    _, mask = _check(B, wl, _variants(B), tunings=((0, 0), (256, 1000)))
+    assert list(mask[:3]) == [1, 1, 1] and 0.1 < mask.mean() < 0.95
+    _check(B, W.sort_candidates_by_author(wl), [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED)])
+
+
+@pytest.mark.parametrize("key_dist", ["clustered", "pareto"])
+def test_batched_shape_with_non_uniform_keys_first_and_second_degree(B, key_dist):
+    for second in (False, True):
+        wl = W.config1(n_docs=200_000, n_req=16, n_cand=12_000, second_degree=second, key_dist=key_dist)
+        _, mask = _check(B, wl, [("auto", 0), ("2phase", B.CCR_FLAG_TWO_PHASE), ("sampled", B.CCR_FLAG_FORCE_SAMPLED),
+                                 ("global", B.CCR_FLAG_FORCE_GLOBAL)])
+        assert 0.2 < (mask & 1).mean() < 0.7
+
+
+def test_sorted_candidates_with_unresolved_positions_inside(B):
+    """CCR_FLAG_CANDS_SORTED binds the resolved candidates only: -1 and out-of-range positions sit at the start,
+    in the middle and at the end of sorted requests, alone and in runs, at sub-tile boundaries too."""
+    wl = W.sort_candidates_by_author(W.config1(n_docs=60_000, n_req=5, n_cand=7_000))
+    b = wl.batch
+    rng = np.random.default_rng(11)
+    cand = b.cand_idx.copy()
+    for r in range(b.n_req):
+        c0, c1 = int(b.cand_offsets[r]), int(b.cand_offsets[r + 1])
+        holes = np.concatenate([rng.integers(c0, c1, size=40), [c0, c1 - 1, c0 + 1023, c0 + 1024, c0 + 2047],
+                                np.arange(c0 + 3000, c0 + 3040)])
+        cand[holes] = np.where(rng.random(len(holes)) < 0.5, -1, wl.store.n_docs + 5)
+    cand[int(b.cand_offsets[3]):int(b.cand_offsets[3]) + 1500] = -1  # a whole sub-tile without a single author
+    wl2 = W.Workload("sorted+holes", 0, wl.store, W.Batch(**{**b.__dict__, "cand_idx": cand}))
+    _check(B, wl2, [("merge", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE), ("ws+sorted", B.CCR_FLAG_CANDS_SORTED),
+                    ("merge+global", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE | B.CCR_FLAG_FORCE_GLOBAL),
+                    ("merge+validate", B.CCR_FLAG_CANDS_SORTED | B.CCR_FLAG_TWO_PHASE | B.CCR_FLAG_VALIDATE)],
+           tunings=((0, 0), (256, 64)))
+
+
 def test_many_small_requests_in_one_launch(B):
     # hundreds of requests of 0..40 candidates: most blocks serve many request segments
     wl = tiny_workload(7, n_docs=3000, alphabet=900, n_req=700, kmax=300, nmax=40, second=False, req_dim=4,
@@ -335,6 +386,59 @@ def test_argument_errors_on_a_live_store(B):
     h = ctypes.c_void_p(store.handle.value)
     store.free()
     assert L.ccr_docstore_free(h) == B.CCR_ERR_BAD_HANDLE  # double free
+
+
+def test_store_larger_than_device_memory_is_refused_before_any_allocation(B):
+    free0 = torch.cuda.mem_get_info()[0]
+    with pytest.raises(B.CcrError) as e:
+        B.Docstore(2_000_000_000, 128, np.float16, 32)  # 512 GB of rows
+    assert e.value.status == B.CCR_ERR_OOM
+    with pytest.raises(B.CcrError) as e:
+        B.Docstore(1_500_000_000, 128, np.float16, 32, max_actors=4)
+    assert e.value.status == B.CCR_ERR_OOM
+    assert abs(torch.cuda.mem_get_info()[0] - free0) < (64 << 20)  # nothing was allocated and kept
+
+
+def test_joins_from_two_host_threads_on_one_store(B):
+    """The launch counter is atomic and hands every launch its own scheduling words: two host threads join
+    against one store at the same time, each on its own stream and into its own buffers."""
+    import threading
+
+    wl = W.config1(n_docs=200_000, n_req=16, n_cand=20_000)
+    b = wl.batch
+    store = B.store_from_workload(wl)
+    db = B.DeviceBatch(b)
+    want_rows, want_mask = oracle.join_workload(wl, n_threads=4)
+    n_calls = 40
+    outs = [[(torch.full((b.total_cands, 384), 0x11, dtype=torch.uint8, device="cuda"),
+              torch.full((b.total_cands,), 0x11, dtype=torch.uint8, device="cuda")) for _ in range(3)] for _ in range(2)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    before = store.launch_count()
+    errors = []
+
+    def worker(t):
+        try:
+            for i in range(n_calls):
+                rows, mask = outs[t][i % 3]
+                B.ccr_join_batch(store, db.n_req, b.total_cands, db.max_edge_len, db.edge_keys, db.edge_feats,
+                                 db.edge_offsets, db.cand_idx, db.cand_offsets, db.req_feats, rows, mask, 0, streams[t])
+        except Exception as exc:  # pragma: no cover
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(2)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    torch.cuda.synchronize()
+    assert not errors
+    assert store.launch_count() == before + 2 * n_calls  # no increment was lost
+    for t in range(2):
+        for rows, mask in outs[t]:
+            assert np.array_equal(mask.cpu().numpy(), want_mask) and np.array_equal(rows.cpu().numpy(), want_rows)
+    assert store.device_status() == B.CCR_OK
+    store.free()
 
 
 def test_expired_device_wait_is_reported_and_the_store_stays_usable(B):

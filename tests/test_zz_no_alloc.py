@@ -3,14 +3,17 @@
 Such callers (a request handler inside a server that has already given all device memory to its own pool, or
 one that cannot afford the device-wide stall of cudaMalloc / cudaFree) hand the request payload over in host
 memory; the library copies it into a fixed 16 MiB device block that is part of its image and launches the
-same kernel as ccr_join_batch.  The check: byte-identical rows and masks to ccr_join_batch (the existing
-entry, device inputs) on two different batches called back to back — the second is smaller, so stale bytes
-of the first would show — plus the refusal of a payload that does not fit the block.
+same kernel as ccr_join_batch.  The checks: rows and masks byte-identical to the CPU oracle and to
+ccr_join_batch (the existing entry, device inputs) on two different batches called back to back — the second is
+smaller, so stale bytes of the first would show —, no change of the device's free memory across the calls, the
+refusal of a payload that does not fit the block, the refusal of scalars that disagree with the host offsets,
+and that a device-side status raised while the entry is in use is still reported through the store.
 
 Collected last on purpose: if it fails, a run that stops at the first failure has already run everything else."""
 import numpy as np
 import pytest
 
+from oracle import oracle
 from paper_2609_22441_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -45,25 +48,55 @@ def test_static_payload_entry_matches_join_batch_twice_in_a_row():
     store = B.store_from_workload(first)
     assert B.lib().ccr_static_payload_capacity() == (16 << 20) - 256
     try:
+        # first use on the device: looks up the block's address (and makes sure the library image is loaded)
+        hb = first.batch
+        warm = [_pinned(hb.edge_keys), _pinned(hb.edge_feats.view(np.uint8)), _pinned(hb.edge_offsets),
+                _pinned(hb.cand_idx), _pinned(hb.cand_offsets), _pinned(hb.req_feats.view(np.uint8))]
+        r0 = torch.empty((hb.total_cands, store.out_row_bytes()), dtype=torch.uint8, device="cuda")
+        m0 = torch.empty((hb.total_cands,), dtype=torch.uint8, device="cuda")
+        B.ccr_join_payload_static(store, hb.n_req, hb.total_cands, hb.max_edge_len, len(hb.edge_keys), *warm, r0, m0)
+        torch.cuda.synchronize()
         for wl in (first, second):
             b = wl.batch
+            oracle_rows, oracle_mask = oracle.join_workload(wl, n_threads=4)
             want_rows, want_mask = B.join_batch(store, B.DeviceBatch(b))
             torch.cuda.synchronize()
             rows = torch.full_like(want_rows, 0x5A)
             mask = torch.full_like(want_mask, 0x5A)
             host = [_pinned(b.edge_keys), _pinned(b.edge_feats.view(np.uint8)), _pinned(b.edge_offsets),
                     _pinned(b.cand_idx), _pinned(b.cand_offsets), _pinned(b.req_feats.view(np.uint8))]
+            torch.cuda.synchronize()
             before = store.launch_count()
+            free_before = torch.cuda.mem_get_info()[0]
             B.ccr_join_payload_static(store, b.n_req, b.total_cands, b.max_edge_len, len(b.edge_keys), *host, rows, mask)
             torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before  # the call took no device memory
             assert store.launch_count() == before + 1
+            assert np.array_equal(mask.cpu().numpy(), oracle_mask)
+            assert np.array_equal(rows.cpu().numpy(), oracle_rows)
             assert torch.equal(mask, want_mask)
             assert torch.equal(rows, want_rows)
         # a payload that cannot fit the fixed block is refused before anything is enqueued
+        big_co = _pinned(np.array([0, 5_000_000], np.int64))
+        one_eo = _pinned(np.array([0, 10], np.int64))
         with pytest.raises(B.CcrError) as e:
-            B.ccr_join_payload_static(store, 1, 5_000_000, 10, 10, host[0], host[1], host[2], host[3], host[4], host[5],
+            B.ccr_join_payload_static(store, 1, 5_000_000, 10, 10, host[0], host[1], one_eo, host[3], big_co, host[5],
                                       rows, mask)
         assert e.value.status == B.CCR_ERR_UNSUPPORTED
+        # scalars that disagree with the (host-readable) offsets are refused as well
+        with pytest.raises(B.CcrError) as e:
+            B.ccr_join_payload_static(store, b.n_req, b.total_cands - 1, b.max_edge_len, len(b.edge_keys), *host, rows, mask)
+        assert e.value.status == B.CCR_ERR_INVALID_ARG
+        with pytest.raises(B.CcrError) as e:
+            B.ccr_join_payload_static(store, b.n_req, b.total_cands, b.max_edge_len, len(b.edge_keys) - 1, *host, rows, mask)
+        assert e.value.status == B.CCR_ERR_INVALID_ARG
         assert store.device_status() == B.CCR_OK
+        # the entry keeps the store's own status word: a wait that ran out (here: the self-test's) is still
+        # reported after a static call, not cleared by it
+        store.selftest_wait()
+        B.ccr_join_payload_static(store, b.n_req, b.total_cands, b.max_edge_len, len(b.edge_keys), *host, rows, mask)
+        assert store.device_status() == B.CCR_ERR_DEVICE_WAIT
+        assert store.device_status() == B.CCR_OK
+        assert torch.equal(rows, want_rows) and torch.equal(mask, want_mask)
     finally:
         store.free()
