@@ -42,9 +42,23 @@ UNIT = "candidates/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
-# summarised under profiles/ (bytes per launch; None until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {"config1": 1184300000, "config2b": 1454900000}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic_per_launch.txt")
+
+
+def ncu_traffic(workload: str, flags: int):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on `workload`, as recorded
+    from an ncu capture in profiles/ncu_dram_traffic_per_launch.txt (columns: workload, flags, kernel, bytes per
+    launch, commit the capture was taken at, summary file).  Returns (bytes, record) or (None, None) when no
+    capture of that workload / flag set is on record."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                line = line.split("#", 1)[0].split()
+                if len(line) >= 6 and line[0] == workload and int(line[1]) == int(flags):
+                    return int(line[3]), {"kernel": line[2], "commit": line[4], "summary": line[5]}
+    except (OSError, ValueError):
+        pass
+    return None, None
 
 
 def parse_args():
@@ -73,24 +87,28 @@ def parse_args():
                    help="time the padded batch layout: ccr_compact_valid + ccr_join_batch_padded into T[n_req, n_max]")
     p.add_argument("--cosine", action="store_true",
                    help="add the derived cosine section (3 medoids x 50 values against elements 8..57 of the document row)")
+    p.add_argument("--keys", default="uniform", choices=["uniform", "clustered", "pareto"],
+                   help="how the viewers' author ids are spread (configs 1 and 2b): uniform over the id range (what the benchmark "
+                        "configurations describe), clustered (a block of consecutive ids plus one far outlier) or pareto "
+                        "(heavy-tailed gaps)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--timed-only", action="store_true",
                    help="only warm-up and the timed region (for profiler captures): no sustain loop, e2e, latency or CPU legs")
     return p.parse_args()
 
 
-def make_workload(config: str, rank: int, c3_docs: int = 50_000_000, c3_requests: int = 256):
+def make_workload(config: str, rank: int, c3_docs: int = 50_000_000, c3_requests: int = 256, keys: str = "uniform"):
     """(workload, extra join flags) of a benchmark configuration; rank shifts the seed so replicas differ."""
     from paper_2609_22441_b200 import binding as B
     from paper_2609_22441_b200 import replicas
     from paper_2609_22441_b200 import workloads as W
 
     if config == "1":
-        return W.config1(seed=W.config_seed(1, 0) + replicas.rank_seed_offset(rank)), 0
+        return W.config1(seed=W.config_seed(1, 0) + replicas.rank_seed_offset(rank), key_dist=keys), 0
     if config == "2b":
-        return W.config1(seed=W.config_seed(2, 1) + replicas.rank_seed_offset(rank), second_degree=True), 0
+        return W.config1(seed=W.config_seed(2, 1) + replicas.rank_seed_offset(rank), second_degree=True, key_dist=keys), 0
     wl = W.config3(seed=W.config_seed(3, 0) + replicas.rank_seed_offset(rank), n_docs=c3_docs, n_req=c3_requests,
-                   extra_pools=160 if c3_docs >= 50_000_000 else 0)
+                   extra_pools=160 if c3_docs >= 50_000_000 else 0, key_dist=keys)
     if config == "3":
         return wl, B.CCR_FLAG_FIRST_DEGREE_ONLY
     if config == "3b":  # sorted candidates: default kernel; add --flags 128 for the merge-path kernel
@@ -188,6 +206,80 @@ class ClockSampler:
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
 
 
+class NvmlClock:
+    """SM clock samples straight from NVML (read-only), every few milliseconds in a thread: the latency sweep's
+    cells last tens of milliseconds, too short for nvidia-smi's sampling loop."""
+
+    def __init__(self, gpu_index: int, period_s: float = 0.005):
+        self.samples = []
+        self._stop = threading.Event()
+        self.thread = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            # NVML orders devices by PCI bus id, CUDA_VISIBLE_DEVICES may remap: resolve through the CUDA device's bus id
+            import torch
+
+            bus = torch.cuda.get_device_properties(gpu_index).pci_bus_id if hasattr(
+                torch.cuda.get_device_properties(gpu_index), "pci_bus_id") else None
+            h = None
+            if bus is not None:
+                for i in range(pynvml.nvmlDeviceGetCount()):
+                    hi = pynvml.nvmlDeviceGetHandleByIndex(i)
+                    if pynvml.nvmlDeviceGetPciInfo(hi).bus == bus:
+                        h = hi
+                        break
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(gpu_index)
+
+            def loop():
+                while not self._stop.is_set():
+                    try:
+                        self.samples.append((time.time(), pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                    except Exception:
+                        return
+                    time.sleep(period_s)
+
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.thread = None
+
+    def median_mhz(self, t0: float, t1: float):
+        v = [c for t, c in self.samples if t0 <= t <= t1]
+        return float(np.median(v)) if v else None
+
+    def stop(self):
+        self._stop.set()
+
+
+def sustain(fn, sync, t_start: float, seconds: float = 1.5):
+    """Keep the measured kernels running until the loaded window is long enough for clock samples."""
+    while time.time() - t_start < seconds:
+        for i in range(20):
+            fn(i)
+        sync()
+
+
+def input_checksums(wl):
+    """64-bit digests of the generated inputs (same seed -> same digests on every box)."""
+    from paper_2609_22441_b200 import workloads as W
+
+    s, b = wl.store, wl.batch
+    return {"author_ids": W.checksum64(s.author_ids), "doc_feats": W.checksum64(s.doc_feats) if s.doc_feats is not None else "device-generated",
+            "edge_keys": W.checksum64(b.edge_keys), "edge_feats": W.checksum64(b.edge_feats), "cand_idx": W.checksum64(b.cand_idx),
+            "cand_offsets": W.checksum64(b.cand_offsets)}
+
+
+def config_dict(wl, bc, flags: int, args, world: int, n_buf: int = 2):
+    """The `config` object of the JSON line; both arms (ours, reference) print the same one for the same run."""
+    return {"workload": workload_label(wl), "l2": "inputs and outputs of a step (%.2f GB) exceed the 126 MB L2; "
+            "outputs rotate over %d buffers" % (bc["compulsory"] / 1e9, n_buf),
+            "match_rate": bc["match_rate"], "seed": wl.seed, "tile": args.tile or "default", "key_cap": args.key_cap or "default",
+            "flags": flags, "replicas": world, "keys": args.keys}
+
+
 def measured_peak_gbs():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -259,7 +351,15 @@ def latency_sweep(args, B, device: int):
     per_k = 32
     tpl = W.make_latency_templates(s, W.config_seed(4), k_values, per_k, first_pool=256, n_pools=wl.meta["n_pools"],
                                    forced_per_template=70_000, edge_dim=wl.batch.edge_dim, n_authors=wl.meta["n_authors"])
-    store, _, _ = B.store_from_generated(wl, device=device)
+    store, _, full = B.store_from_generated(wl, device=device, keep_all=True)  # `full`: the input matrix, for the oracle's rows
+    from oracle import oracle
+
+    oracle.build()
+    cores = host_cores()
+    n_oracle = 0 if args.no_cpu_baseline else min(100, args.sweep_requests)
+    sampler, fine = ClockSampler(device), NvmlClock(device)
+    t_sweep0 = time.time()
+    oracle_cands, oracle_s = 0, 0.0
     flags = B.CCR_FLAG_FIRST_DEGREE_ONLY | args.flags
     out_b = store.out_row_bytes(flags)
     rows = torch.empty((max(n_values), out_b), dtype=torch.uint8, device=dev)
@@ -287,7 +387,10 @@ def latency_sweep(args, B, device: int):
                 cand[i] = row
             cand_dev = torch.from_numpy(cand).to(dev)
             ev, wall = [], []
+            t_cell0 = None
             for i in range(-50, n_per_cell):  # 50 warm-up requests per cell
+                if i == 0:
+                    t_cell0 = time.time()
                 j = i % n_per_cell
                 keys, feats, eo = dev_tpl[j % per_k]
                 a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -301,16 +404,49 @@ def latency_sweep(args, B, device: int):
                 if i >= 0:
                     ev.append(a.elapsed_time(z))
                     wall.append((t1 - t0) * 1e3)
+            t_cell1 = time.time()
             ev.sort()
             wall.sort()
             q = lambda v, p: float(v[max(0, int(np.ceil(p * len(v))) - 1)])
-            cells.append({"candidates": n, "edge_len": k, "event_ms_p50": q(ev, 0.5), "event_ms_p99": q(ev, 0.99),
-                          "host_ms_p50": q(wall, 0.5), "host_ms_p99": q(wall, 0.99)})
+            mhz = fine.median_mhz(t_cell0, t_cell1)
+            cell = {"candidates": n, "edge_len": k, "event_ms_p50": q(ev, 0.5), "event_ms_p99": q(ev, 0.99),
+                    "host_ms_p50": q(wall, 0.5), "host_ms_p99": q(wall, 0.99), "sm_mhz": mhz,
+                    # time x clock: device cycles of the median request, comparable across runs at different clocks
+                    "event_p50_kcycles": None if mhz is None else q(ev, 0.5) * mhz}
             t_all += sum(ev) * 1e-3
             c_all += n * n_per_cell
             del cand_dev
+            # the oracle on the first requests of the cell, one request per call: its rows come from the generated
+            # input matrix, the request becomes a compact problem (store = the request's rows) as in the parity tests
+            o1, oT = [], []
+            for i in range(n_oracle):
+                t = tpl[k][i % per_k]
+                docs = torch.from_numpy(cand[i].astype(np.int64)).to(dev)
+                rows_h = full.index_select(0, docs).cpu().numpy()
+                auth_h = s.author_ids[cand[i].astype(np.int64)]
+                a_ = (rows_h, auth_h, t.keys, t.feats, np.array([0, len(t.keys)], np.int64), np.arange(n, dtype=np.int32),
+                      np.array([0, n], np.int64))
+                for threads, acc in ((1, o1), (cores, oT)):
+                    t0 = time.perf_counter()
+                    oracle.join(*a_, n_threads=threads)
+                    acc.append((time.perf_counter() - t0) * 1e3)
+                oracle_cands += n
+                oracle_s += oT[-1] * 1e-3
+            if o1:
+                o1.sort()
+                oT.sort()
+                cell.update({"oracle_ms_p50_1_thread": q(o1, 0.5), "oracle_ms_p99_1_thread": q(o1, 0.99),
+                             "oracle_ms_p50_all_cores": q(oT, 0.5), "oracle_ms_p99_all_cores": q(oT, 0.99)})
+            cells.append(cell)
     if store.device_status() != B.CCR_OK:
         raise SystemExit("device status not clean after the sweep")
+    sampler.stop()
+    fine.stop()
+    cpu_baseline = None
+    if oracle_cands:
+        cpu_baseline = {"value": oracle_cands / oracle_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": "the first %d requests of each of the 25 cells, one request per call, against a compacted copy of "
+                                  "the request's document rows; per-cell p50 / p99 in latency_sweep (1 thread and all cores)" % n_oracle}
     print(json.dumps({
         "metric": METRIC, "value": c_all / t_all, "unit": UNIT, "n_gpus": 1, "steps": n_per_cell * len(cells), "warmup": 50,
         "ms_per_step": 1e3 * t_all / (n_per_cell * len(cells)), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -319,6 +455,8 @@ def latency_sweep(args, B, device: int):
                    "384-byte rows, %d requests per cell (32 viewer templates per edge-list length, 70%% forced matches)" % n_per_cell,
                    "flags": flags},
         "latency_sweep": cells, "gpu_launches": int(store.launch_count() - launches0),
+        "clocks": sampler.summary(t_sweep0, time.time()), "cpu_baseline": cpu_baseline,
+        "input_checksums": input_checksums(wl),
         "paper_context": "the paper quotes 5-10 ms for its join on unstated Hopper-class hardware (abstract)",
     }))
     store.free()
@@ -344,6 +482,8 @@ def resolve_bench(args, B, device: int):
     rng = np.random.default_rng(W.config_seed(5, 1))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     cells = []
+    sampler = ClockSampler(device)
+    t_leg0 = time.time()
     for b in (1, 8, 64):
         nq = b * 30_000
         present = host[rng.integers(0, n, size=nq)]
@@ -368,6 +508,8 @@ def resolve_bench(args, B, device: int):
             z2.record()
             torch.cuda.synchronize(dev)
             warm.append(a2.elapsed_time(z2))
+        t_busy = time.time()
+        sustain(lambda i: ix.resolve(q_dev, out), lambda: torch.cuda.synchronize(dev), t_busy, 0.7)
         t0 = time.perf_counter()
         want = oracle.resolve_ids(host, q)
         t_cpu = time.perf_counter() - t0
@@ -378,7 +520,11 @@ def resolve_bench(args, B, device: int):
                       "oracle_ms_1_core": 1e3 * t_cpu, "matches_oracle": bool(np.array_equal(out.cpu().numpy(), want)),
                       "found_fraction": float((want >= 0).mean())})
     head = cells[1]
+    sampler.stop()
     print(json.dumps({
+        "clocks": sampler.summary(t_leg0, time.time()),
+        "cpu_baseline": {"value": head["ids"] / (head["oracle_ms_1_core"] * 1e-3), "unit": "ids/s", "cores": 1, "kind": "oracle",
+                         "sample": "the headline batch (8 x 30,000 ids) once"},
         "metric": "document_ids_resolved_per_sec", "value": head["ids_per_s"], "unit": "ids/s", "n_gpus": 1, "steps": 100,
         "warmup": 5, "ms_per_step": head["ms_p50_L2_flushed"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int64", "data": "synthetic",
@@ -429,6 +575,8 @@ def ingest_bench(args, B, device: int):
         return a, z
 
     quick = args.timed_only  # profiler captures: a handful of launches per cell
+    sampler = ClockSampler(device)
+    t_leg0 = time.time()
     n_join = 3 if quick else 300
     for i in range(1 if quick else 5):
         join(i)
@@ -478,7 +626,9 @@ def ingest_bench(args, B, device: int):
     if store.device_status() != B.CCR_OK:
         raise SystemExit("device status not clean")
     head = cells[0]
+    sampler.stop()
     print(json.dumps({
+        "clocks": sampler.summary(t_leg0, time.time()),
         "metric": "rows_upserted_per_sec", "value": head["upsert_alone_rows_per_s"], "unit": "rows/s", "n_gpus": 1, "steps": 400,
         "warmup": 5, "ms_per_step": head["upsert_alone_us"] * 1e-3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
@@ -552,6 +702,8 @@ def flow_bench(args, B, device: int):
         return a.elapsed_time(z) * 1e3 / n
 
     n = max(20, args.steps // 10)
+    sampler = ClockSampler(device)
+    t_leg0 = time.time()
     for fn in stages.values():  # once in order: every stage has real inputs
         fn(0)
     per_stage = {name: timed(fn, n) for name, fn in stages.items()}
@@ -561,6 +713,9 @@ def flow_bench(args, B, device: int):
             fn(i)
 
     chain_us = timed(chain, n)
+    sustain(chain, lambda: torch.cuda.synchronize(dev), t_leg0, 1.5)
+    sampler.stop()
+    clocks = sampler.summary(t_leg0, time.time())
     if store.device_status() != B.CCR_OK:
         raise SystemExit("device status not clean")
     valid = int(offs[-1].item())
@@ -571,7 +726,7 @@ def flow_bench(args, B, device: int):
         "config": {"workload": "config-1 shapes: 64 requests x 30,000 candidate ids (3 % unknown) against a 1,000,000-id index and store; "
                    "61,823 unsorted affinity records; padded T[64, 30000, 416 B] with the cosine section; back-to-back launches, "
                    "inputs in HBM (the 15 MB of ids and the payload stay L2-warm between repetitions)"},
-        "stage_us": per_stage, "chain_us": chain_us, "valid_candidates": valid, "gpu_launches": int(n),
+        "stage_us": per_stage, "chain_us": chain_us, "valid_candidates": valid, "gpu_launches": int(n), "clocks": clocks,
     }))
     ix.free()
     store.free()
@@ -589,6 +744,8 @@ def sort_bench(args, B, device: int):
     dev = torch.device("cuda", device)
     peak, peak_kind = measured_peak_gbs()
     results = []
+    sampler = ClockSampler(device)
+    t_leg0 = time.time()
     for name, wl in (("config1 payload", W.config1(n_docs=10_000, n_cand=100)),
                      ("config3 payload", W.config3(n_docs=100_000, n_cand=100, gen_doc_feats=True, extra_pools=0))):
         b = wl.batch
@@ -618,6 +775,8 @@ def sort_bench(args, B, device: int):
             torch.cuda.synchronize(dev)
             times.append(a.elapsed_time(z))
         ms = float(np.median(times))
+        t_busy = time.time()
+        sustain(lambda i: call(), lambda: torch.cuda.synchronize(dev), t_busy, 0.8)
         E = len(keys)
         nbytes = E * (2 * (8 + b.edge_row_bytes) + 4)
         t0 = time.perf_counter()
@@ -630,7 +789,11 @@ def sort_bench(args, B, device: int):
                         "oracle_ms_1_core": 1e3 * t_cpu, "matches_oracle": ok})
         store.free()
     head = results[-1]
+    sampler.stop()
     print(json.dumps({
+        "clocks": sampler.summary(t_leg0, time.time()),
+        "cpu_baseline": {"value": head["records"] / (head["oracle_ms_1_core"] * 1e-3), "unit": "records/s", "cores": 1,
+                         "kind": "oracle", "sample": "the config-3 payload once"},
         "metric": "edge_records_sorted_per_sec", "value": head["records_per_s"], "unit": "records/s", "n_gpus": 1,
         "steps": max(args.steps // 20, 20), "warmup": 3, "ms_per_step": head["ms"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
@@ -654,8 +817,14 @@ def run_reference(args, rank: int):
         print(json.dumps({"impl": "reference", "unavailable": "the CPU oracle cannot hold the 12.8 GB feature matrix of the "
                           "production-scale configurations; it is timed on configs 1 and 2b"}))
         return
-    wl, _ = make_workload(args.config, 0)
+    wl, cfg_flags = make_workload(args.config, 0, keys=args.keys)
     cores = host_cores()
+    # one pass over the whole batch gives the mask, from which the line's config (realised match rate, bytes) is
+    # written exactly as the CUDA arm writes it
+    _, mask_all = oracle.join_workload(wl, n_threads=cores)
+    second = wl.store.max_actors > 0
+    flags = (args.flags | cfg_flags) & ~args.drop_flags
+    bc = byte_counts(wl, mask_all, wl.out_row_bytes(), second)
     t_probe, n_probe = time_oracle(wl, cores, 1, max_cands=200_000)
     rate = n_probe / t_probe
     budget_s = 60.0
@@ -672,7 +841,7 @@ def run_reference(args, rank: int):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": workload_label(wl), "sample": desc},
+        "config": config_dict(wl, bc, flags, args, 1), "input_checksums": input_checksums(wl),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -738,7 +907,7 @@ def main():
         if rank == 0:
             flow_bench(args, B, local_rank)
         return
-    wl, cfg_flags = make_workload(args.config, rank, args.c3_docs, args.c3_requests)
+    wl, cfg_flags = make_workload(args.config, rank, args.c3_docs, args.c3_requests, args.keys)
     b = wl.batch
     second = wl.store.max_actors > 0
     kept = None
@@ -928,16 +1097,16 @@ def main():
         bc = byte_counts(wl, mask_host, out_b, second and not (flags & B.CCR_FLAG_FIRST_DEGREE_ONLY))
         launch_s = ms_per_step * 1e-3  # one kernel launch per step
         achieved = bc["compulsory"] / launch_s / 1e9
+        traffic, traffic_rec = (None, None) if (args.padded or args.cosine or args.keys != "uniform" or args.tile or args.key_cap) \
+            else ncu_traffic(wl.name, flags)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u8", "data": "synthetic",
-            "config": {"workload": workload_label(wl), "l2": "inputs and outputs of a step (%.2f GB) exceed the 126 MB L2; "
-                       "outputs rotate over %d buffers" % (bc["compulsory"] / 1e9, n_buf),
-                       "match_rate": bc["match_rate"], "seed": wl.seed, "tile": args.tile or "default", "key_cap": args.key_cap or "default",
-                       "flags": flags, "replicas": world},
+            "config": config_dict(wl, bc, flags, args, world, n_buf),
+            "input_checksums": input_checksums(wl),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_kind": "of " + peak_kind,
+                         "traffic": traffic, "traffic_capture": traffic_rec, "peak_kind": "of " + peak_kind,
                          "bytes_per_launch": bc["compulsory"], "logical_bytes_per_launch": bc["logical"],
                          "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                          "logical_gbs": bc["logical"] / launch_s / 1e9},
