@@ -90,6 +90,11 @@ enum {
                                            row streaming) instead of the warp-specialised kernel      */
   CCR_FLAG_COSINE            = 1u << 8, /* append the derived cosine section (ccr_docstore_set_cosine,
                                            ccr_join_batch_ex); adds 32 bytes to the row                */
+  CCR_FLAG_NO_REBALANCE      = 1u << 10, /* second-degree joins: keep the 16-warp form of the warp-specialised kernel
+                                           instead of its 20-warp form with registers moved from the search warps to
+                                           the row-streaming warps (comparison aid)                                  */
+  CCR_FLAG_NO_OVERLAP        = 1u << 11, /* do not let this launch move in behind a join that is still draining on the same
+                                           stream (see "Back-to-back joins" at ccr_join_batch)                       */
   CCR_FLAG_WARP_SPECIALISED  = 1u << 9  /* take the warp-specialised kernel whatever the launch size (by default a
                                            ragged launch of at most 131,072 candidates — a single request —
                                            runs on the two-phase kernel, which has the shorter start-up)      */
@@ -168,7 +173,15 @@ size_t ccr_out_row_bytes(const ccr_docstore* store, uint32_t flags);
  * never synchronises.  cand_offsets[0] must be 0 and both offset arrays non-decreasing; they and the
  * key order are trusted unless CCR_FLAG_VALIDATE is given.  With unsorted keys or an untruthful
  * CCR_FLAG_CANDS_SORTED the values are unspecified but every access stays in bounds.
- * The call allocates nothing, clears nothing and is asynchronous: one kernel on `stream`.          */
+ * The call allocates nothing, clears nothing and is asynchronous: one kernel on `stream`.
+ *
+ * Back-to-back joins.  The warp-specialised kernel is launched with programmatic stream serialization: when the
+ * work in front of it on `stream` is another join of this library, its blocks take over each SM as soon as that
+ * join's block there has retired and read their own inputs (offsets, keys, candidate positions, ids) while the
+ * earlier join drains; they write nothing — rows, mask — before the earlier join has completed, so reusing the
+ * output buffers of the previous call is safe, and any other kernel, copy or event on the stream orders the
+ * launch as usual.  What is NOT ordered is a join that reads, as an input, memory the join directly in front of
+ * it writes (its rows or mask reinterpreted as keys or positions): give such a call CCR_FLAG_NO_OVERLAP.          */
 ccr_status ccr_join_batch(const ccr_docstore* store,
                           int32_t n_req, int64_t total_cands, int64_t max_edge_len,
                           const int64_t* edge_keys,    /* DEVICE [E]                               */

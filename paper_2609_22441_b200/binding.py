@@ -39,6 +39,8 @@ CCR_FLAG_STATIC_SPLIT = 1 << 6
 CCR_FLAG_TWO_PHASE = 1 << 7
 CCR_FLAG_COSINE = 1 << 8
 CCR_FLAG_WARP_SPECIALISED = 1 << 9
+CCR_FLAG_NO_REBALANCE = 1 << 10
+CCR_FLAG_NO_OVERLAP = 1 << 11
 
 EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_upsert", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",

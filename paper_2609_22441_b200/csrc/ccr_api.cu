@@ -28,6 +28,7 @@ constexpr uint64_t kWsMagic = 0x4343525753504143ull;     // "CCRWSPAC"
 constexpr uint64_t kIxMagic = 0x4343524944494e44ull;     // "CCRIDIND"
 constexpr int kMaxSmemBytes = 227 * 1024;
 constexpr int kDefaultTileWs = 256;        // candidates per ring slot of the warp-specialised kernel
+constexpr int kDefaultTileWsRebal = 128;   // ... of its register-rebalanced form (a ring twice as deep)
 constexpr int kDefaultTileTwoPhase = 1024; // candidates per search/copy phase pair of the two-phase kernel
 constexpr int kSmemPerSm = 228 * 1024;
 constexpr int kDefaultKeyCap = 4096;
@@ -36,7 +37,8 @@ constexpr int kAutoSmemBudget = 160 * 1024;  // shared memory the warp-specialis
 constexpr int kMaxTile = ccr::kMaxTileCands;
 constexpr size_t kStageBytes = 16u << 20;  // staging block of second-degree stores (ids uploaded from the host)
 constexpr int kSchedRegions = 64;                    // launches of one store that may be in flight at once
-constexpr int kStatusInts = 4 + 2 * kSchedRegions;   // [0] wait expiry, [1] validation code, [4..] scheduling words
+constexpr int kStatusHead = 4;                       // [0] wait expiry, [1] validation code; then the scheduling words:
+                                                     // kSchedRegions regions of sched_stride ints
 
 inline size_t dtype_size(int32_t dt) { return dt == CCR_F16 ? 2 : (dt == CCR_F32 ? 4 : 0); }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -72,6 +74,7 @@ struct ccr_docstore {
   int blocks_per_sm;  // cap on resident blocks per SM of the two-phase kernel (0 = as many as fit)
   int ws_streamers, ws_resolvers;  // warp split of the warp-specialised kernel
   int n_sms;
+  int sched_stride;   // ints per scheduling region (next tile, finished blocks; a region has a 128-byte line to itself)
   int cos_first, cos_dim, cos_chunks;  // derived cosine section (cos_chunks == 0: not configured)
   std::atomic<int64_t> launches;  // kernels launched for this store; also hands out the scheduling-word pairs
 };
@@ -213,7 +216,7 @@ constexpr int kTunedCosPieces = 7;
 struct Variant {
   int doc_ch, edge_ch, req_ch;
   KernelFn first, second, merge;
-  WsKernelFn ws_first, ws_second, ws_first_cos, ws_second_cos;
+  WsKernelFn ws_first, ws_second, ws_first_cos, ws_second_cos, ws_second_rebal;
 };
 
 #define CCR_VARIANT(D, E, R)                                                                                      \
@@ -222,7 +225,8 @@ struct Variant {
         ccr::join_kernel<D, E, R, false, true>,                                                                   \
         ccr::join_ws_kernel<D, E, R, false>, ccr::join_ws_kernel<D, E, R, true>,                                  \
         ccr::join_ws_kernel<D, E, R, false, (D > 0 ? kTunedCosPieces : -1)>,                                      \
-        ccr::join_ws_kernel<D, E, R, true, (D > 0 ? kTunedCosPieces : -1)>                                        \
+        ccr::join_ws_kernel<D, E, R, true, (D > 0 ? kTunedCosPieces : -1)>,                                       \
+        ccr::join_ws_kernel<D, E, R, true, 0, true>                                                               \
   }
 
 const Variant kVariants[] = {
@@ -262,8 +266,8 @@ ccr_status allow_large_smem() {
       cudaGetLastError();
       return CCR_ERR_CUDA;
     }
-    const WsKernelFn ws[4] = {kVariants[i].ws_first, kVariants[i].ws_second, kVariants[i].ws_first_cos,
-                              kVariants[i].ws_second_cos};
+    const WsKernelFn ws[5] = {kVariants[i].ws_first, kVariants[i].ws_second, kVariants[i].ws_first_cos,
+                              kVariants[i].ws_second_cos, kVariants[i].ws_second_rebal};
     for (WsKernelFn f : ws) {
       if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemBytes) != cudaSuccess) {
         cudaGetLastError();
@@ -353,8 +357,10 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   } else {
     ok = ok && cudaMalloc(&s->author_ids, n * 8 + 256) == cudaSuccess;
   }
-  ok = ok && cudaMalloc(&s->status, kStatusInts * sizeof(int)) == cudaSuccess;
-  ok = ok && cudaMemset(s->status, 0, kStatusInts * sizeof(int)) == cudaSuccess;
+  s->sched_stride = 32;
+  const size_t status_ints = kStatusHead + static_cast<size_t>(kSchedRegions) * s->sched_stride;
+  ok = ok && cudaMalloc(&s->status, status_ints * sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemset(s->status, 0, status_ints * sizeof(int)) == cudaSuccess;
   ok = ok && cudaHostAlloc(&s->status_host, 4 * sizeof(int), cudaHostAllocDefault) == cudaSuccess;
   ccr_status st = ok ? allow_large_smem() : CCR_ERR_OOM;
   if (st != CCR_OK) {
@@ -492,7 +498,7 @@ ccr_status ccr_docstore_set_tuning(ccr_docstore* s, const ccr_tuning* t) {
     return CCR_ERR_INVALID_ARG;
   if (t->tile_cands % 256 || t->tile_cands > kMaxTile) return CCR_ERR_INVALID_ARG;
   if (t->key_capacity > 0 &&
-      static_cast<size_t>(ccr::search_bytes(t->key_capacity, true)) + ccr::kSmemHeader > static_cast<size_t>(kMaxSmemBytes))
+      static_cast<size_t>(ccr::search_keys_bytes(t->key_capacity)) + ccr::kSmemHeader > static_cast<size_t>(kMaxSmemBytes))
     return CCR_ERR_INVALID_ARG;
   const int st = t->ws_streamers > 0 ? t->ws_streamers : s->ws_streamers;
   const int rs = t->ws_resolvers > 0 ? t->ws_resolvers : s->ws_resolvers;
@@ -766,19 +772,32 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     if (!use_ws) return CCR_ERR_UNSUPPORTED;  // the derived section is computed by the warp-specialised kernel only
     if (reinterpret_cast<uintptr_t>(member_emb) & 1u) return CCR_ERR_INVALID_ARG;
   }
-  const int n_str = s->ws_streamers > 0 ? s->ws_streamers : 12;
-  const int n_res = s->ws_resolvers > 0 ? s->ws_resolvers : 4;
+  // second-degree joins on the default warp split take the register-rebalanced form (12 + 8 warps); a configured
+  // split, a configured sub-tile and the cosine section keep the 16-warp kernel
+  const bool rebal = use_ws && second && !cos && s->ws_streamers == 0 && s->tile == 0 && !(flags & CCR_FLAG_NO_REBALANCE);
+  const int n_str = rebal ? ccr::kRebalStreamers : (s->ws_streamers > 0 ? s->ws_streamers : 12);
+  const int n_res = rebal ? ccr::kRebalResolvers : (s->ws_resolvers > 0 ? s->ws_resolvers : 4);
   const int cos_stage = cos ? 32 * (((s->cos_dim + 7) / 8) | 1) * 16 : 0;
   const int cos_bytes = cos ? ccr::ws_cos_bytes(n_str, cos_stage) : 0;
-  auto smem_for = [&](int t, int cap) -> size_t {
-    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, cap, n_req <= ccr::kWsMaxCachedReq ? n_req : 0, cos_bytes, n_res).bytes)
-                  : static_cast<size_t>(ccr::TileLayout(t, second, merge, cap).bytes);
+  // Shared memory of a block: the kernel's own arrays for a sub-tile of t candidates plus `area` bytes for the search
+  // (staged keys, hash tables, sampled keys; ccr_search.cuh).
+  auto smem_for = [&](int t, int area) -> size_t {
+    return use_ws ? static_cast<size_t>(ccr::WsLayout(t, second, area, n_req <= ccr::kWsMaxCachedReq ? n_req : 0, cos_bytes, n_res,
+                                                      rebal ? ccr::kRebalSlots : ccr::kWsSlots,
+                                                      rebal ? ccr::kRebalInFlight * 128 : ccr::kWsWorkItems).bytes)
+                  : static_cast<size_t>(ccr::TileLayout(t, second, merge, area).bytes);
   };
-  // Keys staged per request.  The warp-specialised kernel runs one block per SM, so by default it stages
-  // whole lists up to a shared-memory budget (about 13,000 ids for a first-degree join); the kernels that keep
-  // several blocks per SM default to kDefaultKeyCap.  A configured key_capacity overrides both.
-  const int tile_cfg = s->tile > 0 ? s->tile : (use_ws ? kDefaultTileWs : kDefaultTileTwoPhase);
+  // bytes that hold a list of K keys in its best form: staged next to its table (the merge path builds no table)
+  auto best_area = [&](long long K) -> long long {
+    return K <= 0 ? 0 : ccr::search_bytes(static_cast<int>(K), !merge);
+  };
+  // key_cap = the longest list a block stages in full; the area is sized so that a list of key_cap keys has its
+  // best form, capped by the budget.  The warp-specialised kernel runs one block per SM, so by default it serves
+  // whole lists up to a shared-memory budget; the kernels that keep several blocks per SM default to
+  // kDefaultKeyCap.  A configured key_capacity overrides both.
+  const int tile_cfg = s->tile > 0 ? s->tile : (use_ws ? (rebal ? kDefaultTileWsRebal : kDefaultTileWs) : kDefaultTileTwoPhase);
   int tile = tile_cfg;
+  long long budget = kMaxSmemBytes;  // for the whole block
   int key_cap;
   if (flags & CCR_FLAG_FORCE_GLOBAL) {
     key_cap = 0;
@@ -788,21 +807,35 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     const long long cap = s->key_cap > 0 ? s->key_cap : kDefaultKeyCap;
     key_cap = static_cast<int>(max_edge_len < cap ? max_edge_len : cap);
   } else {
-    // Whole lists are staged as long as the block's shared memory stays within kAutoSmemBudget.  What the
-    // block takes from the SM's 228 KB is taken from the L1 that the streamers' loads pass through: the
-    // production-scale join (lists up to 20,000 keys) ran a third slower with every list staged (~205 KB per
-    // block) than with 100-150 KB, while 140 KB with every list staged beats sampling for second-degree joins.  Longer lists get a sampled top of the tree instead.
-    // A launch of a few tiles per block (a single request: the latency case) is bound by the searches, not by
-    // streaming, and keeps every list staged that fits (55.9 us against 70.3 us for 100,000 candidates x 20,000 keys).
+    // What the block takes from the SM's 228 KB is taken from the L1 that the streamers' loads pass through: the
+    // production-scale join (lists up to 20,000 keys) ran a third slower with ~205 KB per block than with
+    // 100-150 KB, hence kAutoSmemBudget for launches that are bound by streaming.  A launch of a few tiles per
+    // block (a single request: the latency case) is bound by the searches and may take all of it.
     key_cap = static_cast<int>(max_edge_len);
     const long long tiles = (total_cands + tile - 1) / tile;
     const bool streaming_bound = tiles >= 2LL * s->n_sms * n_res;
-    const size_t budget = streaming_bound ? static_cast<size_t>(kAutoSmemBudget) : static_cast<size_t>(kMaxSmemBytes);
-    while (key_cap > kDefaultKeyCap && smem_for(tile, key_cap) > budget) key_cap = std::max(kDefaultKeyCap, key_cap - 1024);
+    if (streaming_bound) budget = kAutoSmemBudget;
   }
-  // sub-tile size: the configured one, shrunk (in steps of 256) until the kernel's arrays fit next to the keys
-  while (tile > 256 && smem_for(tile, key_cap) > static_cast<size_t>(kMaxSmemBytes)) tile -= 256;
-  const size_t smem = smem_for(tile, key_cap);
+  // sub-tile size: the configured one, shrunk (in steps of 256) until the kernel's arrays leave room for the keys
+  // of the longest list an explicit capacity promises to stage (the automatic capacity adapts to the room instead)
+  const bool explicit_cap = (flags & CCR_FLAG_FORCE_SMEM) || s->key_cap > 0;
+  const int must_fit = explicit_cap ? ccr::search_keys_bytes(key_cap) : 0;
+  while (tile > 256 && static_cast<long long>(smem_for(tile, must_fit)) > kMaxSmemBytes) tile -= 256;
+  const long long fixed = static_cast<long long>(smem_for(tile, 0));
+  long long area = best_area(key_cap);
+  if (fixed + area > budget) area = budget - fixed;
+  if (area < 0) area = 0;
+  area &= ~15LL;
+  if (explicit_cap) {
+    // an explicit capacity is honoured as long as the bare keys fit in the block at all
+    const long long need = ccr::search_keys_bytes(key_cap);
+    if (area < need) area = need;
+    if (fixed + area > kMaxSmemBytes) return CCR_ERR_UNSUPPORTED;
+  } else if (key_cap > 0) {
+    // automatic: lists longer than what fits in full (next to a table where one is built) are not staged
+    while (key_cap > 1 && best_area(key_cap) > area) key_cap -= std::max(1, key_cap / 64);
+  }
+  const size_t smem = smem_for(tile, static_cast<int>(area));
   if (smem > static_cast<size_t>(kMaxSmemBytes)) return CCR_ERR_UNSUPPORTED;
 
   ccr::JoinArgs a;
@@ -834,6 +867,7 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   a.cos_stage = cos_stage;
   a.tile = tile;
   a.key_cap = key_cap;
+  a.search_area = static_cast<int>(area);
   a.min_stride_log2 = (flags & CCR_FLAG_FORCE_SAMPLED) ? 2 : 0;
   a.status = s->status;
   a.sched = nullptr;
@@ -862,19 +896,36 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     // one persistent warp-specialised block per SM (fewer when there are fewer 32-row groups than SMs)
     long long blocks = s->n_sms;
     if (blocks > groups) blocks = groups;
-    const WsKernelFn fn = cos ? (second ? v.ws_second_cos : v.ws_first_cos) : (second ? v.ws_second : v.ws_first);
+    const WsKernelFn fn = cos ? (second ? v.ws_second_cos : v.ws_first_cos) : (second ? (rebal ? v.ws_second_rebal : v.ws_second) : v.ws_first);
     // dynamic chunk scheduling through a pair of device words; each launch takes the next pair in turn, so
     // up to kSchedRegions launches of one store may be in flight at once (on any streams)
     // Small launches (fewer tiles than two rounds per block) are split evenly instead: drawing whole rounds
     // from the counter would leave most SMs without work, and a single request is the latency-critical case.
-    const int n_res_auto = s->ws_resolvers > 0 ? s->ws_resolvers : 4;
+    const int n_res_auto = n_res;
     const long long n_tiles = (total_cands + a.tile - 1) / a.tile;
     const bool dynamic = !(flags & CCR_FLAG_STATIC_SPLIT) && n_tiles >= 2LL * blocks * n_res_auto;
     // (the pair is drawn from the atomic launch counter, so host threads that join against one store at the
     // same time never share a pair)
     const int64_t seq = s->launches.fetch_add(1);
-    if (dynamic) a.sched = sched_override ? sched_override : s->status + 4 + 2 * static_cast<int>(seq % kSchedRegions);
-    fn<<<static_cast<unsigned>(blocks), (n_str + n_res) * 32, smem, st>>>(a, n_str);
+    if (dynamic) a.sched = sched_override ? sched_override : s->status + kStatusHead + s->sched_stride * static_cast<int>(seq % kSchedRegions);
+    // Launched with programmatic stream serialization: behind another join on the same stream the blocks become
+    // resident as that join's blocks leave their SMs and prepare (barriers, offsets, first keys, first ids and
+    // searches) while it drains; they store nothing before it has completed (griddepcontrol.wait in the kernel).
+    // Behind any other kernel, copy or event the launch is ordered as usual.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+    cfg.blockDim = dim3(static_cast<unsigned>((n_str + n_res) * 32));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (flags & CCR_FLAG_NO_OVERLAP) ? 0 : 1;
+    if (cudaLaunchKernelEx(&cfg, fn, a, n_str) != cudaSuccess) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
   } else {
     // persistent two-phase kernel: as many blocks as stay resident, each with at least 64 candidates (a single
     // small request is spread over many SMs: 21.6 against 23.4 us for 1,000 candidates with 256 per block)
@@ -1133,7 +1184,7 @@ ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t 
 // payload.  In host code the array's name is only a stand-in for the device symbol, so its device address
 // is looked up once per device with cudaGetSymbolAddress and that pointer is what kernels and copies get.
 constexpr size_t kStaticScratchBytes = 16u << 20;  // 16 MiB, held by every GPU that loads the library
-constexpr size_t kStaticControlBytes = 256;        // status + scheduling words in front of the payload
+constexpr size_t kStaticControlBytes = 256;        // scheduling words in front of the payload
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 namespace {

@@ -67,7 +67,8 @@ struct JoinArgs {
   long long n_max;            // 0: ragged output (row j); > 0: padded output, row r * n_max + (j - cand_offsets[r])
   // launch shape
   int tile;                   // candidates per block
-  int key_cap;                // keys (or sampled keys) a block may stage per request; 0 = search global memory
+  int key_cap;                // longest list a block may stage in full per request; 0 = search global memory
+  int search_area;            // bytes of shared memory the search may use for keys, tables or sampled keys
   int min_stride_log2;        // >0 forces sampling with at least this stride (testing aid)
   int* status;                // device status words
   int* sched;                 // two scheduling words (next tile, finished blocks), zero between launches; or null
@@ -114,15 +115,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait: gives up after kWaitTries polls (each poll may itself suspend for a short,
-// hardware-defined time).  Returns false when the phase never completed.
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait: gives up after kWaitTries polls (each poll may itself suspend for a short, hardware-defined
+// time) or after kWaitNanos of wall time, whichever comes first.  Returns false when the phase never completed.
 constexpr int kWaitTries = 1 << 22;
+constexpr unsigned long long kWaitNanos = 2000000000ull;  // two seconds: far beyond any launch of this library
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int tries = kWaitTries) {
+  unsigned long long t0 = 0;
   for (int i = 0; i < tries; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023) == 1023) {  // the clock is read rarely: the common wait ends within a few polls
+      const unsigned long long t = global_timer_ns();
+      if (t0 == 0) t0 = t;
+      else if (t - t0 > kWaitNanos) return false;
+    }
   }
   return false;
 }
+
+// Programmatic dependent launch.  A join launched right behind another join on the same stream may become resident
+// while the earlier one drains (as its blocks leave their SMs) and run everything that only reads its own inputs;
+// pdl_wait() returns once the earlier grid has completed and its writes are visible, and comes before the first
+// global store.  pdl_trigger() tells the runtime that this block no longer needs to hold back a dependent launch.
+// Both are no-ops for a launch without the attribute or without a predecessor that triggers.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ uint4 ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 

@@ -155,14 +155,14 @@ __device__ __forceinline__ int block_lower_bound(const int64_t* g, int K, int64_
 // Shared-memory layout of join_kernel, shared by host (sizing) and device (carving).
 struct TileLayout {
   int off_idx, off_pos, off_apos, off_auth, off_keys, bytes;
-  __host__ __device__ TileLayout(int tile, bool second, bool merge, int key_cap) {
+  __host__ __device__ TileLayout(int tile, bool second, bool merge, int search_area) {
     off_idx = kSmemHeader;
     off_pos = off_idx + tile * 4;
     off_apos = off_pos + tile * 4;
     off_auth = off_apos + (second ? tile * 16 : 0);
     off_keys = off_auth + (merge ? tile * 8 : 0);
     off_keys = (off_keys + 15) & ~15;
-    bytes = off_keys + search_bytes(key_cap, !merge);
+    bytes = off_keys + search_area;
   }
 };
 
@@ -345,12 +345,12 @@ constexpr int kJoinMinBlocks = CCR_JOIN_MIN_BLOCKS;  // resident blocks per SM t
 template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, bool MERGE, bool PADDED = false>
 __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const JoinArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
-  const TileLayout lay(a.tile, SECOND, MERGE, a.key_cap);
+  const TileLayout lay(a.tile, SECOND, MERGE, a.search_area);
   int* s_idx = reinterpret_cast<int*>(smem + lay.off_idx);
   int* s_pos = reinterpret_cast<int*>(smem + lay.off_pos);
   int4* s_apos = reinterpret_cast<int4*>(smem + lay.off_apos);
   int64_t* s_auth = reinterpret_cast<int64_t*>(smem + lay.off_auth);
-  const SearchSmem ssm = carve_search(smem + lay.off_keys, a.key_cap, !MERGE);
+  const SearchSmem ssm = carve_search(smem + lay.off_keys, a.search_area, !MERGE);
   const BlockGroup grp;
   const uint32_t bar = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -386,7 +386,8 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
 
     StagedKeys keys;
     if (!MERGE) {
-      if (!stage_keys(a, ssm, bar, phase, kb, K, true, keys, grp)) {
+      // lookups this block will make against the list: its candidates of the request (second degree: up to five ids each)
+      if (!stage_keys(a, ssm, bar, phase, kb, K, true, (seg_end - seg) * (SECOND ? 3 : 1), keys, grp)) {
         give_up_wait(a, bar, phase);
         return;
       }
@@ -491,9 +492,10 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
         const int lo = block_lower_bound(gk, K, s_auth[0]);
         const int hi = min(K, block_lower_bound(gk, K, s_auth[n - 1]) + 1);
         const int w = max(hi - lo, 0);
-        const bool windowed = (a.key_cap > 0) && (w <= a.key_cap) && (a.min_stride_log2 == 0) && !any_invalid;
+        const bool windowed = (a.key_cap > 0) && (w <= a.key_cap) && (search_keys_bytes(w) <= a.search_area) &&
+                              (a.min_stride_log2 == 0) && !any_invalid;
         // 3. stage the window (or, if it is too long, the request's keys as the binary-search mode does)
-        if (!stage_keys(a, ssm, bar, phase, windowed ? kb + lo : kb, windowed ? w : K, false, keys, grp)) {
+        if (!stage_keys(a, ssm, bar, phase, windowed ? kb + lo : kb, windowed ? w : K, false, 0, keys, grp)) {
           give_up_wait(a, bar, phase);
           return;
         }

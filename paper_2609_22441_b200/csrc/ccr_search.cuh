@@ -1,26 +1,50 @@
 // Key staging and the per-candidate sorted search (Algorithm 1 steps 2-3 of the paper).
 //
-// A request's sorted author ids are staged in shared memory by one 1-D TMA bulk copy (K <= key_cap), or as
-// a sampled top of the search tree (K > key_cap: every 2^s-th key; the last <= 2^s keys of a search are
-// read from global memory / L2), or not at all (key_cap == 0).
+// What a lookup has to decide is "does some key equal this id, and at which index" (Eq. 1); on sorted, unique keys
+// that is exactly the lower bound + equality test of Algorithm 1.  A request's keys are served from this block's
+// shared memory in one of four forms, chosen per request segment from the list's length K, the shared-memory area
+// of the launch and the number of lookups the segment will make:
 //
-// Fully staged lists also get a bucket index over the key range: bucket b = (key - kmin) >> shift, with
-// (first, end) positions of the keys that fall in it.  A lookup is then one index load plus a branch-free
-// lower bound over the few keys of one bucket (about one key per bucket for evenly spread ids, never more
-// than log2 K steps) instead of log2 K dependent shared-memory probes over the whole list.  The bucket
-// function is monotone in the key, so a bucket's keys are contiguous and the result is exactly the lower
-// bound / equality test of Algorithm 1; an id in an empty bucket is simply not found.
+//   staged + table : the keys are brought in by one 1-D TMA bulk copy and a hash table over them is built beside
+//                    them.  A lookup is two 16-byte table reads (two candidate buckets of four slots; a slot holds
+//                    a 13-bit fingerprint of the key and the key's index) and, only when a fingerprint matches, one key
+//                    read to verify: two dependent shared-memory accesses whatever K is and however the ids are
+//                    spread over their range (a map of the key *range* to buckets degenerates for clustered ids:
+//                    one far outlier puts a whole list into one bucket).
+//   table only     : lists too long to stage next to their table keep only the table in shared memory; the
+//                    verifying key read goes to global memory / L2 (hits only: a miss never leaves the SM).
+//   staged         : segments with too few lookups to pay for building a table search the staged keys by a
+//                    branch-free binary search.
+//   sampled        : every 2^s-th key staged as the top of the search tree, the last <= 2^s keys of a search read
+//                    from global memory / L2 (lists beyond everything above); key_cap == 0: the whole search runs
+//                    in global memory.
+//
+// The table is filled with two-choice placement (a key goes to the emptier of its two buckets), at most one key per
+// two slots.  A key that finds both buckets full is simply left out: a lookup that sees two full buckets and no
+// verified match falls back to the binary search, so the table never has to be complete to be exact (simulated on
+// uniform, consecutive and heavy-tailed ids: no key left out in most lists, both buckets full for 0.03 % of ids).
 #pragma once
 
 #include "ccr_device.cuh"
 
 namespace ccr {
 
-// Shared memory a search needs: the key area and the bucket index.
+constexpr int kSlotPosBits = 18;                       // a slot = fingerprint tag (bits 18..31) | (key index + 1); 0 = empty
+constexpr unsigned kSlotPosMask = (1u << kSlotPosBits) - 1u;
+constexpr int kTableMaxKeys = (1 << kSlotPosBits) - 2;  // longer lists take the sampled search
+#ifndef CCR_TABLE_AMORT
+#define CCR_TABLE_AMORT 1
+#endif
+#ifndef CCR_BUILD_ILP
+#define CCR_BUILD_ILP 2
+#endif
+constexpr int kTableAmort = CCR_TABLE_AMORT;  // a table over K keys is built for a segment of at least K / kTableAmort lookups
+
+// Shared memory a search may use: one area that holds [table | keys], [table], [keys] or [sampled keys].
 struct SearchSmem {
-  int64_t* keys;   // key_cap + 2 slots
-  int2* tab;       // tab_cap entries (0 = no index)
-  int tab_cap;     // power of two
+  unsigned char* base;
+  int bytes;     // size of the area
+  bool index;    // tables may be built
 };
 
 __host__ __device__ inline int pow2_ceil(int x) {
@@ -28,51 +52,53 @@ __host__ __device__ inline int pow2_ceil(int x) {
   while (p < x) p <<= 1;
   return p;
 }
-// bytes of the search area for a given key capacity (keys, then the bucket index), 16-byte aligned pieces
-__host__ __device__ inline int search_keys_bytes(int key_cap) { return (key_cap + 2) * 8; }
-constexpr int kMaxBuckets = 4096;  // 32 KB of index at most; longer lists simply get more keys per bucket
-__host__ __device__ inline int search_tab_cap(int key_cap, bool want_index) {
-  if (!want_index || key_cap <= 0) return 0;
-  const int p = pow2_ceil(key_cap);
-  return p < kMaxBuckets ? p : kMaxBuckets;
+// buckets (of four 4-byte slots) of a table over K keys: two slots per key
+__host__ __device__ inline int table_buckets(int K) { return K > 0 ? (K + 1) / 2 : 0; }
+__host__ __device__ inline int search_keys_bytes(int K) { return K > 0 ? (((K + 2) + 1) & ~1) * 8 : 0; }  // K keys + 2, whole 16 bytes
+// bytes that hold a list of K keys staged next to its table
+__host__ __device__ inline int search_bytes(int K, bool want_index) {
+  return search_keys_bytes(K) + (want_index ? table_buckets(K) * 16 : 0);
 }
-__host__ __device__ inline int search_bytes(int key_cap, bool want_index) {
-  return search_keys_bytes(key_cap) + search_tab_cap(key_cap, want_index) * 8;
-}
-__device__ __forceinline__ SearchSmem carve_search(unsigned char* base, int key_cap, bool want_index) {
+__device__ __forceinline__ SearchSmem carve_search(unsigned char* base, int bytes, bool want_index) {
   SearchSmem s;
-  s.keys = reinterpret_cast<int64_t*>(base);
-  s.tab = reinterpret_cast<int2*>(base + search_keys_bytes(key_cap));
-  s.tab_cap = search_tab_cap(key_cap, want_index);
+  s.base = base;
+  s.bytes = bytes;
+  s.index = want_index;
   return s;
+}
+
+// Two bucket indices and the fingerprint tag of an id: 13 hash bits and a set top bit, placed above the index bits
+// of a slot, so that (slot ^ tag) is the stored index + 1 for a slot that holds this fingerprint and at least
+// 2^18 for every other slot, the empty one included.  Three 32-bit multiplies; the two bucket choices come from
+// differently mixed words, so ids that collide in one rarely collide in the other.
+__device__ __forceinline__ void key_hash(long long id, unsigned nbk, unsigned& b1, unsigned& b2, unsigned& tag) {
+  const unsigned lo = static_cast<unsigned>(id), hi = static_cast<unsigned>(static_cast<unsigned long long>(id) >> 32);
+  const unsigned u = lo * 0x9E3779B1u + hi * 0x85EBCA77u;
+  const unsigned v = (u ^ (u >> 15)) * 0x2C1B3C6Du;
+  b1 = __umulhi(u, nbk);
+  b2 = __umulhi(v, nbk);
+  tag = (v << kSlotPosBits) | 0x80000000u;
 }
 
 // Keys of the request a block is currently serving.
 struct StagedKeys {
   const int64_t* sk;  // shared-memory copy (index i = key i when s_log == 0, sample i otherwise)
   const int64_t* gk;  // the request's keys in global memory
-  const int2* tab;    // bucket index over sk (only when nb > 0)
-  long long kmin, kmax;
+  const uint4* tab;   // hash table over the K keys (only when nbk > 0)
   int K;              // keys in the request
   int M;              // staged entries (0 = nothing staged)
   int s_log;          // log2 of the sampling stride
-  int nb;             // buckets in the index (0 = none)
-  int shift;          // bucket = (key - kmin) >> shift
+  unsigned nbk;       // buckets of the table (0 = none)
+  bool declined;      // no table only because the segment it was staged for had too few lookups to pay for one
 
-  // Algorithm 1 steps 2-3 for one id: found = some key equals id; pos = its index (meaningful when found).
+  // Algorithm 1 steps 2-3 for one id by binary search: found = some key equals id; pos = its index (meaningful
+  // when found).  Serves the segments without a table and the rare lookups the table cannot answer.
   __device__ __forceinline__ bool find(int64_t id, int& pos) const {
     pos = 0;
     if (K == 0) return false;
     if (M > 0 && s_log == 0) {
-      int lo = 0, n = M;
-      if (nb > 0) {
-        if (id < kmin || id > kmax) return false;
-        const int2 e = tab[static_cast<unsigned long long>(id - kmin) >> shift];
-        lo = min(max(e.x, 0), M);             // clamps only matter for unsorted (contract-breaking) keys
-        n = min(max(e.y, lo), M) - lo;
-      }
-      pos = lo + lower_bound_smem(sk + lo, n, id);
-      return pos < lo + n && sk[pos] == id;
+      pos = lower_bound_smem(sk, M, id);
+      return pos < M && sk[pos] == id;
     }
     int lo = 0, n = K;
     if (M > 0) {
@@ -85,42 +111,44 @@ struct StagedKeys {
     return pos < K && __ldg(gk + pos) == id;
   }
 
-  // U independent lookups with their shared-memory accesses interleaved: one round of bucket-index loads,
-  // then one round of up to P key loads per id (a bucket of evenly spread ids holds about one key).
-  // Ids whose bucket is longer, and lists without an index, take find().  id < 0 is "nothing to look up".
-  template <int U, int P = 4>
+  // U independent lookups with their memory accesses interleaved: one round of table reads (two buckets per id),
+  // then one round of verifying key reads (only ids with a matching fingerprint).  Lists without a table, and the
+  // ids the table cannot answer, take find().  id < 0 is "nothing to look up".
+  template <int U>
   __device__ __forceinline__ void find_batch(const int64_t (&id)[U], bool (&found)[U], int (&pos)[U]) const {
-    if (!(K > 0 && M > 0 && s_log == 0 && nb > 0)) {
+    if (nbk == 0) {
 #pragma unroll
-      for (int u = 0; u < U; ++u) found[u] = id[u] >= 0 && find(id[u], pos[u]);
+      for (int u = 0; u < U; ++u) {
+        pos[u] = 0;
+        found[u] = id[u] >= 0 && find(id[u], pos[u]);
+      }
       return;
     }
-    int lo[U], n[U];
+    unsigned hit[U];   // index + 1 of the matching slot with the smallest index (>= 2^18: no fingerprint matched)
+    bool full[U];      // both buckets full: the key may have been left out of the table
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const bool in = id[u] >= kmin && id[u] <= kmax;
-      const int2 e = in ? tab[static_cast<unsigned long long>(id[u] - kmin) >> shift] : make_int2(0, 0);
-      lo[u] = min(max(e.x, 0), M);
-      n[u] = min(max(e.y, lo[u]), M) - lo[u];
+      unsigned b1, b2, tag;
+      key_hash(id[u], nbk, b1, b2, tag);
+      const uint4 x = tab[b1], y = tab[b2];
+      hit[u] = min(min(min(x.x ^ tag, x.y ^ tag), min(x.z ^ tag, x.w ^ tag)),
+                   min(min(y.x ^ tag, y.y ^ tag), min(y.z ^ tag, y.w ^ tag)));
+      full[u] = x.w != 0u && y.w != 0u;  // the slots of a bucket fill in order
     }
-    int64_t k[U][P];
+    int64_t kv[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-#pragma unroll
-      for (int j = 0; j < P; ++j) k[u][j] = (j < n[u]) ? sk[lo[u] + j] : 0;  // lo + j < lo + n <= M
+      pos[u] = static_cast<int>(hit[u]) - 1;  // < K for a match: slots only ever hold indices of this list
+      kv[u] = 0;
+      if (hit[u] <= kSlotPosMask && id[u] >= 0) kv[u] = (M > 0) ? sk[pos[u]] : __ldg(gk + pos[u]);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      found[u] = false;
-      pos[u] = 0;
-#pragma unroll
-      for (int j = 0; j < P; ++j) {
-        if (j < n[u] && k[u][j] == id[u]) {
-          found[u] = true;
-          pos[u] = lo[u] + j;
-        }
-      }
-      if (n[u] > P && !found[u]) found[u] = find(id[u], pos[u]);  // long bucket: bounded binary search
+      const bool has = hit[u] <= kSlotPosMask && id[u] >= 0;
+      found[u] = has && kv[u] == id[u];
+      // a matching fingerprint of another key, or no match with nowhere left to look: the exact search decides
+      if (id[u] >= 0 && !found[u] && (has || full[u])) found[u] = find(id[u], pos[u]);
+      if (!found[u]) pos[u] = 0;
     }
   }
 };
@@ -156,80 +184,123 @@ struct NamedGroup {
   }
 };
 
+// One key into the table: the emptier of its two buckets first, the first free slot of it (claimed with a
+// compare-and-swap, so concurrent inserts never share a slot; a slot is only tried after the one before it was
+// seen occupied, so the occupied slots of a bucket are always its first ones); a key that finds both buckets full
+// is left out.
+__device__ __forceinline__ void table_place(unsigned* slots, unsigned b1, unsigned b2, unsigned tag, const uint4& x,
+                                            const uint4& y, int index) {
+  const int c1 = (x.x != 0u) + (x.y != 0u) + (x.z != 0u) + (x.w != 0u);
+  const int c2 = (y.x != 0u) + (y.y != 0u) + (y.z != 0u) + (y.w != 0u);
+  const unsigned val = tag | static_cast<unsigned>(index + 1);
+  const unsigned first = (c1 <= c2) ? b1 : b2, second = (c1 <= c2) ? b2 : b1;
+  bool done = false;
+  for (int j = min(c1, c2); j < 4 && !done; ++j) done = atomicCAS(slots + first * 4 + j, 0u, val) == 0u;
+  for (int j = max(c1, c2); j < 4 && !done; ++j) done = atomicCAS(slots + second * 4 + j, 0u, val) == 0u;
+}
+__device__ __forceinline__ void table_insert(unsigned* slots, unsigned nbk, long long key, int index) {
+  unsigned b1, b2, tag;
+  key_hash(key, nbk, b1, b2, tag);
+  const uint4 x = reinterpret_cast<const uint4*>(slots)[b1], y = reinterpret_cast<const uint4*>(slots)[b2];
+  table_place(slots, b1, b2, tag, x, y, index);
+}
+
 // Stage keys [kb, kb+K) of the key array for the group.  Starts with a group barrier (everyone is done
 // with the previously staged keys) and ends with one.  Returns false, group-uniformly, if the bounded
-// wait for the bulk copy expired.  `index` asks for the bucket index (built only for fully staged lists).
+// wait for the bulk copy expired.  `index` asks for the hash table; `n_lookups` is how many lookups the
+// caller is about to make against these keys (the table is built only when they pay for it).
 template <typename G>
 __device__ __forceinline__ bool stage_keys(const JoinArgs& a, const SearchSmem& sm, uint32_t bar, uint32_t& phase,
-                                           long long kb, int K, bool index, StagedKeys& st, const G& g) {
-  // The key area may hold ordinary (generic-proxy) stores of an earlier staging — sampled keys, the unaligned
-  // head / tail key — at addresses the bulk copy below writes through the async proxy: every thread orders its
-  // own earlier stores against the async proxy before the barrier that precedes the copy.
+                                           long long kb, int K, bool index, long long n_lookups, StagedKeys& st,
+                                           const G& g) {
+  // The area may hold ordinary (generic-proxy) stores of an earlier staging — a table, sampled keys, the
+  // unaligned head / tail key — at addresses the bulk copy below writes through the async proxy: every thread
+  // orders its own earlier stores against the async proxy before the barrier that precedes the copy.
   fence_proxy_async_smem();
   g.sync();
-  int64_t* skeys = sm.keys;
   st.gk = a.edge_keys + kb;
   st.K = K;
   st.M = 0;
   st.s_log = 0;
-  st.sk = skeys;
-  st.tab = sm.tab;
-  st.nb = 0;
-  st.shift = 0;
-  st.kmin = st.kmax = 0;
+  st.nbk = 0;
+  st.declined = false;
+  st.tab = reinterpret_cast<const uint4*>(sm.base);
+  st.sk = reinterpret_cast<const int64_t*>(sm.base);
+  if (a.key_cap <= 0 || K <= 0 || sm.bytes < 16) {
+    g.sync();
+    return true;
+  }
+
+  const bool sampled_forced = a.min_stride_log2 != 0;
+  const bool table_ok = index && sm.index && !sampled_forced && K > 1 && K <= kTableMaxKeys;
+  const bool want_table = table_ok && n_lookups * kTableAmort >= K;
+  st.declined = table_ok && !want_table;
+  const int tab_bytes = table_buckets(K) * 16, key_bytes = search_keys_bytes(K);
+  const bool may_stage = K <= a.key_cap && !sampled_forced;
+  // [table | keys] when both fit; the table alone for a longer list; else the keys alone or a sampled top of the tree
+  const bool both = want_table && may_stage && tab_bytes + key_bytes <= sm.bytes;
+  const bool table = both || (want_table && tab_bytes <= sm.bytes);
+  const bool staged = both || (!table && may_stage && key_bytes <= sm.bytes);
+  int64_t* skeys = reinterpret_cast<int64_t*>(sm.base + (both ? tab_bytes : 0));
+  unsigned* slots = reinterpret_cast<unsigned*>(sm.base);
   bool expired = false;
-  if (a.key_cap > 0 && K > 0) {
-    if (K <= a.key_cap && a.min_stride_log2 == 0) {
-      // slot of key i is i + shift, so that 16-byte aligned global addresses land on 16-byte aligned slots
-      const int shift = static_cast<int>(kb & 1);
-      const int i0 = shift;                       // first key whose address is 16-byte aligned
-      const int nbulk = (K - i0) & ~1;            // keys moved by the bulk copy (even count)
-      st.sk = skeys + shift;
-      st.M = K;
-      if (g.tid == 0 && nbulk > 0) {
-        mbar_arrive_expect_tx(bar, static_cast<uint32_t>(nbulk) * 8u);
-        bulk_copy_g2s(smem_u32(skeys + i0 + shift), a.edge_keys + kb + i0, static_cast<uint32_t>(nbulk) * 8u, bar);
-      }
-      // the (at most one) key before and after the 16-byte aligned middle, by two other threads
-      if (g.tid == 1 && shift) skeys[shift] = __ldg(a.edge_keys + kb);
-      if (g.tid == 2 && ((K - i0) & 1)) skeys[K - 1 + shift] = __ldg(a.edge_keys + kb + K - 1);
-      if (nbulk > 0) {
-        expired = !mbar_wait_bounded(bar, phase);
-        phase ^= 1u;
-      }
-    } else {
-      int s_log = a.min_stride_log2;
-      while ((K >> s_log) > a.key_cap) ++s_log;
-      st.s_log = s_log;
-      st.M = K >> s_log;
-      for (int i = g.tid; i < st.M; i += g.size)
-        skeys[i] = __ldg(a.edge_keys + kb + ((static_cast<long long>(i) + 1) << s_log) - 1);
+
+  if (table) {  // cleared while the copy below is in flight
+    uint4* t4 = reinterpret_cast<uint4*>(slots);
+    for (int b = g.tid; b < table_buckets(K); b += g.size) t4[b] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  if (staged) {
+    // slot of key i is i + shift, so that 16-byte aligned global addresses land on 16-byte aligned slots
+    const int shift = static_cast<int>(kb & 1);
+    const int i0 = shift;                       // first key whose address is 16-byte aligned
+    const int nbulk = (K - i0) & ~1;            // keys moved by the bulk copy (even count)
+    st.sk = skeys + shift;
+    st.M = K;
+    if (g.tid == 0 && nbulk > 0) {
+      mbar_arrive_expect_tx(bar, static_cast<uint32_t>(nbulk) * 8u);
+      bulk_copy_g2s(smem_u32(skeys + i0 + shift), a.edge_keys + kb + i0, static_cast<uint32_t>(nbulk) * 8u, bar);
     }
+    // the (at most one) key before and after the 16-byte aligned middle, by two other threads
+    if (g.tid == 1 && shift) skeys[shift] = __ldg(a.edge_keys + kb);
+    if (g.tid == 2 && ((K - i0) & 1)) skeys[K - 1 + shift] = __ldg(a.edge_keys + kb + K - 1);
+    if (nbulk > 0) {
+      expired = !mbar_wait_bounded(bar, phase);
+      phase ^= 1u;
+    }
+  } else if (!table) {
+    int s_log = a.min_stride_log2;
+    const int cap = min(a.key_cap, sm.bytes / 8);
+    while ((K >> s_log) > cap) ++s_log;
+    st.s_log = s_log;
+    st.M = K >> s_log;
+    for (int i = g.tid; i < st.M; i += g.size)
+      skeys[i] = __ldg(a.edge_keys + kb + ((static_cast<long long>(i) + 1) << s_log) - 1);
   }
   if (g.sync_or(expired)) return false;
 
-  if (index && sm.tab_cap > 0 && st.M > 1 && st.s_log == 0) {
-    const int M = st.M;
+  if (table) {
+    const unsigned nbk = static_cast<unsigned>(table_buckets(K));
     const int64_t* S = st.sk;
-    st.kmin = S[0];
-    st.kmax = S[M - 1];
-    const unsigned long long range = static_cast<unsigned long long>(st.kmax - st.kmin);
-    const int nb = min(sm.tab_cap, pow2_ceil(M));
-    int shift = 0;
-    while ((range >> shift) >= static_cast<unsigned long long>(nb)) ++shift;  // group-uniform, <= 63 steps
-    st.nb = nb;
-    st.shift = shift;
-    int2* tab = sm.tab;
-    for (int b = g.tid; b < nb; b += g.size) tab[b] = make_int2(0, 0);
-    g.sync();
-    for (int i = g.tid; i < M; i += g.size) {
-      const unsigned long long b = static_cast<unsigned long long>(S[i] - st.kmin) >> shift;
-      if (b >= static_cast<unsigned long long>(nb)) continue;  // only possible with unsorted (contract-breaking) keys
-      const bool first = (i == 0) || ((static_cast<unsigned long long>(S[i - 1] - st.kmin) >> shift) != b);
-      const bool last = (i == M - 1) || ((static_cast<unsigned long long>(S[i + 1] - st.kmin) >> shift) != b);
-      if (first) tab[b].x = i;
-      if (last) tab[b].y = i + 1;
+    // several keys of a thread in flight: the bucket reads and compare-and-swaps of one overlap the others'
+    constexpr int kIlp = CCR_BUILD_ILP;
+    int i = g.tid;
+    for (; i + (kIlp - 1) * g.size < K; i += kIlp * g.size) {
+      long long kk[kIlp];
+#pragma unroll
+      for (int q = 0; q < kIlp; ++q) kk[q] = staged ? S[i + q * g.size] : __ldg(st.gk + i + q * g.size);
+      unsigned b1[kIlp], b2[kIlp], tag[kIlp];
+      uint4 x[kIlp], y[kIlp];
+#pragma unroll
+      for (int q = 0; q < kIlp; ++q) {
+        key_hash(kk[q], nbk, b1[q], b2[q], tag[q]);
+        x[q] = reinterpret_cast<const uint4*>(slots)[b1[q]];
+        y[q] = reinterpret_cast<const uint4*>(slots)[b2[q]];
+      }
+#pragma unroll
+      for (int q = 0; q < kIlp; ++q) table_place(slots, b1[q], b2[q], tag[q], x[q], y[q], i + q * g.size);
     }
+    for (; i < K; i += g.size) table_insert(slots, nbk, staged ? S[i] : __ldg(st.gk + i), i);
+    st.nbk = nbk;
     g.sync();
   }
   return true;

@@ -21,7 +21,9 @@
 // as the launch drains (guided self-scheduling), so blocks on slower SMs or with costlier requests simply take
 // fewer chunks and all blocks finish within about one tile of each other.  The last block to finish puts
 // the two scheduling words back to zero for the next launch.  Without a scheduling word every block takes
-// one equal contiguous slice.
+// one equal contiguous slice.  (Contiguous slices with work stealing between them — fewer key stagings per block —
+// were measured and lost 7-9 % on every configuration: all blocks walking one window of the candidate range
+// together is what the memory system likes.)
 #pragma once
 
 #include "ccr_join.cuh"
@@ -30,8 +32,34 @@ namespace ccr {
 
 constexpr int kWsSlots = 8;        // ring depth
 constexpr int kWsMaxThreads = 512;
+// Register-rebalanced form (second-degree joins, whose resolvers are the bottleneck): 12 streamer + 8 resolver
+// warps = 640 threads.  The block is launched with 96 registers per thread (the most 640 threads can have); the
+// resolver warpgroups then give registers back (setmaxnreg.dec) and the streamer warpgroups take them
+// (setmaxnreg.inc).  Registers only move inside the block's own allocation, and an increase waits until they are
+// there, so 384 x kRebalStreamerRegs + 256 x kRebalResolverRegs must not exceed 640 x 96 — more would never
+// arrive.  Eight resolvers fill eight ring slots at a time, so the ring is twice as deep (of half-size slots).
+constexpr int kRebalStreamers = 12, kRebalResolvers = 8;
+constexpr int kRebalThreads = (kRebalStreamers + kRebalResolvers) * 32;
+#ifndef CCR_REBAL_STREAMER_REGS
+#define CCR_REBAL_STREAMER_REGS 104
+#endif
+#ifndef CCR_REBAL_RESOLVER_REGS
+#define CCR_REBAL_RESOLVER_REGS 80
+#endif
+constexpr int kRebalStreamerRegs = CCR_REBAL_STREAMER_REGS, kRebalResolverRegs = CCR_REBAL_RESOLVER_REGS;
+constexpr int kRebalLaunchRegs = 96;  // 65,536 / 640 rounded down to the allocation unit of 8
+static_assert(kRebalStreamers * 32 * kRebalStreamerRegs + kRebalResolvers * 32 * kRebalResolverRegs <= kRebalThreads * kRebalLaunchRegs,
+              "the registers the streamers take must be the ones the resolvers give back");
+static_assert(kRebalStreamerRegs >= kRebalLaunchRegs && kRebalResolverRegs <= kRebalLaunchRegs && kRebalStreamerRegs % 8 == 0 &&
+              kRebalResolverRegs % 8 == 0, "inc raises, dec lowers, both in units of 8");
+static_assert(kRebalStreamers % 4 == 0 && kRebalResolvers % 4 == 0, "setmaxnreg acts on whole warpgroups");
+constexpr int kRebalSlots = 16;
+constexpr int kRebalInFlight = 2;   // candidates a resolver lane keeps in flight (twice the warps, half the registers)
 constexpr int kWsMaxCachedReq = 1024;  // batches up to this many requests keep their offsets in shared memory
-constexpr int kMaxRounds = 4;      // most tiles per resolver warp a block draws at once
+#ifndef CCR_MAX_ROUNDS
+#define CCR_MAX_ROUNDS 4
+#endif
+constexpr int kMaxRounds = CCR_MAX_ROUNDS;  // most tiles per resolver warp a block draws at once
 constexpr int kMaxTileCands = 4096;  // largest sub-tile the host accepts
 constexpr int kWsWorkItems = 4 * 32 * 4;  // engager slots of one resolver batch: 4 candidates per lane x 4 slots
 constexpr int kWsWorkListBytes = kWsWorkItems * (8 + 2);  // ids (int64) + tags (uint16) per resolver warp
@@ -62,39 +90,43 @@ struct WsLayout {
   // cos_bytes: shared memory of the derived cosine section (0 = off): a block of member-embedding floats per
   // ring slot, then one embedding staging block per streamer warp
   // n_res: resolver warps (second-degree joins give each a work list of engager lookups)
-  __host__ __device__ WsLayout(int tile, bool second, int key_cap, int n_req_cached, int cos_bytes, int n_res) {
+  __host__ __device__ WsLayout(int tile, bool second, int search_area, int n_req_cached, int cos_bytes, int n_res,
+                               int n_slots = kWsSlots, int wl_items = kWsWorkItems) {
     off_full = kSmemHeader;                 // after the key-staging mbarrier
-    off_empty = off_full + kWsSlots * 8;
-    off_slots = off_empty + kWsSlots * 8;
-    off_grab = off_slots + kWsSlots * static_cast<int>(sizeof(WsSlot));
+    off_empty = off_full + n_slots * 8;
+    off_slots = off_empty + n_slots * 8;
+    off_grab = off_slots + n_slots * static_cast<int>(sizeof(WsSlot));
     off_offs = off_grab + 16;
     off_idx = off_offs + (n_req_cached > 0 ? 2 * (n_req_cached + 1) * 8 : 0);
     off_idx = (off_idx + 15) & ~15;
-    off_pos = off_idx + kWsSlots * tile * 4;
-    off_apos = off_pos + kWsSlots * tile * 4;
-    off_cos = off_apos + (second ? kWsSlots * tile * 16 : 0);
+    off_pos = off_idx + n_slots * tile * 4;
+    off_apos = off_pos + n_slots * tile * 4;
+    off_cos = off_apos + (second ? n_slots * tile * 16 : 0);
     off_wl = off_cos + cos_bytes;
-    off_keys = off_wl + (second ? n_res * kWsWorkListBytes : 0);
-    bytes = off_keys + search_bytes(key_cap, true);
+    off_keys = off_wl + (second ? n_res * wl_items * (8 + 2) : 0);
+    off_keys = (off_keys + 15) & ~15;
+    bytes = off_keys + search_area;
   }
 };
 
 // CNP: 0 = no derived section; > 0 = the item embedding spans exactly CNP 16-byte pieces (tuned); < 0 = any shape
-template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0>
-__global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArgs a, int n_streamers) {
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0, bool REBAL = false>
+__global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join_ws_kernel(const JoinArgs a, int n_streamers) {
   extern __shared__ __align__(16) unsigned char smem_ws[];
   unsigned char* smem = smem_ws;
   constexpr bool COS = CNP != 0;
+  constexpr int kSlots = REBAL ? kRebalSlots : kWsSlots;
+  static_assert(!(REBAL && COS), "the rebalanced form carries no cosine section");
   const int n_req_cached = a.n_req <= kWsMaxCachedReq ? a.n_req : 0;
-  const WsLayout lay(a.tile, SECOND, a.key_cap, n_req_cached, COS ? ws_cos_bytes(n_streamers, a.cos_stage) : 0,
-                     (static_cast<int>(blockDim.x) >> 5) - n_streamers);
+  const WsLayout lay(a.tile, SECOND, a.search_area, n_req_cached, COS ? ws_cos_bytes(n_streamers, a.cos_stage) : 0,
+                     (static_cast<int>(blockDim.x) >> 5) - n_streamers, kSlots, REBAL ? kRebalInFlight * 128 : kWsWorkItems);
   WsSlot* slots = reinterpret_cast<WsSlot*>(smem + lay.off_slots);
   int* grab = reinterpret_cast<int*>(smem + lay.off_grab);
   int* s_idx = reinterpret_cast<int*>(smem + lay.off_idx);
   int* s_pos = reinterpret_cast<int*>(smem + lay.off_pos);
   int4* s_apos = reinterpret_cast<int4*>(smem + lay.off_apos);
   float4* s_cos = reinterpret_cast<float4*>(smem + lay.off_cos);
-  const SearchSmem ssm = carve_search(smem + lay.off_keys, a.key_cap, true);
+  const SearchSmem ssm = carve_search(smem + lay.off_keys, a.search_area, true);
   const uint32_t bar = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_threads = blockDim.x;
@@ -117,7 +149,7 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   }
   if (tid == 0) {
     mbar_init(bar, 1);
-    for (int s = 0; s < kWsSlots; ++s) {
+    for (int s = 0; s < kSlots; ++s) {
       slots[s].cos_r = -1;
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, static_cast<uint32_t>(n_streamers));
@@ -137,17 +169,19 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   const int role_rank = (n_threads >> 5) - 1 - warp;  // resolvers are the last n_res warps
   if (role_rank >= n_res) {
     // ============================ streamers ============================
+    if constexpr (REBAL) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRebalStreamerRegs));
     // this warp's embedding staging block (derived cosine section), behind the per-slot member blocks
     [[maybe_unused]] uint4* cos_stage = reinterpret_cast<uint4*>(
         smem + lay.off_cos + kWsSlots * kCosSlotFloat4 * 16 + (role_rank - n_res) * (COS ? a.cos_stage : 0));
     for (unsigned it = 0;; ++it) {
-      const int s = it % kWsSlots;
-      if (!mbar_wait_bounded(full0 + 8 * s, (it / kWsSlots) & 1u)) {
+      const int s = it % kSlots;
+      if (!mbar_wait_bounded(full0 + 8 * s, (it / kSlots) & 1u)) {
         if (lane == 0) atomicExch(a.status, kDevWaitExpired);
         return;
       }
       const WsSlot d = slots[s];
       if (d.n == 0) break;
+      if (it == 0) pdl_wait();  // the first rows are about to be written: the launch before this one must be done
       const uint8_t* edge_base = a.edge_feats + d.kb * sh.edge_b;
       const uint8_t* req_src = sh.req_ch ? a.req_feats + static_cast<long long>(d.r) * sh.req_b : nullptr;
       const int* idx = s_idx + s * a.tile;
@@ -171,6 +205,7 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   }
 
   // ============================ resolvers ============================
+  if constexpr (REBAL) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRebalResolverRegs));
   // All resolver warps walk the same sequence of sub-tiles; warp q fills every n_resolvers-th one on its own
   // (own bounded wait for the slot, own publish), so several sub-tiles are being resolved at any time.  They
   // meet on a named barrier only to draw the next chunk and to stage a new request's keys.
@@ -185,14 +220,18 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
   bool dead = false;     // this warp's wait for a free slot expired: keep walking (barriers!), fill nothing
   int staged_r = -1;     // request whose keys are in shared memory
   StagedKeys keys;
+  keys.declined = false;
+  bool pdl_pending = true;  // this warp has not yet waited for the launch before this one
   // this warp's work list of engager lookups (second-degree joins)
-  [[maybe_unused]] int64_t* wl_id = reinterpret_cast<int64_t*>(smem + lay.off_wl + (SECOND ? rwarp * kWsWorkListBytes : 0));
-  [[maybe_unused]] uint16_t* wl_tag = reinterpret_cast<uint16_t*>(wl_id + kWsWorkItems);
+  constexpr int U = SECOND ? (REBAL ? kRebalInFlight : 4) : 8;  // candidates a lane keeps in flight
+  constexpr int FB = U < 4 ? U : 4;                              // lookups interleaved in one find_batch
+  constexpr int kWlItems = U * 32 * 4;                           // every engager slot of one batch
+  [[maybe_unused]] int64_t* wl_id = reinterpret_cast<int64_t*>(smem + lay.off_wl + (SECOND ? rwarp * kWlItems * (8 + 2) : 0));
+  [[maybe_unused]] uint16_t* wl_tag = reinterpret_cast<uint16_t*>(wl_id + kWlItems);
   int cos_r = -1;        // request whose squared member norms lane k < kCosMaxChunks holds in cos_nm
   float cos_nm = 0.0f;
   const long long n_tiles = (a.total + a.tile - 1) / a.tile;
-  constexpr int U = SECOND ? 4 : 8;  // candidates a lane keeps in flight
-  static_assert(!SECOND || U * 32 * 4 == kWsWorkItems, "the work list holds every engager slot of one batch");
+  static_assert(REBAL || !SECOND || kWlItems == kWsWorkItems, "the work list holds every engager slot of one batch");
   static_assert(kMaxTileCands * 4 <= 65536, "work-list tags are 16 bits: candidate index in the tile x 4 + slot");
 
   for (bool more = true; more && !failed;) {
@@ -231,8 +270,12 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
       const long long seg_end = min(rend, j1);
       const long long kb = eo[r];
       const int K = static_cast<int>(min(max(eo[r + 1] - kb, 0LL), static_cast<long long>(a.max_edge_len)));
-      if (r != staged_r) {
-        if (!stage_keys(a, ssm, bar, phase, kb, K, true, keys, grp)) {
+      const long long n_look = (seg_end - seg) * (SECOND ? 3 : 1);
+      // (a list staged without a table for a short tail gets one when a longer run of the same request follows)
+      if (r != staged_r || (keys.declined && n_look * kTableAmort >= K)) {
+        // lookups the resolvers will make against the list before the next staging: this chunk's candidates of the
+        // request (second degree: up to five ids each, about three on the benchmark stores)
+        if (!stage_keys(a, ssm, bar, phase, kb, K, true, n_look, keys, grp)) {
           if (gtid == 0) {
             atomicExch(a.status, kDevWaitExpired);
             mbar_wait_bounded(bar, phase ^ 1u);
@@ -247,8 +290,8 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
       for (long long sub = seg; sub < seg_lim; sub += a.tile, ++it) {
         if (static_cast<int>(it % n_resolvers) != rwarp || dead) continue;
         const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_lim - sub));
-        const int s = it % kWsSlots;
-        if (it >= static_cast<unsigned>(kWsSlots) && !mbar_wait_bounded(empty0 + 8 * s, (it / kWsSlots - 1) & 1u)) {
+        const int s = it % kSlots;
+        if (it >= static_cast<unsigned>(kSlots) && !mbar_wait_bounded(empty0 + 8 * s, (it / kSlots - 1) & 1u)) {
           if (lane == 0) atomicExch(a.status, kDevWaitExpired);
           dead = true;  // the streamers are gone
           continue;
@@ -286,16 +329,23 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
           bool found[U];
           int pos[U];
 #pragma unroll
-          for (int h = 0; h < U; h += 4) {
-            const int64_t id4[4] = {auth[h], auth[h + 1], auth[h + 2], auth[h + 3]};
-            bool f4[4];
-            int p4[4];
-            keys.find_batch<4>(id4, f4, p4);
+          for (int h = 0; h < U; h += FB) {
+            int64_t idq[FB];
+            bool fq[FB];
+            int pq[FB];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              found[h + q] = f4[q];
-              pos[h + q] = p4[q];
+            for (int q = 0; q < FB; ++q) idq[q] = auth[h + q];
+            keys.find_batch<FB>(idq, fq, pq);
+#pragma unroll
+            for (int q = 0; q < FB; ++q) {
+              found[h + q] = fq[q];
+              pos[h + q] = pq[q];
             }
+          }
+          // everything up to here only read this launch's inputs; the mask bytes below are the first global stores
+          if (pdl_pending) {
+            pdl_wait();
+            pdl_pending = false;
           }
           if constexpr (SECOND) {
             // Engager lookups.  Most slots are empty, and which ones differs from lane to lane, so looking up
@@ -333,20 +383,20 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
               }
             }
             __syncwarp();
-            for (int w0 = 0; w0 < total; w0 += 4 * 32) {
-              int64_t id4[4];
+            for (int w0 = 0; w0 < total; w0 += FB * 32) {
+              int64_t idq[FB];
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
+              for (int q = 0; q < FB; ++q) {
                 const int wi = w0 + q * 32 + lane;
-                id4[q] = wi < total ? wl_id[wi] : -1;
+                idq[q] = wi < total ? wl_id[wi] : -1;
               }
-              bool f4[4];
-              int p4[4];
-              keys.find_batch<4>(id4, f4, p4);
+              bool fq[FB];
+              int pq[FB];
+              keys.find_batch<FB>(idq, fq, pq);
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
+              for (int q = 0; q < FB; ++q) {
                 const int wi = w0 + q * 32 + lane;
-                if (wi < total && f4[q]) apos_i[wl_tag[wi]] = p4[q];
+                if (wi < total && fq[q]) apos_i[wl_tag[wi]] = pq[q];
               }
             }
             __syncwarp();
@@ -432,11 +482,14 @@ __global__ void __launch_bounds__(kWsMaxThreads, 1) join_ws_kernel(const JoinArg
     }
   }
 
+  // no more work will be drawn by this block: a join queued behind this one may start to move in
+  if (gtid == 0) pdl_trigger();
+
   // stop slot: published by the warp whose turn it is
   if (static_cast<int>(it % n_resolvers) == rwarp && !dead) {
-    const int s = it % kWsSlots;
+    const int s = it % kSlots;
     bool ok = true;
-    if (it >= static_cast<unsigned>(kWsSlots)) ok = mbar_wait_bounded(empty0 + 8 * s, (it / kWsSlots - 1) & 1u);
+    if (it >= static_cast<unsigned>(kSlots)) ok = mbar_wait_bounded(empty0 + 8 * s, (it / kSlots - 1) & 1u);
     if (lane == 0) {
       if (!ok) atomicExch(a.status, kDevWaitExpired);
       WsSlot d;
