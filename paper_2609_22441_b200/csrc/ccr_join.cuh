@@ -230,8 +230,23 @@ template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0>
 __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND, CNP != 0>& sh,
                                            const int* s_idx, const int* s_pos, const int4* s_apos,
                                            const uint8_t* edge_base, const uint8_t* req_src, uint8_t* out, int cnt,
-                                           int lane, const float4* cosM = nullptr, uint4* stage = nullptr) {
+                                           int lane, const float4* cosM = nullptr, uint4* stage = nullptr,
+                                           uint8_t* mask_out = nullptr, const unsigned* s_types = nullptr) {
   const long long out_b = sh.out_b;
+  // mask bytes of the group (callers that resolved the candidates elsewhere and did not write them): lane = row;
+  // bit 0 author found, bits 1-4 engager slot found, bits 5-7 engagement types of the found slots
+  if (mask_out != nullptr && lane < cnt) {
+    unsigned m = s_pos[lane] >= 0 ? 1u : 0u;
+    if constexpr (SECOND) {
+      const int4 ap4 = s_apos[lane];
+      const int ap[4] = {ap4.x, ap4.y, ap4.z, ap4.w};
+      const unsigned ty = s_types[lane];
+#pragma unroll
+      for (int sl = 0; sl < 4; ++sl)
+        if (ap[sl] >= 0) m |= (1u << (1 + sl)) | (1u << (5 + ((ty >> (8 * sl)) & 0xffu) % 3u));
+    }
+    mask_out[lane] = static_cast<uint8_t>(m);
+  }
   // Derived section: the row streaming below is unchanged; the lanes that hold a piece of the item embedding
   // also drop it into this warp's staging block in shared memory (row-major, an odd number of 16-byte units
   // per row so that the read-back by lane = row is conflict-free), and once the group's stores are issued

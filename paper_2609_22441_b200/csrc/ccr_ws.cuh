@@ -5,10 +5,11 @@
 // share of the memory pipeline idles.  Here the two jobs run concurrently in one persistent block per SM:
 //   resolver warps : take chunks of the flat candidate range, stage each request's keys (TMA bulk copy +
 //                    mbarrier, waited on by the resolvers only), and fill a ring of sub-tile buffers in
-//                    shared memory with (position, match index) per candidate; they also write the mask
-//                    bytes.  Their latency (ids are 8-byte gathers, key staging) hides behind the streaming.
-//   streamer warps : consume the ring; for every 32-row group all loads are issued, then all stores —
-//                    nothing else.  They never touch keys, ids or barriers other than the ring's.
+//                    shared memory with (position, match index) per candidate; they write nothing to global
+//                    memory.  Their latency (ids are 8-byte gathers, key staging) hides behind the streaming.
+//   streamer warps : consume the ring; for every 32-row group the mask bytes are derived from the match
+//                    indices, all loads are issued, then all stores — nothing else.  They never touch keys,
+//                    ids or barriers other than the ring's.
 // Ring slots are handed over with shared-memory mbarriers: full[slot] (one arrival, by the resolvers, once the
 // slot is written) and empty[slot] (one arrival per streamer warp, once it has taken its last group of the
 // slot).  Warps wait on them individually — a streamer warp that is done with a slot moves on to the next
@@ -85,7 +86,7 @@ __host__ __device__ inline int ws_cos_bytes(int n_streamers, int stage_per_warp)
 }
 
 struct WsLayout {
-  int off_full, off_empty, off_slots, off_grab, off_offs, off_idx, off_pos, off_apos, off_cos, off_wl, off_keys, bytes;
+  int off_full, off_empty, off_slots, off_grab, off_offs, off_idx, off_pos, off_apos, off_types, off_cos, off_wl, off_keys, bytes;
   // n_req_cached: requests whose offsets are mirrored in shared memory (0 = read them from global memory)
   // cos_bytes: shared memory of the derived cosine section (0 = off): a block of member-embedding floats per
   // ring slot, then one embedding staging block per streamer warp
@@ -101,7 +102,8 @@ struct WsLayout {
     off_idx = (off_idx + 15) & ~15;
     off_pos = off_idx + n_slots * tile * 4;
     off_apos = off_pos + n_slots * tile * 4;
-    off_cos = off_apos + (second ? n_slots * tile * 16 : 0);
+    off_types = off_apos + (second ? n_slots * tile * 16 : 0);
+    off_cos = off_types + (second ? n_slots * tile * 4 : 0);
     off_wl = off_cos + cos_bytes;
     off_keys = off_wl + (second ? n_res * wl_items * (8 + 2) : 0);
     off_keys = (off_keys + 15) & ~15;
@@ -125,6 +127,7 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
   int* s_idx = reinterpret_cast<int*>(smem + lay.off_idx);
   int* s_pos = reinterpret_cast<int*>(smem + lay.off_pos);
   int4* s_apos = reinterpret_cast<int4*>(smem + lay.off_apos);
+  unsigned* s_types = reinterpret_cast<unsigned*>(smem + lay.off_types);
   float4* s_cos = reinterpret_cast<float4*>(smem + lay.off_cos);
   const SearchSmem ssm = carve_search(smem + lay.off_keys, a.search_area, true);
   const uint32_t bar = smem_u32(smem);
@@ -187,6 +190,7 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
       const int* idx = s_idx + s * a.tile;
       const int* pos = s_pos + s * a.tile;
       const int4* apos = s_apos + s * a.tile;
+      const unsigned* types = s_types + s * a.tile;
       // groups are handed out one at a time, so a warp that finishes early simply takes more
       for (;;) {
         int g = 0;
@@ -196,7 +200,7 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
         emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND, CNP>(a, sh, idx + g, pos + g, apos + g, edge_base, req_src,
                                                          a.out_rows + (d.out0 + g) * sh.out_b, min(32, d.n - g), lane,
                                                          COS ? s_cos + s * kCosSlotFloat4 : nullptr,
-                                                         COS ? cos_stage : nullptr);
+                                                         COS ? cos_stage : nullptr, a.out_mask + d.out0 + g, types + g);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
@@ -221,7 +225,6 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
   int staged_r = -1;     // request whose keys are in shared memory
   StagedKeys keys;
   keys.declined = false;
-  bool pdl_pending = true;  // this warp has not yet waited for the launch before this one
   // this warp's work list of engager lookups (second-degree joins)
   constexpr int U = SECOND ? (REBAL ? kRebalInFlight : 4) : 8;  // candidates a lane keeps in flight
   constexpr int FB = U < 4 ? U : 4;                              // lookups interleaved in one find_batch
@@ -300,6 +303,7 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
         int* out_idx = s_idx + s * a.tile;
         int* out_pos = s_pos + s * a.tile;
         int4* out_apos = s_apos + s * a.tile;
+        [[maybe_unused]] unsigned* out_types = s_types + s * a.tile;
         for (int base = 0; base < n; base += 32 * U) {
           int idx[U];
           int64_t auth[U];
@@ -341,11 +345,6 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
               found[h + q] = fq[q];
               pos[h + q] = pq[q];
             }
-          }
-          // everything up to here only read this launch's inputs; the mask bytes below are the first global stores
-          if (pdl_pending) {
-            pdl_wait();
-            pdl_pending = false;
           }
           if constexpr (SECOND) {
             // Engager lookups.  Most slots are empty, and which ones differs from lane to lane, so looking up
@@ -399,24 +398,13 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
                 if (wi < total && fq[q]) apos_i[wl_tag[wi]] = pq[q];
               }
             }
-            __syncwarp();
 #pragma unroll
             for (int u = 0; u < U; ++u) {
               const int i = base + u * 32 + lane;
               if (i < n) {
-                const int4 ap4 = out_apos[i];
-                const int ap[4] = {ap4.x, ap4.y, ap4.z, ap4.w};
-                unsigned m = found[u] ? 1u : 0u;
-#pragma unroll
-                for (int sl = 0; sl < 4; ++sl) {
-                  if (ap[sl] >= 0) {
-                    m |= 1u << (1 + sl);
-                    m |= 1u << (5 + ((types[u] >> (8 * sl)) & 0xffu) % 3u);
-                  }
-                }
                 out_idx[i] = idx[u];
                 out_pos[i] = found[u] ? pos[u] : -1;
-                a.out_mask[out0 + i] = static_cast<uint8_t>(m);
+                out_types[i] = types[u];  // the streamers derive the mask byte from the match indices and these
               }
             }
           } else {
@@ -426,7 +414,6 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
               if (i < n) {
                 out_idx[i] = idx[u];
                 out_pos[i] = found[u] ? pos[u] : -1;
-                a.out_mask[out0 + i] = found[u] ? 1 : 0;
               }
             }
           }
