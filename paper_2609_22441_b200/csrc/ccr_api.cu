@@ -36,6 +36,7 @@ constexpr long long kSmallLaunchCands = 131072;  // plain launches up to this si
 constexpr int kAutoSmemBudget = 160 * 1024;  // shared memory the warp-specialised kernel takes by default
 constexpr int kMaxTile = ccr::kMaxTileCands;
 constexpr size_t kStageBytes = 16u << 20;  // staging block of second-degree stores (ids uploaded from the host)
+constexpr int kHostGroups = 4;                       // request groups of a pipelined host-buffer join
 constexpr int kSchedRegions = 64;                    // launches of one store that may be in flight at once
 constexpr int kStatusHead = 4;                       // [0] wait expiry, [1] validation code; then the scheduling words:
                                                      // kSchedRegions regions of sched_stride ints
@@ -93,6 +94,14 @@ struct ccr_workspace {
   uint8_t* req_feats;
   uint8_t* out_rows;
   uint8_t* out_mask;
+  // Pipelined host entry: the payload of a large batch crosses PCIe in groups of requests on a stream of the
+  // workspace's own while the groups already there are being joined on the caller's stream.
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_begin;                  // caller's stream -> copy stream: everything queued before the call
+  cudaEvent_t ev_group[4];               // copy stream -> caller's stream: group g has arrived
+  cudaEvent_t ev_offsets[4];             // the pinned offset block of rotation slot k has been read by its copy
+  int64_t* host_offsets;                 // pinned: 4 rotation slots of (max_req + 1 + 4) rebased candidate offsets
+  int64_t calls;
 };
 
 struct ccr_idindex {
@@ -1093,10 +1102,18 @@ ccr_status ccr_workspace_create(const ccr_docstore* s, int32_t max_req, int64_t 
   ok = ok && cudaMalloc(&w->edge_feats, (max_edges + 2) * w->edge_b) == cudaSuccess;
   ok = ok && cudaMalloc(&w->edge_offsets, (max_req + 1) * 8) == cudaSuccess;
   ok = ok && cudaMalloc(&w->cand_idx, max_cands * 4) == cudaSuccess;
-  ok = ok && cudaMalloc(&w->cand_offsets, (max_req + 1) * 8) == cudaSuccess;
+  ok = ok && cudaMalloc(&w->cand_offsets, (max_req + 1 + kHostGroups) * 8) == cudaSuccess;
   ok = ok && cudaMalloc(&w->req_feats, (max_req + 1) * (w->req_b ? w->req_b : 16)) == cudaSuccess;
   ok = ok && cudaMalloc(&w->out_rows, max_cands * w->out_b_max) == cudaSuccess;
   ok = ok && cudaMalloc(&w->out_mask, max_cands) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&w->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&w->ev_begin, cudaEventDisableTiming) == cudaSuccess;
+  for (int g = 0; g < kHostGroups; ++g) {
+    ok = ok && cudaEventCreateWithFlags(&w->ev_group[g], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&w->ev_offsets[g], cudaEventDisableTiming) == cudaSuccess;
+  }
+  ok = ok && cudaHostAlloc(&w->host_offsets, static_cast<size_t>(kHostGroups) * (max_req + 1 + kHostGroups) * 8,
+                           cudaHostAllocDefault) == cudaSuccess;
   w->magic = kWsMagic;
   handle_add(w);
   if (!ok) {
@@ -1120,6 +1137,13 @@ ccr_status ccr_workspace_free(ccr_workspace* w) {
   cudaFree(w->req_feats);
   cudaFree(w->out_rows);
   cudaFree(w->out_mask);
+  if (w->copy_stream) cudaStreamDestroy(w->copy_stream);
+  if (w->ev_begin) cudaEventDestroy(w->ev_begin);
+  for (int g = 0; g < kHostGroups; ++g) {
+    if (w->ev_group[g]) cudaEventDestroy(w->ev_group[g]);
+    if (w->ev_offsets[g]) cudaEventDestroy(w->ev_offsets[g]);
+  }
+  if (w->host_offsets) cudaFreeHost(w->host_offsets);
   delete w;
   return CCR_OK;
 }
@@ -1149,23 +1173,91 @@ ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t out_b = out_row_bytes(s, flags);
   bool ok = true;
-  if (total_edges > 0) {
-    ok = ok && cudaMemcpyAsync(w->edge_keys, edge_keys, total_edges * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(w->edge_feats, edge_feats, total_edges * w->edge_b, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  // A batch of several large requests is pipelined: its requests are cut into up to kHostGroups groups of about
+  // equal candidate counts; group g + 1 crosses PCIe on the workspace's copy stream while group g is joined on the
+  // caller's stream (each group is an ordinary ccr_join_batch over its own requests, candidates renumbered from 0).
+  int n_groups = 1;
+  if (n_req >= kHostGroups && total_cands >= static_cast<int64_t>(kHostGroups) * 2 * kSmallLaunchCands && !(flags & CCR_FLAG_VALIDATE))
+    n_groups = kHostGroups;
+  if (n_groups == 1) {
+    if (total_edges > 0) {
+      ok = ok && cudaMemcpyAsync(w->edge_keys, edge_keys, total_edges * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+      ok = ok && cudaMemcpyAsync(w->edge_feats, edge_feats, total_edges * w->edge_b, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    }
+    ok = ok && cudaMemcpyAsync(w->edge_offsets, edge_offsets, (n_req + 1) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(w->cand_idx, cand_idx, total_cands * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(w->cand_offsets, cand_offsets, (n_req + 1) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (s->req_b > 0)
+      ok = ok && cudaMemcpyAsync(w->req_feats, req_feats, static_cast<size_t>(n_req) * w->req_b, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
+    const ccr_status js = ccr_join_batch(s, n_req, total_cands, max_edge_len, w->edge_keys, w->edge_feats, w->edge_offsets,
+                                         w->cand_idx, w->cand_offsets, s->req_b ? w->req_feats : nullptr, w->out_rows,
+                                         w->out_mask, flags, stream);
+    if (js != CCR_OK) return js;
+  } else {
+    // group boundaries: request ranges [first[g], first[g + 1]) with about total_cands / n_groups candidates each
+    int32_t first[kHostGroups + 1];
+    first[0] = 0;
+    int32_t r = 0;
+    for (int g = 1; g < n_groups; ++g) {
+      const int64_t want = total_cands * g / n_groups;
+      while (r < n_req && cand_offsets[r] < want) ++r;
+      if (r > n_req - (n_groups - g)) r = n_req - (n_groups - g);  // leave a request for every later group
+      if (r <= first[g - 1]) r = first[g - 1] + 1;
+      first[g] = r;
+    }
+    first[n_groups] = n_req;
+    // rebased candidate offsets of every group, in a pinned block of this call's rotation slot (a slot is reused
+    // four calls later; should its copy still be pending then, the host waits for it)
+    const int slot = static_cast<int>(w->calls++ % kHostGroups);
+    int64_t* h_off = w->host_offsets + static_cast<size_t>(slot) * (w->max_req + 1 + kHostGroups);
+    ok = ok && cudaEventSynchronize(w->ev_offsets[slot]) == cudaSuccess;
+    size_t k = 0;
+    size_t group_off[kHostGroups];
+    for (int g = 0; g < n_groups; ++g) {
+      group_off[g] = k;
+      for (int32_t q = first[g]; q <= first[g + 1]; ++q) h_off[k++] = cand_offsets[q] - cand_offsets[first[g]];
+    }
+    // the copy stream starts behind everything already queued on the caller's stream (earlier calls may still
+    // be reading the workspace)
+    ok = ok && cudaEventRecord(w->ev_begin, st) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(w->copy_stream, w->ev_begin, 0) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(w->cand_offsets, h_off, k * 8, cudaMemcpyHostToDevice, w->copy_stream) == cudaSuccess;
+    ok = ok && cudaEventRecord(w->ev_offsets[slot], w->copy_stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(w->edge_offsets, edge_offsets, (n_req + 1) * 8, cudaMemcpyHostToDevice, w->copy_stream) == cudaSuccess;
+    for (int g = 0; g < n_groups && ok; ++g) {
+      const int32_t r0 = first[g], r1 = first[g + 1];
+      const int64_t c0 = cand_offsets[r0], c1 = cand_offsets[r1], e0 = edge_offsets[r0], e1 = edge_offsets[r1];
+      if (e1 > e0) {
+        ok = ok && cudaMemcpyAsync(w->edge_keys + e0, edge_keys + e0, (e1 - e0) * 8, cudaMemcpyHostToDevice, w->copy_stream) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(w->edge_feats + e0 * w->edge_b, static_cast<const uint8_t*>(edge_feats) + e0 * w->edge_b,
+                                   (e1 - e0) * w->edge_b, cudaMemcpyHostToDevice, w->copy_stream) == cudaSuccess;
+      }
+      if (c1 > c0)
+        ok = ok && cudaMemcpyAsync(w->cand_idx + c0, cand_idx + c0, (c1 - c0) * 4, cudaMemcpyHostToDevice, w->copy_stream) == cudaSuccess;
+      if (s->req_b > 0)
+        ok = ok && cudaMemcpyAsync(w->req_feats + static_cast<size_t>(r0) * w->req_b,
+                                   static_cast<const uint8_t*>(req_feats) + static_cast<size_t>(r0) * w->req_b,
+                                   static_cast<size_t>(r1 - r0) * w->req_b, cudaMemcpyHostToDevice, w->copy_stream) == cudaSuccess;
+      ok = ok && cudaEventRecord(w->ev_group[g], w->copy_stream) == cudaSuccess;
+      ok = ok && cudaStreamWaitEvent(st, w->ev_group[g], 0) == cudaSuccess;
+      if (!ok) break;
+      if (c1 > c0) {
+        const ccr_status js = ccr_join_batch(s, r1 - r0, c1 - c0, max_edge_len, w->edge_keys, w->edge_feats, w->edge_offsets + r0,
+                                             w->cand_idx + c0, w->cand_offsets + group_off[g],
+                                             s->req_b ? w->req_feats + static_cast<size_t>(r0) * w->req_b : nullptr,
+                                             w->out_rows + static_cast<size_t>(c0) * out_b, w->out_mask + c0, flags, stream);
+        if (js != CCR_OK) return js;
+      }
+    }
+    if (!ok) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
   }
-  ok = ok && cudaMemcpyAsync(w->edge_offsets, edge_offsets, (n_req + 1) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(w->cand_idx, cand_idx, total_cands * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(w->cand_offsets, cand_offsets, (n_req + 1) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (s->req_b > 0)
-    ok = ok && cudaMemcpyAsync(w->req_feats, req_feats, static_cast<size_t>(n_req) * w->req_b, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (!ok) {
-    cudaGetLastError();
-    return CCR_ERR_CUDA;
-  }
-  const ccr_status js = ccr_join_batch(s, n_req, total_cands, max_edge_len, w->edge_keys, w->edge_feats, w->edge_offsets,
-                                       w->cand_idx, w->cand_offsets, s->req_b ? w->req_feats : nullptr, w->out_rows,
-                                       w->out_mask, flags, stream);
-  if (js != CCR_OK) return js;
   if (out_rows != nullptr)  // NULL: the rows stay in the workspace for a consumer on the device (ccr_workspace_outputs)
     ok = ok && cudaMemcpyAsync(out_rows, w->out_rows, total_cands * out_b, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(out_mask, w->out_mask, total_cands, cudaMemcpyDeviceToHost, st) == cudaSuccess;

@@ -226,7 +226,9 @@ __device__ __forceinline__ uint4 cosine_section(const JoinArgs& a, const uint4* 
   return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), 0u, 0u);
 }
 
-template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0>
+// SPLIT: the document pieces are loaded and stored before the edge pieces are requested (16 instead of 24 values of
+// a thread in flight: for kernels whose register budget the wide-row variants would otherwise overrun).
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0, bool SPLIT = false>
 __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND, CNP != 0>& sh,
                                            const int* s_idx, const int* s_pos, const int4* s_apos,
                                            const uint8_t* edge_base, const uint8_t* req_src, uint8_t* out, int cnt,
@@ -266,12 +268,14 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       dv[i] = make_uint4(0u, 0u, 0u, 0u);
       if (ridx >= 0) dv[i] = ldg128(a.doc_feats + static_cast<long long>(ridx) * (DOC_CH * 16) + piece * 16);
     }
+    if constexpr (!SPLIT) {
 #pragma unroll
-    for (int i = 0; i < EDGE_CH; ++i) {
-      const int c = i * 32 + lane, row = c / EDGE_CH, piece = c % EDGE_CH;
-      const int rpos = row < cnt ? s_pos[row] : -1;
-      ev[i] = make_uint4(0u, 0u, 0u, 0u);
-      if (rpos >= 0) ev[i] = ldg128(edge_base + static_cast<long long>(rpos) * (EDGE_CH * 16) + piece * 16);
+      for (int i = 0; i < EDGE_CH; ++i) {
+        const int c = i * 32 + lane, row = c / EDGE_CH, piece = c % EDGE_CH;
+        const int rpos = row < cnt ? s_pos[row] : -1;
+        ev[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (rpos >= 0) ev[i] = ldg128(edge_base + static_cast<long long>(rpos) * (EDGE_CH * 16) + piece * 16);
+      }
     }
 #pragma unroll
     for (int i = 0; i < DOC_CH; ++i) {
@@ -280,6 +284,15 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       if constexpr (kCos) {
         const int q = piece - p0;
         if (q >= 0 && q < np) stage[row * sstride + q] = dv[i];
+      }
+    }
+    if constexpr (SPLIT) {
+#pragma unroll
+      for (int i = 0; i < EDGE_CH; ++i) {
+        const int c = i * 32 + lane, row = c / EDGE_CH, piece = c % EDGE_CH;
+        const int rpos = row < cnt ? s_pos[row] : -1;
+        ev[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (rpos >= 0) ev[i] = ldg128(edge_base + static_cast<long long>(rpos) * (EDGE_CH * 16) + piece * 16);
       }
     }
 #pragma unroll
@@ -349,7 +362,7 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
   }
 }
 
-constexpr int kUnroll = 8;  // candidates a thread keeps in flight in phase A
+constexpr int kUnrollMax = 8;  // candidates a thread keeps in flight in phase A (4 in the variants that would spill with 8)
 #ifndef CCR_JOIN_MIN_BLOCKS
 #define CCR_JOIN_MIN_BLOCKS 2
 #endif
@@ -370,6 +383,9 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
   const uint32_t bar = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND> sh(a);
+  // (the generic-width and the wide-row second-degree variants would spill with eight candidates of a thread in
+  // flight in phase A)
+  constexpr int kUnroll = (SECOND && (DOC_CH == 0 || EDGE_CH >= 8)) ? 4 : kUnrollMax;
 
   if (tid == 0) {
     mbar_init(bar, 1);
@@ -557,8 +573,8 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
 
       // ================= phase B: stream the rows =================
       for (int g = warp * 32; g < n; g += kWarps * 32) {
-        emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND>(a, sh, s_idx + g, s_pos + g, s_apos + g, edge_base, req_src,
-                                                    a.out_rows + (out0 + g) * sh.out_b, min(32, n - g), lane);
+        emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND, 0, (EDGE_CH >= 8)>(a, sh, s_idx + g, s_pos + g, s_apos + g, edge_base, req_src,
+                                                                       a.out_rows + (out0 + g) * sh.out_b, min(32, n - g), lane);
       }
       __syncthreads();  // phase A of the next sub-tile overwrites the resolved arrays (and, in merge mode, the keys)
     }

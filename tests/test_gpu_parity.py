@@ -308,6 +308,61 @@ def test_host_buffer_entry_matches_device_entry(B):
     store.free()
 
 
+def test_host_buffer_entry_pipelines_a_large_batch_in_request_groups(B):
+    """Batches of several large requests cross PCIe in groups of requests while earlier groups are joined: very
+    unequal requests (one of them empty, one holding a third of the candidates), twice in a row on one workspace,
+    rows left on the device and rows copied back."""
+    base = W.config1(n_docs=400_000, n_req=24, n_cand=60_000)
+    b0 = base.batch
+    rng = np.random.default_rng(3)
+    sizes = rng.integers(5_000, 60_001, size=b0.n_req)
+    sizes[5] = 0
+    sizes[17] = 60_000
+    keys_l, feats_l, cands_l = [], [], []
+    for r in range(b0.n_req):
+        e0, e1 = int(b0.edge_offsets[r]), int(b0.edge_offsets[r + 1])
+        c0 = int(b0.cand_offsets[r])
+        keys_l.append(b0.edge_keys[e0:e1])
+        feats_l.append(b0.edge_feats[e0:e1])
+        cands_l.append(b0.cand_idx[c0:c0 + int(sizes[r])])
+    # one request of a third of all candidates (repeats are fine)
+    cands_l[2] = np.concatenate([b0.cand_idx[int(b0.cand_offsets[2]):int(b0.cand_offsets[3])]] * 8)
+    wl = W.Workload("ragged-large", 0, base.store, W.assemble_batch(keys_l, feats_l, cands_l, b0.req_feats, b0.edge_dim,
+                                                                   b0.edge_dtype, b0.req_dim, b0.req_dtype))
+    b = wl.batch
+    assert b.total_cands > 1_100_000
+    want_rows, want_mask = oracle.join_workload(wl, n_threads=4)
+    store = B.store_from_workload(wl)
+    ws = B.Workspace(store, b.n_req, b.total_cands, len(b.edge_keys))
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    args = [pin(b.edge_keys), pin(b.edge_feats.view(np.uint8)), pin(b.edge_offsets), pin(b.cand_idx),
+            pin(b.cand_offsets), pin(b.req_feats.view(np.uint8))]
+    out_b = store.out_row_bytes()
+    out_mask = torch.empty((b.total_cands,), dtype=torch.uint8).pin_memory()
+    rows_ptr, _ = ws.outputs()
+
+    class _View:  # the workspace's device buffer seen as a tensor (CUDA array interface)
+        __cuda_array_interface__ = {"shape": (b.total_cands * out_b,), "typestr": "|u1", "data": (rows_ptr, False), "version": 2}
+
+    dev_rows = torch.as_tensor(_View(), device="cuda").view(b.total_cands, out_b)
+    for _ in range(2):
+        out_mask.fill_(9)
+        dev_rows.fill_(7)
+        torch.cuda.synchronize()
+        B.ccr_join_batch_host(store, ws, b.n_req, b.total_cands, b.max_edge_len, len(b.edge_keys), *args, None, out_mask)
+        torch.cuda.synchronize()
+        assert np.array_equal(out_mask.numpy(), want_mask)
+        assert np.array_equal(dev_rows.cpu().numpy(), want_rows)
+    out_rows = torch.empty((b.total_cands, out_b), dtype=torch.uint8).pin_memory()
+    out_mask.fill_(9)
+    B.ccr_join_batch_host(store, ws, b.n_req, b.total_cands, b.max_edge_len, len(b.edge_keys), *args, out_rows, out_mask)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_rows.numpy(), want_rows) and np.array_equal(out_mask.numpy(), want_mask)
+    assert store.device_status() == B.CCR_OK
+    ws.free()
+    store.free()
+
+
 def test_validate_flag_reports_broken_preconditions(B):
     wl = W.config1(n_docs=20_000, n_req=4, n_cand=500)
     store = B.store_from_workload(wl)
