@@ -46,7 +46,9 @@ typedef enum {
   CCR_ERR_CUDA = 4,        /* a CUDA runtime call failed, or no usable device                      */
   CCR_ERR_BAD_HANDLE = 5,  /* handle is NULL, freed or not one of ours                             */
   CCR_ERR_VALIDATION = 6,  /* CCR_FLAG_VALIDATE found a broken precondition                        */
-  CCR_ERR_DEVICE_WAIT = 7  /* a bounded device-side wait ran out (reported by device_status)       */
+  CCR_ERR_DEVICE_WAIT = 7, /* a bounded device-side wait ran out (reported by device_status)       */
+  CCR_ERR_BOUNDS = 8       /* bounds-checked build only (-DCCR_DEBUG_BOUNDS): a join kernel computed an address outside
+                              the buffers of its launch; the access was skipped (reported by device_status)          */
 } ccr_status;
 
 typedef enum { CCR_F16 = 0, CCR_F32 = 1 } ccr_dtype;
@@ -95,6 +97,9 @@ enum {
                                            the row-streaming warps (comparison aid)                                  */
   CCR_FLAG_NO_OVERLAP        = 1u << 11, /* do not let this launch move in behind a join that is still draining on the same
                                            stream (see "Back-to-back joins" at ccr_join_batch)                       */
+  CCR_FLAG_WARP_SEARCH       = 1u << 12, /* lists that are searched in global memory (CCR_FLAG_FORCE_GLOBAL, key capacity 0)
+                                           use the warp-cooperative 32-ary search: one id at a time, 32 pivots per round
+                                           picked by ballot (comparison aid: the lane-per-id binary search is faster)     */
   CCR_FLAG_WARP_SPECIALISED  = 1u << 9  /* take the warp-specialised kernel whatever the launch size (by default a
                                            ragged launch of at most 131,072 candidates — a single request —
                                            runs on the two-phase kernel, which has the shorter start-up)      */
@@ -400,7 +405,11 @@ ccr_status ccr_join_payload_static(const ccr_docstore* store,
 
 /* Synchronise `stream` and report the store's device-side status word: CCR_OK, or
  * CCR_ERR_DEVICE_WAIT if a kernel gave up a bounded wait for a shared-memory bulk copy since the
- * last call (the affected rows of that launch were not written).  Clears the word.                 */
+ * last call (the affected rows of that launch were not written).  Clears the word.
+ * The bounds-checked build of the library (compiled with -DCCR_DEBUG_BOUNDS; `python -m paper_2609_22441_b200.build
+ * --debug-bounds` writes it next to the release build) checks every global address the join kernels compute against
+ * the extents of the launch's buffers, leaves out an access that falls outside (never a trap) and reports
+ * CCR_ERR_BOUNDS here; it synchronises after every join and is meant for tests, not for serving.            */
 ccr_status ccr_docstore_device_status(ccr_docstore* store, void* stream);
 
 /* Self-test of the failure-reporting path (no fault, trap or hang is involved): enqueues a one-block kernel
@@ -428,6 +437,11 @@ int64_t ccr_docstore_launch_count(const ccr_docstore* store);
 
 const char* ccr_status_str(ccr_status s);
 int         ccr_version(void);
+/* 1 in the bounds-checked build, 0 in the release build. */
+int         ccr_debug_bounds_enabled(void);
+/* Bounds-checked build only (no-op otherwise): pretend that the output buffers of the following joins on this store
+ * end `rows` rows early, so that the mechanism itself can be tested without a real out-of-range access.   */
+ccr_status  ccr_debug_shrink_outputs(ccr_docstore* store, int64_t rows);
 
 #ifdef __cplusplus
 }

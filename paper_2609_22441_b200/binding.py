@@ -25,6 +25,7 @@ CCR_ERR_CUDA = 4
 CCR_ERR_BAD_HANDLE = 5
 CCR_ERR_VALIDATION = 6
 CCR_ERR_DEVICE_WAIT = 7
+CCR_ERR_BOUNDS = 8
 
 CCR_F16 = 0
 CCR_F32 = 1
@@ -41,6 +42,7 @@ CCR_FLAG_COSINE = 1 << 8
 CCR_FLAG_WARP_SPECIALISED = 1 << 9
 CCR_FLAG_NO_REBALANCE = 1 << 10
 CCR_FLAG_NO_OVERLAP = 1 << 11
+CCR_FLAG_WARP_SEARCH = 1 << 12
 
 EXPORTS = (
     "ccr_docstore_create", "ccr_docstore_upload", "ccr_docstore_upsert", "ccr_docstore_free", "ccr_out_row_bytes", "ccr_join_batch",
@@ -49,6 +51,7 @@ EXPORTS = (
     "ccr_docstore_set_tuning", "ccr_docstore_launch_count", "ccr_status_str", "ccr_version",
     "ccr_static_payload_capacity", "ccr_join_payload_static", "ccr_docstore_selftest_wait",
     "ccr_sort_edges", "ccr_idindex_create", "ccr_idindex_free", "ccr_resolve_ids",
+    "ccr_debug_bounds_enabled", "ccr_debug_shrink_outputs",
 )
 
 
@@ -154,6 +157,10 @@ def lib() -> ctypes.CDLL:
     L.ccr_status_str.argtypes = [ctypes.c_int]
     L.ccr_version.restype = ctypes.c_int
     L.ccr_version.argtypes = []
+    L.ccr_debug_bounds_enabled.restype = ctypes.c_int
+    L.ccr_debug_bounds_enabled.argtypes = []
+    L.ccr_debug_shrink_outputs.restype = ctypes.c_int
+    L.ccr_debug_shrink_outputs.argtypes = [vp, i64]
     _lib = L
     return L
 

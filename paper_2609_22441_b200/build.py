@@ -31,6 +31,21 @@ def is_stale() -> bool:
     return any(os.path.getmtime(p) > t for p in _deps())
 
 
+DEBUG_LIB = os.path.join(HERE, "libccr_debug.so")
+
+
+def build_debug(force: bool = False) -> str:
+    """The bounds-checked build (-DCCR_DEBUG_BOUNDS): every global address of the join kernels is checked against the
+    launch's buffers; load it through CCR_LIB_OVERRIDE.  For tests, not for serving."""
+    if not force and os.path.exists(DEBUG_LIB) and all(os.path.getmtime(p) <= os.path.getmtime(DEBUG_LIB) for p in _deps()):
+        return DEBUG_LIB
+    nvcc = os.environ.get("NVCC", "nvcc")
+    tmp = DEBUG_LIB + ".tmp.%d" % os.getpid()
+    subprocess.run([nvcc] + NVCC_FLAGS + ["-DCCR_DEBUG_BOUNDS", "-o", tmp] + SOURCES, check=True)
+    os.replace(tmp, DEBUG_LIB)
+    return DEBUG_LIB
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not is_stale():
         return LIB
@@ -43,4 +58,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--debug-bounds" in sys.argv:
+        print(build_debug(force="--force" in sys.argv))
+    else:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

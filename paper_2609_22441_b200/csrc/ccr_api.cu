@@ -77,6 +77,7 @@ struct ccr_docstore {
   int n_sms;
   int sched_stride;   // ints per scheduling region (next tile, finished blocks; a region has a 128-byte line to itself)
   int cos_first, cos_dim, cos_chunks;  // derived cosine section (cos_chunks == 0: not configured)
+  int64_t dbg_shrink_rows;             // bounds-checked build: rows cut off the registered output extents
   std::atomic<int64_t> launches;  // kernels launched for this store; also hands out the scheduling-word pairs
 };
 
@@ -222,6 +223,13 @@ using WsKernelFn = void (*)(const ccr::JoinArgs, int);
 // pieces (the paper's 50 values span 7); any other shape runs on the generic variant.
 constexpr int kTunedCosPieces = 7;
 
+// The bounds-checked build leaves the register-rebalanced form out: its checks do not fit the fixed register split.
+#ifdef CCR_DEBUG_BOUNDS
+constexpr bool kRebalBuilt = false;
+#else
+constexpr bool kRebalBuilt = true;
+#endif
+
 struct Variant {
   int doc_ch, edge_ch, req_ch;
   KernelFn first, second, merge;
@@ -235,7 +243,7 @@ struct Variant {
         ccr::join_ws_kernel<D, E, R, false>, ccr::join_ws_kernel<D, E, R, true>,                                  \
         ccr::join_ws_kernel<D, E, R, false, (D > 0 ? kTunedCosPieces : -1)>,                                      \
         ccr::join_ws_kernel<D, E, R, true, (D > 0 ? kTunedCosPieces : -1)>,                                       \
-        ccr::join_ws_kernel<D, E, R, true, 0, true>                                                               \
+        ccr::join_ws_kernel<D, E, R, true, 0, kRebalBuilt>                                                        \
   }
 
 const Variant kVariants[] = {
@@ -287,6 +295,24 @@ ccr_status allow_large_smem() {
   return CCR_OK;
 }
 
+#ifdef CCR_DEBUG_BOUNDS
+// Bounds-checked build: the extents of every buffer a join launch may touch, registered before the launch.
+struct DbgRegistrar {
+  ccr::DbgTable t;
+  DbgRegistrar() { std::memset(&t, 0, sizeof(t)); }
+  void add(const void* p, size_t bytes) {
+    if (p == nullptr || bytes == 0 || t.n >= 16) return;
+    t.r[t.n].lo = reinterpret_cast<unsigned long long>(p);
+    t.r[t.n].hi = t.r[t.n].lo + bytes;
+    ++t.n;
+  }
+  bool commit(int* word) {
+    t.word = word;
+    return cudaMemcpyToSymbol(ccr::g_dbg, &t, sizeof(t)) == cudaSuccess;
+  }
+};
+#endif
+
 size_t out_row_bytes(const ccr_docstore* s, uint32_t flags) {
   const bool second = s->desc.max_actors > 0 && !(flags & CCR_FLAG_FIRST_DEGREE_ONLY);
   return static_cast<size_t>(s->doc_b) + s->edge_b * (second ? 2 : 1) + s->req_b + ((flags & CCR_FLAG_COSINE) ? ccr::kCosSectionBytes : 0);
@@ -298,6 +324,20 @@ extern "C" {
 
 int ccr_version(void) { return 100; }
 
+int ccr_debug_bounds_enabled(void) {
+#ifdef CCR_DEBUG_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+ccr_status ccr_debug_shrink_outputs(ccr_docstore* s, int64_t rows) {
+  if (!good(s)) return CCR_ERR_BAD_HANDLE;
+  s->dbg_shrink_rows = rows < 0 ? 0 : rows;
+  return CCR_OK;
+}
+
 const char* ccr_status_str(ccr_status s) {
   switch (s) {
     case CCR_OK: return "ok";
@@ -308,6 +348,7 @@ const char* ccr_status_str(ccr_status s) {
     case CCR_ERR_BAD_HANDLE: return "bad handle";
     case CCR_ERR_VALIDATION: return "input validation failed";
     case CCR_ERR_DEVICE_WAIT: return "a bounded device-side wait expired";
+    case CCR_ERR_BOUNDS: return "bounds-checked build: an address outside the launch's buffers was skipped";
   }
   return "unknown status";
 }
@@ -536,6 +577,7 @@ ccr_status ccr_docstore_device_status(ccr_docstore* s, void* stream) {
     cudaGetLastError();
     return CCR_ERR_CUDA;
   }
+  if (s->status_host[2] != 0) return CCR_ERR_BOUNDS;  // only the bounds-checked build ever sets this word
   return s->status_host[0] == ccr::kDevWaitExpired ? CCR_ERR_DEVICE_WAIT : CCR_OK;
 }
 
@@ -783,7 +825,7 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   }
   // second-degree joins on the default warp split take the register-rebalanced form (12 + 8 warps); a configured
   // split, a configured sub-tile and the cosine section keep the 16-warp kernel
-  const bool rebal = use_ws && second && !cos && s->ws_streamers == 0 && s->tile == 0 && !(flags & CCR_FLAG_NO_REBALANCE);
+  const bool rebal = kRebalBuilt && use_ws && second && !cos && s->ws_streamers == 0 && s->tile == 0 && !(flags & CCR_FLAG_NO_REBALANCE);
   const int n_str = rebal ? ccr::kRebalStreamers : (s->ws_streamers > 0 ? s->ws_streamers : 12);
   const int n_res = rebal ? ccr::kRebalResolvers : (s->ws_resolvers > 0 ? s->ws_resolvers : 4);
   const int cos_stage = cos ? 32 * (((s->cos_dim + 7) / 8) | 1) * 16 : 0;
@@ -878,12 +920,42 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   a.key_cap = key_cap;
   a.search_area = static_cast<int>(area);
   a.min_stride_log2 = (flags & CCR_FLAG_FORCE_SAMPLED) ? 2 : 0;
+  a.warp_search = ((flags & CCR_FLAG_WARP_SEARCH) && use_ws) ? 1 : 0;  // its callers there are converged warps
   a.status = s->status;
   a.sched = nullptr;
 
   DeviceScope scope(s->desc.device);
   if (!scope.ok) return CCR_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+#ifdef CCR_DEBUG_BOUNDS
+  {
+    // the true sizes of the ragged arrays are on the device: read them back (this build synchronises anyway)
+    int64_t C = 0, E = 0;
+    if (cudaStreamSynchronize(st) != cudaSuccess ||
+        cudaMemcpy(&C, cand_offsets + n_req, 8, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(&E, edge_offsets + n_req, 8, cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
+    const size_t out_b = out_row_bytes(s, flags);
+    int64_t rows = n_max > 0 ? static_cast<int64_t>(n_req) * n_max : C;
+    rows = rows > s->dbg_shrink_rows ? rows - s->dbg_shrink_rows : 0;
+    DbgRegistrar reg;
+    reg.add(s->doc_feats, static_cast<size_t>(s->desc.n_docs) * s->doc_b);
+    reg.add(s->author_ids, static_cast<size_t>(s->desc.n_docs) * 8);
+    reg.add(s->id_recs, static_cast<size_t>(s->desc.n_docs) * sizeof(ccr::IdRec));
+    reg.add(edge_keys, static_cast<size_t>(E) * 8);
+    reg.add(edge_feats, static_cast<size_t>(E) * s->edge_b);
+    reg.add(edge_offsets, static_cast<size_t>(n_req + 1) * 8);
+    reg.add(cand_idx, static_cast<size_t>(C) * 4);
+    reg.add(cand_offsets, static_cast<size_t>(n_req + 1) * 8);
+    reg.add(req_feats, static_cast<size_t>(n_req) * s->req_b);
+    if (cos) reg.add(member_emb, static_cast<size_t>(n_req) * s->cos_chunks * s->cos_dim * 2);
+    reg.add(out_rows, static_cast<size_t>(rows) * out_b);
+    reg.add(out_mask, static_cast<size_t>(rows));
+    if (!reg.commit(s->status + 2)) return CCR_ERR_CUDA;
+  }
+#endif
 
   if (flags & CCR_FLAG_VALIDATE) {
     validate_kernel<<<n_req, 256, 0, st>>>(a, (flags & CCR_FLAG_CANDS_SORTED) ? 1 : 0, s->status + 1);
@@ -952,6 +1024,9 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
     s->launches++;
   }
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+#ifdef CCR_DEBUG_BOUNDS
+  if (cudaStreamSynchronize(st) != cudaSuccess) return CCR_ERR_CUDA;  // the table is one per process: no overlap
+#endif
   return CCR_OK;
 }
 
@@ -985,6 +1060,16 @@ ccr_status padded_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cand
   {
     DeviceScope scope(s->desc.device);
     if (!scope.ok) return CCR_ERR_CUDA;
+#ifdef CCR_DEBUG_BOUNDS
+    {
+      DbgRegistrar reg;
+      const size_t out_b = out_row_bytes(s, flags);
+      reg.add(cand_offsets, static_cast<size_t>(n_req + 1) * 8);
+      reg.add(out_rows, static_cast<size_t>(n_req) * n_max * out_b);
+      reg.add(out_mask, static_cast<size_t>(n_req) * n_max);
+      if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess || !reg.commit(s->status + 2)) return CCR_ERR_CUDA;
+    }
+#endif
     // enough blocks to fill the device however few requests there are
     const unsigned slices = static_cast<unsigned>(std::max(1, std::min(64, (2 * s->n_sms + n_req - 1) / n_req)));
     ccr::pad_fill_kernel<<<dim3(static_cast<unsigned>(n_req), slices), ccr::kPadThreads, 0,

@@ -70,6 +70,7 @@ struct JoinArgs {
   int key_cap;                // longest list a block may stage in full per request; 0 = search global memory
   int search_area;            // bytes of shared memory the search may use for keys, tables or sampled keys
   int min_stride_log2;        // >0 forces sampling with at least this stride (testing aid)
+  int warp_search;            // searches that run in global memory use the warp-cooperative 32-ary search (comparison aid)
   int* status;                // device status words
   int* sched;                 // two scheduling words (next tile, finished blocks), zero between launches; or null
 };
@@ -146,16 +147,55 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-__device__ __forceinline__ uint4 ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+// ---- bounds-checked build (-DCCR_DEBUG_BOUNDS) ------------------------------------------------------------------
+// Every global load and store of the join kernels goes through gload / gstore / ldg128 / st128_stream.  In the
+// checked build the host registers the extent of every buffer of the launch in g_dbg; an access that does not lie
+// inside one of them is not made (loads give zero), and a code is left in the store's third status word, which
+// ccr_docstore_device_status reports as CCR_ERR_BOUNDS.  Nothing traps.  The release build compiles the checks away.
+#ifdef CCR_DEBUG_BOUNDS
+struct DbgRange {
+  unsigned long long lo, hi;
+};
+struct DbgTable {
+  DbgRange r[16];
+  int n;
+  int* word;
+};
+__device__ DbgTable g_dbg;
+__device__ __noinline__ bool dbg_in_bounds(const void* p, int bytes) {
+  const unsigned long long q = reinterpret_cast<unsigned long long>(p);
+  for (int i = 0; i < g_dbg.n; ++i)
+    if (q >= g_dbg.r[i].lo && q + static_cast<unsigned long long>(bytes) <= g_dbg.r[i].hi) return true;
+  if (g_dbg.word != nullptr) atomicCAS(g_dbg.word, 0, 1);
+  return false;
+}
+#define CCR_CHK(p, bytes) ::ccr::dbg_in_bounds((p), (bytes))
+#else
+#define CCR_CHK(p, bytes) true
+#endif
+
+template <typename T>
+__device__ __forceinline__ T gload(const T* p) {
+  if (!CCR_CHK(p, static_cast<int>(sizeof(T)))) return T{};
+  return __ldg(p);
+}
+template <typename T, typename V>
+__device__ __forceinline__ void gstore(T* p, V v) {
+  if (CCR_CHK(p, static_cast<int>(sizeof(T)))) *p = static_cast<T>(v);
+}
+__device__ __forceinline__ uint4 ldg128(const void* p) {
+  if (!CCR_CHK(p, 16)) return make_uint4(0u, 0u, 0u, 0u);
+  return __ldg(reinterpret_cast<const uint4*>(p));
+}
 
 // Author id of the document at position idx (0 <= idx < n_docs).
 __device__ __forceinline__ long long load_author(const JoinArgs& a, int idx) {
-  return a.id_recs != nullptr ? __ldg(&a.id_recs[idx].author) : __ldg(a.author_ids + idx);
+  return a.id_recs != nullptr ? gload(&a.id_recs[idx].author) : gload(a.author_ids + idx);
 }
 // Engager ids and types (one byte per slot, packed little-endian) of the document at position idx.
 __device__ __forceinline__ void load_actors(const JoinArgs& a, int idx, long long (&act)[4], unsigned& types) {
   const uint4* r = reinterpret_cast<const uint4*>(a.id_recs + idx);
-  const uint4 w0 = __ldg(r), w1 = __ldg(r + 1), w2 = __ldg(r + 2);  // author|a0, a1|a2, a3|types
+  const uint4 w0 = gload(r), w1 = gload(r + 1), w2 = gload(r + 2);  // author|a0, a1|a2, a3|types
   act[0] = static_cast<long long>(w0.z | (static_cast<unsigned long long>(w0.w) << 32));
   act[1] = static_cast<long long>(w1.x | (static_cast<unsigned long long>(w1.y) << 32));
   act[2] = static_cast<long long>(w1.z | (static_cast<unsigned long long>(w1.w) << 32));
@@ -165,7 +205,9 @@ __device__ __forceinline__ void load_actors(const JoinArgs& a, int idx, long lon
 
 // Output rows are written once and never read back by the kernel: streaming (evict-first) stores keep
 // them from displacing the keys, edge tables and id arrays that live in L2.
-__device__ __forceinline__ void st128_stream(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
+__device__ __forceinline__ void st128_stream(void* p, uint4 v) {
+  if (CCR_CHK(p, 16)) __stcs(reinterpret_cast<uint4*>(p), v);
+}
 
 // Branch-free lower bound over n ascending keys: number of keys < id.  Every lane of a warp runs the
 // same trip count when n is warp-uniform.
@@ -184,10 +226,10 @@ __device__ __forceinline__ int lower_bound_global(const int64_t* g, int n, int64
   int lo = 0;
   while (n > 1) {
     const int half = n >> 1;
-    lo = (__ldg(g + lo + half - 1) < id) ? lo + half : lo;
+    lo = (gload(g + lo + half - 1) < id) ? lo + half : lo;
     n -= half;
   }
-  if (n == 1) lo += (__ldg(g + lo) < id) ? 1 : 0;
+  if (n == 1) lo += (gload(g + lo) < id) ? 1 : 0;
   return lo;
 }
 

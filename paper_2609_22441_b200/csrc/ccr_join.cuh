@@ -120,8 +120,8 @@ __device__ __forceinline__ int request_of(const int64_t* co, int n_req, long lon
 
 // Key count of request r, clamped to what the host promised (so a malformed offset cannot widen a search).
 __device__ __forceinline__ int request_keys(const JoinArgs& a, int r, long long& kb) {
-  kb = __ldg(a.edge_offsets + r);
-  long long K = __ldg(a.edge_offsets + r + 1) - kb;
+  kb = gload(a.edge_offsets + r);
+  long long K = gload(a.edge_offsets + r + 1) - kb;
   K = K < 0 ? 0 : (K > a.max_edge_len ? a.max_edge_len : K);
   return static_cast<int>(K);
 }
@@ -143,7 +143,7 @@ __device__ __forceinline__ int block_lower_bound(const int64_t* g, int K, int64_
   while (n > 0) {
     const int step = (n + kThreads - 1) / kThreads;
     const long long p = static_cast<long long>(lo) + static_cast<long long>(threadIdx.x + 1) * step - 1;
-    const int below = (p < lo + n) && (__ldg(g + p) < id);
+    const int below = (p < lo + n) && (gload(g + p) < id);
     const int c = __syncthreads_count(below);
     const int nlo = min(lo + c * step, lo + n);
     n = min(step - 1, lo + n - nlo);
@@ -226,9 +226,7 @@ __device__ __forceinline__ uint4 cosine_section(const JoinArgs& a, const uint4* 
   return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), 0u, 0u);
 }
 
-// SPLIT: the document pieces are loaded and stored before the edge pieces are requested (16 instead of 24 values of
-// a thread in flight: for kernels whose register budget the wide-row variants would otherwise overrun).
-template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0, bool SPLIT = false>
+template <int DOC_CH, int EDGE_CH, int REQ_CH, bool SECOND, int CNP = 0>
 __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC_CH, EDGE_CH, REQ_CH, SECOND, CNP != 0>& sh,
                                            const int* s_idx, const int* s_pos, const int4* s_apos,
                                            const uint8_t* edge_base, const uint8_t* req_src, uint8_t* out, int cnt,
@@ -247,7 +245,7 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       for (int sl = 0; sl < 4; ++sl)
         if (ap[sl] >= 0) m |= (1u << (1 + sl)) | (1u << (5 + ((ty >> (8 * sl)) & 0xffu) % 3u));
     }
-    mask_out[lane] = static_cast<uint8_t>(m);
+    gstore(mask_out + lane, m);
   }
   // Derived section: the row streaming below is unchanged; the lanes that hold a piece of the item embedding
   // also drop it into this warp's staging block in shared memory (row-major, an odd number of 16-byte units
@@ -268,14 +266,12 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       dv[i] = make_uint4(0u, 0u, 0u, 0u);
       if (ridx >= 0) dv[i] = ldg128(a.doc_feats + static_cast<long long>(ridx) * (DOC_CH * 16) + piece * 16);
     }
-    if constexpr (!SPLIT) {
 #pragma unroll
-      for (int i = 0; i < EDGE_CH; ++i) {
-        const int c = i * 32 + lane, row = c / EDGE_CH, piece = c % EDGE_CH;
-        const int rpos = row < cnt ? s_pos[row] : -1;
-        ev[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (rpos >= 0) ev[i] = ldg128(edge_base + static_cast<long long>(rpos) * (EDGE_CH * 16) + piece * 16);
-      }
+    for (int i = 0; i < EDGE_CH; ++i) {
+      const int c = i * 32 + lane, row = c / EDGE_CH, piece = c % EDGE_CH;
+      const int rpos = row < cnt ? s_pos[row] : -1;
+      ev[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (rpos >= 0) ev[i] = ldg128(edge_base + static_cast<long long>(rpos) * (EDGE_CH * 16) + piece * 16);
     }
 #pragma unroll
     for (int i = 0; i < DOC_CH; ++i) {
@@ -284,15 +280,6 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       if constexpr (kCos) {
         const int q = piece - p0;
         if (q >= 0 && q < np) stage[row * sstride + q] = dv[i];
-      }
-    }
-    if constexpr (SPLIT) {
-#pragma unroll
-      for (int i = 0; i < EDGE_CH; ++i) {
-        const int c = i * 32 + lane, row = c / EDGE_CH, piece = c % EDGE_CH;
-        const int rpos = row < cnt ? s_pos[row] : -1;
-        ev[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (rpos >= 0) ev[i] = ldg128(edge_base + static_cast<long long>(rpos) * (EDGE_CH * 16) + piece * 16);
       }
     }
 #pragma unroll
@@ -404,7 +391,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
 
   long long seg = j0;
   while (seg < j1 && r < a.n_req) {
-    const long long rend = __ldg(a.cand_offsets + r + 1);
+    const long long rend = gload(a.cand_offsets + r + 1);
     if (rend <= seg) {  // request without candidates here
       ++r;
       continue;
@@ -425,7 +412,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
     }
 
     // padded output: a request's candidates behind its n_max-th have no slot and are dropped
-    const long long r_first = PADDED ? __ldg(a.cand_offsets + r) : 0;
+    const long long r_first = PADDED ? gload(a.cand_offsets + r) : 0;
     const long long seg_lim = PADDED ? min(seg_end, r_first + a.n_max) : seg_end;
     for (long long sub = seg; sub < seg_lim; sub += a.tile) {
       const int n = static_cast<int>(min(static_cast<long long>(a.tile), seg_lim - sub));
@@ -439,7 +426,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
 #pragma unroll
           for (int u = 0; u < kUnroll; ++u) {
             const int i = base + u * kThreads + tid;
-            idx[u] = i < n ? __ldg(a.cand_idx + sub + i) : -1;
+            idx[u] = i < n ? gload(a.cand_idx + sub + i) : -1;
           }
 #pragma unroll
           for (int u = 0; u < kUnroll; ++u) {
@@ -491,7 +478,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
             }
             s_idx[i] = idx[u];
             s_pos[i] = found[u] ? pos[u] : -1;
-            a.out_mask[out0 + i] = static_cast<uint8_t>(m);
+            gstore(a.out_mask + out0 + i, m);
           }
         }
       } else {
@@ -502,7 +489,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
 #pragma unroll
           for (int u = 0; u < kUnroll; ++u) {
             const int i = base + u * kThreads + tid;
-            idx[u] = i < n ? __ldg(a.cand_idx + sub + i) : -1;
+            idx[u] = i < n ? gload(a.cand_idx + sub + i) : -1;
           }
 #pragma unroll
           for (int u = 0; u < kUnroll; ++u) {
@@ -558,14 +545,14 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
             int p = s_pos[i];
             if (p >= K) p = -1;
             s_pos[i] = p;
-            a.out_mask[out0 + i] = p >= 0 ? 1 : 0;
+            gstore(a.out_mask + out0 + i, p >= 0 ? 1 : 0);
           }
         } else {
           for (int i = tid; i < n; i += kThreads) {
             int pos = 0;
             const bool found = s_idx[i] >= 0 && keys.find(s_auth[i], pos);
             s_pos[i] = found ? pos : -1;
-            a.out_mask[out0 + i] = found ? 1 : 0;
+            gstore(a.out_mask + out0 + i, found ? 1 : 0);
           }
         }
       }
@@ -573,7 +560,7 @@ __global__ void __launch_bounds__(kThreads, kJoinMinBlocks) join_kernel(const Jo
 
       // ================= phase B: stream the rows =================
       for (int g = warp * 32; g < n; g += kWarps * 32) {
-        emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND, 0, (EDGE_CH >= 8)>(a, sh, s_idx + g, s_pos + g, s_apos + g, edge_base, req_src,
+        emit_group<DOC_CH, EDGE_CH, REQ_CH, SECOND>(a, sh, s_idx + g, s_pos + g, s_apos + g, edge_base, req_src,
                                                                        a.out_rows + (out0 + g) * sh.out_b, min(32, n - g), lane);
       }
       __syncthreads();  // phase A of the next sub-tile overwrites the resolved arrays (and, in merge mode, the keys)

@@ -11,6 +11,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "ccr_device.cuh"
+
 namespace ccr {
 
 constexpr int kPadThreads = 1024;
@@ -157,8 +159,8 @@ pad_fill_kernel(const int64_t* cand_offsets, long long n_max, long long out_b, u
   const long long chunks = pads * (out_b / 16);
   const long long t = static_cast<long long>(blockIdx.y) * kPadThreads + threadIdx.x;
   const long long stride = static_cast<long long>(gridDim.y) * kPadThreads;
-  for (long long c = t; c < chunks; c += stride) __stcs(rows + c, make_uint4(0u, 0u, 0u, 0u));
-  for (long long i = t; i < pads; i += stride) out_mask[first + i] = 0;
+  for (long long c = t; c < chunks; c += stride) st128_stream(rows + c, make_uint4(0u, 0u, 0u, 0u));
+  for (long long i = t; i < pads; i += stride) gstore(out_mask + first + i, 0);
 }
 
 }  // namespace ccr

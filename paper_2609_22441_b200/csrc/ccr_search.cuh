@@ -89,6 +89,7 @@ struct StagedKeys {
   int M;              // staged entries (0 = nothing staged)
   int s_log;          // log2 of the sampling stride
   unsigned nbk;       // buckets of the table (0 = none)
+  bool warp_search;   // global-memory searches run warp-cooperatively (find_batch_warp)
   bool declined;      // no table only because the segment it was staged for had too few lookups to pay for one
 
   // Algorithm 1 steps 2-3 for one id by binary search: found = some key equals id; pos = its index (meaningful
@@ -108,14 +109,76 @@ struct StagedKeys {
       n = min(1 << s_log, K - lo);
     }
     pos = lo + lower_bound_global(gk + lo, n, id);
-    return pos < K && __ldg(gk + pos) == id;
+    return pos < K && gload(gk + pos) == id;
   }
 
   // U independent lookups with their memory accesses interleaved: one round of table reads (two buckets per id),
   // then one round of verifying key reads (only ids with a matching fingerprint).  Lists without a table, and the
   // ids the table cannot answer, take find().  id < 0 is "nothing to look up".
+  // The warp-cooperative form of the search in global memory (all 32 lanes must call, converged): the warp serves
+  // one id at a time — 32 pivots spread over the remaining range are read by the 32 lanes, a ballot counts the
+  // pivots below the id and picks the sub-range, so a list of 20,000 keys takes 3 rounds (+ 1 read for the
+  // equality test) instead of 15 dependent probes, and the last round's 32 keys are one coalesced 256-byte read.
+  // Four ids are in flight at once.  The price is that the 32 x U ids of a batch are served one after the other
+  // rather than side by side.
+  template <int U>
+  __device__ __forceinline__ void find_batch_warp(const int64_t (&id)[U], bool (&found)[U], int (&pos)[U]) const {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      found[u] = false;
+      pos[u] = 0;
+    }
+    if (K == 0) return;
+#pragma unroll 1
+    for (int u = 0; u < U; ++u) {
+#pragma unroll 1
+      for (int src = 0; src < 32; src += 4) {
+        long long q[4];
+        int lo[4], n[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          q[t] = __shfl_sync(kFull, id[u], src + t);
+          lo[t] = 0;
+          n[t] = q[t] >= 0 ? K : 0;
+        }
+        while (n[0] > 0 || n[1] > 0 || n[2] > 0 || n[3] > 0) {  // warp-uniform: q, lo and n are the same in every lane
+          long long kv[4];
+          int step[4];
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            step[t] = (n[t] + 31) >> 5;
+            const long long p = static_cast<long long>(lo[t]) + static_cast<long long>(lane + 1) * step[t] - 1;
+            kv[t] = (n[t] > 0 && p < lo[t] + n[t]) ? gload(gk + p) : 0x7fffffffffffffffLL;
+          }
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            if (n[t] > 0) {
+              const int c = __popc(__ballot_sync(kFull, kv[t] < q[t]));
+              const int nlo = min(lo[t] + c * step[t], lo[t] + n[t]);
+              n[t] = min(step[t] - 1, lo[t] + n[t] - nlo);
+              lo[t] = nlo;
+            }
+          }
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const bool f = q[t] >= 0 && lo[t] < K && gload(gk + lo[t]) == q[t];
+          if (lane == src + t) {
+            found[u] = f;
+            pos[u] = f ? lo[t] : 0;
+          }
+        }
+      }
+    }
+  }
+
   template <int U>
   __device__ __forceinline__ void find_batch(const int64_t (&id)[U], bool (&found)[U], int (&pos)[U]) const {
+    if (nbk == 0 && warp_search && M == 0) {
+      find_batch_warp<U>(id, found, pos);
+      return;
+    }
     if (nbk == 0) {
 #pragma unroll
       for (int u = 0; u < U; ++u) {
@@ -140,7 +203,7 @@ struct StagedKeys {
     for (int u = 0; u < U; ++u) {
       pos[u] = static_cast<int>(hit[u]) - 1;  // < K for a match: slots only ever hold indices of this list
       kv[u] = 0;
-      if (hit[u] <= kSlotPosMask && id[u] >= 0) kv[u] = (M > 0) ? sk[pos[u]] : __ldg(gk + pos[u]);
+      if (hit[u] <= kSlotPosMask && id[u] >= 0) kv[u] = (M > 0) ? sk[pos[u]] : gload(gk + pos[u]);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -224,6 +287,7 @@ __device__ __forceinline__ bool stage_keys(const JoinArgs& a, const SearchSmem& 
   st.s_log = 0;
   st.nbk = 0;
   st.declined = false;
+  st.warp_search = a.warp_search != 0;
   st.tab = reinterpret_cast<const uint4*>(sm.base);
   st.sk = reinterpret_cast<const int64_t*>(sm.base);
   if (a.key_cap <= 0 || K <= 0 || sm.bytes < 16) {
@@ -253,7 +317,8 @@ __device__ __forceinline__ bool stage_keys(const JoinArgs& a, const SearchSmem& 
     // slot of key i is i + shift, so that 16-byte aligned global addresses land on 16-byte aligned slots
     const int shift = static_cast<int>(kb & 1);
     const int i0 = shift;                       // first key whose address is 16-byte aligned
-    const int nbulk = (K - i0) & ~1;            // keys moved by the bulk copy (even count)
+    int nbulk = (K - i0) & ~1;                  // keys moved by the bulk copy (even count)
+    if (nbulk > 0 && !CCR_CHK(a.edge_keys + kb + i0, nbulk * 8)) nbulk = 0;  // (checked build: the copy is left out)
     st.sk = skeys + shift;
     st.M = K;
     if (g.tid == 0 && nbulk > 0) {
@@ -261,8 +326,8 @@ __device__ __forceinline__ bool stage_keys(const JoinArgs& a, const SearchSmem& 
       bulk_copy_g2s(smem_u32(skeys + i0 + shift), a.edge_keys + kb + i0, static_cast<uint32_t>(nbulk) * 8u, bar);
     }
     // the (at most one) key before and after the 16-byte aligned middle, by two other threads
-    if (g.tid == 1 && shift) skeys[shift] = __ldg(a.edge_keys + kb);
-    if (g.tid == 2 && ((K - i0) & 1)) skeys[K - 1 + shift] = __ldg(a.edge_keys + kb + K - 1);
+    if (g.tid == 1 && shift) skeys[shift] = gload(a.edge_keys + kb);
+    if (g.tid == 2 && ((K - i0) & 1)) skeys[K - 1 + shift] = gload(a.edge_keys + kb + K - 1);
     if (nbulk > 0) {
       expired = !mbar_wait_bounded(bar, phase);
       phase ^= 1u;
@@ -274,7 +339,7 @@ __device__ __forceinline__ bool stage_keys(const JoinArgs& a, const SearchSmem& 
     st.s_log = s_log;
     st.M = K >> s_log;
     for (int i = g.tid; i < st.M; i += g.size)
-      skeys[i] = __ldg(a.edge_keys + kb + ((static_cast<long long>(i) + 1) << s_log) - 1);
+      skeys[i] = gload(a.edge_keys + kb + ((static_cast<long long>(i) + 1) << s_log) - 1);
   }
   if (g.sync_or(expired)) return false;
 
@@ -287,7 +352,7 @@ __device__ __forceinline__ bool stage_keys(const JoinArgs& a, const SearchSmem& 
     for (; i + (kIlp - 1) * g.size < K; i += kIlp * g.size) {
       long long kk[kIlp];
 #pragma unroll
-      for (int q = 0; q < kIlp; ++q) kk[q] = staged ? S[i + q * g.size] : __ldg(st.gk + i + q * g.size);
+      for (int q = 0; q < kIlp; ++q) kk[q] = staged ? S[i + q * g.size] : gload(st.gk + i + q * g.size);
       unsigned b1[kIlp], b2[kIlp], tag[kIlp];
       uint4 x[kIlp], y[kIlp];
 #pragma unroll
@@ -299,7 +364,7 @@ __device__ __forceinline__ bool stage_keys(const JoinArgs& a, const SearchSmem& 
 #pragma unroll
       for (int q = 0; q < kIlp; ++q) table_place(slots, b1[q], b2[q], tag[q], x[q], y[q], i + q * g.size);
     }
-    for (; i < K; i += g.size) table_insert(slots, nbk, staged ? S[i] : __ldg(st.gk + i), i);
+    for (; i < K; i += g.size) table_insert(slots, nbk, staged ? S[i] : gload(st.gk + i), i);
     st.nbk = nbk;
     g.sync();
   }

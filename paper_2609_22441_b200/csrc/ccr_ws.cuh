@@ -144,8 +144,8 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
     int64_t* s_co = reinterpret_cast<int64_t*>(smem + lay.off_offs);
     int64_t* s_eo = s_co + (a.n_req + 1);
     for (int i = tid; i <= a.n_req; i += n_threads) {
-      s_co[i] = __ldg(a.cand_offsets + i);
-      s_eo[i] = __ldg(a.edge_offsets + i);
+      s_co[i] = gload(a.cand_offsets + i);
+      s_eo[i] = gload(a.edge_offsets + i);
     }
     co = s_co;
     eo = s_eo;
@@ -310,7 +310,7 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
 #pragma unroll
           for (int u = 0; u < U; ++u) {
             const int i = base + u * 32 + lane;
-            idx[u] = i < n ? __ldg(a.cand_idx + sub + i) : -1;
+            idx[u] = i < n ? gload(a.cand_idx + sub + i) : -1;
           }
           // every id of the U candidates is requested before the first one is used
           int64_t act[SECOND ? U : 1][4];
@@ -429,7 +429,7 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
               if (e < a.cos_dim) {
 #pragma unroll
                 for (int k = 0; k < kCosMaxChunks; ++k)
-                  if (k < a.cos_chunks) m[k] = __half2float(__ushort_as_half(__ldg(mem + k * a.cos_dim + e)));
+                  if (k < a.cos_chunks) m[k] = __half2float(__ushort_as_half(gload(mem + k * a.cos_dim + e)));
               }
               M[e] = make_float4(m[0], m[1], m[2], m[3]);
             }
@@ -437,7 +437,7 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
               cos_nm = 0.0f;
               if (lane < a.cos_chunks) {
                 for (int e = 0; e < a.cos_dim; ++e) {
-                  const float v = __half2float(__ushort_as_half(__ldg(mem + lane * a.cos_dim + e)));
+                  const float v = __half2float(__ushort_as_half(gload(mem + lane * a.cos_dim + e)));
                   cos_nm = fmaf(v, v, cos_nm);
                 }
               }

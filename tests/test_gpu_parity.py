@@ -34,6 +34,7 @@ def _variants(B, include_smem=True):
     if include_smem:
         v.append(("smem", B.CCR_FLAG_FORCE_SMEM))
     # without a kernel flag a small launch takes the two-phase kernel and a large one the warp-specialised kernel
+    v.append(("global+warp-search", B.CCR_FLAG_FORCE_GLOBAL | B.CCR_FLAG_WARP_SEARCH))
     return (v + [(n + "+2phase", f | B.CCR_FLAG_TWO_PHASE) for n, f in v] +
             [(n + "+ws", f | B.CCR_FLAG_WARP_SPECIALISED) for n, f in v] +
             [(n + "+static", f | B.CCR_FLAG_STATIC_SPLIT) for n, f in v])
