@@ -264,7 +264,7 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       const int c = i * 32 + lane, row = c / DOC_CH, piece = c % DOC_CH;
       const int ridx = row < cnt ? s_idx[row] : -1;
       dv[i] = make_uint4(0u, 0u, 0u, 0u);
-      if (ridx >= 0) dv[i] = ldg128(a.doc_feats + static_cast<long long>(ridx) * (DOC_CH * 16) + piece * 16);
+      if (ridx >= 0) dv[i] = ldg128_once(a.doc_feats + static_cast<long long>(ridx) * (DOC_CH * 16) + piece * 16);
     }
 #pragma unroll
     for (int i = 0; i < EDGE_CH; ++i) {
@@ -292,7 +292,7 @@ __device__ __forceinline__ void emit_group(const JoinArgs& a, const RowShape<DOC
       const int c = i * 32 + lane, row = c / sh.doc_ch, piece = c - row * sh.doc_ch;
       const int ridx = row < cnt ? s_idx[row] : -1;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (ridx >= 0) v = ldg128(a.doc_feats + static_cast<long long>(ridx) * sh.doc_b + piece * 16);
+      if (ridx >= 0) v = ldg128_once(a.doc_feats + static_cast<long long>(ridx) * sh.doc_b + piece * 16);
       if (row < cnt) st128_stream(out + row * out_b + piece * 16, v);
       if constexpr (kCos) {
         const int q = piece - p0;

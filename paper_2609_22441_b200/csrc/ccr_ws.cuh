@@ -318,16 +318,19 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
 #pragma unroll
           for (int u = 0; u < U; ++u) {
             if (idx[u] < 0 || idx[u] >= a.n_docs) idx[u] = -1;  // unresolved / out-of-range position
-            auth[u] = idx[u] >= 0 ? load_author(a, idx[u]) : -1;
             if constexpr (SECOND) {
+              auth[u] = -1;
               act[u][0] = act[u][1] = act[u][2] = act[u][3] = -1;
               types[u] = 0;
               if (idx[u] >= 0) {
-                long long rec[4];
-                load_actors(a, idx[u], rec, types[u]);
+                long long rec[4], au;
+                load_record(a, idx[u], au, rec, types[u]);
+                auth[u] = au;
 #pragma unroll
                 for (int sl = 0; sl < 4; ++sl) act[u][sl] = sl < a.max_actors ? rec[sl] : -1;
               }
+            } else {
+              auth[u] = idx[u] >= 0 ? load_author(a, idx[u]) : -1;
             }
           }
           bool found[U];
