@@ -228,6 +228,7 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
   // this warp's work list of engager lookups (second-degree joins)
   constexpr int U = SECOND ? (REBAL ? kRebalInFlight : 4) : 8;  // candidates a lane keeps in flight
   constexpr int FB = U < 4 ? U : 4;                              // lookups interleaved in one find_batch
+  constexpr int FBW = FB;                                        // ... of the engager work list (wider was slower)
   constexpr int kWlItems = U * 32 * 4;                           // every engager slot of one batch
   [[maybe_unused]] int64_t* wl_id = reinterpret_cast<int64_t*>(smem + lay.off_wl + (SECOND ? rwarp * kWlItems * (8 + 2) : 0));
   [[maybe_unused]] uint16_t* wl_tag = reinterpret_cast<uint16_t*>(wl_id + kWlItems);
@@ -385,18 +386,18 @@ __global__ void __launch_bounds__(REBAL ? kRebalThreads : kWsMaxThreads, 1) join
               }
             }
             __syncwarp();
-            for (int w0 = 0; w0 < total; w0 += FB * 32) {
-              int64_t idq[FB];
+            for (int w0 = 0; w0 < total; w0 += FBW * 32) {
+              int64_t idq[FBW];
 #pragma unroll
-              for (int q = 0; q < FB; ++q) {
+              for (int q = 0; q < FBW; ++q) {
                 const int wi = w0 + q * 32 + lane;
                 idq[q] = wi < total ? wl_id[wi] : -1;
               }
-              bool fq[FB];
-              int pq[FB];
-              keys.find_batch<FB>(idq, fq, pq);
+              bool fq[FBW];
+              int pq[FBW];
+              keys.find_batch<FBW>(idq, fq, pq);
 #pragma unroll
-              for (int q = 0; q < FB; ++q) {
+              for (int q = 0; q < FBW; ++q) {
                 const int wi = w0 + q * 32 + lane;
                 if (wi < total && fq[q]) apos_i[wl_tag[wi]] = pq[q];
               }

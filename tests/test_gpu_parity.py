@@ -535,6 +535,51 @@ def test_joins_in_flight_on_several_streams(B):
     store.free()
 
 
+def test_back_to_back_joins_overlap_without_breaking_stream_order(B):
+    """Consecutive joins on one stream move in behind each other (programmatic dependent launch).  What stream order
+    promises must still hold: two different batches joined alternately into the SAME output buffers leave the last
+    batch's rows (nothing of an earlier launch lands after a later one's); a kernel that rewrites the candidate
+    positions between two joins is seen by the second join; and the result equals CCR_FLAG_NO_OVERLAP's."""
+    wl_a = W.config1(n_docs=300_000, n_req=16, n_cand=30_000)
+    rng = np.random.default_rng(9)
+    b = wl_a.batch
+    cand_b = b.cand_idx.copy()
+    rng.shuffle(cand_b)
+    wl_b = W.Workload("b", 0, wl_a.store, W.Batch(**{**b.__dict__, "cand_idx": cand_b}))
+    want_a = oracle.join_workload(wl_a, n_threads=4)
+    want_b = oracle.join_workload(wl_b, n_threads=4)
+    store = B.store_from_workload(wl_a)
+    da, db = B.DeviceBatch(wl_a.batch), B.DeviceBatch(wl_b.batch)
+    rows = torch.empty((b.total_cands, 384), dtype=torch.uint8, device="cuda")
+    mask = torch.empty((b.total_cands,), dtype=torch.uint8, device="cuda")
+
+    def call(d, flags=0):
+        B.ccr_join_batch(store, d.n_req, d.total_cands, d.max_edge_len, d.edge_keys, d.edge_feats, d.edge_offsets, d.cand_idx,
+                         d.cand_offsets, d.req_feats, rows, mask, flags)
+
+    for flags in (0, B.CCR_FLAG_NO_OVERLAP):
+        for i in range(41):  # a, b, a, ... a
+            call(da if i % 2 == 0 else db, flags)
+        torch.cuda.synchronize()
+        assert np.array_equal(mask.cpu().numpy(), want_a[1]) and np.array_equal(rows.cpu().numpy(), want_a[0])
+        call(db, flags)
+        torch.cuda.synchronize()
+        assert np.array_equal(mask.cpu().numpy(), want_b[1]) and np.array_equal(rows.cpu().numpy(), want_b[0])
+    # a torch kernel between two joins rewrites the second join's input: ordinary stream order applies to it
+    scratch = da.cand_idx.clone()
+    dc = B.DeviceBatch(wl_a.batch)
+    dc.cand_idx = scratch
+    for _ in range(10):
+        call(da)
+        scratch.copy_(db.cand_idx)   # now holds batch b's positions
+        call(dc)
+        torch.cuda.synchronize()
+        assert np.array_equal(rows.cpu().numpy(), want_b[0])
+        scratch.copy_(da.cand_idx)
+    assert store.device_status() == B.CCR_OK
+    store.free()
+
+
 def test_upload_in_pieces_from_device_memory(B):
     wl = W.config0(n_docs=10_000, n_cand=3000, k=200, second_degree=True)
     s = wl.store
