@@ -38,6 +38,19 @@ struct ResolveArgs {
   int32_t* out_pos;
 };
 
+// 16-byte window piece of a level that does not stay in any cache between queries (the three lowest levels of a
+// large index): read past L1.
+__device__ __forceinline__ longlong2 resolve_load(const longlong2* p, bool once) {
+#ifndef CCR_RESOLVE_L1
+  if (once) {
+    longlong2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.s64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p));
+    return v;
+  }
+#endif
+  return __ldg(p);
+}
+
 __global__ void build_level_kernel(const int64_t* below, long long n_below, int64_t* above, long long n_above) {
   for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n_above;
        i += static_cast<long long>(gridDim.x) * blockDim.x)
@@ -92,7 +105,7 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
       const longlong2* lev = reinterpret_cast<const longlong2*>(a.level[l]);
       longlong2 k[kResolveUnroll];
 #pragma unroll
-      for (int u = 0; u < kResolveUnroll; ++u) k[u] = __ldg(lev + (static_cast<size_t>(c[u]) * G + sub));
+      for (int u = 0; u < kResolveUnroll; ++u) k[u] = resolve_load(lev + (static_cast<size_t>(c[u]) * G + sub), l <= 2);
 #pragma unroll
       for (int u = 0; u < kResolveUnroll; ++u) {
         unsigned v = (k[u].x < q[u] ? 1u : 0u) + (k[u].y < q[u] ? 1u : 0u);
@@ -105,7 +118,7 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
       const longlong2* lev = reinterpret_cast<const longlong2*>(a.level[0]);
       longlong2 k[kResolveUnroll];
 #pragma unroll
-      for (int u = 0; u < kResolveUnroll; ++u) k[u] = __ldg(lev + (static_cast<size_t>(c[u]) * G + sub));
+      for (int u = 0; u < kResolveUnroll; ++u) k[u] = resolve_load(lev + (static_cast<size_t>(c[u]) * G + sub), true);
 #pragma unroll
       for (int u = 0; u < kResolveUnroll; ++u) {
         unsigned v = (k[u].x < q[u] ? 1u : 0u) + (k[u].y < q[u] ? 1u : 0u) + ((k[u].x == q[u] || k[u].y == q[u]) ? 256u : 0u);
