@@ -313,6 +313,23 @@ struct DbgRegistrar {
 };
 #endif
 
+// Launch of a kernel that belongs to a chain of small launches (its first statement is chain_enter()): with
+// programmatic stream serialization the launch is set up while the kernel in front of it still runs.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*fn)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, fn, static_cast<KArgs>(args)...);
+}
+
 size_t out_row_bytes(const ccr_docstore* s, uint32_t flags) {
   const bool second = s->desc.max_actors > 0 && !(flags & CCR_FLAG_FIRST_DEGREE_ONLY);
   return static_cast<size_t>(s->doc_b) + s->edge_b * (second ? 2 : 1) + s->req_b + ((flags & CCR_FLAG_COSINE) ? ccr::kCosSectionBytes : 0);
@@ -738,28 +755,31 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
     // largest block most partners lie beyond the list, which is why half as many would not do)
     const unsigned pair_blocks = static_cast<unsigned>((n_chunks * static_cast<long long>(ccr::kSortChunk) + pairs_per_block - 1) / pairs_per_block);
     const dim3 per_chunk(static_cast<unsigned>(n_req), n_chunks), per_pairs(static_cast<unsigned>(n_req), pair_blocks);
-    ccr::sort_chunks_kernel<<<per_chunk, ccr::kSortThreads, 0, st>>>(a);
+    a.more_follow = 1;  // every kernel of the call but the last lets the next one be set up early
+    launch_chained(ccr::sort_chunks_kernel, per_chunk, dim3(ccr::kSortThreads), 0, st, a);
     s->launches++;
     for (long long k = 2LL * ccr::kSortChunk; (k >> 1) < max_edge_len; k <<= 1) {
-      ccr::sort_global_step_kernel<<<per_pairs, ccr::kSortThreads, 0, st>>>(a, static_cast<int>(k), static_cast<int>(k - 1));
+      launch_chained(ccr::sort_global_step_kernel, per_pairs, dim3(ccr::kSortThreads), 0, st, a, static_cast<int>(k), static_cast<int>(k - 1));
       s->launches++;
       for (long long d = k >> 2; d >= ccr::kSortChunk; d >>= 1) {
-        ccr::sort_global_step_kernel<<<per_pairs, ccr::kSortThreads, 0, st>>>(a, static_cast<int>(k), static_cast<int>(d));
+        launch_chained(ccr::sort_global_step_kernel, per_pairs, dim3(ccr::kSortThreads), 0, st, a, static_cast<int>(k), static_cast<int>(d));
         s->launches++;
       }
-      ccr::sort_chunk_finish_kernel<<<per_chunk, ccr::kSortThreads, 0, st>>>(a, static_cast<int>(k));
+      launch_chained(ccr::sort_chunk_finish_kernel, per_chunk, dim3(ccr::kSortThreads), 0, st, a, static_cast<int>(k));
       s->launches++;
     }
-    ccr::sort_unpack_kernel<<<per_chunk, ccr::kSortThreads, 0, st>>>(a);
+    launch_chained(ccr::sort_unpack_kernel, per_chunk, dim3(ccr::kSortThreads), 0, st, a);
     s->launches++;
   }
   // short or unpackable lists (all lists without perm_out): one block per list
-  ccr::sort_edges_kernel<<<static_cast<unsigned>(n_req), ccr::kSortThreads, smem, st>>>(a);
+  a.more_follow = a.multi ? 1 : 0;
+  launch_chained(ccr::sort_edges_kernel, dim3(static_cast<unsigned>(n_req)), dim3(ccr::kSortThreads), smem, st, a);
   s->launches++;
   if (a.multi) {
     const long long per_block = static_cast<long long>(ccr::kSortThreads) * ccr::kSortGatherUnroll;
     const unsigned row_blocks = static_cast<unsigned>((max_edge_len * a.row_ch + per_block - 1) / per_block);
-    ccr::gather_all_kernel<<<dim3(static_cast<unsigned>(n_req), row_blocks), ccr::kSortThreads, 0, st>>>(a);
+    a.more_follow = 0;
+    launch_chained(ccr::gather_all_kernel, dim3(static_cast<unsigned>(n_req), row_blocks), dim3(ccr::kSortThreads), 0, st, a);
     s->launches++;
   }
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
@@ -1143,14 +1163,14 @@ ccr_status ccr_compact_valid(const ccr_docstore* cs, int32_t n_req, int64_t tota
   if (!scope.ok) return CCR_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const long long n_docs = s->desc.n_docs;
-  ccr::count_valid_kernel<<<static_cast<unsigned>(n_req), ccr::kPadThreads, 0, st>>>(cand_idx, cand_offsets, n_docs,
-                                                                                      offsets_out);
-  ccr::scan_counts_kernel<<<1, ccr::kPadThreads, 0, st>>>(offsets_out, n_req);
+  launch_chained(ccr::count_valid_kernel, dim3(static_cast<unsigned>(n_req)), dim3(ccr::kPadThreads), 0, st, cand_idx, cand_offsets,
+                 n_docs, offsets_out);
+  launch_chained(ccr::scan_counts_kernel, dim3(1), dim3(ccr::kPadThreads), 0, st, offsets_out, n_req);
   // slices per request: about one round of the compaction each, bounded so that the re-count stays small
   const long long per_round = static_cast<long long>(ccr::kPadThreads) * ccr::kPadItems;
   const long long avg = (total_cands + n_req - 1) / n_req;
   const unsigned slices = static_cast<unsigned>(std::max(1LL, std::min(8LL, (avg + per_round - 1) / per_round)));
-  ccr::compact_valid_kernel<<<dim3(static_cast<unsigned>(n_req), slices), ccr::kPadThreads, 0, st>>>(
+  launch_chained(ccr::compact_valid_kernel, dim3(static_cast<unsigned>(n_req), slices), dim3(ccr::kPadThreads), 0, st,
       cand_idx, cand_offsets, n_docs, offsets_out, idx_out, src_out);
   s->launches += 3;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;

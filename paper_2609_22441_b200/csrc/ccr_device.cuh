@@ -147,6 +147,16 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// First statement of the kernels that run as a chain of small launches (sort, compaction).  This kernel touches
+// memory only after the launch in front of it has completed; when another kernel of the same chain follows
+// (more_follow), that launch may be set up right away and will wait in the same way, so the launch gaps inside the
+// chain overlap.  The LAST kernel of a chain never lets its successor in early: whatever is launched behind the chain
+// (a join, whose resolver warps read their inputs without waiting) starts only after the whole chain has completed.
+__device__ __forceinline__ void chain_enter(bool more_follow) {
+  if (more_follow) pdl_trigger();
+  pdl_wait();
+}
+
 // ---- bounds-checked build (-DCCR_DEBUG_BOUNDS) ------------------------------------------------------------------
 // Every global load and store of the join kernels goes through gload / gstore / ldg128 / st128_stream.  In the
 // checked build the host registers the extent of every buffer of the launch in g_dbg; an access that does not lie

@@ -65,6 +65,7 @@ __device__ __forceinline__ int block_count_valid(const int32_t* cand_idx, long l
 // Step 1a: valid candidates per request -> counts[r + 1] (counts[0] = 0).  One block per request.
 __global__ void __launch_bounds__(kPadThreads)
 count_valid_kernel(const int32_t* cand_idx, const int64_t* cand_offsets, long long n_docs, int64_t* counts) {
+  chain_enter(true);
   __shared__ int warp_sums[kPadThreads / 32];
   const int r = blockIdx.x;
   const int total = block_count_valid(cand_idx, cand_offsets[r], cand_offsets[r + 1], n_docs, warp_sums);
@@ -76,6 +77,7 @@ count_valid_kernel(const int32_t* cand_idx, const int64_t* cand_offsets, long lo
 
 // Step 1b: in-place inclusive scan of counts[1 .. n_req] (one block; n_req is a batch size, a few hundred).
 __global__ void __launch_bounds__(kPadThreads) scan_counts_kernel(int64_t* counts, int n_req) {
+  chain_enter(true);
   __shared__ int warp_sums[kPadThreads / 32];
   __shared__ long long carry_s;
   if (threadIdx.x == 0) carry_s = 0;
@@ -103,6 +105,7 @@ __global__ void __launch_bounds__(kPadThreads) scan_counts_kernel(int64_t* count
 __global__ void __launch_bounds__(kPadThreads)
 compact_valid_kernel(const int32_t* cand_idx, const int64_t* cand_offsets, long long n_docs, const int64_t* offsets_out,
                      int32_t* idx_out, int32_t* src_out) {
+  chain_enter(false);
   __shared__ int warp_sums[kPadThreads / 32];
   const int r = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

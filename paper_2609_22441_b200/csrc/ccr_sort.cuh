@@ -180,6 +180,7 @@ __device__ __forceinline__ void gather_rows(const uint4* src, uint4* dst, long l
 }
 
 struct SortArgs {
+  int more_follow;           // another kernel of the same ccr_sort_edges call is launched behind this one
   int n_req;
   const int64_t* keys_in;
   const uint8_t* feats_in;
@@ -220,6 +221,7 @@ __device__ __forceinline__ bool list_is_packable(const int64_t* keys, int K, int
 }
 
 __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortArgs a) {
+  chain_enter(a.more_follow != 0);
   extern __shared__ __align__(16) unsigned char smem_sort[];
   const int r = blockIdx.x;
   const long long e0 = __ldg(a.edge_offsets + r);
@@ -307,6 +309,7 @@ __device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, lon
 
 // grid (n_req, chunks of the longest list): sort chunk blockIdx.y of list blockIdx.x
 __global__ void __launch_bounds__(kSortThreads, 1) sort_chunks_kernel(const SortArgs a) {
+  chain_enter(a.more_follow != 0);
   __shared__ unsigned long long w[kSortChunk];
   const int r = blockIdx.x;
   const long long e0 = __ldg(a.edge_offsets + r);
@@ -360,6 +363,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_chunks_kernel(const Sort
 // power of two >= kSortChunk (disperse) — for the lists that have a block of size k to sort.
 constexpr int kSortPairsPerThread = 4;
 __global__ void __launch_bounds__(kSortThreads) sort_global_step_kernel(const SortArgs a, int k, int j) {
+  chain_enter(a.more_follow != 0);
   long long e0;
   int K;
   if (!list_on_multi_path(a, blockIdx.x, e0, K) || (k >> 1) >= K) return;
@@ -381,6 +385,7 @@ __global__ void __launch_bounds__(kSortThreads) sort_global_step_kernel(const So
 
 // grid (n_req, chunks): the disperse steps at distances kSortChunk / 2 ... 1 of phase k, per chunk in shared memory
 __global__ void __launch_bounds__(kSortThreads, 1) sort_chunk_finish_kernel(const SortArgs a, int k) {
+  chain_enter(a.more_follow != 0);
   __shared__ unsigned long long w[kSortChunk];
   long long e0;
   int K;
@@ -403,6 +408,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_chunk_finish_kernel(cons
 
 // grid (n_req, chunks): words -> keys (in place) and source indices
 __global__ void __launch_bounds__(kSortThreads) sort_unpack_kernel(const SortArgs a) {
+  chain_enter(a.more_follow != 0);
   long long e0;
   int K;
   const int c0 = blockIdx.y * kSortChunk;
@@ -420,6 +426,7 @@ __global__ void __launch_bounds__(kSortThreads) sort_unpack_kernel(const SortArg
 // grid (n_req, row blocks): rows follow their keys, for every list of the batch, kSortGatherUnroll 16-byte chunks
 // per thread in flight
 __global__ void __launch_bounds__(kSortThreads) gather_all_kernel(const SortArgs a) {
+  chain_enter(a.more_follow != 0);
   const int r = blockIdx.x;
   const long long e0 = __ldg(a.edge_offsets + r);
   const long long K = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
