@@ -421,13 +421,17 @@ ccr_status ccr_docstore_selftest_wait(ccr_docstore* store, void* stream);
 /* Tuning knobs of the join kernels; a field that is 0 keeps the store's current value.              */
 typedef struct {
   int32_t tile_cands;         /* candidates per ring slot / search-copy phase pair: multiple of 256, <= 4096;
-                                 unset = 256 (warp-specialised kernel) / 1024 (two-phase kernel)               */
-  int32_t key_capacity;       /* most keys (or sampled keys) a block stages in shared memory per request;
-                                 unset = whole lists up to a 160 KB shared-memory budget per block
-                                 (warp-specialised kernel) or 4096 (the others)                              */
+                                 unset = 256 (warp-specialised kernel; 128 in its 20-warp second-degree form, which
+                                 a configured value switches off) / 1024 (two-phase kernel)                    */
+  int32_t key_capacity;       /* longest list a block stages in full in shared memory (next to its hash table
+                                 while both fit; longer lists keep a table only, or a sampled top of the tree);
+                                 unset = what fits a 160 KB shared-memory budget per block (warp-specialised
+                                 kernel) or 4096 (the others)                                                */
   int32_t ws_streamers;       /* warp-specialised kernel: row-streaming warps per block (1..14)              */
   int32_t ws_resolvers;       /* warp-specialised kernel: search warps per block (1..8); sum <= 16; set both
-                                 or neither (unset = 12 + 4)              */
+                                 or neither (unset = 12 + 4; second-degree joins: 12 + 8 in the 20-warp form with
+                                 registers moved from the search warps to the streaming warps, which a configured
+                                 split switches off)                                                           */
   int32_t blocks_per_sm;      /* two-phase kernel: cap on resident blocks per SM (1..8)                      */
 } ccr_tuning;
 ccr_status ccr_docstore_set_tuning(ccr_docstore* store, const ccr_tuning* tuning);
