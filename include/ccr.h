@@ -300,10 +300,12 @@ ccr_status ccr_join_batch_ex(const ccr_docstore* store, const ccr_join_io* io, u
  * one 1024-thread block in shared memory (one kernel); lists of more than 19,000 records then have no place to
  * be sorted in and the call returns CCR_ERR_INVALID_ARG.  With perm_out, and max_edge_len above 4,096, lists
  * whose keys leave room for the record index in one 64-bit word (non-negative, below 2^(63 - index bits): every
- * realistic id) are sorted in chunks of 4,096 records by one block each and merged by grid-wide passes of the
- * same sorting network over the key output array, so that a single long list is spread over many SMs instead
- * of one (a batch whose long lists would keep the SMs busy one list each stays on the one-block path), and the
- * rows of all lists are moved by one grid-wide gather: up to ~14 small kernels on `stream`.
+ * realistic id) are sorted in chunks of 4,096 records by one block each and the sorted chunks merged pairwise,
+ * one grid-wide launch per doubling of the run length (the merged words alternate between keys_out and the
+ * list's own part of feats_out, which therefore holds scratch data until the end of the call), so that a long
+ * list is spread over many SMs instead of one, and the rows of all lists are moved by one grid-wide gather:
+ * 4 + ceil(log2(max_edge_len / 4096)) small kernels on `stream` (CCR_ERR_UNSUPPORTED if n_req x the tiles of
+ * max_edge_len records exceed the 2^31 - 1 blocks of a grid).
  * max_edge_len (HOST) must be at least the longest list; a longer list is cut there (its first max_edge_len
  * records are sorted among themselves, the rest of its output is left unwritten) and no access leaves the arrays.
  * All pointers DEVICE; no allocation, no synchronisation.

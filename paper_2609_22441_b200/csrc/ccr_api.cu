@@ -748,27 +748,23 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   // Lists longer than one chunk are spread over many blocks when the caller provides perm_out (the row gather
   // of that path reads the source indices from it).
   a.multi = (perm_out != nullptr && max_edge_len > ccr::kSortChunk) ? 1 : 0;
+  // grids of the chunked path: one block per tile of every list, sized for the longest list
+  auto tiles_grid = [&](long long per_list_units, long long tile) -> long long {
+    return static_cast<long long>(n_req) * ((per_list_units + tile - 1) / tile);
+  };
+  const long long g_chunk = tiles_grid(max_edge_len, ccr::kSortChunk), g_merge = tiles_grid(max_edge_len, ccr::kSortMergeTile);
+  const long long g_unpack = tiles_grid(max_edge_len, ccr::kSortUnpackTile);
+  const long long g_gather = tiles_grid(max_edge_len * a.row_ch, ccr::kSortGatherTile);
   if (a.multi) {
-    const unsigned n_chunks = static_cast<unsigned>((max_edge_len + ccr::kSortChunk - 1) / ccr::kSortChunk);
-    const long long pairs_per_block = static_cast<long long>(ccr::kSortThreads) * ccr::kSortPairsPerThread;
-    // pair number p maps to a lower partner i >= p, so p < max_edge_len covers every pair (in the flip of the
-    // largest block most partners lie beyond the list, which is why half as many would not do)
-    const unsigned pair_blocks = static_cast<unsigned>((n_chunks * static_cast<long long>(ccr::kSortChunk) + pairs_per_block - 1) / pairs_per_block);
-    const dim3 per_chunk(static_cast<unsigned>(n_req), n_chunks), per_pairs(static_cast<unsigned>(n_req), pair_blocks);
+    if (g_merge > 0x7fffffffLL || g_unpack > 0x7fffffffLL || g_gather > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;
     a.more_follow = 1;  // every kernel of the call but the last lets the next one be set up early
-    launch_chained(ccr::sort_chunks_kernel, per_chunk, dim3(ccr::kSortThreads), 0, st, a);
+    launch_chained(ccr::sort_chunks_kernel, dim3(static_cast<unsigned>(g_chunk)), dim3(ccr::kSortChunkThreads), 0, st, a);
     s->launches++;
-    for (long long k = 2LL * ccr::kSortChunk; (k >> 1) < max_edge_len; k <<= 1) {
-      launch_chained(ccr::sort_global_step_kernel, per_pairs, dim3(ccr::kSortThreads), 0, st, a, static_cast<int>(k), static_cast<int>(k - 1));
-      s->launches++;
-      for (long long d = k >> 2; d >= ccr::kSortChunk; d >>= 1) {
-        launch_chained(ccr::sort_global_step_kernel, per_pairs, dim3(ccr::kSortThreads), 0, st, a, static_cast<int>(k), static_cast<int>(d));
-        s->launches++;
-      }
-      launch_chained(ccr::sort_chunk_finish_kernel, per_chunk, dim3(ccr::kSortThreads), 0, st, a, static_cast<int>(k));
+    for (int phase = 1; phase <= ccr::sort_merge_phases(max_edge_len); ++phase) {
+      launch_chained(ccr::sort_merge_kernel, dim3(static_cast<unsigned>(g_merge)), dim3(ccr::kSortMergeThreads), 0, st, a, phase);
       s->launches++;
     }
-    launch_chained(ccr::sort_unpack_kernel, per_chunk, dim3(ccr::kSortThreads), 0, st, a);
+    launch_chained(ccr::sort_unpack_kernel, dim3(static_cast<unsigned>(g_unpack)), dim3(ccr::kSortUnpackThreads), 0, st, a);
     s->launches++;
   }
   // short or unpackable lists (all lists without perm_out): one block per list
@@ -776,10 +772,8 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   launch_chained(ccr::sort_edges_kernel, dim3(static_cast<unsigned>(n_req)), dim3(ccr::kSortThreads), smem, st, a);
   s->launches++;
   if (a.multi) {
-    const long long per_block = static_cast<long long>(ccr::kSortThreads) * ccr::kSortGatherUnroll;
-    const unsigned row_blocks = static_cast<unsigned>((max_edge_len * a.row_ch + per_block - 1) / per_block);
     a.more_follow = 0;
-    launch_chained(ccr::gather_all_kernel, dim3(static_cast<unsigned>(n_req), row_blocks), dim3(ccr::kSortThreads), 0, st, a);
+    launch_chained(ccr::gather_all_kernel, dim3(static_cast<unsigned>(g_gather)), dim3(ccr::kSortGatherThreads), 0, st, a);
     s->launches++;
   }
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;

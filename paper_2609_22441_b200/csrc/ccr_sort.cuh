@@ -1,12 +1,16 @@
 // Algorithm 1 step 1 of the paper on the device: per request, sort the viewer's affinity records by author
 // id (a_sorted, idx = sort(a); F_sorted = gather(F, idx)) so that unsorted request payloads can be joined.
 //
-// One 1024-thread block per request.  Keys and record indices are sorted together in shared memory with a
-// bitonic network written for arbitrary n (flip + disperse steps, every compare-exchange ascending, partners
-// beyond n skipped — equivalent to padding with +infinity); the order is on (key, index), which makes the
-// result the stable sort.  Keys that leave room for the index in the same 64-bit word (the usual case) take 8
-// bytes per record, so lists of up to ~29,000 records are sorted in shared memory; other keys take 12 bytes
-// (~19,000 records).  Longer lists are sorted by the same network directly on the output arrays in global memory (L2).  The rows then follow their keys in 16-byte chunks.
+// The order is on (key, index of the record in its list), which makes the result the stable sort.  Keys that leave
+// room for the index in the same 64-bit word (the usual case) are sorted as single words, key << bits | index.
+// With a permutation output the lists are cut into chunks of 4,096 records, one block sorts a chunk in shared
+// memory (a merge sort: four words per thread in registers, then runs doubled per pass along merge paths), the
+// sorted chunks are merged pairwise by grid-wide launches (merge path again, one output tile per block), and the
+// rows follow their keys in one grid-wide gather.  Without a permutation output, or for keys that do not leave
+// room for the index, one 1024-thread block sorts a whole list in shared memory (merge sort up to 16,384 packed
+// words, a bitonic network written for arbitrary n beyond that and for the 12-byte (key, index) records of
+// unpackable keys; lists that do not fit shared memory are sorted by the network on the output arrays in L2) and
+// moves its rows itself.
 #pragma once
 
 #include "ccr_device.cuh"
@@ -156,6 +160,60 @@ __device__ __forceinline__ void sort_words_bitonic(unsigned long long* w, int n)
   }
 }
 
+// Merge sort of n <= IPT * blockDim.x distinct words in shared memory: every thread sorts IPT consecutive words in
+// registers, then sorted runs are merged pairwise, doubling per pass; in a pass a thread produces IPT consecutive
+// output words, from the point of its pair of runs that the merge path (a binary search along its diagonal)
+// assigns to it, into registers, and writes them back after a barrier.  log2(n / IPT) passes of two barriers
+// each, against the ~n log^2 n / 2 compare-exchanges and ~25 barriers of the network for 4,096 words.
+template <int IPT>
+__device__ __forceinline__ void sort_words_merge(unsigned long long* w, int n) {
+  const int t0 = static_cast<int>(threadIdx.x) * IPT;
+  unsigned long long v[IPT];
+#pragma unroll
+  for (int u = 0; u < IPT; ++u) v[u] = t0 + u < n ? w[t0 + u] : ~0ull;
+  // odd-even transposition sort of the thread's words (IPT rounds)
+#pragma unroll
+  for (int rd = 0; rd < IPT; ++rd) {
+#pragma unroll
+    for (int u = rd & 1; u + 1 < IPT; u += 2) {
+      const unsigned long long lo = min(v[u], v[u + 1]), hi = max(v[u], v[u + 1]);
+      v[u] = lo;
+      v[u + 1] = hi;
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < IPT; ++u)
+    if (t0 + u < n) w[t0 + u] = v[u];
+  __syncthreads();
+  for (int run = IPT; run < n; run <<= 1) {
+    const int pb = (t0 / (2 * run)) * (2 * run);
+    const int lenA = max(0, min(run, n - pb)), lenB = max(0, min(run, n - pb - run));
+    const unsigned long long* A = w + pb;
+    const unsigned long long* B = A + run;
+    const int d = min(t0 - pb, lenA + lenB);
+    int lo = max(0, d - lenB), hi = min(d, lenA);
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (A[mid] < B[d - 1 - mid]) lo = mid + 1; else hi = mid;
+    }
+    int i = lo, j = d - lo;
+#pragma unroll
+    for (int u = 0; u < IPT; ++u) {
+      const bool has_a = i < lenA, has_b = j < lenB;
+      const unsigned long long va = has_a ? A[i] : ~0ull, vb = has_b ? B[j] : ~0ull;
+      const bool take_a = has_a && (!has_b || va < vb);
+      v[u] = take_a ? va : vb;
+      i += take_a ? 1 : 0;
+      j += take_a ? 0 : 1;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < IPT; ++u)
+      if (t0 + u < n) w[t0 + u] = v[u];
+    __syncthreads();
+  }
+}
+
 // Rows follow their keys: output chunk c (16 bytes) comes from row source_of(c / row_ch) of the input.  One block
 // moves a whole list, so every thread keeps kSortGatherUnroll loads in flight.
 constexpr int kSortGatherUnroll = 8;
@@ -196,9 +254,18 @@ struct SortArgs {
                          //    rows of every list are moved by gather_all_kernel (perm_out is then required)
 };
 
-constexpr int kSortChunkLog = 12;
+#ifndef CCR_SORT_CHUNK_LOG
+#define CCR_SORT_CHUNK_LOG 12
+#endif
+#ifndef CCR_SORT_CHUNK_THREADS
+#define CCR_SORT_CHUNK_THREADS 1024
+#endif
+#ifndef CCR_SORT_CHUNK_BLOCKS
+#define CCR_SORT_CHUNK_BLOCKS 2  // resident per SM: one block's loads hide behind the other's merging (32 registers, no spill)
+#endif
+constexpr int kSortChunkLog = CCR_SORT_CHUNK_LOG;
 constexpr int kSortChunk = 1 << kSortChunkLog;  // records one block of the multi-block path sorts in shared memory
-constexpr int kSortMultiBalance = 64;  // long lists are spread over blocks while their total length is at most this many times the longest
+constexpr int kSortChunkThreads = CCR_SORT_CHUNK_THREADS;
 constexpr int kSortMultiFlag = 0x5a17ed01;      // "this list is on the multi-block path", kept in the list's first output row
 
 __device__ __forceinline__ int sort_index_bits(int K) {
@@ -212,6 +279,7 @@ __device__ __forceinline__ int sort_index_bits(int K) {
 __device__ __forceinline__ bool list_is_packable(const int64_t* keys, int K, int idx_bits) {
   long long kmax = 0;
   int negative = 0;
+#pragma unroll 8
   for (int i = threadIdx.x; i < K; i += blockDim.x) {
     const long long k = __ldg(keys + i);
     kmax = max(kmax, k);
@@ -244,7 +312,11 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
     for (int i = threadIdx.x; i < K; i += blockDim.x)
       w[i] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
     __syncthreads();
-    sort_words_bitonic(w, K);
+    // merge sort while a thread's share of the list fits its registers, the network beyond
+    if (K <= 4 * kSortThreads) sort_words_merge<4>(w, K);
+    else if (K <= 8 * kSortThreads) sort_words_merge<8>(w, K);
+    else if (K <= 16 * kSortThreads) sort_words_merge<16>(w, K);
+    else sort_words_bitonic(w, K);
     const unsigned long long low = (1ull << idx_bits) - 1;
     for (int i = threadIdx.x; i < K; i += blockDim.x) {
       const unsigned long long v = w[i];
@@ -291,13 +363,12 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
 
 
 // ---------------------------------------------------------------------------------------------------
-// Multi-block path for long lists.  One block per list leaves a 19,000-record list to a single SM (264 us,
-// instruction-bound) while the others idle.  Here the same network runs over the packed words in global
-// memory (the key output array): chunks of kSortChunk records are sorted in shared memory by one block each;
-// then, for every larger block size k, the steps whose partner distance reaches across chunks (the flip, and
-// disperse steps at distances >= kSortChunk) run as grid-wide passes, one launch each, and the remaining steps
-// of the phase run per chunk in shared memory again.  A flag in the list's first output row (written by the
-// chunk kernel, overwritten by the final row gather) tells the later kernels that the list is packable.
+// Multi-block path.  One block per list leaves a 19,000-record list to a single SM while the others idle.  Here
+// chunks of kSortChunk records are sorted in shared memory by one block each (packed words, written to the key
+// output array) and the sorted chunks are then merged pairwise, one launch per doubling of the run length, every
+// block producing kSortMergeTile consecutive output words from the two stretches of its pair of runs that the
+// merge path assigns to them.  A flag in the list's first output row (written by the chunk kernel, overwritten by
+// the final row gather) tells the later kernels that the list is on this path.
 
 __device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, long long& e0, int& K) {
   e0 = __ldg(a.edge_offsets + r);
@@ -307,131 +378,181 @@ __device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, lon
   return *reinterpret_cast<const volatile int*>(a.feats_out + e0 * a.row_ch * 16) == kSortMultiFlag;
 }
 
-// grid (n_req, chunks of the longest list): sort chunk blockIdx.y of list blockIdx.x
-__global__ void __launch_bounds__(kSortThreads, 1) sort_chunks_kernel(const SortArgs a) {
+// Block b of a grid of n_req x tiles-of-the-longest-list blocks: its list and its tile within the list.
+__device__ __forceinline__ void sort_block_item(const SortArgs& a, int tile, int& r, long long& y) {
+  const unsigned per = static_cast<unsigned>((static_cast<long long>(a.max_len) + tile - 1) / tile);
+  r = static_cast<int>(blockIdx.x / per);
+  y = blockIdx.x - static_cast<unsigned>(r) * per;
+}
+
+// One block per chunk of kSortChunk records of a list: the chunk sorted in shared memory, as packed words
+__global__ void __launch_bounds__(kSortChunkThreads, CCR_SORT_CHUNK_BLOCKS) sort_chunks_kernel(const SortArgs a) {
   chain_enter(a.more_follow != 0);
   __shared__ unsigned long long w[kSortChunk];
-  const int r = blockIdx.x;
+  int r;
+  long long y;
+  sort_block_item(a, kSortChunk, r, y);
   const long long e0 = __ldg(a.edge_offsets + r);
   const int K = static_cast<int>(min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len)));
-  const int c0 = blockIdx.y * kSortChunk;
-  if (c0 >= K) return;  // also K <= 0
+  if (y * kSortChunk >= K) return;  // also K <= 0
+  const int c0 = static_cast<int>(y) * kSortChunk;
   const int idx_bits = sort_index_bits(K);
-  bool take = list_is_packable(a.keys_in + e0, K, idx_bits);
-  if (K > kSortChunk) {
-    // Spreading a long list over many blocks costs more SM time than sorting it in one block, so it pays only
-    // while the batch's long lists would not keep the SMs busy one list each.
-    // every block sizes up the batch's long lists for itself (the same numbers in all of them): their total
-    // length against the longest one — one block per list takes about 14 ns per record of the longest list,
-    // the chunked path about 0.2 ns per record of all long lists (measured)
-    __shared__ unsigned long long sum_long_s;
-    __shared__ int max_long_s;
-    if (threadIdx.x == 0) {
-      sum_long_s = 0;
-      max_long_s = 0;
-    }
-    __syncthreads();
-    unsigned long long sum = 0;
-    int longest = 0;
-    for (int q = threadIdx.x; q < a.n_req; q += blockDim.x) {
-      const long long len = min(static_cast<long long>(__ldg(a.edge_offsets + q + 1) - __ldg(a.edge_offsets + q)), static_cast<long long>(a.max_len));
-      if (len > kSortChunk) {
-        sum += static_cast<unsigned long long>(len);
-        longest = max(longest, static_cast<int>(min(len, 0x7fffffffLL)));
-      }
-    }
-    if (sum) {
-      atomicAdd(&sum_long_s, sum);
-      atomicMax(&max_long_s, longest);
-    }
-    __syncthreads();
-    take = take && sum_long_s <= static_cast<unsigned long long>(kSortMultiBalance) * max_long_s;
-  }
-  if (blockIdx.y == 0 && threadIdx.x == 0)
+  const bool take = list_is_packable(a.keys_in + e0, K, idx_bits);
+  if (y == 0 && threadIdx.x == 0)
     *reinterpret_cast<int*>(a.feats_out + e0 * a.row_ch * 16) = take ? kSortMultiFlag : 0;
   if (!take) return;
   const int n = min(kSortChunk, K - c0);
   for (int t = threadIdx.x; t < n; t += blockDim.x)
     w[t] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + c0 + t)) << idx_bits) | static_cast<unsigned>(c0 + t);
   __syncthreads();
-  sort_words_bitonic(w, n);
+  static_assert(kSortChunk % kSortChunkThreads == 0, "every thread of a chunk block owns the same number of words");
+  sort_words_merge<kSortChunk / kSortChunkThreads>(w, n);
   unsigned long long* W = reinterpret_cast<unsigned long long*>(a.keys_out + e0);
   for (int t = threadIdx.x; t < n; t += blockDim.x) W[c0 + t] = w[t];
 }
 
-// grid (n_req, pair blocks): one step of the network across chunks — partner mask j = k - 1 (flip) or a
-// power of two >= kSortChunk (disperse) — for the lists that have a block of size k to sort.
-constexpr int kSortPairsPerThread = 4;
-__global__ void __launch_bounds__(kSortThreads) sort_global_step_kernel(const SortArgs a, int k, int j) {
+// Merging the sorted chunks.  Phase p = 1, 2, ... merges neighbouring runs of kSortChunk << (p - 1) words into
+// runs of twice that length, out of place: the words alternate between the key output array and a scratch area
+// inside the list's own output rows (8 bytes per record behind the flag's 16 bytes; a row has at least 16), which
+// nothing else uses until the rows are gathered at the end.  A list takes part in a phase while it is longer than
+// the phase's input runs, so a list of K records goes through sort_merge_phases(K) phases and its words end in the
+// scratch area when that number is odd.
+__device__ __host__ __forceinline__ int sort_merge_phases(long long K) {
+  int p = 0;
+  while ((static_cast<long long>(kSortChunk) << p) < K) ++p;
+  return p;
+}
+__device__ __forceinline__ unsigned long long* sort_words_at(const SortArgs& a, long long e0, bool scratch) {
+  return scratch ? reinterpret_cast<unsigned long long*>(a.feats_out + e0 * a.row_ch * 16 + 16)
+                 : reinterpret_cast<unsigned long long*>(a.keys_out + e0);
+}
+
+// Merge path, warp-cooperative: how many of the first d words of merge(A, B) come from A.  All words are distinct
+// (the record index is part of the word).  A[i] is among the first d exactly when A[i] < B[d - 1 - i]; that holds for
+// i below the answer and fails from it on, so the warp probes the last element of up to 32 equal sub-ranges at once
+// and narrows the range by a factor of 32 per round trip to memory (three rounds for runs of 16,384).
+__device__ __forceinline__ int merge_path_warp(const unsigned long long* A, int lenA, const unsigned long long* B, int lenB,
+                                               int d, int lane) {
+  int lo = max(0, d - lenB), hi = min(d, lenA);
+  while (lo < hi) {
+    const int span = hi - lo, s = (span + 31) >> 5;
+    const int i = lo + lane * s + s - 1;
+    const bool before = i < hi && A[i] < B[d - 1 - i];
+    const int cnt = __popc(__ballot_sync(0xffffffffu, before));  // the predicate is monotone: the first cnt probes hold
+    const int first_fail = lo + cnt * s + s - 1;                 // probe number cnt failed or lies beyond the range
+    lo += cnt * s;
+    hi = min(hi, first_fail);
+  }
+  return lo;
+}
+
+// One block per kSortMergeTile consecutive output words of phase `phase` of a list.  Small blocks, several per
+// SM: the grid is sized for the longest list, and the blocks beyond the end of a shorter one leave after reading
+// the offsets — side by side rather than one after the other.
+constexpr int kSortMergeThreads = 256;
+constexpr int kSortMergePerThread = 4;
+constexpr int kSortMergeTile = kSortMergeThreads * kSortMergePerThread;
+__global__ void __launch_bounds__(kSortMergeThreads) sort_merge_kernel(const SortArgs a, int phase) {
   chain_enter(a.more_follow != 0);
-  long long e0;
-  int K;
-  if (!list_on_multi_path(a, blockIdx.x, e0, K) || (k >> 1) >= K) return;
-  unsigned long long* W = reinterpret_cast<unsigned long long*>(a.keys_out + e0);
-  const int top = 31 - __clz(j);
+  __shared__ unsigned long long w[kSortMergeTile];
+  __shared__ int split[2];
+  long long e0, y;
+  int K, r;
+  sort_block_item(a, kSortMergeTile, r, y);
+  const long long run = static_cast<long long>(kSortChunk) << (phase - 1);
+  if (!list_on_multi_path(a, r, e0, K) || run >= K || y * kSortMergeTile >= K) return;
+  const int o0 = static_cast<int>(y) * kSortMergeTile;  // first output word of this block, within the list
+  const unsigned long long* src = sort_words_at(a, e0, (phase & 1) == 0);
+  unsigned long long* dst = sort_words_at(a, e0, (phase & 1) != 0);
+  const int pb = static_cast<int>((o0 / (2 * run)) * (2 * run));  // the pair of runs this block's words belong to
+  const int lenA = static_cast<int>(min(run, static_cast<long long>(K - pb)));
+  const int lenB = static_cast<int>(min(run, static_cast<long long>(K - pb - lenA)));
+  const unsigned long long* A = src + pb;
+  const unsigned long long* B = A + lenA;
+  const int d0 = o0 - pb, d1 = min(d0 + kSortMergeTile, lenA + lenB);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp < 2) {
+    const int ia = merge_path_warp(A, lenA, B, lenB, warp == 0 ? d0 : d1, lane);
+    if (lane == 0) split[warp] = ia;
+  }
+  __syncthreads();
+  const int ia0 = split[0], ia1 = split[1], ib0 = d0 - ia0, ib1 = d1 - ia1;
+  const int nA = ia1 - ia0, nB = ib1 - ib0, n = nA + nB;
+  if (nA < 0 || nB < 0 || n > kSortMergeTile) return;  // only if the runs were not sorted: touch nothing out of range
+  for (int t = threadIdx.x; t < n; t += kSortMergeThreads) w[t] = t < nA ? A[ia0 + t] : B[ib0 + t - nA];
+  __syncthreads();
+  // every thread merges kSortMergePerThread consecutive output words: its own split of the tile by binary search
+  const unsigned long long* sa = w;
+  const unsigned long long* sb = w + nA;
+  const int d = min(static_cast<int>(threadIdx.x) * kSortMergePerThread, n);
+  int lo = max(0, d - nB), hi = min(d, nA);
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (sa[mid] < sb[d - 1 - mid]) lo = mid + 1; else hi = mid;
+  }
+  int i = lo, j = d - lo;
+  unsigned long long out[kSortMergePerThread];
 #pragma unroll
-  for (int u = 0; u < kSortPairsPerThread; ++u) {
-    const int p = (blockIdx.y * kSortPairsPerThread + u) * kSortThreads + threadIdx.x;
-    const int i = pair_low_index(p, top), l = i ^ j;
-    if (i < K && l < K) {
-      const unsigned long long wi = W[i], wl = W[l];
-      if (wi > wl) {
-        W[i] = wl;
-        W[l] = wi;
-      }
+  for (int u = 0; u < kSortMergePerThread; ++u) {
+    const bool has_a = i < nA, has_b = j < nB;
+    const unsigned long long va = has_a ? sa[i] : ~0ull, vb = has_b ? sb[j] : ~0ull;
+    const bool take_a = has_a && (!has_b || va < vb);
+    out[u] = take_a ? va : vb;
+    i += take_a ? 1 : 0;
+    j += take_a ? 0 : 1;
+  }
+#pragma unroll
+  for (int u = 0; u < kSortMergePerThread; ++u)
+    if (d + u < n) dst[pb + d0 + d + u] = out[u];
+}
+
+// One block per kSortUnpackTile words of a list: words -> keys and source indices
+constexpr int kSortUnpackThreads = 256;
+constexpr int kSortUnpackTile = 4 * kSortUnpackThreads;
+__global__ void __launch_bounds__(kSortUnpackThreads) sort_unpack_kernel(const SortArgs a) {
+  chain_enter(a.more_follow != 0);
+  long long e0, y;
+  int K, r;
+  sort_block_item(a, kSortUnpackTile, r, y);
+  if (!list_on_multi_path(a, r, e0, K) || y * kSortUnpackTile >= K) return;
+  const int c0 = static_cast<int>(y) * kSortUnpackTile;
+  const int idx_bits = sort_index_bits(K);
+  const unsigned long long low = (1ull << idx_bits) - 1;
+  const int n = min(kSortUnpackTile, K - c0);
+  const unsigned long long* W = sort_words_at(a, e0, (sort_merge_phases(K) & 1) != 0);
+  unsigned long long v[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int t = u * kSortUnpackThreads + threadIdx.x;
+    if (t < n) v[u] = W[c0 + t];
+  }
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int t = u * kSortUnpackThreads + threadIdx.x;
+    if (t < n) {  // (when the words are in the key array, a thread overwrites only words it has read itself)
+      a.keys_out[e0 + c0 + t] = static_cast<long long>(v[u] >> idx_bits);
+      a.perm_out[e0 + c0 + t] = static_cast<int>(v[u] & low);
     }
   }
 }
 
-// grid (n_req, chunks): the disperse steps at distances kSortChunk / 2 ... 1 of phase k, per chunk in shared memory
-__global__ void __launch_bounds__(kSortThreads, 1) sort_chunk_finish_kernel(const SortArgs a, int k) {
+// One block per kSortGatherTile 16-byte chunks of a list's rows: rows follow their keys, for every list of the
+// batch, kSortGatherUnroll chunks per thread in flight; small blocks for the same reason as in the merge kernel
+constexpr int kSortGatherThreads = 256;
+constexpr int kSortGatherTile = kSortGatherThreads * kSortGatherUnroll;
+__global__ void __launch_bounds__(kSortGatherThreads) gather_all_kernel(const SortArgs a) {
   chain_enter(a.more_follow != 0);
-  __shared__ unsigned long long w[kSortChunk];
-  long long e0;
-  int K;
-  const int c0 = blockIdx.y * kSortChunk;
-  if (!list_on_multi_path(a, blockIdx.x, e0, K) || (k >> 1) >= K || c0 >= K) return;
-  unsigned long long* W = reinterpret_cast<unsigned long long*>(a.keys_out + e0);
-  const int n = min(kSortChunk, K - c0);
-  for (int t = threadIdx.x; t < n; t += blockDim.x) w[t] = W[c0 + t];
-  __syncthreads();
-  for (int b = kSortChunkLog - 1; b >= 5;) {
-    const int m = b - 4 >= 3 ? 3 : b - 4;
-    if (m == 3) disperse_fused<3>(w, n, b);
-    else if (m == 2) disperse_fused<2>(w, n, b);
-    else disperse_fused<1>(w, n, b);
-    b -= m;
+  int r;
+  long long y;
+  {
+    const unsigned per = static_cast<unsigned>((static_cast<long long>(a.max_len) * a.row_ch + kSortGatherTile - 1) / kSortGatherTile);
+    r = static_cast<int>(blockIdx.x / per);
+    y = blockIdx.x - static_cast<unsigned>(r) * per;
   }
-  warp_steps<false>(w, n);
-  for (int t = threadIdx.x; t < n; t += blockDim.x) W[c0 + t] = w[t];
-}
-
-// grid (n_req, chunks): words -> keys (in place) and source indices
-__global__ void __launch_bounds__(kSortThreads) sort_unpack_kernel(const SortArgs a) {
-  chain_enter(a.more_follow != 0);
-  long long e0;
-  int K;
-  const int c0 = blockIdx.y * kSortChunk;
-  if (!list_on_multi_path(a, blockIdx.x, e0, K) || c0 >= K) return;
-  const int idx_bits = sort_index_bits(K);
-  const unsigned long long low = (1ull << idx_bits) - 1;
-  const int n = min(kSortChunk, K - c0);
-  for (int t = threadIdx.x; t < n; t += blockDim.x) {
-    const unsigned long long v = reinterpret_cast<const unsigned long long*>(a.keys_out + e0)[c0 + t];
-    a.keys_out[e0 + c0 + t] = static_cast<long long>(v >> idx_bits);
-    a.perm_out[e0 + c0 + t] = static_cast<int>(v & low);
-  }
-}
-
-// grid (n_req, row blocks): rows follow their keys, for every list of the batch, kSortGatherUnroll 16-byte chunks
-// per thread in flight
-__global__ void __launch_bounds__(kSortThreads) gather_all_kernel(const SortArgs a) {
-  chain_enter(a.more_follow != 0);
-  const int r = blockIdx.x;
   const long long e0 = __ldg(a.edge_offsets + r);
   const long long K = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   const long long chunks = K * a.row_ch;
-  const long long first = static_cast<long long>(blockIdx.y) * kSortThreads * kSortGatherUnroll;
+  const long long first = y * kSortGatherTile;
   if (first >= chunks) return;
   const uint4* src = reinterpret_cast<const uint4*>(a.feats_in) + e0 * a.row_ch;
   uint4* dst = reinterpret_cast<uint4*>(a.feats_out) + e0 * a.row_ch;
@@ -439,7 +560,7 @@ __global__ void __launch_bounds__(kSortThreads) gather_all_kernel(const SortArgs
   uint4 v[kSortGatherUnroll];
 #pragma unroll
   for (int u = 0; u < kSortGatherUnroll; ++u) {
-    const long long c = first + static_cast<long long>(u) * kSortThreads + threadIdx.x;
+    const long long c = first + static_cast<long long>(u) * kSortGatherThreads + threadIdx.x;
     if (c < chunks) {
       const int row = static_cast<int>(c / a.row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * a.row_ch);
       v[u] = __ldg(src + static_cast<long long>(__ldg(perm + row)) * a.row_ch + piece);
@@ -447,8 +568,8 @@ __global__ void __launch_bounds__(kSortThreads) gather_all_kernel(const SortArgs
   }
 #pragma unroll
   for (int u = 0; u < kSortGatherUnroll; ++u) {
-    const long long c = first + static_cast<long long>(u) * kSortThreads + threadIdx.x;
-    if (c < chunks) dst[c] = v[u];
+    const long long c = first + static_cast<long long>(u) * kSortGatherThreads + threadIdx.x;
+    if (c < chunks) __stcs(dst + c, v[u]);  // written once, read by a later kernel at the earliest
   }
 }
 

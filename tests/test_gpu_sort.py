@@ -114,12 +114,13 @@ def test_sort_with_keys_that_cannot_share_a_word_with_the_index(B):
     store.free()
 
 
-@pytest.mark.parametrize("case", ["few_long", "many_long", "mixed_unpackable", "powers_of_two"])
-def test_sort_chunked_path_and_its_policy(B, case):
-    """With perm_out, lists longer than 4,096 records are sorted in chunks by many blocks and merged by grid-wide
-    passes — unless the batch's long lists add up to more than 64 times the longest, or a list's keys cannot
-    share a word with the index; those stay on the one-block path inside the same launch sequence."""
-    rng = np.random.default_rng({"few_long": 1, "many_long": 2, "mixed_unpackable": 3, "powers_of_two": 4}[case])
+@pytest.mark.parametrize("case", ["few_long", "many_long", "mixed_unpackable", "powers_of_two", "very_long"])
+def test_sort_chunked_path(B, case):
+    """With perm_out, lists are sorted in chunks of 4,096 records by one block each and the chunks merged pairwise,
+    one launch per doubling of the run length (a list of K records takes ceil(log2(K / 4096)) merges and its words
+    end in the key array or in the scratch area accordingly) — unless a list's keys cannot share a word with the
+    index; those stay on the one-block path inside the same launch sequence."""
+    rng = np.random.default_rng({"few_long": 1, "many_long": 2, "mixed_unpackable": 3, "powers_of_two": 4, "very_long": 5}[case])
     imax = np.iinfo(np.int64).max
     if case == "few_long":
         lens = [4097, 9000, 20_000, 3, 0, 12_288, 4096, 16_385]
@@ -132,9 +133,13 @@ def test_sort_chunked_path_and_its_policy(B, case):
         keyf = [lambda n: rng.integers(0, 1 << 40, size=n), lambda n: imax - rng.integers(0, 1 << 20, size=n),
                 lambda n: rng.integers(-1000, 1000, size=n), lambda n: rng.integers(0, 1000, size=n),  # many ties
                 lambda n: rng.integers(0, 1 << 40, size=n)]
-    else:
+    elif case == "powers_of_two":
         lens = [8192, 16_384, 32_768, 8193, 16_383]
         keyf = [lambda n: rng.integers(0, 1 << 45, size=n)] * len(lens)
+    else:  # four, five and six merges; few distinct keys in the longest (ties across every run boundary)
+        lens = [131_073, 70_000, 12_289, 65_536]
+        keyf = [lambda n: rng.integers(0, 97, size=n), lambda n: rng.integers(0, 1 << 44, size=n),
+                lambda n: rng.integers(0, 1 << 20, size=n), lambda n: np.arange(n)[::-1].copy()]
     keys = np.concatenate([f(n) for f, n in zip(keyf, lens)] + [np.empty(0, np.int64)]).astype(np.int64)
     feats = rng.standard_normal((len(keys), 64)).astype(np.float16)
     eo = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
