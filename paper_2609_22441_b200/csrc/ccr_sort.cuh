@@ -378,11 +378,12 @@ __device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, lon
   return *reinterpret_cast<const volatile int*>(a.feats_out + e0 * a.row_ch * 16) == kSortMultiFlag;
 }
 
-// Block b of a grid of n_req x tiles-of-the-longest-list blocks: its list and its tile within the list.
-__device__ __forceinline__ void sort_block_item(const SortArgs& a, int tile, int& r, long long& y) {
-  const unsigned per = static_cast<unsigned>((static_cast<long long>(a.max_len) + tile - 1) / tile);
-  r = static_cast<int>(blockIdx.x / per);
-  y = blockIdx.x - static_cast<unsigned>(r) * per;
+// Block b of a grid of (tiles of the longest list) x n_req blocks: its list and its tile within the list.  Lists
+// vary fastest, so the blocks that have work (every list has a first tile, few have a twentieth) come first and
+// the ones that leave at once are the tail of the launch.
+__device__ __forceinline__ void sort_block_item(const SortArgs& a, int& r, long long& y) {
+  y = blockIdx.x / static_cast<unsigned>(a.n_req);
+  r = static_cast<int>(blockIdx.x - static_cast<unsigned>(y) * static_cast<unsigned>(a.n_req));
 }
 
 // One block per chunk of kSortChunk records of a list: the chunk sorted in shared memory, as packed words
@@ -391,7 +392,7 @@ __global__ void __launch_bounds__(kSortChunkThreads, CCR_SORT_CHUNK_BLOCKS) sort
   __shared__ unsigned long long w[kSortChunk];
   int r;
   long long y;
-  sort_block_item(a, kSortChunk, r, y);
+  sort_block_item(a, r, y);
   const long long e0 = __ldg(a.edge_offsets + r);
   const int K = static_cast<int>(min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len)));
   if (y * kSortChunk >= K) return;  // also K <= 0
@@ -458,7 +459,7 @@ __global__ void __launch_bounds__(kSortMergeThreads) sort_merge_kernel(const Sor
   __shared__ int split[2];
   long long e0, y;
   int K, r;
-  sort_block_item(a, kSortMergeTile, r, y);
+  sort_block_item(a, r, y);
   const long long run = static_cast<long long>(kSortChunk) << (phase - 1);
   if (!list_on_multi_path(a, r, e0, K) || run >= K || y * kSortMergeTile >= K) return;
   const int o0 = static_cast<int>(y) * kSortMergeTile;  // first output word of this block, within the list
@@ -513,7 +514,7 @@ __global__ void __launch_bounds__(kSortUnpackThreads) sort_unpack_kernel(const S
   chain_enter(a.more_follow != 0);
   long long e0, y;
   int K, r;
-  sort_block_item(a, kSortUnpackTile, r, y);
+  sort_block_item(a, r, y);
   if (!list_on_multi_path(a, r, e0, K) || y * kSortUnpackTile >= K) return;
   const int c0 = static_cast<int>(y) * kSortUnpackTile;
   const int idx_bits = sort_index_bits(K);
@@ -544,11 +545,7 @@ __global__ void __launch_bounds__(kSortGatherThreads) gather_all_kernel(const So
   chain_enter(a.more_follow != 0);
   int r;
   long long y;
-  {
-    const unsigned per = static_cast<unsigned>((static_cast<long long>(a.max_len) * a.row_ch + kSortGatherTile - 1) / kSortGatherTile);
-    r = static_cast<int>(blockIdx.x / per);
-    y = blockIdx.x - static_cast<unsigned>(r) * per;
-  }
+  sort_block_item(a, r, y);
   const long long e0 = __ldg(a.edge_offsets + r);
   const long long K = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   const long long chunks = K * a.row_ch;
