@@ -748,23 +748,27 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   // Lists longer than one chunk are spread over many blocks when the caller provides perm_out (the row gather
   // of that path reads the source indices from it).
   a.multi = (perm_out != nullptr && max_edge_len > ccr::kSortChunk) ? 1 : 0;
-  // grids of the chunked path: one block per tile of every list, sized for the longest list
-  auto tiles_grid = [&](long long per_list_units, long long tile) -> long long {
-    return static_cast<long long>(n_req) * ((per_list_units + tile - 1) / tile);
+  // grids of the chunked path: one block per tile of every list, sized for the longest list, folded into one
+  // dimension; the row gather takes lists x tiles when the tiles fit a grid's second dimension (x = 0: too many blocks)
+  auto tiles_grid = [&](long long per_list_units, long long tile, bool two_d) -> dim3 {
+    const long long tiles = (per_list_units + tile - 1) / tile;
+    if (two_d && tiles <= 65535) return dim3(static_cast<unsigned>(n_req), static_cast<unsigned>(tiles));
+    const long long blocks = static_cast<long long>(n_req) * tiles;
+    return dim3(blocks <= 0x7fffffffLL ? static_cast<unsigned>(blocks) : 0u);
   };
-  const long long g_chunk = tiles_grid(max_edge_len, ccr::kSortChunk), g_merge = tiles_grid(max_edge_len, ccr::kSortMergeTile);
-  const long long g_unpack = tiles_grid(max_edge_len, ccr::kSortUnpackTile);
-  const long long g_gather = tiles_grid(max_edge_len * a.row_ch, ccr::kSortGatherTile);
+  const dim3 g_chunk = tiles_grid(max_edge_len, ccr::kSortChunk, false), g_merge = tiles_grid(max_edge_len, ccr::kSortMergeTile, false);
+  const dim3 g_unpack = tiles_grid(max_edge_len, ccr::kSortUnpackTile, false);
+  const dim3 g_gather = tiles_grid(max_edge_len * a.row_ch, ccr::kSortGatherTile, true);
   if (a.multi) {
-    if (g_merge > 0x7fffffffLL || g_unpack > 0x7fffffffLL || g_gather > 0x7fffffffLL) return CCR_ERR_UNSUPPORTED;
+    if (g_chunk.x == 0 || g_merge.x == 0 || g_unpack.x == 0 || g_gather.x == 0) return CCR_ERR_UNSUPPORTED;
     a.more_follow = 1;  // every kernel of the call but the last lets the next one be set up early
-    launch_chained(ccr::sort_chunks_kernel, dim3(static_cast<unsigned>(g_chunk)), dim3(ccr::kSortChunkThreads), 0, st, a);
+    launch_chained(ccr::sort_chunks_kernel, g_chunk, dim3(ccr::kSortChunkThreads), 0, st, a);
     s->launches++;
     for (int phase = 1; phase <= ccr::sort_merge_phases(max_edge_len); ++phase) {
-      launch_chained(ccr::sort_merge_kernel, dim3(static_cast<unsigned>(g_merge)), dim3(ccr::kSortMergeThreads), 0, st, a, phase);
+      launch_chained(ccr::sort_merge_kernel, g_merge, dim3(ccr::kSortMergeThreads), 0, st, a, phase);
       s->launches++;
     }
-    launch_chained(ccr::sort_unpack_kernel, dim3(static_cast<unsigned>(g_unpack)), dim3(ccr::kSortUnpackThreads), 0, st, a);
+    launch_chained(ccr::sort_unpack_kernel, g_unpack, dim3(ccr::kSortUnpackThreads), 0, st, a);
     s->launches++;
   }
   // short or unpackable lists (all lists without perm_out): one block per list
@@ -773,7 +777,7 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   s->launches++;
   if (a.multi) {
     a.more_follow = 0;
-    launch_chained(ccr::gather_all_kernel, dim3(static_cast<unsigned>(g_gather)), dim3(ccr::kSortGatherThreads), 0, st, a);
+    launch_chained(ccr::gather_all_kernel, g_gather, dim3(ccr::kSortGatherThreads), 0, st, a);
     s->launches++;
   }
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;

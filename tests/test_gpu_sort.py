@@ -182,3 +182,39 @@ def test_sort_with_an_untruthful_length_bound_stays_in_bounds(B):
                 assert (k[a + m:a + n] == -7).all() and (p[a + m:a + n] == -7).all() and (f[a + m:a + n] == 7).all()
     finally:
         store.free()
+
+
+def test_sort_a_list_with_more_row_tiles_than_a_grid_has_rows(B):
+    """16.8M records of 128-byte rows: the row gather needs more than 65,535 tiles for the list, so its grid (and
+    only its grid) takes the folded one-dimensional form; a short list rides along.  Keys and permutation are
+    compared in full, the rows on 200,000 sampled records and the short list."""
+    if torch.cuda.mem_get_info()[0] < 12 * 2**30:
+        pytest.skip("needs ~6 GB of free device memory")
+    rng = np.random.default_rng(77)
+    lens = [16_800_000, 5000]
+    E = sum(lens)
+    keys = rng.integers(0, 1 << 34, size=E, dtype=np.int64)
+    eo = np.array([0, lens[0], E], dtype=np.int64)
+    wl = W.config3(n_docs=1000, n_req=1, n_cand=10, gen_doc_feats=True, extra_pools=0)
+    store = B.store_from_workload(wl)
+    try:
+        k_in = torch.from_numpy(keys).cuda()
+        # rows made on the device: row i = 16 int32 lanes of (i * 2654435761 + lane) — 128 bytes like the store's edge rows
+        i = torch.arange(E, dtype=torch.int64, device="cuda").unsqueeze(1)
+        f_in = ((i * 2654435761 + torch.arange(32, dtype=torch.int64, device="cuda")) & 0x7fffffff).to(torch.int32)
+        assert f_in.shape[1] * 4 == wl.batch.edge_row_bytes
+        k_out, f_out = torch.empty_like(k_in), torch.empty_like(f_in)
+        p_out = torch.empty(E, dtype=torch.int32, device="cuda")
+        B.ccr_sort_edges(store, 2, lens[0], k_in, f_in, torch.from_numpy(eo).cuda(), k_out, f_out, p_out)
+        torch.cuda.synchronize()
+        k, p = k_out.cpu().numpy(), p_out.cpu().numpy()
+        want_k, _, want_p = oracle.sort_edges(keys, np.zeros((E, 1), np.uint8), eo)  # one-byte rows: keys and order only
+        assert np.array_equal(k, want_k) and np.array_equal(p, want_p)
+        sample = np.concatenate([rng.integers(0, lens[0], size=200_000), np.arange(lens[0], E),
+                                 np.array([0, 1, lens[0] - 1])]).astype(np.int64)
+        src = np.where(sample < lens[0], p[sample], lens[0] + p[sample])
+        got = f_out[torch.from_numpy(sample).cuda()].cpu().numpy()
+        want = f_in[torch.from_numpy(src).cuda()].cpu().numpy()
+        assert np.array_equal(got, want)
+    finally:
+        store.free()
