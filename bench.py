@@ -766,6 +766,7 @@ def sort_bench(args, B, device: int):
             call()
         torch.cuda.synchronize(dev)
         times = []
+        launches0 = store.launch_count()
         for _ in range(max(args.steps // 20, 20)):
             flush.fill_(1)
             a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -775,6 +776,7 @@ def sort_bench(args, B, device: int):
             torch.cuda.synchronize(dev)
             times.append(a.elapsed_time(z))
         ms = float(np.median(times))
+        kernels = int(store.launch_count() - launches0)  # this library's kernels inside the timed calls of the payload
         t_busy = time.time()
         sustain(lambda i: call(), lambda: torch.cuda.synchronize(dev), t_busy, 0.8)
         E = len(keys)
@@ -786,7 +788,8 @@ def sort_bench(args, B, device: int):
         results.append({"payload": name, "requests": b.n_req, "records": E, "longest_list": b.max_edge_len,
                         "row_bytes": b.edge_row_bytes, "ms": ms, "records_per_s": E / (ms * 1e-3),
                         "algorithmic_gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / peak,
-                        "oracle_ms_1_core": 1e3 * t_cpu, "matches_oracle": ok})
+                        "oracle_ms_1_core": 1e3 * t_cpu, "matches_oracle": ok,
+                        "kernels_per_call": kernels // max(args.steps // 20, 20), "gpu_launches": kernels})
         store.free()
     head = results[-1]
     sampler.stop()
@@ -801,8 +804,9 @@ def sort_bench(args, B, device: int):
                    "peak_kind": "of " + peak_kind},
         "roofline": {"bound": "hbm", "achieved": head["algorithmic_gbs"], "peak": peak, "unit": "GB/s",
                      "frac": head["frac_of_hbm_peak"], "traffic": None,
-                     "note": "bound by the sorting network of the longest lists (instruction issue), not by HBM"},
-        "payloads": results, "gpu_launches": max(args.steps // 20, 20),
+                     "note": "seven dependent kernels per call, each starting on flushed caches, and the shared-memory merge "
+                             "sort of the chunks: latency- and instruction-bound, not by HBM"},
+        "payloads": results, "gpu_launches": head["gpu_launches"],
     }))
 
 

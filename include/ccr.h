@@ -304,7 +304,7 @@ ccr_status ccr_join_batch_ex(const ccr_docstore* store, const ccr_join_io* io, u
  * one grid-wide launch per doubling of the run length (the merged words alternate between keys_out and the
  * list's own part of feats_out, which therefore holds scratch data until the end of the call), so that a long
  * list is spread over many SMs instead of one, and the rows of all lists are moved by one grid-wide gather:
- * 4 + ceil(log2(max_edge_len / 4096)) small kernels on `stream` (CCR_ERR_UNSUPPORTED if n_req x the tiles of
+ * 3 + ceil(log2(max_edge_len / 4096)) small kernels on `stream` (CCR_ERR_UNSUPPORTED if n_req x the tiles of
  * max_edge_len records exceed the 2^31 - 1 blocks of a grid).
  * max_edge_len (HOST) must be at least the longest list; a longer list is cut there (its first max_edge_len
  * records are sorted among themselves, the rest of its output is left unwritten) and no access leaves the arrays.

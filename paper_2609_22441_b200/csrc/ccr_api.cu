@@ -757,10 +757,9 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
     return dim3(blocks <= 0x7fffffffLL ? static_cast<unsigned>(blocks) : 0u);
   };
   const dim3 g_chunk = tiles_grid(max_edge_len, ccr::kSortChunk, false), g_merge = tiles_grid(max_edge_len, ccr::kSortMergeTile, false);
-  const dim3 g_unpack = tiles_grid(max_edge_len, ccr::kSortUnpackTile, false);
   const dim3 g_gather = tiles_grid(max_edge_len * a.row_ch, ccr::kSortGatherTile, true);
   if (a.multi) {
-    if (g_chunk.x == 0 || g_merge.x == 0 || g_unpack.x == 0 || g_gather.x == 0) return CCR_ERR_UNSUPPORTED;
+    if (g_chunk.x == 0 || g_merge.x == 0 || g_gather.x == 0) return CCR_ERR_UNSUPPORTED;
     a.more_follow = 1;  // every kernel of the call but the last lets the next one be set up early
     launch_chained(ccr::sort_chunks_kernel, g_chunk, dim3(ccr::kSortChunkThreads), 0, st, a);
     s->launches++;
@@ -768,8 +767,6 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
       launch_chained(ccr::sort_merge_kernel, g_merge, dim3(ccr::kSortMergeThreads), 0, st, a, phase);
       s->launches++;
     }
-    launch_chained(ccr::sort_unpack_kernel, g_unpack, dim3(ccr::kSortUnpackThreads), 0, st, a);
-    s->launches++;
   }
   // short or unpackable lists (all lists without perm_out): one block per list
   a.more_follow = a.multi ? 1 : 0;

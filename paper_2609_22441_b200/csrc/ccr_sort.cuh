@@ -382,8 +382,8 @@ __device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, lon
 // varying fastest, or lists along x and tiles along y.  Either way the blocks that have work (every list has a
 // first tile, few have a twentieth) come first and the ones that leave at once are the tail of the launch.  Which
 // form a kernel gets is a measurement on a 256-list batch: the row gather was 9 us faster on the two-dimensional
-// grid (it falls back to the folded one when a list has more tiles than a grid has rows), the chunk, merge and
-// unpack kernels together 6 us faster on the folded one.
+// grid (it falls back to the folded one when a list has more tiles than a grid has rows), the chunk and merge kernels
+// together 6 us faster on the folded one.
 __device__ __forceinline__ void sort_block_item(const SortArgs& a, int& r, long long& y) {
   if (gridDim.y > 1) {
     r = static_cast<int>(blockIdx.x);
@@ -392,6 +392,24 @@ __device__ __forceinline__ void sort_block_item(const SortArgs& a, int& r, long 
     y = blockIdx.x / static_cast<unsigned>(a.n_req);
     r = static_cast<int>(blockIdx.x - static_cast<unsigned>(y) * static_cast<unsigned>(a.n_req));
   }
+}
+
+// Merging the sorted chunks.  Phase p = 1, 2, ... merges neighbouring runs of kSortChunk << (p - 1) words into
+// runs of twice that length, out of place: the words alternate between the key output array and a scratch area
+// inside the list's own output rows (8 bytes per record behind the flag's 16 bytes; a row has at least 16), which
+// nothing else uses until the rows are gathered at the end.  A list takes part in a phase while it is longer than
+// the phase's input runs, so a list of K records goes through P = sort_merge_phases(K) phases.  Its last phase
+// writes keys and source indices instead of words (a single-chunk list gets them from the chunk kernel), and so
+// that this never overwrites words another block still has to read, the last phase must read from the scratch
+// area: phase p reads it when P - p is even, and the chunk kernel writes there when P is odd.
+__device__ __host__ __forceinline__ int sort_merge_phases(long long K) {
+  int p = 0;
+  while ((static_cast<long long>(kSortChunk) << p) < K) ++p;
+  return p;
+}
+__device__ __forceinline__ unsigned long long* sort_words_at(const SortArgs& a, long long e0, bool scratch) {
+  return scratch ? reinterpret_cast<unsigned long long*>(a.feats_out + e0 * a.row_ch * 16 + 16)
+                 : reinterpret_cast<unsigned long long*>(a.keys_out + e0);
 }
 
 // One block per chunk of kSortChunk records of a list: the chunk sorted in shared memory, as packed words
@@ -416,24 +434,17 @@ __global__ void __launch_bounds__(kSortChunkThreads, CCR_SORT_CHUNK_BLOCKS) sort
   __syncthreads();
   static_assert(kSortChunk % kSortChunkThreads == 0, "every thread of a chunk block owns the same number of words");
   sort_words_merge<kSortChunk / kSortChunkThreads>(w, n);
-  unsigned long long* W = reinterpret_cast<unsigned long long*>(a.keys_out + e0);
+  const int P = sort_merge_phases(K);
+  if (P == 0) {  // the whole list: done
+    const unsigned long long low = (1ull << idx_bits) - 1;
+    for (int t = threadIdx.x; t < n; t += blockDim.x) {
+      a.keys_out[e0 + t] = static_cast<long long>(w[t] >> idx_bits);
+      a.perm_out[e0 + t] = static_cast<int>(w[t] & low);
+    }
+    return;
+  }
+  unsigned long long* W = sort_words_at(a, e0, (P & 1) != 0);
   for (int t = threadIdx.x; t < n; t += blockDim.x) W[c0 + t] = w[t];
-}
-
-// Merging the sorted chunks.  Phase p = 1, 2, ... merges neighbouring runs of kSortChunk << (p - 1) words into
-// runs of twice that length, out of place: the words alternate between the key output array and a scratch area
-// inside the list's own output rows (8 bytes per record behind the flag's 16 bytes; a row has at least 16), which
-// nothing else uses until the rows are gathered at the end.  A list takes part in a phase while it is longer than
-// the phase's input runs, so a list of K records goes through sort_merge_phases(K) phases and its words end in the
-// scratch area when that number is odd.
-__device__ __host__ __forceinline__ int sort_merge_phases(long long K) {
-  int p = 0;
-  while ((static_cast<long long>(kSortChunk) << p) < K) ++p;
-  return p;
-}
-__device__ __forceinline__ unsigned long long* sort_words_at(const SortArgs& a, long long e0, bool scratch) {
-  return scratch ? reinterpret_cast<unsigned long long*>(a.feats_out + e0 * a.row_ch * 16 + 16)
-                 : reinterpret_cast<unsigned long long*>(a.keys_out + e0);
 }
 
 // Merge path, warp-cooperative: how many of the first d words of merge(A, B) come from A.  All words are distinct
@@ -471,8 +482,9 @@ __global__ void __launch_bounds__(kSortMergeThreads) sort_merge_kernel(const Sor
   const long long run = static_cast<long long>(kSortChunk) << (phase - 1);
   if (!list_on_multi_path(a, r, e0, K) || run >= K || y * kSortMergeTile >= K) return;
   const int o0 = static_cast<int>(y) * kSortMergeTile;  // first output word of this block, within the list
-  const unsigned long long* src = sort_words_at(a, e0, (phase & 1) == 0);
-  unsigned long long* dst = sort_words_at(a, e0, (phase & 1) != 0);
+  const int P = sort_merge_phases(K);
+  const unsigned long long* src = sort_words_at(a, e0, ((P - phase) & 1) == 0);
+  unsigned long long* dst = sort_words_at(a, e0, ((P - phase) & 1) != 0);
   const int pb = static_cast<int>((o0 / (2 * run)) * (2 * run));  // the pair of runs this block's words belong to
   const int lenA = static_cast<int>(min(run, static_cast<long long>(K - pb)));
   const int lenB = static_cast<int>(min(run, static_cast<long long>(K - pb - lenA)));
@@ -510,39 +522,21 @@ __global__ void __launch_bounds__(kSortMergeThreads) sort_merge_kernel(const Sor
     i += take_a ? 1 : 0;
     j += take_a ? 0 : 1;
   }
+  if (phase == P) {  // the list's last merge: keys and source indices (src is the scratch area here)
+    const int idx_bits = sort_index_bits(K);
+    const unsigned long long low = (1ull << idx_bits) - 1;
+#pragma unroll
+    for (int u = 0; u < kSortMergePerThread; ++u) {
+      if (d + u < n) {
+        a.keys_out[e0 + o0 + d + u] = static_cast<long long>(out[u] >> idx_bits);
+        a.perm_out[e0 + o0 + d + u] = static_cast<int>(out[u] & low);
+      }
+    }
+    return;
+  }
 #pragma unroll
   for (int u = 0; u < kSortMergePerThread; ++u)
-    if (d + u < n) dst[pb + d0 + d + u] = out[u];
-}
-
-// One block per kSortUnpackTile words of a list: words -> keys and source indices
-constexpr int kSortUnpackThreads = 256;
-constexpr int kSortUnpackTile = 4 * kSortUnpackThreads;
-__global__ void __launch_bounds__(kSortUnpackThreads) sort_unpack_kernel(const SortArgs a) {
-  chain_enter(a.more_follow != 0);
-  long long e0, y;
-  int K, r;
-  sort_block_item(a, r, y);
-  if (!list_on_multi_path(a, r, e0, K) || y * kSortUnpackTile >= K) return;
-  const int c0 = static_cast<int>(y) * kSortUnpackTile;
-  const int idx_bits = sort_index_bits(K);
-  const unsigned long long low = (1ull << idx_bits) - 1;
-  const int n = min(kSortUnpackTile, K - c0);
-  const unsigned long long* W = sort_words_at(a, e0, (sort_merge_phases(K) & 1) != 0);
-  unsigned long long v[4];
-#pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    const int t = u * kSortUnpackThreads + threadIdx.x;
-    if (t < n) v[u] = W[c0 + t];
-  }
-#pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    const int t = u * kSortUnpackThreads + threadIdx.x;
-    if (t < n) {  // (when the words are in the key array, a thread overwrites only words it has read itself)
-      a.keys_out[e0 + c0 + t] = static_cast<long long>(v[u] >> idx_bits);
-      a.perm_out[e0 + c0 + t] = static_cast<int>(v[u] & low);
-    }
-  }
+    if (d + u < n) dst[o0 + d + u] = out[u];
 }
 
 // One block per kSortGatherTile 16-byte chunks of a list's rows: rows follow their keys, for every list of the
