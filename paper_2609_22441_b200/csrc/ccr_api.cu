@@ -79,6 +79,7 @@ struct ccr_docstore {
   int cos_first, cos_dim, cos_chunks;  // derived cosine section (cos_chunks == 0: not configured)
   int64_t dbg_shrink_rows;             // bounds-checked build: rows cut off the registered output extents
   std::atomic<int64_t> launches;  // kernels launched for this store; also hands out the scheduling-word pairs
+  std::atomic<int64_t> sort_calls;  // chunked ccr_sort_edges calls; hands out their flag words
 };
 
 struct ccr_workspace {
@@ -402,6 +403,7 @@ ccr_status ccr_docstore_create(const ccr_docstore_desc* d, ccr_docstore** out) {
   ccr_docstore* s = new (std::nothrow) ccr_docstore();  // value-initialised: every field zero
   if (s == nullptr) return CCR_ERR_OOM;
   s->launches.store(0);
+  s->sort_calls.store(0);
   s->desc = *d;
   s->doc_b = static_cast<int>(doc_b);
   s->edge_b = static_cast<int>(edge_b);
@@ -748,6 +750,9 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   // Lists longer than one chunk are spread over many blocks when the caller provides perm_out (the row gather
   // of that path reads the source indices from it).
   a.multi = (perm_out != nullptr && max_edge_len > ccr::kSortChunk) ? 1 : 0;
+  // the call's flag word: word 8 of a scheduling region (the joins use words 0 and 1), regions taken in turn, so up
+  // to kSchedRegions chunked sorts of one store may be in flight at once
+  a.call_flag = a.multi ? s->status + kStatusHead + s->sched_stride * static_cast<int>(s->sort_calls.fetch_add(1) % kSchedRegions) + 8 : nullptr;
   // grids of the chunked path: one block per tile of every list, sized for the longest list, folded into one
   // dimension; the row gather takes lists x tiles when the tiles fit a grid's second dimension (x = 0: too many blocks)
   auto tiles_grid = [&](long long per_list_units, long long tile, bool two_d) -> dim3 {

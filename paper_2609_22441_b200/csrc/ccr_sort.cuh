@@ -238,6 +238,7 @@ __device__ __forceinline__ void gather_rows(const uint4* src, uint4* dst, long l
 }
 
 struct SortArgs {
+  int* call_flag;          // multi: device word, zero between calls; set when a key of the batch cannot share a word with its index
   int more_follow;           // another kernel of the same ccr_sort_edges call is launched behind this one
   int n_req;
   const int64_t* keys_in;
@@ -266,7 +267,6 @@ struct SortArgs {
 constexpr int kSortChunkLog = CCR_SORT_CHUNK_LOG;
 constexpr int kSortChunk = 1 << kSortChunkLog;  // records one block of the multi-block path sorts in shared memory
 constexpr int kSortChunkThreads = CCR_SORT_CHUNK_THREADS;
-constexpr int kSortMultiFlag = 0x5a17ed01;      // "this list is on the multi-block path", kept in the list's first output row
 
 __device__ __forceinline__ int sort_index_bits(int K) {
   int idx_bits = 1;
@@ -299,8 +299,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
   // keys that leave room for the record index in one 64-bit word (non-negative, below 2^(63 - index bits)) are
   // sorted as single words: key << shift | index orders like (key, index), needs 8 bytes per record and no
   // index array at all (the word's low bits are the index)
-  if (a.multi && *reinterpret_cast<const volatile int*>(a.feats_out + e0 * a.row_ch * 16) == kSortMultiFlag)
-    return;  // the chunked kernels have sorted this list
+  if (a.multi && __ldg(a.call_flag) == 0) return;  // the chunked kernels have sorted every list
   const int idx_bits = sort_index_bits(K);
   const bool packable = list_is_packable(a.keys_in + e0, K, idx_bits);
   const long long chunks = a.multi ? 0 : static_cast<long long>(K) * a.row_ch;  // multi: rows move in gather_all_kernel
@@ -364,18 +363,21 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
 
 // ---------------------------------------------------------------------------------------------------
 // Multi-block path.  One block per list leaves a 19,000-record list to a single SM while the others idle.  Here
-// chunks of kSortChunk records are sorted in shared memory by one block each (packed words, written to the key
-// output array) and the sorted chunks are then merged pairwise, one launch per doubling of the run length, every
-// block producing kSortMergeTile consecutive output words from the two stretches of its pair of runs that the
-// merge path assigns to them.  A flag in the list's first output row (written by the chunk kernel, overwritten by
-// the final row gather) tells the later kernels that the list is on this path.
+// chunks of kSortChunk records are sorted in shared memory by one block each (packed words) and the sorted chunks
+// are then merged pairwise, one launch per doubling of the run length, every block producing kSortMergeTile
+// consecutive output words from the two stretches of its pair of runs that the merge path assigns to them.
+// Packing needs keys that leave room for the index (non-negative, below 2^(63 - index bits)).  Every chunk block
+// checks the keys it loads; one that cannot be packed sets the call's flag word, and the batch is then sorted
+// list by list by sort_edges_kernel instead (what the chunked kernels wrote is overwritten).  The row gather at the
+// end of the call puts the word back to zero.
 
 __device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, long long& e0, int& K) {
   e0 = __ldg(a.edge_offsets + r);
   const long long Kl = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   K = Kl > 0 ? static_cast<int>(Kl) : 0;
-  if (K == 0) return false;
-  return *reinterpret_cast<const volatile int*>(a.feats_out + e0 * a.row_ch * 16) == kSortMultiFlag;
+  // (read-only in every kernel that tests it, so the load may be cached: ten thousand blocks reading one word
+  // past L1 queue up at a single L2 slice — 15 us on a 256-list batch)
+  return K > 0 && __ldg(a.call_flag) == 0;
 }
 
 // The grids of this path have one block per (list, tile of the longest list), either folded into x with lists
@@ -396,7 +398,7 @@ __device__ __forceinline__ void sort_block_item(const SortArgs& a, int& r, long 
 
 // Merging the sorted chunks.  Phase p = 1, 2, ... merges neighbouring runs of kSortChunk << (p - 1) words into
 // runs of twice that length, out of place: the words alternate between the key output array and a scratch area
-// inside the list's own output rows (8 bytes per record behind the flag's 16 bytes; a row has at least 16), which
+// inside the list's own output rows (8 bytes per record; a row has at least 16), which
 // nothing else uses until the rows are gathered at the end.  A list takes part in a phase while it is longer than
 // the phase's input runs, so a list of K records goes through P = sort_merge_phases(K) phases.  Its last phase
 // writes keys and source indices instead of words (a single-chunk list gets them from the chunk kernel), and so
@@ -408,7 +410,7 @@ __device__ __host__ __forceinline__ int sort_merge_phases(long long K) {
   return p;
 }
 __device__ __forceinline__ unsigned long long* sort_words_at(const SortArgs& a, long long e0, bool scratch) {
-  return scratch ? reinterpret_cast<unsigned long long*>(a.feats_out + e0 * a.row_ch * 16 + 16)
+  return scratch ? reinterpret_cast<unsigned long long*>(a.feats_out + e0 * a.row_ch * 16)
                  : reinterpret_cast<unsigned long long*>(a.keys_out + e0);
 }
 
@@ -424,14 +426,17 @@ __global__ void __launch_bounds__(kSortChunkThreads, CCR_SORT_CHUNK_BLOCKS) sort
   if (y * kSortChunk >= K) return;  // also K <= 0
   const int c0 = static_cast<int>(y) * kSortChunk;
   const int idx_bits = sort_index_bits(K);
-  const bool take = list_is_packable(a.keys_in + e0, K, idx_bits);
-  if (y == 0 && threadIdx.x == 0)
-    *reinterpret_cast<int*>(a.feats_out + e0 * a.row_ch * 16) = take ? kSortMultiFlag : 0;
-  if (!take) return;
   const int n = min(kSortChunk, K - c0);
-  for (int t = threadIdx.x; t < n; t += blockDim.x)
-    w[t] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + c0 + t)) << idx_bits) | static_cast<unsigned>(c0 + t);
-  __syncthreads();
+  int bad = 0;
+  for (int t = threadIdx.x; t < n; t += blockDim.x) {
+    const long long k = __ldg(a.keys_in + e0 + c0 + t);
+    bad |= (k < 0 || (k >> (63 - idx_bits)) != 0) ? 1 : 0;
+    w[t] = (static_cast<unsigned long long>(k) << idx_bits) | static_cast<unsigned>(c0 + t);
+  }
+  if (__syncthreads_or(bad)) {  // a key that cannot share a word with its index: the batch goes to the one-block path
+    if (threadIdx.x == 0) atomicOr(a.call_flag, 1);
+    return;
+  }
   static_assert(kSortChunk % kSortChunkThreads == 0, "every thread of a chunk block owns the same number of words");
   sort_words_merge<kSortChunk / kSortChunkThreads>(w, n);
   const int P = sort_merge_phases(K);
@@ -548,6 +553,7 @@ __global__ void __launch_bounds__(kSortGatherThreads) gather_all_kernel(const So
   int r;
   long long y;
   sort_block_item(a, r, y);
+  if (r == 0 && y == 0 && threadIdx.x == 0) *a.call_flag = 0;  // every reader of the word has finished: ready for the next call
   const long long e0 = __ldg(a.edge_offsets + r);
   const long long K = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   const long long chunks = K * a.row_ch;
