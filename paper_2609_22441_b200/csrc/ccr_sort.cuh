@@ -160,32 +160,15 @@ __device__ __forceinline__ void sort_words_bitonic(unsigned long long* w, int n)
   }
 }
 
-// Merge sort of n <= IPT * blockDim.x distinct words in shared memory: every thread sorts IPT consecutive words in
-// registers, then sorted runs are merged pairwise, doubling per pass; in a pass a thread produces IPT consecutive
-// output words, from the point of its pair of runs that the merge path (a binary search along its diagonal)
-// assigns to it, into registers, and writes them back after a barrier.  log2(n / IPT) passes of two barriers
-// each, against the ~n log^2 n / 2 compare-exchanges and ~25 barriers of the network for 4,096 words.
+// Merge passes over sorted runs of `run` words in shared memory (n <= IPT * blockDim.x distinct words): runs are
+// merged pairwise, doubling per pass; in a pass a thread produces IPT consecutive output words, from the point of
+// its pair of runs that the merge path (a binary search along its diagonal) assigns to it, into registers, and
+// writes them back after a barrier.  Two barriers per pass.
 template <int IPT>
-__device__ __forceinline__ void sort_words_merge(unsigned long long* w, int n) {
+__device__ __forceinline__ void merge_passes(unsigned long long* w, int n, int run) {
   const int t0 = static_cast<int>(threadIdx.x) * IPT;
   unsigned long long v[IPT];
-#pragma unroll
-  for (int u = 0; u < IPT; ++u) v[u] = t0 + u < n ? w[t0 + u] : ~0ull;
-  // odd-even transposition sort of the thread's words (IPT rounds)
-#pragma unroll
-  for (int rd = 0; rd < IPT; ++rd) {
-#pragma unroll
-    for (int u = rd & 1; u + 1 < IPT; u += 2) {
-      const unsigned long long lo = min(v[u], v[u + 1]), hi = max(v[u], v[u + 1]);
-      v[u] = lo;
-      v[u + 1] = hi;
-    }
-  }
-#pragma unroll
-  for (int u = 0; u < IPT; ++u)
-    if (t0 + u < n) w[t0 + u] = v[u];
-  __syncthreads();
-  for (int run = IPT; run < n; run <<= 1) {
+  for (; run < n; run <<= 1) {
     const int pb = (t0 / (2 * run)) * (2 * run);
     const int lenA = max(0, min(run, n - pb)), lenB = max(0, min(run, n - pb - run));
     const unsigned long long* A = w + pb;
@@ -212,6 +195,94 @@ __device__ __forceinline__ void sort_words_merge(unsigned long long* w, int n) {
       if (t0 + u < n) w[t0 + u] = v[u];
     __syncthreads();
   }
+}
+
+// Merge sort of n <= IPT * blockDim.x distinct words in shared memory: every thread sorts IPT consecutive words in
+// registers (odd-even transposition), then log2(n / IPT) merge passes.
+template <int IPT>
+__device__ __forceinline__ void sort_words_merge(unsigned long long* w, int n) {
+  const int t0 = static_cast<int>(threadIdx.x) * IPT;
+  unsigned long long v[IPT];
+#pragma unroll
+  for (int u = 0; u < IPT; ++u) v[u] = t0 + u < n ? w[t0 + u] : ~0ull;
+#pragma unroll
+  for (int rd = 0; rd < IPT; ++rd) {
+#pragma unroll
+    for (int u = rd & 1; u + 1 < IPT; u += 2) {
+      const unsigned long long lo = min(v[u], v[u + 1]), hi = max(v[u], v[u + 1]);
+      v[u] = lo;
+      v[u + 1] = hi;
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < IPT; ++u)
+    if (t0 + u < n) w[t0 + u] = v[u];
+  __syncthreads();
+  merge_passes<IPT>(w, n, IPT);
+}
+
+// The same for n <= 4 * blockDim.x with the first seven doublings in registers: a warp holds 128 consecutive words,
+// lane-strided (word e in register e / 32 of lane e % 32, so its loads and stores are to consecutive words), and
+// sorts them with a bitonic network whose steps at distances 32 and 64 pair registers of one lane and the others
+// lanes (shuffles): no shared memory, no barriers.  Measured per 4,096-word chunk (two blocks resident per SM):
+// 8 us for this start + 13 us for the five merge passes behind it, against 30 us for ten merge passes from runs of
+// four, and 23 us with the merge passes done warp-wise on strided registers as well (bitonic merges of 128).
+template <int J, typename Up>
+__device__ __forceinline__ void warp128_step(unsigned long long (&v)[4], int lane, Up up) {
+  if constexpr (J >= 32) {
+    constexpr int dr = J >> 5;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      if ((r & dr) == 0) {
+        const unsigned long long lo = min(v[r], v[r | dr]), hi = max(v[r], v[r | dr]);
+        const bool u = up((r << 5) | lane);  // the pair holding word e goes in ascending order
+        v[r] = u ? lo : hi;
+        v[r | dr] = u ? hi : lo;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const unsigned long long pv = __shfl_xor_sync(0xffffffffu, v[r], J);
+      const bool keep_min = ((lane & J) == 0) == up((r << 5) | lane);
+      v[r] = keep_min ? min(v[r], pv) : max(v[r], pv);
+    }
+  }
+}
+// the steps of one block size K of the network: partner distances K/2 ... 1
+template <int K, typename Up>
+__device__ __forceinline__ void warp128_block(unsigned long long (&v)[4], int lane, Up up) {
+  if constexpr (K >= 128) warp128_step<64>(v, lane, up);
+  if constexpr (K >= 64) warp128_step<32>(v, lane, up);
+  if constexpr (K >= 32) warp128_step<16>(v, lane, up);
+  if constexpr (K >= 16) warp128_step<8>(v, lane, up);
+  if constexpr (K >= 8) warp128_step<4>(v, lane, up);
+  if constexpr (K >= 4) warp128_step<2>(v, lane, up);
+  warp128_step<1>(v, lane, up);
+}
+__device__ __forceinline__ void sort_words_merge128(unsigned long long* w, int n) {
+  const int lane = threadIdx.x & 31, o = (static_cast<int>(threadIdx.x) >> 5) * 128;
+  unsigned long long v[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = o + (r << 5) + lane;
+    v[r] = i < n ? w[i] : ~0ull;  // padding sorts last
+  }
+  // blocks of K words alternate in direction until the last, which is ascending
+  warp128_block<2>(v, lane, [](int e) { return (e & 2) == 0; });
+  warp128_block<4>(v, lane, [](int e) { return (e & 4) == 0; });
+  warp128_block<8>(v, lane, [](int e) { return (e & 8) == 0; });
+  warp128_block<16>(v, lane, [](int e) { return (e & 16) == 0; });
+  warp128_block<32>(v, lane, [](int e) { return (e & 32) == 0; });
+  warp128_block<64>(v, lane, [](int e) { return (e & 64) == 0; });
+  warp128_block<128>(v, lane, [](int) { return true; });
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = o + (r << 5) + lane;
+    if (i < n) w[i] = v[r];
+  }
+  __syncthreads();
+  merge_passes<4>(w, n, 128);
 }
 
 // Rows follow their keys: output chunk c (16 bytes) comes from row source_of(c / row_ch) of the input.  One block
@@ -312,7 +383,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
       w[i] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
     __syncthreads();
     // merge sort while a thread's share of the list fits its registers, the network beyond
-    if (K <= 4 * kSortThreads) sort_words_merge<4>(w, K);
+    if (K <= 4 * kSortThreads) sort_words_merge128(w, K);
     else if (K <= 8 * kSortThreads) sort_words_merge<8>(w, K);
     else if (K <= 16 * kSortThreads) sort_words_merge<16>(w, K);
     else sort_words_bitonic(w, K);
@@ -437,8 +508,8 @@ __global__ void __launch_bounds__(kSortChunkThreads, CCR_SORT_CHUNK_BLOCKS) sort
     if (threadIdx.x == 0) atomicOr(a.call_flag, 1);
     return;
   }
-  static_assert(kSortChunk % kSortChunkThreads == 0, "every thread of a chunk block owns the same number of words");
-  sort_words_merge<kSortChunk / kSortChunkThreads>(w, n);
+  static_assert(kSortChunk == 4 * kSortChunkThreads, "a warp of a chunk block owns 128 words");
+  sort_words_merge128(w, n);
   const int P = sort_merge_phases(K);
   if (P == 0) {  // the whole list: done
     const unsigned long long low = (1ull << idx_bits) - 1;
