@@ -342,12 +342,12 @@ ccr_status ccr_workspace_outputs(const ccr_workspace* ws, void** rows, uint8_t**
  * copies the inputs to the workspace, runs ccr_join_batch, copies rows and mask back — all enqueued
  * on `stream`, nothing synchronised.  Pinned host memory makes the copies asynchronous.
  * total_edges = edge_offsets[n_req].  Sizes beyond the workspace give CCR_ERR_INVALID_ARG.
- * A batch of at least four requests and about a million candidates is pipelined: the requests are cut into four
+ * A batch of at least three requests and 786,432 candidates is pipelined: the requests are cut into three
  * groups of about equal candidate counts, and a group's payload crosses PCIe on a stream the workspace owns while
  * the groups already on the device are joined on `stream` (events order the two; results are those of one
  * ccr_join_batch over the whole batch).  For that the rebased offsets of the groups pass through a small pinned
- * block of the workspace with four rotation slots; a call only ever waits on the host when the copy of the call
- * four calls back has not yet run.  One workspace serves one stream at a time.
+ * block of the workspace with three rotation slots; a call only ever waits on the host when the copy of the call
+ * three calls back has not yet run.  One workspace serves one stream at a time.
  * out_rows may be NULL: the rows then stay in the workspace's device buffer, where the ranking model reads them
  * (ccr_workspace_outputs gives the DEVICE pointers; valid until the next call on this workspace), and only the
  * mask travels back — the serving case, in which the rows never leave the GPU.                      */

@@ -36,7 +36,13 @@ constexpr long long kSmallLaunchCands = 131072;  // plain launches up to this si
 constexpr int kAutoSmemBudget = 160 * 1024;  // shared memory the warp-specialised kernel takes by default
 constexpr int kMaxTile = ccr::kMaxTileCands;
 constexpr size_t kStageBytes = 16u << 20;  // staging block of second-degree stores (ids uploaded from the host)
-constexpr int kHostGroups = 4;                       // request groups of a pipelined host-buffer join
+#ifndef CCR_HOST_GROUPS
+#define CCR_HOST_GROUPS 3  // config 1, rows staying on the device: 1 group 0.514 ms, 2 0.431, 3 0.413, 4 0.437, 6 0.456, 8 0.495
+#endif
+#ifndef CCR_HOST_GROUP_CANDS
+#define CCR_HOST_GROUP_CANDS (2 * kSmallLaunchCands)
+#endif
+constexpr int kHostGroups = CCR_HOST_GROUPS;         // most request groups of a pipelined host-buffer join
 constexpr int kSchedRegions = 64;                    // launches of one store that may be in flight at once
 constexpr int kStatusHead = 4;                       // [0] wait expiry, [1] validation code; then the scheduling words:
                                                      // kSchedRegions regions of sched_stride ints
@@ -100,8 +106,8 @@ struct ccr_workspace {
   // workspace's own while the groups already there are being joined on the caller's stream.
   cudaStream_t copy_stream;
   cudaEvent_t ev_begin;                  // caller's stream -> copy stream: everything queued before the call
-  cudaEvent_t ev_group[4];               // copy stream -> caller's stream: group g has arrived
-  cudaEvent_t ev_offsets[4];             // the pinned offset block of rotation slot k has been read by its copy
+  cudaEvent_t ev_group[kHostGroups];               // copy stream -> caller's stream: group g has arrived
+  cudaEvent_t ev_offsets[kHostGroups];             // the pinned offset block of rotation slot k has been read by its copy
   int64_t* host_offsets;                 // pinned: 4 rotation slots of (max_req + 1 + 4) rebased candidate offsets
   int64_t calls;
 };
@@ -1282,8 +1288,12 @@ ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t 
   // equal candidate counts; group g + 1 crosses PCIe on the workspace's copy stream while group g is joined on the
   // caller's stream (each group is an ordinary ccr_join_batch over its own requests, candidates renumbered from 0).
   int n_groups = 1;
-  if (n_req >= kHostGroups && total_cands >= static_cast<int64_t>(kHostGroups) * 2 * kSmallLaunchCands && !(flags & CCR_FLAG_VALIDATE))
-    n_groups = kHostGroups;
+  if (!(flags & CCR_FLAG_VALIDATE)) {
+    const int64_t by_size = total_cands / (CCR_HOST_GROUP_CANDS);
+    n_groups = static_cast<int>(by_size < kHostGroups ? by_size : kHostGroups);
+    if (n_groups > n_req) n_groups = n_req;
+    if (n_groups < kHostGroups) n_groups = 1;
+  }
   if (n_groups == 1) {
     if (total_edges > 0) {
       ok = ok && cudaMemcpyAsync(w->edge_keys, edge_keys, total_edges * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -1316,7 +1326,7 @@ ccr_status ccr_join_batch_host(const ccr_docstore* s, ccr_workspace* w, int32_t 
     }
     first[n_groups] = n_req;
     // rebased candidate offsets of every group, in a pinned block of this call's rotation slot (a slot is reused
-    // four calls later; should its copy still be pending then, the host waits for it)
+    // kHostGroups calls later; should its copy still be pending then, the host waits for it)
     const int slot = static_cast<int>(w->calls++ % kHostGroups);
     int64_t* h_off = w->host_offsets + static_cast<size_t>(slot) * (w->max_req + 1 + kHostGroups);
     ok = ok && cudaEventSynchronize(w->ev_offsets[slot]) == cudaSuccess;
