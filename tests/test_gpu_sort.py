@@ -218,3 +218,33 @@ def test_sort_a_list_with_more_row_tiles_than_a_grid_has_rows(B):
         assert np.array_equal(got, want)
     finally:
         store.free()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_sort_random_batches(B, seed):
+    """Random batches: list lengths drawn around every boundary of the chunked path (empty, a few records, one
+    chunk, one record more, two / four / eight chunks +- 1, tens of thousands), key ranges from a handful of
+    distinct values (ties across every run boundary) to 2^44, with and without the permutation output."""
+    rng = np.random.default_rng(1000 + seed)
+    n_req = int(rng.integers(1, 40))
+    with_perm = bool(seed % 3 != 2)
+    pools = [lambda: 0, lambda: int(rng.integers(1, 50)), lambda: int(rng.integers(1000, 6000)),
+             lambda: int(rng.integers(4090, 4103)), lambda: int(rng.integers(8185, 8200)),
+             lambda: int(rng.integers(16380, 16390)), lambda: int(rng.integers(10_000, 19_000)),
+             lambda: int(rng.integers(32_760, 32_775)) if with_perm else int(rng.integers(18_000, 19_000))]
+    lens = [pools[int(rng.integers(0, len(pools)))]() for _ in range(n_req)]
+    hi = [3, 100, 1 << 20, 1 << 44][int(rng.integers(0, 4))]
+    keys = rng.integers(0, hi, size=sum(lens), dtype=np.int64)
+    feats = rng.standard_normal((len(keys), 64)).astype(np.float16)
+    eo = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    want_k, want_f, want_p = oracle.sort_edges(keys, feats, eo)
+    wl = W.config3(n_docs=1000, n_req=1, n_cand=10, gen_doc_feats=True, extra_pools=0)
+    store = B.store_from_workload(wl)
+    try:
+        k, f, p = _gpu_sort(B, store, keys, feats, eo, with_perm=with_perm)
+        assert np.array_equal(k.cpu().numpy(), want_k)
+        assert np.array_equal(f.cpu().numpy().view(np.uint16), want_f.view(np.uint16))
+        if with_perm:
+            assert np.array_equal(p.cpu().numpy(), want_p)
+    finally:
+        store.free()
