@@ -677,7 +677,9 @@ ccr_status ccr_idindex_create(int32_t device, int64_t n_ids, const int64_t* sort
     ok = cudaGetLastError() == cudaSuccess;
   }
   ok = ok && cudaDeviceSynchronize() == cudaSuccess;
-  ok = ok && cudaFuncSetAttribute(ccr::resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  ok = ok && cudaFuncSetAttribute(ccr::resolve_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  ccr::kResolveTopMax * 8 + 256) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(ccr::resolve_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   ccr::kResolveTopMax * 8 + 256) == cudaSuccess;
   ix->magic = kIxMagic;
   handle_add(ix);
@@ -716,7 +718,10 @@ ccr_status ccr_resolve_ids(const ccr_idindex* cix, int64_t n_queries, const int6
   const long long cap = static_cast<long long>(ix->n_sms) * ccr::kResolveBlocksPerSm;  // the top level is re-read by every block
   if (blocks > cap) blocks = cap;
   const size_t smem = static_cast<size_t>(ix->count[ix->n_levels - 1]) * 8 + 16;
-  ccr::resolve_kernel<<<static_cast<unsigned>(blocks), ccr::kResolveThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  if (n_queries >= ccr::kResolveWarpMin)
+    ccr::resolve_kernel<true><<<static_cast<unsigned>(blocks), ccr::kResolveThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  else
+    ccr::resolve_kernel<false><<<static_cast<unsigned>(blocks), ccr::kResolveThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
   ix->launches++;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
   return CCR_OK;

@@ -50,6 +50,26 @@ def test_resolve_matches_oracle(B, n_ids, with_positions):
     ix.free()
 
 
+@pytest.mark.parametrize("n_ids", [0, 1, 9, 2048, 2049, 16385, 8 * 16384 + 5, 3_000_000])
+@pytest.mark.parametrize("n_q", [(1 << 20), (1 << 20) + 37])
+def test_resolve_large_batches_take_the_lane_per_query_top_search(B, n_ids, n_q):
+    """From 2^20 queries on the kernel searches the top level a lane per query and hands the queries to the lane
+    groups by shuffles: same results, ragged last warp included, the largest int64 among the queries."""
+    rng = np.random.default_rng(n_ids + n_q)
+    ids = (np.cumsum(rng.integers(1, 6, size=n_ids)) * 2).astype(np.int64)
+    pos = rng.permutation(n_ids).astype(np.int32) if n_ids % 2 else None
+    q = _queries(rng, ids, n_q)
+    want = oracle.resolve_ids(ids, q, pos)
+    ix = B.IdIndex(ids, pos)
+    out = torch.full((len(q) + 64,), -7, dtype=torch.int32, device="cuda")
+    ix.resolve(torch.from_numpy(q).cuda(), out[32:32 + len(q)])
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    assert (got[:32] == -7).all() and (got[32 + len(q):] == -7).all()
+    assert np.array_equal(got[32:32 + len(q)], want)
+    ix.free()
+
+
 @pytest.mark.parametrize("n_ids", [5, 8, 13, 2048, 2051, 40_001])
 def test_resolve_with_the_largest_int64_as_an_id(B, n_ids):
     """Keys beyond the end of a level count as +infinity inside the kernel; an id equal to that value is still
