@@ -39,7 +39,13 @@ constexpr int kWsMaxThreads = 512;
 // (setmaxnreg.inc).  Registers only move inside the block's own allocation, and an increase waits until they are
 // there, so 384 x kRebalStreamerRegs + 256 x kRebalResolverRegs must not exceed 640 x 96 — more would never
 // arrive.  Eight resolvers fill eight ring slots at a time, so the ring is twice as deep (of half-size slots).
-constexpr int kRebalStreamers = 12, kRebalResolvers = 8;
+#ifndef CCR_REBAL_STREAMERS
+#define CCR_REBAL_STREAMERS 12
+#endif
+#ifndef CCR_REBAL_RESOLVERS
+#define CCR_REBAL_RESOLVERS 8
+#endif
+constexpr int kRebalStreamers = CCR_REBAL_STREAMERS, kRebalResolvers = CCR_REBAL_RESOLVERS;
 constexpr int kRebalThreads = (kRebalStreamers + kRebalResolvers) * 32;
 #ifndef CCR_REBAL_STREAMER_REGS
 #define CCR_REBAL_STREAMER_REGS 104
