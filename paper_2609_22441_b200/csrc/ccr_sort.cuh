@@ -322,8 +322,8 @@ struct SortArgs {
   int smem_keys;         // (key, index) records the dynamic shared memory can hold: 12 bytes each
   int smem_words;        // packed key|index words it can hold: 8 bytes each
   int max_len;           // the host's bound on the list length: longer lists are cut there (their tail is left alone)
-  int multi;             // 1: packable lists longer than kSortChunk are sorted by the multi-block kernels, and the
-                         //    rows of every list are moved by gather_all_kernel (perm_out is then required)
+  int multi;             // 1: the chunked kernels sort every list (sort_edges_kernel only when a key of the batch cannot be
+                         //    packed), and the rows of every list are moved by gather_all_kernel (perm_out is then required)
 };
 
 #ifndef CCR_SORT_CHUNK_LOG
