@@ -47,8 +47,9 @@ typedef enum {
   CCR_ERR_BAD_HANDLE = 5,  /* handle is NULL, freed or not one of ours                             */
   CCR_ERR_VALIDATION = 6,  /* CCR_FLAG_VALIDATE found a broken precondition                        */
   CCR_ERR_DEVICE_WAIT = 7, /* a bounded device-side wait ran out (reported by device_status)       */
-  CCR_ERR_BOUNDS = 8       /* bounds-checked build only (-DCCR_DEBUG_BOUNDS): a join kernel computed an address outside
-                              the buffers of its launch; the access was skipped (reported by device_status)          */
+  CCR_ERR_BOUNDS = 8       /* bounds-checked build only (-DCCR_DEBUG_BOUNDS): a kernel computed an address outside the
+                              buffers of its launch; the access was skipped (joins: reported by device_status; sort,
+                              resolve, compaction and upsert calls wait for their kernels and return it themselves)   */
 } ccr_status;
 
 typedef enum { CCR_F16 = 0, CCR_F32 = 1 } ccr_dtype;
@@ -409,9 +410,10 @@ ccr_status ccr_join_payload_static(const ccr_docstore* store,
  * CCR_ERR_DEVICE_WAIT if a kernel gave up a bounded wait for a shared-memory bulk copy since the
  * last call (the affected rows of that launch were not written).  Clears the word.
  * The bounds-checked build of the library (compiled with -DCCR_DEBUG_BOUNDS; `python -m paper_2609_22441_b200.build
- * --debug-bounds` writes it next to the release build) checks every global address the join kernels compute against
- * the extents of the launch's buffers, leaves out an access that falls outside (never a trap) and reports
- * CCR_ERR_BOUNDS here; it synchronises after every join and is meant for tests, not for serving.            */
+ * --debug-bounds` writes it next to the release build) checks every global address the join, sort, resolve,
+ * compaction and upsert kernels compute against the extents of the launch's buffers and leaves out an access that
+ * falls outside (never a trap).  A join reports CCR_ERR_BOUNDS here; the other calls wait for their kernels and
+ * return it as their own status.  The build synchronises in every call and is meant for tests, not for serving.   */
 ccr_status ccr_docstore_device_status(ccr_docstore* store, void* stream);
 
 /* Self-test of the failure-reporting path (no fault, trap or hang is involved): enqueues a one-block kernel
@@ -445,8 +447,8 @@ const char* ccr_status_str(ccr_status s);
 int         ccr_version(void);
 /* 1 in the bounds-checked build, 0 in the release build. */
 int         ccr_debug_bounds_enabled(void);
-/* Bounds-checked build only (no-op otherwise): pretend that the output buffers of the following joins on this store
- * end `rows` rows early, so that the mechanism itself can be tested without a real out-of-range access.   */
+/* Bounds-checked build only (no-op otherwise): pretend that the output rows of the following joins and sorts on this
+ * store (and the store's own rows, for upserts) end `rows` rows early, so that the mechanism itself can be tested without a real out-of-range access.   */
 ccr_status  ccr_debug_shrink_outputs(ccr_docstore* store, int64_t rows);
 
 #ifdef __cplusplus

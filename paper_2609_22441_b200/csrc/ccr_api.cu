@@ -121,6 +121,7 @@ struct ccr_idindex {
   int64_t* level[ccr::kResolveMaxLevels];  // level[0] = sorted ids (owned copy)
   long long count[ccr::kResolveMaxLevels];
   int32_t* positions;                      // owned copy, or null
+  int* dbg_word;                           // bounds-checked build: set by a kernel whose access left the registered buffers
   int64_t launches;
 };
 
@@ -318,6 +319,20 @@ struct DbgRegistrar {
     return cudaMemcpyToSymbol(ccr::g_dbg, &t, sizeof(t)) == cudaSuccess;
   }
 };
+// End of a checked call outside the joins: wait for its kernels and report a flagged address as the call's status
+// (the joins leave that to ccr_docstore_device_status).
+ccr_status dbg_finish(int* word, cudaStream_t st) {
+  int v = 0;
+  if (cudaStreamSynchronize(st) != cudaSuccess || cudaMemcpy(&v, word, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return CCR_ERR_CUDA;
+  }
+  if (v != 0) {
+    cudaMemset(word, 0, 4);
+    return CCR_ERR_BOUNDS;
+  }
+  return CCR_OK;
+}
 #endif
 
 // Launch of a kernel that belongs to a chain of small launches (its first statement is chain_enter()): with
@@ -553,6 +568,25 @@ ccr_status ccr_docstore_upsert(ccr_docstore* s, int64_t n, const int32_t* positi
   a.dst_author = s->author_ids;
   a.dst_recs = ma > 0 ? s->id_recs : nullptr;
   a.max_actors = ma;
+#ifdef CCR_DEBUG_BOUNDS
+  {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
+    const int64_t rows = s->desc.n_docs > s->dbg_shrink_rows ? s->desc.n_docs - s->dbg_shrink_rows : 0;
+    DbgRegistrar reg;
+    reg.add(positions, static_cast<size_t>(n) * 4);
+    reg.add(doc_feats, static_cast<size_t>(n) * s->doc_b);
+    reg.add(author_ids, static_cast<size_t>(n) * 8);
+    reg.add(actor_ids, static_cast<size_t>(n) * ma * 8);
+    reg.add(actor_types, static_cast<size_t>(n) * ma);
+    reg.add(s->doc_feats, static_cast<size_t>(rows) * s->doc_b);
+    reg.add(s->author_ids, static_cast<size_t>(rows) * 8);
+    reg.add(s->id_recs, static_cast<size_t>(rows) * sizeof(ccr::IdRec));
+    if (!reg.commit(s->status + 2)) return CCR_ERR_CUDA;
+  }
+#endif
   const long long work = doc_feats ? n * a.row_ch : n;
   const long long per_block = static_cast<long long>(ccr::kUpsertThreads) * ccr::kUpsertUnroll;
   long long blocks = (work + per_block - 1) / per_block;
@@ -561,7 +595,11 @@ ccr_status ccr_docstore_upsert(ccr_docstore* s, int64_t n, const int32_t* positi
   ccr::upsert_kernel<<<static_cast<unsigned>(blocks), ccr::kUpsertThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
   s->launches++;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+#ifdef CCR_DEBUG_BOUNDS
+  return dbg_finish(s->status + 2, static_cast<cudaStream_t>(stream));
+#else
   return CCR_OK;
+#endif
 }
 
 size_t ccr_out_row_bytes(const ccr_docstore* s, uint32_t flags) { return good(s) ? out_row_bytes(s, flags) : 0; }
@@ -612,6 +650,7 @@ ccr_status ccr_idindex_free(ccr_idindex* ix) {
   ix->magic = 0;
   for (int l = 0; l < ccr::kResolveMaxLevels; ++l) cudaFree(ix->level[l]);
   cudaFree(ix->positions);
+  cudaFree(ix->dbg_word);
   delete ix;
   return CCR_OK;
 }
@@ -676,6 +715,9 @@ ccr_status ccr_idindex_create(int32_t device, int64_t n_ids, const int64_t* sort
     ix->launches++;
     ok = cudaGetLastError() == cudaSuccess;
   }
+#ifdef CCR_DEBUG_BOUNDS
+  ok = ok && cudaMalloc(&ix->dbg_word, 256) == cudaSuccess && cudaMemset(ix->dbg_word, 0, 256) == cudaSuccess;
+#endif
   ok = ok && cudaDeviceSynchronize() == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(ccr::resolve_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   ccr::kResolveTopMax * 8 + 256) == cudaSuccess;
@@ -712,6 +754,20 @@ ccr_status ccr_resolve_ids(const ccr_idindex* cix, int64_t n_queries, const int6
   a.n_queries = n_queries;
   a.queries = query_ids;
   a.out_pos = out_pos;
+#ifdef CCR_DEBUG_BOUNDS
+  {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
+    DbgRegistrar reg;
+    for (int l = 0; l < ix->n_levels; ++l) reg.add(ix->level[l], static_cast<size_t>(ix->count[l] + ccr::kResolvePad) * 8);
+    reg.add(ix->positions, static_cast<size_t>(ix->n_ids) * 4);
+    reg.add(query_ids, static_cast<size_t>(n_queries) * 8);
+    reg.add(out_pos, static_cast<size_t>(n_queries) * 4);
+    if (!reg.commit(ix->dbg_word)) return CCR_ERR_CUDA;
+  }
+#endif
   const long long per_block = static_cast<long long>(ccr::kResolveThreads);
   const long long lanes = 1LL << (ccr::kResolveFanLog2 - 1);  // lanes that share a query
   long long blocks = (n_queries * lanes + per_block - 1) / per_block;
@@ -724,7 +780,11 @@ ccr_status ccr_resolve_ids(const ccr_idindex* cix, int64_t n_queries, const int6
     ccr::resolve_kernel<false><<<static_cast<unsigned>(blocks), ccr::kResolveThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
   ix->launches++;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+#ifdef CCR_DEBUG_BOUNDS
+  return dbg_finish(ix->dbg_word, static_cast<cudaStream_t>(stream));  // an index has no status call of its own
+#else
   return CCR_OK;
+#endif
 }
 
 ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edge_len, const int64_t* keys_in,
@@ -764,6 +824,27 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
   // the call's flag word: word 8 of a scheduling region (the joins use words 0 and 1), regions taken in turn, so up
   // to kSchedRegions chunked sorts of one store may be in flight at once
   a.call_flag = a.multi ? s->status + kStatusHead + s->sched_stride * static_cast<int>(s->sort_calls.fetch_add(1) % kSchedRegions) + 8 : nullptr;
+#ifdef CCR_DEBUG_BOUNDS
+  {
+    // the record count is on the device: read it back (this build synchronises anyway)
+    int64_t E = 0;
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaMemcpy(&E, edge_offsets + n_req, 8, cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
+    const size_t row_b = static_cast<size_t>(a.row_ch) * 16;
+    const int64_t out_rows_n = E > s->dbg_shrink_rows ? E - s->dbg_shrink_rows : 0;
+    DbgRegistrar reg;
+    reg.add(keys_in, static_cast<size_t>(E) * 8);
+    reg.add(feats_in, static_cast<size_t>(E) * row_b);
+    reg.add(edge_offsets, static_cast<size_t>(n_req + 1) * 8);
+    reg.add(keys_out, static_cast<size_t>(E) * 8);
+    reg.add(feats_out, static_cast<size_t>(out_rows_n) * row_b);
+    reg.add(perm_out, static_cast<size_t>(E) * 4);
+    reg.add(a.call_flag, 4);
+    if (!reg.commit(s->status + 2)) return CCR_ERR_CUDA;
+  }
+#endif
   // grids of the chunked path: one block per tile of every list, sized for the longest list, folded into one
   // dimension; the row gather takes lists x tiles when the tiles fit a grid's second dimension (x = 0: too many blocks)
   auto tiles_grid = [&](long long per_list_units, long long tile, bool two_d) -> dim3 {
@@ -794,7 +875,11 @@ ccr_status ccr_sort_edges(const ccr_docstore* cs, int32_t n_req, int64_t max_edg
     s->launches++;
   }
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+#ifdef CCR_DEBUG_BOUNDS
+  return dbg_finish(s->status + 2, st);
+#else
   return CCR_OK;
+#endif
 }
 
 ccr_status ccr_docstore_selftest_wait(ccr_docstore* s, void* stream) {
@@ -1174,6 +1259,21 @@ ccr_status ccr_compact_valid(const ccr_docstore* cs, int32_t n_req, int64_t tota
   if (!scope.ok) return CCR_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const long long n_docs = s->desc.n_docs;
+#ifdef CCR_DEBUG_BOUNDS
+  {
+    if (cudaStreamSynchronize(st) != cudaSuccess) {
+      cudaGetLastError();
+      return CCR_ERR_CUDA;
+    }
+    DbgRegistrar reg;
+    reg.add(cand_idx, static_cast<size_t>(total_cands) * 4);
+    reg.add(cand_offsets, static_cast<size_t>(n_req + 1) * 8);
+    reg.add(offsets_out, static_cast<size_t>(n_req + 1) * 8);
+    reg.add(idx_out, static_cast<size_t>(total_cands) * 4);
+    reg.add(src_out, static_cast<size_t>(total_cands) * 4);
+    if (!reg.commit(s->status + 2)) return CCR_ERR_CUDA;
+  }
+#endif
   launch_chained(ccr::count_valid_kernel, dim3(static_cast<unsigned>(n_req)), dim3(ccr::kPadThreads), 0, st, cand_idx, cand_offsets,
                  n_docs, offsets_out);
   launch_chained(ccr::scan_counts_kernel, dim3(1), dim3(ccr::kPadThreads), 0, st, offsets_out, n_req);
@@ -1185,7 +1285,11 @@ ccr_status ccr_compact_valid(const ccr_docstore* cs, int32_t n_req, int64_t tota
       cand_idx, cand_offsets, n_docs, offsets_out, idx_out, src_out);
   s->launches += 3;
   if (cudaGetLastError() != cudaSuccess) return CCR_ERR_CUDA;
+#ifdef CCR_DEBUG_BOUNDS
+  return dbg_finish(s->status + 2, st);
+#else
   return CCR_OK;
+#endif
 }
 
 ccr_status ccr_workspace_create(const ccr_docstore* s, int32_t max_req, int64_t max_cands, int64_t max_edges,

@@ -158,7 +158,7 @@ __device__ __forceinline__ void chain_enter(bool more_follow) {
 }
 
 // ---- bounds-checked build (-DCCR_DEBUG_BOUNDS) ------------------------------------------------------------------
-// Every global load and store of the join kernels goes through gload / gstore / ldg128 / st128_stream.  In the
+// Every global load and store of the kernels goes through gload / gstore / ldg128 / st128_stream and their kin.  In the
 // checked build the host registers the extent of every buffer of the launch in g_dbg; an access that does not lie
 // inside one of them is not made (loads give zero), and a code is left in the store's third status word, which
 // ccr_docstore_device_status reports as CCR_ERR_BOUNDS.  Nothing traps.  The release build compiles the checks away.
@@ -192,6 +192,15 @@ __device__ __forceinline__ T gload(const T* p) {
 template <typename T, typename V>
 __device__ __forceinline__ void gstore(T* p, V v) {
   if (CCR_CHK(p, static_cast<int>(sizeof(T)))) *p = static_cast<T>(v);
+}
+// load of data that an earlier part of the same kernel may have written (no read-only path)
+template <typename T>
+__device__ __forceinline__ T gload_rw(const T* p) {
+  if (!CCR_CHK(p, static_cast<int>(sizeof(T)))) return T{};
+  return *p;
+}
+__device__ __forceinline__ void gatomic_or(int* p, int v) {
+  if (CCR_CHK(p, 4)) atomicOr(p, v);
 }
 __device__ __forceinline__ uint4 ldg128(const void* p) {
   if (!CCR_CHK(p, 16)) return make_uint4(0u, 0u, 0u, 0u);

@@ -51,7 +51,7 @@ __device__ __forceinline__ int block_count_valid(const int32_t* cand_idx, long l
 #pragma unroll
     for (int k = 0; k < kPadItems; ++k) {
       const long long j = base + static_cast<long long>(k) * kPadThreads;
-      p[k] = j < j1 ? __ldg(cand_idx + j) : -1;
+      p[k] = j < j1 ? gload(cand_idx + j) : -1;
     }
 #pragma unroll
     for (int k = 0; k < kPadItems; ++k) c += position_valid(p[k], n_docs) ? 1 : 0;
@@ -68,10 +68,10 @@ count_valid_kernel(const int32_t* cand_idx, const int64_t* cand_offsets, long lo
   chain_enter(true);
   __shared__ int warp_sums[kPadThreads / 32];
   const int r = blockIdx.x;
-  const int total = block_count_valid(cand_idx, cand_offsets[r], cand_offsets[r + 1], n_docs, warp_sums);
+  const int total = block_count_valid(cand_idx, gload(cand_offsets + r), gload(cand_offsets + r + 1), n_docs, warp_sums);
   if (threadIdx.x == 0) {
-    counts[r + 1] = total;
-    if (r == 0) counts[0] = 0;
+    gstore(counts + r + 1, total);
+    if (r == 0) gstore(counts, 0);
   }
 }
 
@@ -84,11 +84,11 @@ __global__ void __launch_bounds__(kPadThreads) scan_counts_kernel(int64_t* count
   __syncthreads();
   for (int base = 0; base < n_req; base += kPadThreads) {
     const int r = base + threadIdx.x;
-    const int v = r < n_req ? static_cast<int>(counts[r + 1]) : 0;
+    const int v = r < n_req ? static_cast<int>(gload_rw(counts + r + 1)) : 0;
     int total;
     const int inc = block_scan_inclusive(v, warp_sums, total);
     const long long carry = carry_s;
-    if (r < n_req) counts[r + 1] = carry + inc;
+    if (r < n_req) gstore(counts + r + 1, carry + inc);
     __syncthreads();
     if (threadIdx.x == 0) carry_s = carry + total;
     __syncthreads();
@@ -109,16 +109,16 @@ compact_valid_kernel(const int32_t* cand_idx, const int64_t* cand_offsets, long 
   __shared__ int warp_sums[kPadThreads / 32];
   const int r = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const long long j0 = cand_offsets[r], j1 = cand_offsets[r + 1];
+  const long long j0 = gload(cand_offsets + r), j1 = gload(cand_offsets + r + 1);
   const long long slice = (((j1 - j0) + gridDim.y - 1) / gridDim.y + 31) / 32 * 32;
   const long long s0 = min(j1, j0 + blockIdx.y * slice), s1 = min(j1, s0 + slice);
   if (s0 >= s1) return;
-  long long out = offsets_out[r] + block_count_valid(cand_idx, j0, s0, n_docs, warp_sums);
+  long long out = gload(offsets_out + r) + block_count_valid(cand_idx, j0, s0, n_docs, warp_sums);
   for (long long base = s0; base < s1; base += kPadThreads * kPadItems) {
     const long long jw = base + static_cast<long long>(warp) * (32 * kPadItems) + lane;
     int p[kPadItems];
 #pragma unroll
-    for (int k = 0; k < kPadItems; ++k) p[k] = jw + 32 * k < s1 ? __ldg(cand_idx + jw + 32 * k) : -1;
+    for (int k = 0; k < kPadItems; ++k) p[k] = jw + 32 * k < s1 ? gload(cand_idx + jw + 32 * k) : -1;
     unsigned votes[kPadItems];
     int warp_total = 0;
 #pragma unroll
@@ -140,8 +140,8 @@ compact_valid_kernel(const int32_t* cand_idx, const int64_t* cand_offsets, long 
     for (int k = 0; k < kPadItems; ++k) {
       if ((votes[k] >> lane) & 1u) {
         const long long w = w0 + __popc(votes[k] & ((1u << lane) - 1u));
-        idx_out[w] = p[k];
-        if (src_out != nullptr) src_out[w] = static_cast<int32_t>(jw + 32 * k);
+        gstore(idx_out + w, p[k]);
+        if (src_out != nullptr) gstore(src_out + w, jw + 32 * k);
       }
       w0 += __popc(votes[k]);
     }
@@ -155,7 +155,7 @@ compact_valid_kernel(const int32_t* cand_idx, const int64_t* cand_offsets, long 
 __global__ void __launch_bounds__(kPadThreads)
 pad_fill_kernel(const int64_t* cand_offsets, long long n_max, long long out_b, uint8_t* out_rows, uint8_t* out_mask) {
   const int r = blockIdx.x;
-  long long n_r = cand_offsets[r + 1] - cand_offsets[r];
+  long long n_r = gload(cand_offsets + r + 1) - gload(cand_offsets + r);
   n_r = n_r < 0 ? 0 : (n_r > n_max ? n_max : n_r);
   const long long first = r * n_max + n_r, pads = n_max - n_r;
   uint4* rows = reinterpret_cast<uint4*>(out_rows + first * out_b);

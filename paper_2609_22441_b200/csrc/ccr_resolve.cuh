@@ -47,6 +47,7 @@ struct ResolveArgs {
 // 16-byte window piece of a level that does not stay in any cache between queries (the three lowest levels of a
 // large index): read past L1.
 __device__ __forceinline__ longlong2 resolve_load(const longlong2* p, bool once) {
+  if (!CCR_CHK(p, 16)) return make_longlong2(kResolveInf, kResolveInf);  // reads like the padding behind a level
 #ifndef CCR_RESOLVE_L1
   if (once) {
     longlong2 v;
@@ -80,7 +81,7 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
   int64_t* top = reinterpret_cast<int64_t*>(smem_res);
   const int top_l = a.n_levels - 1;
   const int n_top = static_cast<int>(a.count[top_l]);
-  for (int i = threadIdx.x; i < n_top; i += blockDim.x) top[i] = __ldg(a.level[top_l] + i);
+  for (int i = threadIdx.x; i < n_top; i += blockDim.x) top[i] = gload(a.level[top_l] + i);
   __syncthreads();
   constexpr int G = 1 << (kResolveFanLog2 - 1);  // lanes that share a query: one 16-byte load each per window
   if constexpr (WARP_TOP) {
@@ -93,7 +94,7 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
     // kResolveWarpUnroll x 8 at a time, to groups of G lanes by shuffles.
     for (long long first = warp_id * 32; first < a.n_queries; first += n_warps * 32) {  // warp-uniform
       const long long mine = first + lane;
-      const int64_t q_own = mine < a.n_queries ? __ldg(a.queries + mine) : 0;
+      const int64_t q_own = mine < a.n_queries ? gload(a.queries + mine) : 0;
       unsigned c_own = 0;  // number of keys of the current level that are below q (an index has < 2^31 ids)
       {
         int n = n_top;
@@ -142,8 +143,8 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
             const long long j = first + src[u];
             if (sub == 0 && j < a.n_queries) {
               int pos = -1;
-              if (v >= 256u && c[u] < a.count[0]) pos = a.positions ? __ldg(a.positions + c[u]) : static_cast<int>(c[u]);
-              a.out_pos[j] = pos;
+              if (v >= 256u && c[u] < a.count[0]) pos = a.positions ? gload(a.positions + c[u]) : static_cast<int>(c[u]);
+              gstore(a.out_pos + j, pos);
             }
           }
         }
@@ -162,7 +163,7 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
 #pragma unroll
     for (int u = 0; u < kResolveUnroll; ++u) {
       const long long j = base + static_cast<long long>(u) * groups;
-      q[u] = j < a.n_queries ? __ldg(a.queries + j) : 0;
+      q[u] = j < a.n_queries ? gload(a.queries + j) : 0;
       c[u] = 0;
     }
     {  // the group's searches of the top level step together, so their shared-memory reads overlap
@@ -206,8 +207,8 @@ __global__ void __launch_bounds__(kResolveThreads) resolve_kernel(const ResolveA
         const long long j = base + static_cast<long long>(u) * groups;
         if (sub == 0 && j < a.n_queries) {
           int pos = -1;
-          if (v >= 256u && c[u] < a.count[0]) pos = a.positions ? __ldg(a.positions + c[u]) : static_cast<int>(c[u]);
-          a.out_pos[j] = pos;
+          if (v >= 256u && c[u] < a.count[0]) pos = a.positions ? gload(a.positions + c[u]) : static_cast<int>(c[u]);
+          gstore(a.out_pos + j, pos);
         }
       }
     }

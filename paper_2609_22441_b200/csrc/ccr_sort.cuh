@@ -297,13 +297,13 @@ __device__ __forceinline__ void gather_rows(const uint4* src, uint4* dst, long l
       const long long c = c0 + static_cast<long long>(u) * blockDim.x;
       if (c < chunks) {
         const int row = static_cast<int>(c / row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * row_ch);
-        v[u] = __ldg(src + source_of(row) * row_ch + piece);
+        v[u] = ldg128(src + source_of(row) * row_ch + piece);
       }
     }
 #pragma unroll
     for (int u = 0; u < kSortGatherUnroll; ++u) {
       const long long c = c0 + static_cast<long long>(u) * blockDim.x;
-      if (c < chunks) dst[c] = v[u];
+      if (c < chunks) st128_stream(dst + c, v[u]);
     }
   }
 }
@@ -352,7 +352,7 @@ __device__ __forceinline__ bool list_is_packable(const int64_t* keys, int K, int
   int negative = 0;
 #pragma unroll 8
   for (int i = threadIdx.x; i < K; i += blockDim.x) {
-    const long long k = __ldg(keys + i);
+    const long long k = gload(keys + i);
     kmax = max(kmax, k);
     negative |= (k < 0);
   }
@@ -363,14 +363,14 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
   chain_enter(a.more_follow != 0);
   extern __shared__ __align__(16) unsigned char smem_sort[];
   const int r = blockIdx.x;
-  const long long e0 = __ldg(a.edge_offsets + r);
-  const long long Kl = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
+  const long long e0 = gload(a.edge_offsets + r);
+  const long long Kl = min(static_cast<long long>(gload(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   if (Kl <= 0) return;
   const int K = static_cast<int>(Kl);
   // keys that leave room for the record index in one 64-bit word (non-negative, below 2^(63 - index bits)) are
   // sorted as single words: key << shift | index orders like (key, index), needs 8 bytes per record and no
   // index array at all (the word's low bits are the index)
-  if (a.multi && __ldg(a.call_flag) == 0) return;  // the chunked kernels have sorted every list
+  if (a.multi && gload(a.call_flag) == 0) return;  // the chunked kernels have sorted every list
   const int idx_bits = sort_index_bits(K);
   const bool packable = list_is_packable(a.keys_in + e0, K, idx_bits);
   const long long chunks = a.multi ? 0 : static_cast<long long>(K) * a.row_ch;  // multi: rows move in gather_all_kernel
@@ -380,7 +380,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
   if (packable && K <= a.smem_words) {
     unsigned long long* w = reinterpret_cast<unsigned long long*>(smem_sort);
     for (int i = threadIdx.x; i < K; i += blockDim.x)
-      w[i] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
+      w[i] = (static_cast<unsigned long long>(gload(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
     __syncthreads();
     // merge sort while a thread's share of the list fits its registers, the network beyond
     if (K <= 4 * kSortThreads) sort_words_merge128(w, K);
@@ -390,8 +390,8 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
     const unsigned long long low = (1ull << idx_bits) - 1;
     for (int i = threadIdx.x; i < K; i += blockDim.x) {
       const unsigned long long v = w[i];
-      a.keys_out[e0 + i] = static_cast<long long>(v >> idx_bits);
-      if (a.perm_out) a.perm_out[e0 + i] = static_cast<int>(v & low);
+      gstore(a.keys_out + e0 + i, v >> idx_bits);
+      if (a.perm_out) gstore(a.perm_out + e0 + i, v & low);
     }
     gather_rows(src, dst, chunks, a.row_ch, [&](int row) { return static_cast<long long>(w[row] & low); });
     return;
@@ -404,7 +404,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
   if (packable) {  // only reached by lists too long for shared memory: the words live in the key output array
     unsigned long long* w = reinterpret_cast<unsigned long long*>(keys);
     for (int i = threadIdx.x; i < K; i += blockDim.x)
-      w[i] = (static_cast<unsigned long long>(__ldg(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
+      w[i] = (static_cast<unsigned long long>(gload(a.keys_in + e0 + i)) << idx_bits) | static_cast<unsigned>(i);
     __syncthreads();
     sort_words_bitonic(w, K);
     const unsigned long long low = (1ull << idx_bits) - 1;
@@ -416,7 +416,7 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
     __syncthreads();
   } else {
     for (int i = threadIdx.x; i < K; i += blockDim.x) {
-      keys[i] = __ldg(a.keys_in + e0 + i);
+      keys[i] = gload(a.keys_in + e0 + i);
       idx[i] = i;
     }
     __syncthreads();
@@ -424,8 +424,8 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
   }
   if (in_smem) {
     for (int i = threadIdx.x; i < K; i += blockDim.x) {
-      a.keys_out[e0 + i] = keys[i];
-      if (a.perm_out) a.perm_out[e0 + i] = idx[i];
+      gstore(a.keys_out + e0 + i, keys[i]);
+      if (a.perm_out) gstore(a.perm_out + e0 + i, idx[i]);
     }
   }
   gather_rows(src, dst, chunks, a.row_ch, [&](int row) { return static_cast<long long>(idx[row]); });
@@ -443,12 +443,12 @@ __global__ void __launch_bounds__(kSortThreads, 1) sort_edges_kernel(const SortA
 // end of the call puts the word back to zero.
 
 __device__ __forceinline__ bool list_on_multi_path(const SortArgs& a, int r, long long& e0, int& K) {
-  e0 = __ldg(a.edge_offsets + r);
-  const long long Kl = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
+  e0 = gload(a.edge_offsets + r);
+  const long long Kl = min(static_cast<long long>(gload(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   K = Kl > 0 ? static_cast<int>(Kl) : 0;
   // (read-only in every kernel that tests it, so the load may be cached: ten thousand blocks reading one word
   // past L1 queue up at a single L2 slice — 15 us on a 256-list batch)
-  return K > 0 && __ldg(a.call_flag) == 0;
+  return K > 0 && gload(a.call_flag) == 0;
 }
 
 // The grids of this path have one block per (list, tile of the longest list), either folded into x with lists
@@ -492,20 +492,20 @@ __global__ void __launch_bounds__(kSortChunkThreads, CCR_SORT_CHUNK_BLOCKS) sort
   int r;
   long long y;
   sort_block_item(a, r, y);
-  const long long e0 = __ldg(a.edge_offsets + r);
-  const int K = static_cast<int>(min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len)));
+  const long long e0 = gload(a.edge_offsets + r);
+  const int K = static_cast<int>(min(static_cast<long long>(gload(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len)));
   if (y * kSortChunk >= K) return;  // also K <= 0
   const int c0 = static_cast<int>(y) * kSortChunk;
   const int idx_bits = sort_index_bits(K);
   const int n = min(kSortChunk, K - c0);
   int bad = 0;
   for (int t = threadIdx.x; t < n; t += blockDim.x) {
-    const long long k = __ldg(a.keys_in + e0 + c0 + t);
+    const long long k = gload(a.keys_in + e0 + c0 + t);
     bad |= (k < 0 || (k >> (63 - idx_bits)) != 0) ? 1 : 0;
     w[t] = (static_cast<unsigned long long>(k) << idx_bits) | static_cast<unsigned>(c0 + t);
   }
   if (__syncthreads_or(bad)) {  // a key that cannot share a word with its index: the batch goes to the one-block path
-    if (threadIdx.x == 0) atomicOr(a.call_flag, 1);
+    if (threadIdx.x == 0) gatomic_or(a.call_flag, 1);
     return;
   }
   static_assert(kSortChunk == 4 * kSortChunkThreads, "a warp of a chunk block owns 128 words");
@@ -514,13 +514,13 @@ __global__ void __launch_bounds__(kSortChunkThreads, CCR_SORT_CHUNK_BLOCKS) sort
   if (P == 0) {  // the whole list: done
     const unsigned long long low = (1ull << idx_bits) - 1;
     for (int t = threadIdx.x; t < n; t += blockDim.x) {
-      a.keys_out[e0 + t] = static_cast<long long>(w[t] >> idx_bits);
-      a.perm_out[e0 + t] = static_cast<int>(w[t] & low);
+      gstore(a.keys_out + e0 + t, w[t] >> idx_bits);
+      gstore(a.perm_out + e0 + t, w[t] & low);
     }
     return;
   }
   unsigned long long* W = sort_words_at(a, e0, (P & 1) != 0);
-  for (int t = threadIdx.x; t < n; t += blockDim.x) W[c0 + t] = w[t];
+  for (int t = threadIdx.x; t < n; t += blockDim.x) gstore(W + c0 + t, w[t]);
 }
 
 // Merge path, warp-cooperative: how many of the first d words of merge(A, B) come from A.  All words are distinct
@@ -533,7 +533,7 @@ __device__ __forceinline__ int merge_path_warp(const unsigned long long* A, int 
   while (lo < hi) {
     const int span = hi - lo, s = (span + 31) >> 5;
     const int i = lo + lane * s + s - 1;
-    const bool before = i < hi && A[i] < B[d - 1 - i];
+    const bool before = i < hi && gload(A + i) < gload(B + d - 1 - i);
     const int cnt = __popc(__ballot_sync(0xffffffffu, before));  // the predicate is monotone: the first cnt probes hold
     const int first_fail = lo + cnt * s + s - 1;                 // probe number cnt failed or lies beyond the range
     lo += cnt * s;
@@ -576,7 +576,7 @@ __global__ void __launch_bounds__(kSortMergeThreads) sort_merge_kernel(const Sor
   const int ia0 = split[0], ia1 = split[1], ib0 = d0 - ia0, ib1 = d1 - ia1;
   const int nA = ia1 - ia0, nB = ib1 - ib0, n = nA + nB;
   if (nA < 0 || nB < 0 || n > kSortMergeTile) return;  // only if the runs were not sorted: touch nothing out of range
-  for (int t = threadIdx.x; t < n; t += kSortMergeThreads) w[t] = t < nA ? A[ia0 + t] : B[ib0 + t - nA];
+  for (int t = threadIdx.x; t < n; t += kSortMergeThreads) w[t] = t < nA ? gload(A + ia0 + t) : gload(B + ib0 + t - nA);
   __syncthreads();
   // every thread merges kSortMergePerThread consecutive output words: its own split of the tile by binary search
   const unsigned long long* sa = w;
@@ -604,15 +604,15 @@ __global__ void __launch_bounds__(kSortMergeThreads) sort_merge_kernel(const Sor
 #pragma unroll
     for (int u = 0; u < kSortMergePerThread; ++u) {
       if (d + u < n) {
-        a.keys_out[e0 + o0 + d + u] = static_cast<long long>(out[u] >> idx_bits);
-        a.perm_out[e0 + o0 + d + u] = static_cast<int>(out[u] & low);
+        gstore(a.keys_out + e0 + o0 + d + u, out[u] >> idx_bits);
+        gstore(a.perm_out + e0 + o0 + d + u, out[u] & low);
       }
     }
     return;
   }
 #pragma unroll
   for (int u = 0; u < kSortMergePerThread; ++u)
-    if (d + u < n) dst[o0 + d + u] = out[u];
+    if (d + u < n) gstore(dst + o0 + d + u, out[u]);
 }
 
 // One block per kSortGatherTile 16-byte chunks of a list's rows: rows follow their keys, for every list of the
@@ -624,9 +624,9 @@ __global__ void __launch_bounds__(kSortGatherThreads) gather_all_kernel(const So
   int r;
   long long y;
   sort_block_item(a, r, y);
-  if (r == 0 && y == 0 && threadIdx.x == 0) *a.call_flag = 0;  // every reader of the word has finished: ready for the next call
-  const long long e0 = __ldg(a.edge_offsets + r);
-  const long long K = min(static_cast<long long>(__ldg(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
+  if (r == 0 && y == 0 && threadIdx.x == 0) gstore(a.call_flag, 0);  // every reader of the word has finished: ready for the next call
+  const long long e0 = gload(a.edge_offsets + r);
+  const long long K = min(static_cast<long long>(gload(a.edge_offsets + r + 1) - e0), static_cast<long long>(a.max_len));
   const long long chunks = K * a.row_ch;
   const long long first = y * kSortGatherTile;
   if (first >= chunks) return;
@@ -639,13 +639,13 @@ __global__ void __launch_bounds__(kSortGatherThreads) gather_all_kernel(const So
     const long long c = first + static_cast<long long>(u) * kSortGatherThreads + threadIdx.x;
     if (c < chunks) {
       const int row = static_cast<int>(c / a.row_ch), piece = static_cast<int>(c - static_cast<long long>(row) * a.row_ch);
-      v[u] = __ldg(src + static_cast<long long>(__ldg(perm + row)) * a.row_ch + piece);
+      v[u] = ldg128(src + static_cast<long long>(gload(perm + row)) * a.row_ch + piece);
     }
   }
 #pragma unroll
   for (int u = 0; u < kSortGatherUnroll; ++u) {
     const long long c = first + static_cast<long long>(u) * kSortGatherThreads + threadIdx.x;
-    if (c < chunks) __stcs(dst + c, v[u]);  // written once, read by a later kernel at the earliest
+    if (c < chunks) st128_stream(dst + c, v[u]);  // written once, read by a later kernel at the earliest
   }
 }
 

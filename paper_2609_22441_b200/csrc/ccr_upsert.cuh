@@ -48,33 +48,34 @@ __global__ void __launch_bounds__(kUpsertThreads) upsert_kernel(const UpsertArgs
         target[u] = -1;
         if (c < chunks) {
           const long long i = c / a.row_ch;
-          const int p = __ldg(a.positions + i);
+          const int p = gload(a.positions + i);
           if (p >= 0 && p < a.n_docs) target[u] = static_cast<long long>(p) * a.row_ch + (c - i * a.row_ch);
-          v[u] = __ldcs(src + c);
+          v[u] = CCR_CHK(src + c, 16) ? __ldcs(src + c) : make_uint4(0u, 0u, 0u, 0u);
         }
       }
 #pragma unroll
       for (int u = 0; u < kUpsertUnroll; ++u)
-        if (target[u] >= 0) dst[target[u]] = v[u];
+        if (target[u] >= 0 && CCR_CHK(dst + target[u], 16)) dst[target[u]] = v[u];
     }
   }
   if (a.src_author == nullptr && a.src_actor == nullptr && a.src_type == nullptr) return;
   for (long long i = tid; i < a.n; i += stride) {
-    const int p = __ldg(a.positions + i);
+    const int p = gload(a.positions + i);
     if (p < 0 || p >= a.n_docs) continue;
     if (a.dst_recs == nullptr) {
-      if (a.src_author) a.dst_author[p] = a.src_author[i];
+      if (a.src_author) gstore(a.dst_author + p, gload(a.src_author + i));
       continue;
     }
+    if (!CCR_CHK(a.dst_recs + p, static_cast<int>(sizeof(IdRec)))) continue;
     IdRec& r = a.dst_recs[p];
-    if (a.src_author) r.author = a.src_author[i];
+    if (a.src_author) r.author = gload(a.src_author + i);
     if (a.src_actor) {
 #pragma unroll
-      for (int s = 0; s < 4; ++s) r.actor[s] = s < a.max_actors ? a.src_actor[i * a.max_actors + s] : -1;
+      for (int s = 0; s < 4; ++s) r.actor[s] = s < a.max_actors ? gload(a.src_actor + i * a.max_actors + s) : -1;
     }
     if (a.src_type) {
 #pragma unroll
-      for (int s = 0; s < 4; ++s) r.type[s] = s < a.max_actors ? a.src_type[i * a.max_actors + s] : 0;
+      for (int s = 0; s < 4; ++s) r.type[s] = s < a.max_actors ? gload(a.src_type + i * a.max_actors + s) : 0;
     }
   }
 }
