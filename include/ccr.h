@@ -307,6 +307,9 @@ ccr_status ccr_join_batch_ex(const ccr_docstore* store, const ccr_join_io* io, u
  * list is spread over many SMs instead of one, and the rows of all lists are moved by one grid-wide gather:
  * 3 + ceil(log2(max_edge_len / 4096)) small kernels on `stream` (CCR_ERR_UNSUPPORTED if n_req x the tiles of
  * max_edge_len records exceed the 2^31 - 1 blocks of a grid).
+ * A batch in which some key does not leave that room is sorted list by list by the one-block kernel inside the same
+ * call (a device-side flag word of the store, taken in turn from 64 such words: at most 64 calls with perm_out may be
+ * in flight on one store at once, on any streams).
  * max_edge_len (HOST) must be at least the longest list; a longer list is cut there (its first max_edge_len
  * records are sorted among themselves, the rest of its output is left unwritten) and no access leaves the arrays.
  * All pointers DEVICE; no allocation, no synchronisation.
