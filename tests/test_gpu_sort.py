@@ -72,7 +72,8 @@ def test_sort_matches_oracle_on_config1_and_the_join_accepts_it(B, dups):
     store.free()
 
 
-@pytest.mark.parametrize("lens", [[0, 1, 2, 3, 31, 32, 33, 1023, 1024, 1025, 4097], [18_999, 19_000, 7], [19_001, 40_000, 5, 0, 65_537]])
+@pytest.mark.parametrize("lens", [[0, 1, 2, 3, 31, 32, 33, 1023, 1024, 1025, 4097], [18_999, 19_000, 7], [19_001, 40_000, 5, 0, 65_537],
+                                  [4096, 100, 0, 4095, 129, 128, 127]])  # the last: no list beyond one chunk, one block per list
 def test_sort_lengths_around_the_block_and_shared_memory_limits(B, lens):
     rng = np.random.default_rng(sum(lens))
     keys = np.concatenate([rng.integers(0, 10 * max(n, 1), size=n) for n in lens] + [np.empty(0, np.int64)]).astype(np.int64)
