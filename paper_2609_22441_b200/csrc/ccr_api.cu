@@ -34,6 +34,7 @@ constexpr int kSmemPerSm = 228 * 1024;
 constexpr int kDefaultKeyCap = 4096;
 constexpr long long kSmallLaunchCands = 131072;  // plain launches up to this size default to the two-phase kernel
 constexpr int kAutoSmemBudget = 160 * 1024;  // shared memory the warp-specialised kernel takes by default
+constexpr long long kIdsInL2Bytes = 64LL << 20;  // an author-id array up to this size is taken to stay in the 126 MB L2
 constexpr int kMaxTile = ccr::kMaxTileCands;
 constexpr size_t kStageBytes = 16u << 20;  // staging block of second-degree stores (ids uploaded from the host)
 #ifndef CCR_HOST_GROUPS
@@ -942,8 +943,13 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   // second-degree joins on the default warp split take the register-rebalanced form (12 + 8 warps); a configured
   // split, a configured sub-tile and the cosine section keep the 16-warp kernel
   const bool rebal = kRebalBuilt && use_ws && second && !cos && s->ws_streamers == 0 && s->tile == 0 && !(flags & CCR_FLAG_NO_REBALANCE);
-  const int n_str = rebal ? ccr::kRebalStreamers : (s->ws_streamers > 0 ? s->ws_streamers : 12);
-  const int n_res = rebal ? ccr::kRebalResolvers : (s->ws_resolvers > 0 ? s->ws_resolvers : 4);
+  // Default split of the 16-warp kernel: 12 streamers + 4 resolvers; over a store whose author ids do not stay in L2
+  // (8 bytes x n_docs beyond kIdsInL2Bytes) every candidate's id is a trip to HBM and a fifth resolver pays for the
+  // streamer it replaces (50M documents: 1666 -> 1639 us, sorted candidates 1643 -> 1615 us; 10 + 6: 1643 us; on the
+  // 1M-document store 11 + 5 costs 2 %: 207.0 against 202.9 us).
+  const bool ids_beyond_l2 = !second && static_cast<long long>(s->desc.n_docs) * 8 > kIdsInL2Bytes;
+  const int n_str = rebal ? ccr::kRebalStreamers : (s->ws_streamers > 0 ? s->ws_streamers : (ids_beyond_l2 ? 11 : 12));
+  const int n_res = rebal ? ccr::kRebalResolvers : (s->ws_resolvers > 0 ? s->ws_resolvers : (ids_beyond_l2 ? 5 : 4));
   const int cos_stage = cos ? 32 * (((s->cos_dim + 7) / 8) | 1) * 16 : 0;
   const int cos_bytes = cos ? ccr::ws_cos_bytes(n_str, cos_stage) : 0;
   // Shared memory of a block: the kernel's own arrays for a sub-tile of t candidates plus `area` bytes for the search
