@@ -944,10 +944,11 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   // split, a configured sub-tile and the cosine section keep the 16-warp kernel
   const bool rebal = kRebalBuilt && use_ws && second && !cos && s->ws_streamers == 0 && s->tile == 0 && !(flags & CCR_FLAG_NO_REBALANCE);
   // Default split of the 16-warp kernel: 12 streamers + 4 resolvers; over a store whose author ids do not stay in L2
-  // (8 bytes x n_docs beyond kIdsInL2Bytes) every candidate's id is a trip to HBM and a fifth resolver pays for the
+  // (the id array, or the 64-byte id records of a store with engagers, beyond kIdsInL2Bytes) every candidate's id is a trip to HBM and a fifth resolver pays for the
   // streamer it replaces (50M documents: 1666 -> 1639 us, sorted candidates 1643 -> 1615 us; 10 + 6: 1643 us; on the
   // 1M-document store 11 + 5 costs 2 %: 207.0 against 202.9 us).
-  const bool ids_beyond_l2 = !second && static_cast<long long>(s->desc.n_docs) * 8 > kIdsInL2Bytes;
+  const long long id_bytes = s->id_recs != nullptr ? static_cast<long long>(sizeof(ccr::IdRec)) : 8;  // what holds a document's author id
+  const bool ids_beyond_l2 = !second && static_cast<long long>(s->desc.n_docs) * id_bytes > kIdsInL2Bytes;
   const int n_str = rebal ? ccr::kRebalStreamers : (s->ws_streamers > 0 ? s->ws_streamers : (ids_beyond_l2 ? 11 : 12));
   const int n_res = rebal ? ccr::kRebalResolvers : (s->ws_resolvers > 0 ? s->ws_resolvers : (ids_beyond_l2 ? 5 : 4));
   const int cos_stage = cos ? 32 * (((s->cos_dim + 7) / 8) | 1) * 16 : 0;
