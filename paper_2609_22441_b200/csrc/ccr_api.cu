@@ -949,8 +949,12 @@ ccr_status join_impl(const ccr_docstore* cs, int32_t n_req, int64_t total_cands,
   // 1M-document store 11 + 5 costs 2 %: 207.0 against 202.9 us).
   const long long id_bytes = s->id_recs != nullptr ? static_cast<long long>(sizeof(ccr::IdRec)) : 8;  // what holds a document's author id
   const bool ids_beyond_l2 = !second && static_cast<long long>(s->desc.n_docs) * id_bytes > kIdsInL2Bytes;
-  const int n_str = rebal ? ccr::kRebalStreamers : (s->ws_streamers > 0 ? s->ws_streamers : (ids_beyond_l2 ? 11 : 12));
-  const int n_res = rebal ? ccr::kRebalResolvers : (s->ws_resolvers > 0 ? s->ws_resolvers : (ids_beyond_l2 ? 5 : 4));
+  // With the cosine section the streamers carry the arithmetic tail of every group as well, and a first-degree join
+  // over a store whose ids stay in L2 does better with one resolver less (config 1: 13 + 3 242 us, 12 + 4 251 us,
+  // 11 + 5 265 us, 14 + 2 269 us).
+  const bool cos_first = cos && !second && !ids_beyond_l2;
+  const int n_str = rebal ? ccr::kRebalStreamers : (s->ws_streamers > 0 ? s->ws_streamers : (ids_beyond_l2 ? 11 : (cos_first ? 13 : 12)));
+  const int n_res = rebal ? ccr::kRebalResolvers : (s->ws_resolvers > 0 ? s->ws_resolvers : (ids_beyond_l2 ? 5 : (cos_first ? 3 : 4)));
   const int cos_stage = cos ? 32 * (((s->cos_dim + 7) / 8) | 1) * 16 : 0;
   const int cos_bytes = cos ? ccr::ws_cos_bytes(n_str, cos_stage) : 0;
   // Shared memory of a block: the kernel's own arrays for a sub-tile of t candidates plus `area` bytes for the search
