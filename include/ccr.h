@@ -436,9 +436,9 @@ typedef struct {
                                  kernel) or 4096 (the others)                                                */
   int32_t ws_streamers;       /* warp-specialised kernel: row-streaming warps per block (1..14)              */
   int32_t ws_resolvers;       /* warp-specialised kernel: search warps per block (1..8); sum <= 16; set both
-                                 or neither (unset = 12 + 4; 11 + 5 over a store whose author ids — 8 bytes per document,
-                                 64 with engager slots — exceed 64 MB and do not stay in L2; 13 + 3 for a first-degree
-                                 join with the cosine section over a smaller store; second-degree joins: 12 + 8 in the 20-warp form with
+                                 or neither (unset = 12 + 4; one warp moves to the resolvers over a store whose author
+                                 ids — 8 bytes per document, 64 with engager slots — exceed 64 MB and do not stay in
+                                 L2, one to the streamers for a first-degree join with the cosine section; second-degree joins: 12 + 8 in the 20-warp form with
                                  registers moved from the search warps to the streaming warps, which a configured
                                  split switches off)                                                           */
   int32_t blocks_per_sm;      /* two-phase kernel: cap on resident blocks per SM (1..8)                      */
